@@ -1,0 +1,259 @@
+/*
+ * NOVA-KV CPU oracle (TEST INFRASTRUCTURE ONLY).
+ *
+ * A plain, slow, float64 restatement of what the decode and append paths compute, written
+ * from the paper.  It is used by the tests, by the smoke check and by the benchmark's CPU
+ * baseline; the product path never calls it.  It shares no code with the CUDA library.
+ *
+ *   encode  : Algorithm 1 line 7 and Sec. 2.2 ("Quantization"): coefficients
+ *             r = (k - kbar) R_K, s = (v - vbar) R_V, then per group of g coefficients the
+ *             index of the nearest codeword (exact Euclidean search, App. B "Calibration").
+ *   decode  : Sec. 2.2 reconstruction k^ = Q(r) R_K^{-1} + kbar (Theorem 1 text), v^ = Q(s) R_V^T
+ *             + vbar (Corollary 1), followed by textbook attention, Eq. "scores":
+ *             softmax(q k^T / sqrt(d)) v.  Keys and values are dequantised EXPLICITLY; the
+ *             query fold, the dropped mean (Lemma S1) and the transform-domain value
+ *             accumulation used on the GPU are deliberately NOT used here.
+ *   R_K^{-1} is taken from the stored synthesis matrix: R_K^{-1} = (R_K^{-T})^T.
+ *
+ * Precision: everything is float64, except the one place where floating point decides an
+ * integer.  The library boundary fixes that decision's arithmetic (see the encode entry of
+ * the public header): the float64 coefficient is rounded once to binary32 and the squared
+ * distance to each codeword is evaluated in binary32 as
+ *      fma(e3,e3, fma(e2,e2, fma(e1,e1, e0*e0))),   e_i = coef_i - codeword_i,
+ * visiting codewords in ascending index and keeping the first minimum.  The oracle takes the
+ * decision in that same precision and, beside it, reports the float64 decision and the
+ * float64 relative gap (d2 - d1) / d1 between the two smallest distances, which is how
+ * near-ties are counted.
+ *
+ * Pins (tests/test_oracle_pins.py): exact invariance of the attention products when the
+ * quantiser is the identity, generalised Parseval relation (Prop. 1), Lemma S1, one-token
+ * and equal-logit caches, brute force against an independently written search, hand-built
+ * tie cases, split invariance, planted needle.  No end-to-end numeric value is printed in
+ * the paper, so the numeric end-to-end parity is pinned by those identities only.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <float.h>
+
+typedef struct {
+    int n_kv_heads, head_dim, group_size, codebook_size;
+    const double* rk;        /* [Hkv][d][d]  analysis  R_K            */
+    const double* rk_inv_t;  /* [Hkv][d][d]  R_K^{-T}                 */
+    const double* rv;        /* [Hkv][d][d]  R_V (orthogonal)         */
+    const double* k_mean;    /* [Hkv][d]                              */
+    const double* v_mean;    /* [Hkv][d]                              */
+    const double* cb_k;      /* [Hkv][L][C][g]                        */
+    const double* cb_v;      /* [Hkv][L][C][g]                        */
+} oracle_tables;
+
+/* row vector times matrix: y[c] = sum_r x[r] M[r][c] */
+static void rowvec_mat(const double* x, const double* m, int d, double* y)
+{
+    for (int c = 0; c < d; ++c) y[c] = 0.0;
+    for (int r = 0; r < d; ++r)
+        for (int c = 0; c < d; ++c) y[c] += x[r] * m[r * d + c];
+}
+
+/* row vector times transposed matrix: y[r] = sum_c x[c] M[r][c] */
+static void rowvec_mat_t(const double* x, const double* m, int d, double* y)
+{
+    for (int r = 0; r < d; ++r) {
+        double s = 0.0;
+        for (int c = 0; c < d; ++c) s += x[c] * m[r * d + c];
+        y[r] = s;
+    }
+}
+
+/* Transform coefficients of one vector: (x - mean) M. */
+void oracle_coefficients(const double* x, const double* mean, const double* m, int d, double* out)
+{
+    double* xc = (double*)malloc(sizeof(double) * d);
+    for (int i = 0; i < d; ++i) xc[i] = x[i] - mean[i];
+    rowvec_mat(xc, m, d, out);
+    free(xc);
+}
+
+/*
+ * Nearest-codeword search for one group (Sec. 2.2; lowest index wins ties).
+ * coef: g float64 coefficients.  cb: [C][g] float64 holding binary32-representable values.
+ * Returns the binary32 decision; *idx64 gets the float64 decision and *gap the float64
+ * relative gap between the two smallest float64 distances (DBL_MAX if d1 == 0 and d2 > 0,
+ * 0 if both are 0).
+ */
+static int search_group(const double* coef, const double* cb, int g, int C, int* idx64, double* gap)
+{
+    float best32 = 0.f;
+    int bi32 = -1;
+    double d1 = DBL_MAX, d2 = DBL_MAX;
+    int bi64 = -1;
+    for (int c = 0; c < C; ++c) {
+        const double* cw = cb + (long)c * g;
+        /* binary32 decision, the arithmetic the library boundary documents */
+        float acc = 0.f;
+        for (int i = 0; i < g; ++i) {
+            float e = (float)coef[i] - (float)cw[i];
+            acc = (i == 0) ? e * e : fmaf(e, e, acc);
+        }
+        if (bi32 < 0 || acc < best32) { best32 = acc; bi32 = c; }
+        /* float64 distances for the near-tie accounting */
+        double s = 0.0;
+        for (int i = 0; i < g; ++i) {
+            double e = coef[i] - cw[i];
+            s += e * e;
+        }
+        if (s < d1) { d2 = d1; d1 = s; bi64 = c; }
+        else if (s < d2) { d2 = s; }
+    }
+    if (idx64) *idx64 = bi64;
+    if (gap) *gap = (d1 > 0.0) ? (d2 - d1) / d1 : (d2 > 0.0 ? DBL_MAX : 0.0);
+    return bi32;
+}
+
+/*
+ * Encode from coefficients that are already given (float64 holding the values to search).
+ * coef: [n][d]; cb: [L][C][g]; idx: [n][L].  idx64 / gap may be NULL.
+ */
+void oracle_search(const double* coef, long n, int d, int g, int C, const double* cb,
+                   uint8_t* idx, uint8_t* idx64, double* gap)
+{
+    int L = d / g;
+#pragma omp parallel for schedule(static)
+    for (long j = 0; j < n; ++j) {
+        for (int l = 0; l < L; ++l) {
+            int i64; double gp;
+            int i32 = search_group(coef + j * d + l * g, cb + (long)l * C * g, g, C, &i64, &gp);
+            idx[j * L + l] = (uint8_t)i32;
+            if (idx64) idx64[j * L + l] = (uint8_t)i64;
+            if (gap) gap[j * L + l] = gp;
+        }
+    }
+}
+
+/*
+ * Write path for n tokens: k, v [n][Hkv][d] -> kidx, vidx [n][Hkv][L] (+ float64 decision and
+ * gap arrays of the same shape, may be NULL).
+ */
+void oracle_encode(const oracle_tables* t, const double* k, const double* v, long n,
+                   uint8_t* kidx, uint8_t* vidx, uint8_t* kidx64, uint8_t* vidx64,
+                   double* kgap, double* vgap)
+{
+    const int d = t->head_dim, g = t->group_size, C = t->codebook_size, H = t->n_kv_heads;
+    const int L = d / g;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long j = 0; j < n; ++j) {
+        for (int h = 0; h < H; ++h) {
+            double* coef = (double*)malloc(sizeof(double) * d);
+            long o = (j * H + h);
+            /* keys */
+            oracle_coefficients(k + o * d, t->k_mean + (long)h * d, t->rk + (long)h * d * d, d, coef);
+            for (int l = 0; l < L; ++l) {
+                int i64; double gp;
+                int i32 = search_group(coef + l * g, t->cb_k + ((long)h * L + l) * C * g, g, C, &i64, &gp);
+                kidx[o * L + l] = (uint8_t)i32;
+                if (kidx64) kidx64[o * L + l] = (uint8_t)i64;
+                if (kgap) kgap[o * L + l] = gp;
+            }
+            /* values */
+            oracle_coefficients(v + o * d, t->v_mean + (long)h * d, t->rv + (long)h * d * d, d, coef);
+            for (int l = 0; l < L; ++l) {
+                int i64; double gp;
+                int i32 = search_group(coef + l * g, t->cb_v + ((long)h * L + l) * C * g, g, C, &i64, &gp);
+                vidx[o * L + l] = (uint8_t)i32;
+                if (vidx64) vidx64[o * L + l] = (uint8_t)i64;
+                if (vgap) vgap[o * L + l] = gp;
+            }
+            free(coef);
+        }
+    }
+}
+
+/* Dequantise one key: r^ = concat_l cb_k[l][idx[l]];  k^ = r^ (R_K^{-T})^T + kbar. */
+static void reconstruct_key(const oracle_tables* t, int h, const uint8_t* idx, double* out)
+{
+    const int d = t->head_dim, g = t->group_size, C = t->codebook_size, L = d / g;
+    double* r = (double*)malloc(sizeof(double) * d);
+    for (int l = 0; l < L; ++l)
+        for (int i = 0; i < g; ++i)
+            r[l * g + i] = t->cb_k[(((long)h * L + l) * C + idx[l]) * g + i];
+    rowvec_mat_t(r, t->rk_inv_t + (long)h * d * d, d, out);   /* r (R_K^{-T})^T = r R_K^{-1} */
+    for (int i = 0; i < d; ++i) out[i] += t->k_mean[(long)h * d + i];
+    free(r);
+}
+
+/* Dequantise one value: s^ = concat_l cb_v[l][idx[l]];  v^ = s^ R_V^T + vbar. */
+static void reconstruct_value(const oracle_tables* t, int h, const uint8_t* idx, double* out)
+{
+    const int d = t->head_dim, g = t->group_size, C = t->codebook_size, L = d / g;
+    double* s = (double*)malloc(sizeof(double) * d);
+    for (int l = 0; l < L; ++l)
+        for (int i = 0; i < g; ++i)
+            s[l * g + i] = t->cb_v[(((long)h * L + l) * C + idx[l]) * g + i];
+    rowvec_mat_t(s, t->rv + (long)h * d * d, d, out);         /* s R_V^T */
+    for (int i = 0; i < d; ++i) out[i] += t->v_mean[(long)h * d + i];
+    free(s);
+}
+
+/* kidx, vidx: [S][Hkv][L] -> k_hat, v_hat: [S][Hkv][d] */
+void oracle_reconstruct(const oracle_tables* t, const uint8_t* kidx, const uint8_t* vidx, long S,
+                        double* k_hat, double* v_hat)
+{
+    const int d = t->head_dim, H = t->n_kv_heads, L = d / t->group_size;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long j = 0; j < S; ++j)
+        for (int h = 0; h < H; ++h) {
+            long o = j * H + h;
+            if (k_hat) reconstruct_key(t, h, kidx + o * L, k_hat + o * d);
+            if (v_hat) reconstruct_value(t, h, vidx + o * L, v_hat + o * d);
+        }
+}
+
+/*
+ * Textbook single-query attention over explicit keys and values (Eq. "scores"):
+ * q: [Hq][d];  k, v: [S][Hkv][d];  out: [Hq][d].  Query head h reads KV head h / (Hq/Hkv).
+ */
+void oracle_attention(const double* q, const double* k, const double* v, long S, int Hq, int Hkv,
+                      int d, double sm_scale, double* out)
+{
+    const int hg = Hq / Hkv;
+#pragma omp parallel for schedule(static)
+    for (int h = 0; h < Hq; ++h) {
+        const int kv = h / hg;
+        double* z = (double*)malloc(sizeof(double) * (S > 0 ? S : 1));
+        double zmax = -DBL_MAX;
+        for (long j = 0; j < S; ++j) {
+            const double* kj = k + (j * Hkv + kv) * d;
+            double s = 0.0;
+            for (int i = 0; i < d; ++i) s += q[(long)h * d + i] * kj[i];
+            z[j] = s * sm_scale;
+            if (z[j] > zmax) zmax = z[j];
+        }
+        double den = 0.0;
+        for (long j = 0; j < S; ++j) { z[j] = exp(z[j] - zmax); den += z[j]; }
+        for (int i = 0; i < d; ++i) out[(long)h * d + i] = 0.0;
+        for (long j = 0; j < S; ++j) {
+            const double p = z[j] / den;
+            const double* vj = v + (j * Hkv + kv) * d;
+            for (int i = 0; i < d; ++i) out[(long)h * d + i] += p * vj[i];
+        }
+        free(z);
+    }
+}
+
+/*
+ * Decode step for one sequence: dequantise the whole cache, then textbook attention.
+ * q: [Hq][d]; kidx, vidx: [S][Hkv][L]; out: [Hq][d].  S == 0 gives zeros.
+ */
+void oracle_decode(const oracle_tables* t, const double* q, const uint8_t* kidx,
+                   const uint8_t* vidx, long S, int Hq, double sm_scale, double* out)
+{
+    const int d = t->head_dim, H = t->n_kv_heads;
+    if (S <= 0) { memset(out, 0, sizeof(double) * (size_t)Hq * d); return; }
+    double* k_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
+    double* v_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
+    oracle_reconstruct(t, kidx, vidx, S, k_hat, v_hat);
+    oracle_attention(q, k_hat, v_hat, S, Hq, H, d, sm_scale, out);
+    free(k_hat);
+    free(v_hat);
+}

@@ -1,0 +1,180 @@
+"""ctypes wrapper around the float64 CPU oracle (TEST INFRASTRUCTURE ONLY).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline / reference arm may import
+this module.  It builds ``novakv_oracle.c`` with gcc next to the source and exposes the
+oracle's functions on numpy arrays.  It imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_DIR = Path(__file__).resolve().parent
+_SRC = _DIR / "novakv_oracle.c"
+_LIB = _DIR / "libnovakv_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    if not force and _LIB.exists() and _LIB.stat().st_mtime >= _SRC.stat().st_mtime:
+        return _LIB
+    flags = ["-O2", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC"]
+    try:
+        with open("/proc/cpuinfo") as f:
+            if " fma " in f.read():
+                flags.append("-mfma")     # fmaf() becomes one instruction; results are identical
+    except OSError:
+        pass
+    res = subprocess.run(["gcc", *flags, str(_SRC), "-lm", "-o", str(_LIB)],
+                         capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("gcc failed building the oracle:\n" + res.stdout + res.stderr)
+    return _LIB
+
+
+class _Tables(ctypes.Structure):
+    _fields_ = [("n_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int),
+                ("group_size", ctypes.c_int), ("codebook_size", ctypes.c_int),
+                ("rk", ctypes.c_void_p), ("rk_inv_t", ctypes.c_void_p), ("rv", ctypes.c_void_p),
+                ("k_mean", ctypes.c_void_p), ("v_mean", ctypes.c_void_p),
+                ("cb_k", ctypes.c_void_p), ("cb_v", ctypes.c_void_p)]
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(str(build()))
+        for name in ("oracle_coefficients", "oracle_search", "oracle_encode", "oracle_reconstruct",
+                     "oracle_attention", "oracle_decode"):
+            getattr(_lib, name).restype = None
+    return _lib
+
+
+def cpu_threads() -> int:
+    """Threads the oracle's OpenMP loops will use (affinity-limited core count)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env)
+    return len(os.sched_getaffinity(0))
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _u8(a):
+    return np.ascontiguousarray(a, dtype=np.uint8)
+
+
+class Oracle:
+    """The oracle bound to one layer's calibration tables (float32 values widened to float64)."""
+
+    def __init__(self, rk, rk_inv_t, rv, k_mean, v_mean, cb_k, cb_v):
+        self.rk, self.rk_inv_t, self.rv = _f64(rk), _f64(rk_inv_t), _f64(rv)
+        self.k_mean, self.v_mean = _f64(k_mean), _f64(v_mean)
+        self.cb_k, self.cb_v = _f64(cb_k), _f64(cb_v)
+        self.n_kv_heads, self.d = self.rk.shape[0], self.rk.shape[1]
+        self.n_groups, self.codebook_size, self.g = self.cb_k.shape[1:]
+        assert self.n_groups * self.g == self.d
+        self._t = _Tables(self.n_kv_heads, self.d, self.g, self.codebook_size,
+                          self.rk.ctypes.data, self.rk_inv_t.ctypes.data, self.rv.ctypes.data,
+                          self.k_mean.ctypes.data, self.v_mean.ctypes.data,
+                          self.cb_k.ctypes.data, self.cb_v.ctypes.data)
+
+    @classmethod
+    def from_calibration(cls, cal):
+        return cls(cal.rk, cal.rk_inv_t, cal.rv, cal.k_mean, cal.v_mean, cal.cb_k, cal.cb_v)
+
+    # -- write path -------------------------------------------------------------------
+    def coefficients(self, x, which: str):
+        """(x - mean) R for x of shape [n][Hkv][d]; which in {"k", "v"}."""
+        x = _f64(x)
+        n = x.shape[0]
+        out = np.empty_like(x)
+        m, mean = (self.rk, self.k_mean) if which == "k" else (self.rv, self.v_mean)
+        lib = _load()
+        for j in range(n):
+            for h in range(self.n_kv_heads):
+                lib.oracle_coefficients(ctypes.c_void_p(x[j, h].ctypes.data),
+                                        ctypes.c_void_p(mean[h].ctypes.data),
+                                        ctypes.c_void_p(m[h].ctypes.data), self.d,
+                                        ctypes.c_void_p(out[j, h].ctypes.data))
+        return out
+
+    def search(self, coef, kvh: int, which: str):
+        """Nearest-codeword search of given coefficients [n][d] against one head's codebooks.
+
+        Returns (idx binary32 decision, idx float64 decision, float64 relative gap), each [n][L].
+        """
+        coef = _f64(coef)
+        n = coef.shape[0]
+        cb = (self.cb_k if which == "k" else self.cb_v)[kvh]
+        idx = np.empty((n, self.n_groups), np.uint8)
+        idx64 = np.empty_like(idx)
+        gap = np.empty((n, self.n_groups), np.float64)
+        _load().oracle_search(ctypes.c_void_p(coef.ctypes.data), ctypes.c_long(n), self.d, self.g,
+                              self.codebook_size, ctypes.c_void_p(cb.ctypes.data),
+                              ctypes.c_void_p(idx.ctypes.data), ctypes.c_void_p(idx64.ctypes.data),
+                              ctypes.c_void_p(gap.ctypes.data))
+        return idx, idx64, gap
+
+    def encode(self, k, v, with_gaps: bool = True):
+        """k, v: [n][Hkv][d] -> dict(kidx, vidx[, kidx64, vidx64, kgap, vgap]), each [n][Hkv][L]."""
+        k, v = _f64(k), _f64(v)
+        n = k.shape[0]
+        shp = (n, self.n_kv_heads, self.n_groups)
+        res = dict(kidx=np.empty(shp, np.uint8), vidx=np.empty(shp, np.uint8))
+        if with_gaps:
+            res.update(kidx64=np.empty(shp, np.uint8), vidx64=np.empty(shp, np.uint8),
+                       kgap=np.empty(shp, np.float64), vgap=np.empty(shp, np.float64))
+
+        def p(name):
+            return ctypes.c_void_p(res[name].ctypes.data) if name in res else ctypes.c_void_p(0)
+
+        _load().oracle_encode(ctypes.byref(self._t), ctypes.c_void_p(k.ctypes.data),
+                              ctypes.c_void_p(v.ctypes.data), ctypes.c_long(n), p("kidx"), p("vidx"),
+                              p("kidx64"), p("vidx64"), p("kgap"), p("vgap"))
+        return res
+
+    # -- read path --------------------------------------------------------------------
+    def reconstruct(self, kidx, vidx):
+        """Explicit dequantisation: indices [S][Hkv][L] -> (k_hat, v_hat) [S][Hkv][d]."""
+        kidx, vidx = _u8(kidx), _u8(vidx)
+        s = kidx.shape[0]
+        k_hat = np.empty((s, self.n_kv_heads, self.d))
+        v_hat = np.empty((s, self.n_kv_heads, self.d))
+        _load().oracle_reconstruct(ctypes.byref(self._t), ctypes.c_void_p(kidx.ctypes.data),
+                                   ctypes.c_void_p(vidx.ctypes.data), ctypes.c_long(s),
+                                   ctypes.c_void_p(k_hat.ctypes.data), ctypes.c_void_p(v_hat.ctypes.data))
+        return k_hat, v_hat
+
+    def decode(self, q, kidx, vidx, sm_scale: float | None = None):
+        """One decode step of one sequence: q [Hq][d], indices [S][Hkv][L] -> out [Hq][d]."""
+        q = _f64(q)
+        kidx, vidx = _u8(kidx), _u8(vidx)
+        hq = q.shape[0]
+        s = kidx.shape[0]
+        scale = 1.0 / np.sqrt(self.d) if sm_scale is None else float(sm_scale)
+        out = np.empty((hq, self.d))
+        _load().oracle_decode(ctypes.byref(self._t), ctypes.c_void_p(q.ctypes.data),
+                              ctypes.c_void_p(kidx.ctypes.data), ctypes.c_void_p(vidx.ctypes.data),
+                              ctypes.c_long(s), hq, ctypes.c_double(scale),
+                              ctypes.c_void_p(out.ctypes.data))
+        return out
+
+
+def attention(q, k, v, sm_scale: float | None = None):
+    """Textbook attention on explicit float64 keys/values: q [Hq][d], k/v [S][Hkv][d]."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    hq, d = q.shape
+    s, hkv, _ = k.shape
+    scale = 1.0 / np.sqrt(d) if sm_scale is None else float(sm_scale)
+    out = np.empty((hq, d))
+    _load().oracle_attention(ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(k.ctypes.data),
+                             ctypes.c_void_p(v.ctypes.data), ctypes.c_long(s), hq, hkv, d,
+                             ctypes.c_double(scale), ctypes.c_void_p(out.ctypes.data))
+    return out
