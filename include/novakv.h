@@ -1,0 +1,214 @@
+/*
+ * novakv — decode-step attention over a 2-bit, fixed-width, vector-quantised KV cache, and the
+ * append-time encoder that fills it (NOVA-KV, arxiv 2608.04074).  C ABI, CUDA sm_100a.
+ *
+ * Notation (App. A of the paper): row vectors, linear maps act on the right (x R).  B sequences,
+ * Hq query heads, Hkv KV heads, Hg = Hq/Hkv, d head dimension, g = 4 coefficients per group,
+ * L = d/g groups, C = 256 codewords per group.  Query head h reads KV head h / Hg.
+ *
+ * Cache format (Sec. 2.2 "Quantization", Sec. 5 "Bit rate"): per token and KV head, L uint8
+ * codeword indices for the key and L for the value: 8/g = 2 bits per cached element, no
+ * per-token metadata.  Pages hold 64 tokens.  Two caller-owned device pools of equal geometry:
+ *     key pool    uint8 [n_pages][Hkv][64][L]        token-major
+ *     value pool  uint8 [n_pages][Hkv][4][L][16]     four 16-token blocks, group-major in a block
+ * page_table[seq][i] (int32, row length max_pages_per_seq) names the page of tokens 64i..64i+63.
+ *
+ * Ownership: the context owns device copies of the calibration tables and one device status
+ * word.  Pools, page tables, lengths, queries, outputs and workspaces are the caller's device
+ * memory (device pointers unless a parameter says "host").  Calls are asynchronous on `stream`
+ * unless stated.  A context is used from one host thread at a time.
+ *
+ * Errors: every entry point validates its arguments on the host and returns a status; nothing
+ * aborts.  Faults only the device can see (page id out of range, length beyond the page table, a
+ * pipeline wait that ran out) set bits in the device status word, skip the offending work and
+ * never trap; read them with novakv_last_device_status.
+ *
+ * Determinism: for fixed inputs, shapes and device, outputs are bitwise reproducible.
+ */
+#ifndef NOVAKV_H
+#define NOVAKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct novakv_ctx novakv_ctx;        /* opaque */
+typedef void* novakv_stream;                 /* a cudaStream_t; NULL is the default stream */
+
+typedef enum {
+    NOVAKV_OK = 0,
+    NOVAKV_EINVAL = 1,        /* NULL / negative / inconsistent argument */
+    NOVAKV_ESHAPE = 2,        /* geometry this build has no kernel for */
+    NOVAKV_ENOCALIB = 3,      /* layer has no calibration loaded */
+    NOVAKV_EPAGE = 4,         /* page-table geometry inconsistent */
+    NOVAKV_EWORKSPACE = 5,    /* workspace NULL or too small */
+    NOVAKV_ECUDA = 6,         /* a CUDA runtime call failed */
+    NOVAKV_EUNSUPPORTED = 7   /* value codebook not binary16-representable, etc. */
+} novakv_status;
+
+/* Bits of the device status word. */
+#define NOVAKV_DEV_BAD_PAGE      1u   /* a page id was outside [0, n_pages) */
+#define NOVAKV_DEV_BAD_LENGTH    2u   /* a sequence length exceeded 64 * max_pages_per_seq */
+#define NOVAKV_DEV_WAIT_TIMEOUT  4u   /* an in-kernel pipeline wait hit its iteration limit */
+#define NOVAKV_DEV_BAD_TOKEN     8u   /* an appended token named a sequence slot or position out of range */
+
+typedef struct {
+    int n_layers;
+    int n_q_heads;       /* Hq */
+    int n_kv_heads;      /* Hkv, divides Hq; Hq/Hkv in {1,2,4,8} */
+    int head_dim;        /* d in {64, 128}; (d = 128, Hq/Hkv = 8) is not supported */
+    int group_size;      /* must be 4   */
+    int codebook_size;   /* must be 256 */
+    int page_tokens;     /* must be 64  */
+    int device;          /* CUDA device ordinal */
+} novakv_config;
+
+/*
+ * Calibration tables of one layer (App. B "Bits per element": per (layer, KV head) the three
+ * d x d transforms, the mean and L codebooks; value codebooks and a value mean are added here
+ * because values are vector-quantised too, App. B "Value quantizer").  HOST pointers, float32,
+ * row-major, the equal-volume grouping of Sec. 4 already folded into the columns, so that
+ * group l owns coefficient columns [4l, 4l+4).
+ *   rk        [Hkv][d][d]   analysis    r = (k - k_mean) rk          (Theorem 1)
+ *   rk_inv_t  [Hkv][d][d]   R_K^{-T}    q' = q rk_inv_t; also the synthesis matrix (k^ = r^ rk_inv_t^T + k_mean)
+ *   rv        [Hkv][d][d]   orthogonal  s = (v - v_mean) rv,  v^ = s^ rv^T + v_mean   (Corollary 1)
+ *   k_mean    [Hkv][d]      may be NULL (= 0)
+ *   v_mean    [Hkv][d]      may be NULL (= 0)
+ *   cb_k      [Hkv][L][256][4]
+ *   cb_v      [Hkv][L][256][4]   every entry must be exactly representable in IEEE binary16
+ */
+typedef struct {
+    const float* rk;
+    const float* rk_inv_t;
+    const float* rv;
+    const float* k_mean;
+    const float* v_mean;
+    const float* cb_k;
+    const float* cb_v;
+} novakv_calibration;
+
+novakv_status novakv_create(novakv_ctx** out, const novakv_config* cfg);
+novakv_status novakv_destroy(novakv_ctx* ctx);
+const char* novakv_status_string(novakv_status s);
+
+/*
+ * Algorithm 1 lines 1-6 produce these tables offline; this call copies them to the device
+ * (synchronous; the caller keeps its memory).  Returns NOVAKV_EUNSUPPORTED if cb_v holds a value
+ * that binary16 cannot represent exactly (the decode kernel keeps value codewords in binary16;
+ * snap them offline, as the paper does for its codebooks, so that encoder and decoder agree).
+ */
+novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, const novakv_calibration* host);
+
+/* Bytes of one page of the key pool (= of the value pool), all KV heads: Hkv * 64 * L. */
+size_t novakv_page_bytes(const novakv_ctx* ctx);
+
+/* Workspace bytes novakv_decode_attention needs for `batch` sequences (device memory, 256-byte aligned). */
+size_t novakv_decode_workspace_bytes(const novakv_ctx* ctx, int batch);
+
+/*
+ * Write path (Algorithm 1 line 7; Sec. 4 "Complexity"): for each new token t and KV head,
+ *     r = (k_t - k_mean) rk,   s = (v_t - v_mean) rv          accumulated in binary64,
+ * each coefficient rounded once to binary32, then for every group l the index of the nearest
+ * codeword (exact Euclidean search, App. B "Calibration").  The squared distance is evaluated
+ * in binary32 as fma(e3,e3, fma(e2,e2, fma(e1,e1, e0*e0))), e_i = coef_i - codeword_i, visiting
+ * codewords in ascending index and keeping the first minimum (lowest index wins a tie).
+ * The 2L index bytes go to page page_table[tok_seq[t]][tok_pos[t]/64] at slot tok_pos[t]%64, and
+ * seq_lens[tok_seq[t]] becomes max(seq_lens[tok_seq[t]], tok_pos[t]+1).
+ *   k_new, v_new  bf16 [n_tokens][Hkv][d]
+ *   tok_seq, tok_pos  int32 [n_tokens]; two tokens of one call must not share (seq, pos)
+ *   n_tokens = 0 is a no-op.  Out-of-range tokens/pages set device status bits and are skipped.
+ */
+novakv_status novakv_encode_append(novakv_ctx* ctx, int layer,
+    const void* k_new, const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos,
+    int n_tokens, uint8_t* k_pages, uint8_t* v_pages, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
+    novakv_stream stream);
+
+/*
+ * Read path (Algorithm 1 line 8; App. B "Decoding kernel and read path"): one decode step for
+ * `batch` sequences directly on the index cache, never materialising keys or values:
+ *     q'_h = q_h rk_inv_t                                     one d x d product per head
+ *     z_hj = sm_scale * sum_l < q'_h[4l..4l+3], cb_k[l][kidx_j[l]] >     (k_mean dropped: Lemma S1)
+ *     p_h  = softmax_j(z_hj)  over positions 0 .. seq_lens[b]-1
+ *     o_h  = ( sum_j p_hj concat_l cb_v[l][vidx_j[l]] ) rv^T + v_mean    (Remark after Corollary 1)
+ * computed split over the sequence with an exact log-sum-exp merge, binary32 accumulation.
+ *   q    bf16 [batch][Hq][d]
+ *   out  [batch][Hq][d], float32 if out_is_fp32 else bf16; a sequence of length 0 yields zeros
+ *   workspace  at least novakv_decode_workspace_bytes(ctx, batch) bytes; contents are scratch
+ */
+novakv_status novakv_decode_attention(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch,
+    float sm_scale, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
+    novakv_stream stream);
+
+/* Synchronises `stream`, returns the device status word in *word and clears it. */
+novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word);
+
+/*
+ * One serving step from HOST buffers (Fig. 1(b): write path then read path): copies the new
+ * tokens and the queries to the device, appends, decodes and copies the output back, all on
+ * `stream`, then synchronises it.  The index cache itself stays resident on the device.
+ *   k_new_host, v_new_host  bf16 [n_tokens][Hkv][d];  tok_seq_host, tok_pos_host int32 [n_tokens]
+ *   q_host   bf16 [batch][Hq][d];  out_host  float32 [batch][Hq][d]
+ *   staging  device scratch of novakv_step_staging_bytes(ctx, batch, n_tokens) bytes
+ * For pinned host memory the copies are asynchronous until the final synchronise.
+ */
+size_t novakv_step_staging_bytes(const novakv_ctx* ctx, int batch, int n_tokens);
+novakv_status novakv_step_host(novakv_ctx* ctx, int layer,
+    const void* k_new_host, const void* v_new_host, const int32_t* tok_seq_host,
+    const int32_t* tok_pos_host, int n_tokens, const void* q_host,
+    uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int32_t* seq_lens, int batch, float sm_scale, float* out_host,
+    void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+    novakv_stream stream);
+
+/* ---- measurement and staged-parity helpers (not part of the serving contract) ---------------- */
+
+/*
+ * Search only (second half of the write path): coefficients are given, float32 [n][Hkv][d]
+ * (device); writes logical indices uint8 [n][Hkv][L] (device).  which = 0 keys, 1 values.
+ */
+novakv_status novakv_search_coefficients(novakv_ctx* ctx, int layer, int which, const float* coef,
+    int n, uint8_t* idx_out, novakv_stream stream);
+
+/*
+ * Uncompressed comparator: the same decode step on a bf16 paged cache
+ * (pools bf16 [n_pages][Hkv][64][d] for keys and for values), textbook attention with the same
+ * split-and-merge structure.  Used to report the compression speed-up on identical shapes.
+ * window > 0 restricts attention to the last `window` positions (sliding-window layers).
+ */
+size_t novakv_bf16_workspace_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq);
+novakv_status novakv_bf16_decode_attention(novakv_ctx* ctx, const void* q,
+    const void* k_pages_bf16, const void* v_pages_bf16, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch,
+    float sm_scale, int window, void* out, int out_is_fp32, void* workspace,
+    size_t workspace_bytes, novakv_stream stream);
+
+/*
+ * Per-kernel device timing for roofline accounting: when enabled, the library brackets the
+ * dominant kernel of each decode / append call with CUDA events on the call's stream.
+ * novakv_profile_read synchronises, returns the accumulated milliseconds and launch counts since
+ * the last read and resets them.  kind: 0 = decode stage 1 (index scan), 1 = encode kernel,
+ * 2 = bf16 comparator stage 1.
+ */
+novakv_status novakv_profile_enable(novakv_ctx* ctx, int on);
+novakv_status novakv_profile_read(novakv_ctx* ctx, int kind, double* total_ms, long* launches);
+
+/*
+ * Test knob: number of CTAs the decode scan kernel is launched with (0 = one per SM, the default;
+ * values above the SM count are clamped).  The result must not depend on it beyond binary32
+ * rounding, because the split over the sequence is merged exactly (App. B, two-stage split-KV).
+ */
+novakv_status novakv_debug_set_scan_ctas(novakv_ctx* ctx, int n_ctas);
+
+/* Kernels this library launched since the context was created (all kinds). */
+long novakv_launch_count(const novakv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NOVAKV_H */

@@ -1,0 +1,352 @@
+// Host side of the C ABI: context, calibration upload, argument validation, dispatch.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "novakv_internal.cuh"
+
+#define CUDA_OK(expr)                                   \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) return NOVAKV_ECUDA;    \
+    } while (0)
+
+extern "C" const char* novakv_status_string(novakv_status s) {
+    switch (s) {
+        case NOVAKV_OK: return "ok";
+        case NOVAKV_EINVAL: return "invalid argument";
+        case NOVAKV_ESHAPE: return "unsupported shape";
+        case NOVAKV_ENOCALIB: return "layer has no calibration";
+        case NOVAKV_EPAGE: return "inconsistent page geometry";
+        case NOVAKV_EWORKSPACE: return "workspace missing or too small";
+        case NOVAKV_ECUDA: return "CUDA runtime error";
+        case NOVAKV_EUNSUPPORTED: return "unsupported calibration content";
+    }
+    return "unknown status";
+}
+
+static bool shape_supported(const novakv_config& c) {
+    if (c.group_size != NOVAKV_G || c.codebook_size != NOVAKV_C || c.page_tokens != NOVAKV_PAGE_TOKENS) return false;
+    if (c.head_dim != 64 && c.head_dim != 128) return false;
+    if (c.n_kv_heads <= 0 || c.n_q_heads <= 0 || c.n_q_heads % c.n_kv_heads != 0) return false;
+    int hg = c.n_q_heads / c.n_kv_heads;
+    if (hg != 1 && hg != 2 && hg != 4 && hg != 8) return false;
+    if (c.head_dim == 128 && hg == 8) return false;
+    return true;
+}
+
+extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cfg) {
+    if (!out || !cfg) return NOVAKV_EINVAL;
+    *out = nullptr;
+    if (cfg->n_layers <= 0 || cfg->device < 0) return NOVAKV_EINVAL;
+    if (!shape_supported(*cfg)) return NOVAKV_ESHAPE;
+    int ndev = 0;
+    CUDA_OK(cudaGetDeviceCount(&ndev));
+    if (cfg->device >= ndev) return NOVAKV_EINVAL;
+    CUDA_OK(cudaSetDevice(cfg->device));
+    novakv_ctx* ctx = new (std::nothrow) novakv_ctx();
+    if (!ctx) return NOVAKV_EINVAL;
+    ctx->cfg = *cfg;
+    ctx->hg = cfg->n_q_heads / cfg->n_kv_heads;
+    ctx->n_groups = cfg->head_dim / NOVAKV_G;
+    ctx->layers.resize(cfg->n_layers);
+    if (cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess ||
+        cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
+        cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess) {
+        delete ctx;
+        return NOVAKV_ECUDA;
+    }
+    *out = ctx;
+    return NOVAKV_OK;
+}
+
+static void free_layer(novakv_layer& ly) {
+    cudaFree(ly.rk_d); cudaFree(ly.rv_d); cudaFree(ly.k_mean_d); cudaFree(ly.v_mean_d);
+    cudaFree(ly.cb_k); cudaFree(ly.cb_v); cudaFree(ly.rk_inv_t); cudaFree(ly.rv_t);
+    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_half);
+    ly = novakv_layer();
+}
+
+extern "C" novakv_status novakv_destroy(novakv_ctx* ctx) {
+    if (!ctx) return NOVAKV_EINVAL;
+    cudaSetDevice(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    for (auto& ly : ctx->layers) free_layer(ly);
+    for (int k = 0; k < 3; ++k)
+        for (auto& e : ctx->prof[k]) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
+    for (auto& e : ctx->prof_free) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
+    cudaFree(ctx->dev_status);
+    delete ctx;
+    return NOVAKV_OK;
+}
+
+template <typename T>
+static cudaError_t upload(T** dst, const std::vector<T>& host) {
+    cudaError_t e = cudaMalloc(dst, host.size() * sizeof(T));
+    if (e != cudaSuccess) return e;
+    return cudaMemcpy(*dst, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, const novakv_calibration* h) {
+    if (!ctx || !h || layer < 0 || layer >= ctx->cfg.n_layers) return NOVAKV_EINVAL;
+    if (!h->rk || !h->rk_inv_t || !h->rv || !h->cb_k || !h->cb_v) return NOVAKV_EINVAL;
+    const int H = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim, L = ctx->n_groups, C = NOVAKV_C, g = NOVAKV_G;
+    const size_t n_mat = (size_t)H * d * d, n_vec = (size_t)H * d, n_cb = (size_t)H * L * C * g;
+
+    // value codewords must survive the binary16 round trip exactly
+    std::vector<__half> cbv_half((size_t)H * C * 32 * g, __float2half(0.f));
+    for (int hh = 0; hh < H; ++hh)
+        for (int l = 0; l < L; ++l)
+            for (int c = 0; c < C; ++c)
+                for (int i = 0; i < g; ++i) {
+                    float x = h->cb_v[(((size_t)hh * L + l) * C + c) * g + i];
+                    __half hx = __float2half_rn(x);
+                    if (!(__half2float(hx) == x)) return NOVAKV_EUNSUPPORTED;
+                    cbv_half[(((size_t)hh * C + c) * 32 + l) * g + i] = hx;
+                }
+
+    std::vector<double> rk_d(n_mat), rv_d(n_mat), km_d(n_vec, 0.0), vm_d(n_vec, 0.0);
+    std::vector<float> vm_f(n_vec, 0.f);
+    for (size_t i = 0; i < n_mat; ++i) { rk_d[i] = (double)h->rk[i]; rv_d[i] = (double)h->rv[i]; }
+    if (h->k_mean) for (size_t i = 0; i < n_vec; ++i) km_d[i] = (double)h->k_mean[i];
+    if (h->v_mean) for (size_t i = 0; i < n_vec; ++i) { vm_d[i] = (double)h->v_mean[i]; vm_f[i] = h->v_mean[i]; }
+
+    // key codebook in score-table order: [Hkv][plane][code][e = (m%2)*8 + sigma][4],
+    // group l = sigma*GPS + plane*2 + (m%2), GPS = L/8 groups per slot.
+    const int GPS = L / 8, planes = GPS / 2;
+    std::vector<float> cbk_lut((size_t)H * planes * C * 16 * g);
+    for (int hh = 0; hh < H; ++hh)
+        for (int pl = 0; pl < planes; ++pl)
+            for (int c = 0; c < C; ++c)
+                for (int e = 0; e < 16; ++e) {
+                    int sigma = e & 7, mpar = e >> 3;
+                    int l = sigma * GPS + pl * 2 + mpar;
+                    for (int i = 0; i < g; ++i)
+                        cbk_lut[((((size_t)hh * planes + pl) * C + c) * 16 + e) * g + i] =
+                            h->cb_k[(((size_t)hh * L + l) * C + c) * g + i];
+                }
+
+    CUDA_OK(cudaSetDevice(ctx->cfg.device));
+    novakv_layer& ly = ctx->layers[layer];
+    if (ly.loaded) { cudaDeviceSynchronize(); free_layer(ly); }
+    std::vector<float> cbk(h->cb_k, h->cb_k + n_cb), cbv(h->cb_v, h->cb_v + n_cb);
+    std::vector<float> rkinv(h->rk_inv_t, h->rk_inv_t + n_mat), rvt(n_mat);
+    for (int hh = 0; hh < H; ++hh)       // transposed copy: rv_t[c][r] = rv[r][c], so that o = o' rv^T reads rows
+        for (int r = 0; r < d; ++r)
+            for (int c = 0; c < d; ++c) rvt[((size_t)hh * d + c) * d + r] = h->rv[((size_t)hh * d + r) * d + c];
+    bool ok = upload(&ly.rk_d, rk_d) == cudaSuccess && upload(&ly.rv_d, rv_d) == cudaSuccess &&
+              upload(&ly.k_mean_d, km_d) == cudaSuccess && upload(&ly.v_mean_d, vm_d) == cudaSuccess &&
+              upload(&ly.cb_k, cbk) == cudaSuccess && upload(&ly.cb_v, cbv) == cudaSuccess &&
+              upload(&ly.rk_inv_t, rkinv) == cudaSuccess && upload(&ly.rv_t, rvt) == cudaSuccess &&
+              upload(&ly.v_mean, vm_f) == cudaSuccess && upload(&ly.cb_k_lut, cbk_lut) == cudaSuccess &&
+              upload(&ly.cb_v_half, cbv_half) == cudaSuccess;
+    if (!ok) { free_layer(ly); return NOVAKV_ECUDA; }
+    ly.loaded = true;
+    return NOVAKV_OK;
+}
+
+extern "C" size_t novakv_page_bytes(const novakv_ctx* ctx) {
+    if (!ctx) return 0;
+    return (size_t)ctx->cfg.n_kv_heads * NOVAKV_PAGE_TOKENS * ctx->n_groups;
+}
+
+extern "C" size_t novakv_decode_workspace_bytes(const novakv_ctx* ctx, int batch) {
+    if (!ctx || batch <= 0) return 0;
+    return novakv_decode_ws_bytes(ctx, batch);
+}
+
+static novakv_status check_common(const novakv_ctx* ctx, int layer) {
+    if (!ctx) return NOVAKV_EINVAL;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return NOVAKV_EINVAL;
+    if (!ctx->layers[layer].loaded) return NOVAKV_ENOCALIB;
+    return NOVAKV_OK;
+}
+
+extern "C" novakv_status novakv_encode_append(novakv_ctx* ctx, int layer, const void* k_new,
+    const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens, uint8_t* k_pages,
+    uint8_t* v_pages, int n_pages, const int32_t* page_table, int max_pages_per_seq, int n_seq,
+    int32_t* seq_lens, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (n_tokens < 0) return NOVAKV_EINVAL;
+    if (n_tokens == 0) return NOVAKV_OK;
+    if (!k_new || !v_new || !tok_seq || !tok_pos || !k_pages || !v_pages || !page_table || !seq_lens) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0 || n_seq <= 0) return NOVAKV_EPAGE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_encode(ctx, ctx->layers[layer], (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new,
+                                tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages, page_table,
+                                max_pages_per_seq, n_seq, seq_lens, (cudaStream_t)stream);
+}
+
+extern "C" novakv_status novakv_decode_attention(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out, int out_is_fp32,
+    void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!q || !k_pages || !v_pages || !page_table || !seq_lens || !out) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_pages & 15) || ((uintptr_t)v_pages & 15)) return NOVAKV_EINVAL;   // bulk copies need 16-byte alignment
+    if (!(sm_scale == sm_scale)) return NOVAKV_EINVAL;
+    if (!workspace || workspace_bytes < novakv_decode_ws_bytes(ctx, batch) || ((uintptr_t)workspace & 255)) return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_decode(ctx, ctx->layers[layer], (const __nv_bfloat16*)q, k_pages, v_pages, n_pages,
+                                page_table, max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,
+                                workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+extern "C" novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word) {
+    if (!ctx || !word) return NOVAKV_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    CUDA_OK(cudaSetDevice(ctx->cfg.device));
+    CUDA_OK(cudaMemcpyAsync(word, ctx->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+    CUDA_OK(cudaMemsetAsync(ctx->dev_status, 0, sizeof(uint32_t), s));
+    CUDA_OK(cudaStreamSynchronize(s));
+    return NOVAKV_OK;
+}
+
+// ------------------------------------------------------------------ host-buffer step
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+extern "C" size_t novakv_step_staging_bytes(const novakv_ctx* ctx, int batch, int n_tokens) {
+    if (!ctx || batch < 0 || n_tokens < 0) return 0;
+    const size_t d = ctx->cfg.head_dim;
+    size_t kv = align256((size_t)n_tokens * ctx->cfg.n_kv_heads * d * 2);
+    size_t tok = align256((size_t)n_tokens * 4);
+    size_t q = align256((size_t)batch * ctx->cfg.n_q_heads * d * 2);
+    size_t o = align256((size_t)batch * ctx->cfg.n_q_heads * d * 4);
+    return 2 * kv + 2 * tok + q + o + 256;
+}
+
+extern "C" novakv_status novakv_step_host(novakv_ctx* ctx, int layer, const void* k_new_host,
+    const void* v_new_host, const int32_t* tok_seq_host, const int32_t* tok_pos_host, int n_tokens,
+    const void* q_host, uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int32_t* seq_lens, int batch, float sm_scale, float* out_host, void* staging,
+    size_t staging_bytes, void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch <= 0 || n_tokens < 0 || !q_host || !out_host || !staging) return NOVAKV_EINVAL;
+    if (n_tokens > 0 && (!k_new_host || !v_new_host || !tok_seq_host || !tok_pos_host)) return NOVAKV_EINVAL;
+    if (staging_bytes < novakv_step_staging_bytes(ctx, batch, n_tokens) || ((uintptr_t)staging & 255)) return NOVAKV_EWORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    CUDA_OK(cudaSetDevice(ctx->cfg.device));
+    const size_t d = ctx->cfg.head_dim;
+    const size_t kv_b = (size_t)n_tokens * ctx->cfg.n_kv_heads * d * 2, tok_b = (size_t)n_tokens * 4;
+    const size_t q_b = (size_t)batch * ctx->cfg.n_q_heads * d * 2, o_b = (size_t)batch * ctx->cfg.n_q_heads * d * 4;
+    char* p = (char*)staging;
+    char* dk = p; p += align256(kv_b);
+    char* dv = p; p += align256(kv_b);
+    char* dseq = p; p += align256(tok_b);
+    char* dpos = p; p += align256(tok_b);
+    char* dq = p; p += align256(q_b);
+    char* dout = p;
+    if (n_tokens > 0) {
+        CUDA_OK(cudaMemcpyAsync(dk, k_new_host, kv_b, cudaMemcpyHostToDevice, s));
+        CUDA_OK(cudaMemcpyAsync(dv, v_new_host, kv_b, cudaMemcpyHostToDevice, s));
+        CUDA_OK(cudaMemcpyAsync(dseq, tok_seq_host, tok_b, cudaMemcpyHostToDevice, s));
+        CUDA_OK(cudaMemcpyAsync(dpos, tok_pos_host, tok_b, cudaMemcpyHostToDevice, s));
+    }
+    CUDA_OK(cudaMemcpyAsync(dq, q_host, q_b, cudaMemcpyHostToDevice, s));
+    if (n_tokens > 0) {
+        st = novakv_encode_append(ctx, layer, dk, dv, (const int32_t*)dseq, (const int32_t*)dpos, n_tokens,
+                                  k_pages, v_pages, n_pages, page_table, max_pages_per_seq, batch, seq_lens, stream);
+        if (st != NOVAKV_OK) return st;
+    }
+    st = novakv_decode_attention(ctx, layer, dq, k_pages, v_pages, n_pages, page_table, max_pages_per_seq,
+                                 seq_lens, batch, sm_scale, dout, 1, workspace, workspace_bytes, stream);
+    if (st != NOVAKV_OK) return st;
+    CUDA_OK(cudaMemcpyAsync(out_host, dout, o_b, cudaMemcpyDeviceToHost, s));
+    CUDA_OK(cudaStreamSynchronize(s));
+    return NOVAKV_OK;
+}
+
+// ------------------------------------------------------------------ helpers for tests / bench
+extern "C" novakv_status novakv_search_coefficients(novakv_ctx* ctx, int layer, int which, const float* coef,
+    int n, uint8_t* idx_out, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (n < 0 || (which != 0 && which != 1)) return NOVAKV_EINVAL;
+    if (n == 0) return NOVAKV_OK;
+    if (!coef || !idx_out) return NOVAKV_EINVAL;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_search(ctx, ctx->layers[layer], which, coef, n, idx_out, (cudaStream_t)stream);
+}
+
+extern "C" size_t novakv_bf16_workspace_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq) {
+    if (!ctx || batch <= 0 || max_pages_per_seq <= 0) return 0;
+    return novakv_bf16_ws_bytes(ctx, batch, max_pages_per_seq);
+}
+
+extern "C" novakv_status novakv_bf16_decode_attention(novakv_ctx* ctx, const void* q, const void* k_pages_bf16,
+    const void* v_pages_bf16, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+    const int32_t* seq_lens, int batch, float sm_scale, int window, void* out, int out_is_fp32,
+    void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    if (!ctx) return NOVAKV_EINVAL;
+    if (batch < 0 || window < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!q || !k_pages_bf16 || !v_pages_bf16 || !page_table || !seq_lens || !out) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0) return NOVAKV_EPAGE;
+    if (!workspace || workspace_bytes < novakv_bf16_ws_bytes(ctx, batch, max_pages_per_seq) || ((uintptr_t)workspace & 255)) return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_bf16_decode(ctx, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pages_bf16,
+                                     (const __nv_bfloat16*)v_pages_bf16, n_pages, page_table, max_pages_per_seq,
+                                     seq_lens, batch, sm_scale, window, out, out_is_fp32, workspace,
+                                     workspace_bytes, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------ profiling
+novakv_prof_scope::novakv_prof_scope(novakv_ctx* c, int k, cudaStream_t s) : ctx(c), kind(k), stream(s), active(false) {
+    if (!ctx->profile) return;
+    if (!ctx->prof_free.empty()) {
+        ev = ctx->prof_free.back();
+        ctx->prof_free.pop_back();
+    } else {
+        if (cudaEventCreate(&ev.start) != cudaSuccess) return;
+        if (cudaEventCreate(&ev.stop) != cudaSuccess) { cudaEventDestroy(ev.start); return; }
+    }
+    cudaEventRecord(ev.start, stream);
+    active = true;
+}
+
+void novakv_prof_scope::end() {
+    if (!active) return;
+    cudaEventRecord(ev.stop, stream);
+    ctx->prof[kind].push_back(ev);
+    active = false;
+}
+
+extern "C" novakv_status novakv_profile_enable(novakv_ctx* ctx, int on) {
+    if (!ctx) return NOVAKV_EINVAL;
+    ctx->profile = on != 0;
+    return NOVAKV_OK;
+}
+
+extern "C" novakv_status novakv_profile_read(novakv_ctx* ctx, int kind, double* total_ms, long* launches) {
+    if (!ctx || kind < 0 || kind > 2 || !total_ms || !launches) return NOVAKV_EINVAL;
+    CUDA_OK(cudaSetDevice(ctx->cfg.device));
+    double tot = 0.0;
+    long n = 0;
+    for (auto& e : ctx->prof[kind]) {
+        CUDA_OK(cudaEventSynchronize(e.stop));
+        float ms = 0.f;
+        CUDA_OK(cudaEventElapsedTime(&ms, e.start, e.stop));
+        tot += ms;
+        n++;
+        ctx->prof_free.push_back(e);
+    }
+    ctx->prof[kind].clear();
+    *total_ms = tot;
+    *launches = n;
+    return NOVAKV_OK;
+}
+
+extern "C" novakv_status novakv_debug_set_scan_ctas(novakv_ctx* ctx, int n_ctas) {
+    if (!ctx || n_ctas < 0) return NOVAKV_EINVAL;
+    ctx->scan_ctas = n_ctas;
+    return NOVAKV_OK;
+}
+
+extern "C" long novakv_launch_count(const novakv_ctx* ctx) { return ctx ? ctx->launches : 0; }

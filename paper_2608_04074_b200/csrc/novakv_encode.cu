@@ -1,0 +1,261 @@
+// Write path: forward transforms (binary64) + brute-force nearest-codeword search (binary32) +
+// paged store.  One CTA handles a tile of tokens for one (KV head, side); side 0 = keys, 1 = values.
+//
+// The search is ALU-bound (256 distance evaluations per group, per token, per side); the codebook
+// of the CTA's head and side stays in shared memory and every warp reads codewords as broadcasts.
+#include "novakv_internal.cuh"
+
+namespace {
+
+constexpr int ENC_THREADS = 256;
+constexpr int ENC_TILE = 64;   // tokens per tile (search granularity)
+constexpr int ENC_XT = 32;     // tokens per transform pass (bounds the binary64 staging buffer)
+
+template <int D>
+struct EncSmem {
+    static constexpr int L = D / NOVAKV_G;
+    static constexpr int RSTRIDE = D + 4;                       // floats; keeps 128-bit row reads conflict-free
+    static constexpr size_t cb_bytes = (size_t)L * NOVAKV_C * NOVAKV_G * sizeof(float);
+    static constexpr size_t xc_bytes = (size_t)ENC_XT * D * sizeof(double);
+    static constexpr size_t r_bytes = (size_t)ENC_TILE * RSTRIDE * sizeof(float);
+    static constexpr size_t idx_bytes = (size_t)ENC_TILE * L;
+    static constexpr size_t total = cb_bytes + xc_bytes + r_bytes + idx_bytes + 3 * ENC_TILE * sizeof(int);
+};
+
+// Squared distance in the arithmetic the public header fixes: fma(e3,e3,fma(e2,e2,fma(e1,e1,e0*e0))).
+__device__ __forceinline__ float dist4(const float4 r, const float4 c) {
+    const float e0 = __fsub_rn(r.x, c.x), e1 = __fsub_rn(r.y, c.y);
+    const float e2 = __fsub_rn(r.z, c.z), e3 = __fsub_rn(r.w, c.w);
+    return __fmaf_rn(e3, e3, __fmaf_rn(e2, e2, __fmaf_rn(e1, e1, __fmul_rn(e0, e0))));
+}
+
+// Search of the tile's coefficients (r_s, [ENC_TILE][RSTRIDE] float) against cb_s ([L][256] float4).
+// Warp w owns groups w, w+8, ...; lane t owns tokens t and t+32.  Ascending codeword index with a
+// strict '<' keeps the first minimum.
+template <int D>
+__device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s, uint8_t* idx_s, int n_valid) {
+    constexpr int L = D / NOVAKV_G;
+    constexpr int RS = EncSmem<D>::RSTRIDE;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int l = warp; l < L; l += ENC_THREADS / 32) {
+        const float4 ra = *reinterpret_cast<const float4*>(r_s + (size_t)lane * RS + l * 4);
+        const float4 rb = *reinterpret_cast<const float4*>(r_s + (size_t)(lane + 32) * RS + l * 4);
+        float best_a = 0.f, best_b = 0.f;
+        int ia = 0, ib = 0;
+        const float4* cb = cb_s + (size_t)l * NOVAKV_C;
+        {
+            const float4 c0 = cb[0];
+            best_a = dist4(ra, c0);
+            best_b = dist4(rb, c0);
+        }
+#pragma unroll 4
+        for (int c = 1; c < NOVAKV_C; ++c) {
+            const float4 cw = cb[c];
+            const float da = dist4(ra, cw), db = dist4(rb, cw);
+            if (da < best_a) { best_a = da; ia = c; }
+            if (db < best_b) { best_b = db; ib = c; }
+        }
+        if (lane < n_valid) idx_s[lane * L + l] = (uint8_t)ia;
+        if (lane + 32 < n_valid) idx_s[(lane + 32) * L + l] = (uint8_t)ib;
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(ENC_THREADS, 1)
+novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+                     const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
+                     const double* __restrict__ rk_d, const double* __restrict__ rv_d,
+                     const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
+                     const float* __restrict__ cb_k, const float* __restrict__ cb_v,
+                     uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages, int n_pages,
+                     const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
+                     int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
+                     uint32_t* __restrict__ dev_status) {
+    constexpr int L = D / NOVAKV_G;
+    constexpr int RS = EncSmem<D>::RSTRIDE;
+    extern __shared__ __align__(16) unsigned char smem[];
+    float4* cb_s = reinterpret_cast<float4*>(smem);
+    double* xc_s = reinterpret_cast<double*>(smem + EncSmem<D>::cb_bytes);
+    float* r_s = reinterpret_cast<float*>(smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes);
+    uint8_t* idx_s = smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes + EncSmem<D>::r_bytes;
+    int* page_s = reinterpret_cast<int*>(idx_s + EncSmem<D>::idx_bytes);   // [ENC_TILE] page id or -1
+    int* slot_s = page_s + ENC_TILE;                                       // [ENC_TILE] slot in page
+
+    const int kvh = blockIdx.y, side = blockIdx.z;
+    const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
+    const double* R = (side == 0 ? rk_d : rv_d) + (size_t)kvh * D * D;
+    const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
+    const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
+
+    // codebook of this (head, side) -> shared memory, once per CTA
+    for (int i = threadIdx.x; i < L * NOVAKV_C; i += ENC_THREADS) cb_s[i] = cb_g[i];
+
+    const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
+    const int tile0 = blockIdx.x * tiles_per_cta;
+    for (int tile = tile0; tile < min(n_tiles, tile0 + tiles_per_cta); ++tile) {
+        const int t0 = tile * ENC_TILE;
+        const int n_valid = min(ENC_TILE, n_tokens - t0);
+        __syncthreads();   // previous tile's readers are done (also orders the codebook fill)
+
+        // destination of each token (validated once)
+        if (threadIdx.x < ENC_TILE) {
+            const int t = threadIdx.x;
+            int page = -1, slot = 0;
+            if (t < n_valid) {
+                const int s = tok_seq[t0 + t], pos = tok_pos[t0 + t];
+                if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
+                    atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
+                } else {
+                    page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
+                    slot = pos % NOVAKV_PAGE_TOKENS;
+                    if (page < 0 || page >= n_pages) {
+                        atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
+                        page = -1;
+                    } else if (kvh == 0 && side == 0) {
+                        atomicMax(&seq_lens[s], pos + 1);
+                    }
+                }
+            }
+            page_s[t] = page;
+            slot_s[t] = slot;
+        }
+
+        for (int half = 0; half < ENC_TILE / ENC_XT; ++half) {
+            const int tb = half * ENC_XT;
+            if (half > 0) __syncthreads();   // the previous pass no longer reads xc_s
+            // centred inputs in binary64: xc[t][i] = x[t][i] - mean[i]   (exact)
+            for (int i = threadIdx.x; i < ENC_XT * D; i += ENC_THREADS) {
+                const int t = i / D, c = i - t * D;
+                double x = 0.0;
+                if (tb + t < n_valid)
+                    x = (double)__bfloat162float(x_new[((size_t)(t0 + tb + t) * n_kv_heads + kvh) * D + c]) - mean[c];
+                xc_s[i] = x;
+            }
+            __syncthreads();
+            // transform: r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA, rounded once to binary32.
+            // thread -> column c = tid % D, token subset tid / D (stride ENC_THREADS / D).
+            constexpr int TSUB = ENC_THREADS / D;           // 2 (D=128) or 4 (D=64)
+            constexpr int TPT = ENC_XT / TSUB;              // tokens per thread: 16 or 8
+            const int c = threadIdx.x % D, sub = threadIdx.x / D;
+            double acc[TPT];
+#pragma unroll
+            for (int j = 0; j < TPT; ++j) acc[j] = 0.0;
+            for (int i = 0; i < D; ++i) {
+                const double rv = R[(size_t)i * D + c];
+#pragma unroll
+                for (int j = 0; j < TPT; ++j) acc[j] = fma(xc_s[(size_t)(sub + j * TSUB) * D + i], rv, acc[j]);
+            }
+#pragma unroll
+            for (int j = 0; j < TPT; ++j) r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc[j];
+        }
+        __syncthreads();
+
+        search_tile<D>(r_s, cb_s, idx_s, n_valid);
+        __syncthreads();
+
+        // paged store
+        for (int i = threadIdx.x; i < n_valid * L; i += ENC_THREADS) {
+            const int t = i / L, l = i - t * L;
+            const int page = page_s[t];
+            if (page < 0) continue;
+            const int slot = slot_s[t];
+            const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
+            if (side == 0) {
+                k_pages[base + (size_t)slot * L + l] = idx_s[i];
+            } else {
+                v_pages[base + ((size_t)(slot / NOVAKV_VBLOCK) * L + l) * NOVAKV_VBLOCK + (slot % NOVAKV_VBLOCK)] = idx_s[i];
+            }
+        }
+    }
+}
+
+// Search only, from given binary32 coefficients [n][Hkv][D]; logical indices out [n][Hkv][L].
+template <int D>
+__global__ void __launch_bounds__(ENC_THREADS, 1)
+novakv_search_kernel(const float* __restrict__ coef, int n, const float* __restrict__ cb_all, int n_kv_heads,
+                     uint8_t* __restrict__ idx_out) {
+    constexpr int L = D / NOVAKV_G;
+    constexpr int RS = EncSmem<D>::RSTRIDE;
+    extern __shared__ __align__(16) unsigned char smem[];
+    float4* cb_s = reinterpret_cast<float4*>(smem);
+    float* r_s = reinterpret_cast<float*>(smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes);
+    uint8_t* idx_s = smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes + EncSmem<D>::r_bytes;
+    const int kvh = blockIdx.y;
+    const float4* cb_g = reinterpret_cast<const float4*>(cb_all + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
+    for (int i = threadIdx.x; i < L * NOVAKV_C; i += ENC_THREADS) cb_s[i] = cb_g[i];
+    const int n_tiles = (n + ENC_TILE - 1) / ENC_TILE;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int t0 = tile * ENC_TILE;
+        const int n_valid = min(ENC_TILE, n - t0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < ENC_TILE * D; i += ENC_THREADS) {
+            const int t = i / D, c = i - t * D;
+            r_s[(size_t)t * RS + c] = t < n_valid ? coef[((size_t)(t0 + t) * n_kv_heads + kvh) * D + c] : 0.f;
+        }
+        __syncthreads();
+        search_tile<D>(r_s, cb_s, idx_s, n_valid);
+        __syncthreads();
+        for (int i = threadIdx.x; i < n_valid * L; i += ENC_THREADS) {
+            const int t = i / L, l = i - t * L;
+            idx_out[((size_t)(t0 + t) * n_kv_heads + kvh) * L + l] = idx_s[i];
+        }
+    }
+}
+
+template <int D>
+novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* k_new,
+                              const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos,
+                              int n_tokens, uint8_t* k_pages, uint8_t* v_pages, int n_pages,
+                              const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
+                              cudaStream_t stream) {
+    auto kern = novakv_encode_kernel<D>;
+    const size_t smem = EncSmem<D>::total;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;
+    const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
+    const int hs = ctx->cfg.n_kv_heads * 2;
+    // enough CTAs per (head, side) to fill the machine about twice, each amortising its codebook fill
+    int ctas_x = max(1, min(n_tiles, (2 * ctx->n_sm + hs - 1) / hs));
+    const int tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
+    ctas_x = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    dim3 grid(ctas_x, ctx->cfg.n_kv_heads, 2);
+    novakv_prof_scope ps(ctx, 1, stream);
+    kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d, ly.rv_d,
+                                               ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
+                                               page_table, max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads,
+                                               tiles_per_cta, ctx->dev_status);
+    ps.end();
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
+}
+
+template <int D>
+novakv_status launch_search_t(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef, int n,
+                              uint8_t* idx_out, cudaStream_t stream) {
+    auto kern = novakv_search_kernel<D>;
+    const size_t smem = EncSmem<D>::total;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;
+    const int n_tiles = (n + ENC_TILE - 1) / ENC_TILE;
+    dim3 grid(max(1, min(n_tiles, 2 * ctx->n_sm / ctx->cfg.n_kv_heads + 1)), ctx->cfg.n_kv_heads);
+    kern<<<grid, ENC_THREADS, smem, stream>>>(coef, n, which == 0 ? ly.cb_k : ly.cb_v, ctx->cfg.n_kv_heads, idx_out);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
+}
+
+}  // namespace
+
+novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* k_new,
+    const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens,
+    uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream) {
+    if (ctx->cfg.head_dim == 128)
+        return launch_encode_t<128>(ctx, ly, k_new, v_new, tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages,
+                                    page_table, max_pages_per_seq, n_seq, seq_lens, stream);
+    return launch_encode_t<64>(ctx, ly, k_new, v_new, tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages,
+                               page_table, max_pages_per_seq, n_seq, seq_lens, stream);
+}
+
+novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef,
+    int n, uint8_t* idx_out, cudaStream_t stream) {
+    if (ctx->cfg.head_dim == 128) return launch_search_t<128>(ctx, ly, which, coef, n, idx_out, stream);
+    return launch_search_t<64>(ctx, ly, which, coef, n, idx_out, stream);
+}

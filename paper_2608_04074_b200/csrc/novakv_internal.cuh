@@ -1,0 +1,130 @@
+// Internal declarations shared by the translation units of libnovakv (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <vector>
+
+#include "novakv.h"
+
+#define NOVAKV_PAGE_TOKENS 64
+#define NOVAKV_G 4
+#define NOVAKV_C 256
+#define NOVAKV_VBLOCK 16
+
+// Device copies of one layer's tables, in the layouts the kernels read.
+struct novakv_layer {
+    bool loaded = false;
+    // write path (binary64 transforms, see the encode entry of the public header)
+    double* rk_d = nullptr;       // [Hkv][d][d]
+    double* rv_d = nullptr;       // [Hkv][d][d]
+    double* k_mean_d = nullptr;   // [Hkv][d]
+    double* v_mean_d = nullptr;   // [Hkv][d]
+    float* cb_k = nullptr;        // [Hkv][L][256][4]  search layout
+    float* cb_v = nullptr;        // [Hkv][L][256][4]
+    // read path
+    float* rk_inv_t = nullptr;    // [Hkv][d][d]
+    float* rv_t = nullptr;        // [Hkv][d][d]  transposed R_V: rv_t[c][r] = R_V[r][c]
+    float* v_mean = nullptr;      // [Hkv][d]
+    float* cb_k_lut = nullptr;    // [Hkv][plane][256][16][4]  the order the score table is built in
+    __half* cb_v_half = nullptr;  // [Hkv][256][32][4]         row of 256 bytes per code (padded for L=16)
+};
+
+struct novakv_event_pair {
+    cudaEvent_t start, stop;
+};
+
+struct novakv_ctx {
+    novakv_config cfg;
+    int hg = 0, n_groups = 0, n_sm = 0;
+    std::vector<novakv_layer> layers;
+    uint32_t* dev_status = nullptr;
+    bool profile = false;
+    std::vector<novakv_event_pair> prof[3];
+    std::vector<novakv_event_pair> prof_free;
+    long launches = 0;
+    int scan_ctas = 0;            // 0 = one per SM
+};
+
+// RAII-free helper: brackets a launch with events when profiling is on.
+struct novakv_prof_scope {
+    novakv_ctx* ctx;
+    int kind;
+    cudaStream_t stream;
+    novakv_event_pair ev;
+    bool active;
+    novakv_prof_scope(novakv_ctx* c, int k, cudaStream_t s);
+    void end();
+};
+
+// encode
+novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* k_new,
+    const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens,
+    uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream);
+novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef,
+    int n, uint8_t* idx_out, cudaStream_t stream);
+
+// decode
+size_t novakv_decode_ws_bytes(const novakv_ctx* ctx, int batch);
+novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
+    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+// bf16 comparator
+size_t novakv_bf16_ws_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq);
+novakv_status novakv_launch_bf16_decode(novakv_ctx* ctx, const __nv_bfloat16* q,
+    const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch,
+    float sm_scale, int window, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
+    cudaStream_t stream);
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after `limit` polls and reports false (the caller records the fault).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = (1u << 24)) {
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    return false;
+}
+// 1-D bulk asynchronous copy global -> shared of this CTA, completion on an mbarrier.
+// Both addresses 16-byte aligned, size a multiple of 16 bytes.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,301 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Indices are compared bit for bit (a difference is tolerated only where the
+oracle's float64 relative gap between the two nearest codewords is <= 1e-6, and is counted);
+attention outputs within max|delta| <= 2e-3 * ||o||_inf on float32 output."""
+import numpy as np
+import pytest
+
+from gpu_common import Case, check_indices, check_output, NEAR_TIE
+from paper_2608_04074_b200 import synth, workloads
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def _dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    return Case(workloads.tiny())
+
+
+@pytest.fixture(scope="module")
+def qwen():
+    return Case(workloads.qwen3_8b(batch=4, seq_len=4096, calib_tokens=4096, lloyd_iters=6))
+
+
+@pytest.fixture(scope="module")
+def gptoss():
+    return Case(workloads.gpt_oss_20b(batch=2, seq_len=2048, calib_tokens=4096, lloyd_iters=6))
+
+
+def _cache(case, seq_lens, capacity=None, seed=3):
+    from paper_2608_04074_b200.runtime import PagedCache
+    return PagedCache(case.ctx, seq_lens, capacity_tokens=capacity, seed=seed)
+
+
+def _fill_with_oracle(case, cache, seq_lens, seed):
+    """Draw tokens per sequence, encode them with the ORACLE, store the oracle's indices."""
+    encs, items = [], []
+    for b, n in enumerate(seq_lens):
+        k, v, _ = case.draw(seed + 10 * b, int(n), 1)
+        enc = case.oracle.encode(k.astype(np.float64), v.astype(np.float64), with_gaps=False) if n > 0 else \
+            dict(kidx=np.zeros((0, case.ctx.n_kv_heads, case.ctx.n_groups), np.uint8),
+                 vidx=np.zeros((0, case.ctx.n_kv_heads, case.ctx.n_groups), np.uint8))
+        encs.append(enc)
+        if n > 0:
+            items.append((b, 0, enc["kidx"], enc["vidx"]))
+    cache.store_logical_batch(items)
+    return encs
+
+
+# --------------------------------------------------------------------------- T1: search only
+@pytest.mark.parametrize("name", ["tiny", "qwen", "gptoss"])
+def test_search_from_oracle_coefficients_is_exact(name, request):
+    case = request.getfixturevalue(name)
+    n = 777                                        # several 64-token tiles and a ragged tail
+    k, v, _ = case.draw(100, n, 1)
+    for which, x in (("k", k), ("v", v)):
+        coef = case.oracle.coefficients(x.astype(np.float64), which).astype(np.float32)
+        idx_gpu = torch.empty((n, case.ctx.n_kv_heads, case.ctx.n_groups), dtype=torch.uint8, device="cuda")
+        case.ctx.novakv_search_coefficients(0, 0 if which == "k" else 1, _dev(coef), idx_gpu)
+        got = idx_gpu.cpu().numpy()
+        for h in range(case.ctx.n_kv_heads):
+            ref, _, _ = case.oracle.search(coef[:, h].astype(np.float64), h, which)
+            assert np.array_equal(got[:, h], ref), f"{which} head {h}"
+
+
+# --------------------------------------------------------------------------- T2: transform + search + paged store
+@pytest.mark.parametrize("name", ["tiny", "qwen", "gptoss"])
+def test_encode_append_matches_oracle_indices(name, request):
+    case = request.getfixturevalue(name)
+    lens0 = np.array([0, 5, 63, 130], np.int32)          # existing lengths; tokens are appended after them
+    add = np.array([200, 64, 1, 130], np.int32)
+    cache = _cache(case, lens0, capacity=lens0 + add)
+    n = int(add.sum())
+    k, v, _ = case.draw(200, n, 1)
+    tok_seq = np.concatenate([np.full(a, b, np.int32) for b, a in enumerate(add)])
+    tok_pos = np.concatenate([lens0[b] + np.arange(a, dtype=np.int32) for b, a in enumerate(add)])
+    perm = synth.rng(5).permutation(n)                   # tokens of different sequences interleaved
+    k, v, tok_seq, tok_pos = k[perm], v[perm], tok_seq[perm], tok_pos[perm]
+    cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(tok_seq), _dev(tok_pos))
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens0 + add)
+    enc = case.oracle.encode(k.astype(np.float64), v.astype(np.float64))
+    got_k = np.empty_like(enc["kidx"]); got_v = np.empty_like(enc["vidx"])
+    for t in range(n):
+        kk, vv = cache.load_logical(int(tok_seq[t]), int(tok_pos[t]), 1)
+        got_k[t], got_v[t] = kk[0], vv[0]
+    dk, nk = check_indices(got_k, enc, "k")
+    dv, nv = check_indices(got_v, enc, "v")
+    print(f"[{name}] index mismatches K {dk} V {dv}; oracle near-ties (gap<={NEAR_TIE}) K {nk} V {nv} of {got_k.size}")
+    # bytes of positions that were not appended stay untouched (zero)
+    kk, _ = cache.load_logical(1, 0, 5)
+    assert not kk.any()
+
+
+# --------------------------------------------------------------------------- T3/T5: decode on the oracle's indices
+@pytest.mark.parametrize("name,lens", [
+    ("tiny", [1024]),
+    ("tiny", [1]),
+    ("qwen", [1, 63, 64, 65, 1000, 0, 3001]),
+    ("gptoss", [2048, 77, 640]),
+])
+def test_decode_matches_oracle(name, lens, request):
+    case = request.getfixturevalue(name)
+    lens = np.array(lens, np.int32)
+    cache = _cache(case, lens)
+    encs = _fill_with_oracle(case, cache, lens, 300)
+    _, _, q = case.draw(301, 1, len(lens))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    worst = 0.0
+    for b, n in enumerate(lens):
+        ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
+        if n == 0:
+            assert not out[b].any()
+            continue
+        worst = max(worst, check_output(out[b], ref))
+    print(f"[{name} {lens.tolist()}] max|delta|/||o||inf = {worst:.3e}")
+
+
+# --------------------------------------------------------------------------- T4: split invariance, determinism
+def test_split_count_invariance_and_determinism(qwen):
+    case = qwen
+    lens = np.array([4096, 900, 2500], np.int32)
+    cache = _cache(case, lens)
+    encs = _fill_with_oracle(case, cache, lens, 400)
+    _, _, q = case.draw(401, 1, len(lens))
+    qd = _dev(q, torch.bfloat16)
+    outs = {}
+    for n_ctas in (1, 2, 7, 0):
+        case.ctx.novakv_debug_set_scan_ctas(n_ctas)
+        outs[n_ctas] = cache.decode(0, qd).cpu().numpy()
+        again = cache.decode(0, qd).cpu().numpy()
+        assert np.array_equal(outs[n_ctas], again), "same launch configuration must be bitwise reproducible"
+    case.ctx.novakv_debug_set_scan_ctas(0)
+    for b in range(len(lens)):
+        ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
+        for n_ctas, o in outs.items():
+            check_output(o[b], ref)
+        scale = np.abs(ref).max()
+        for n_ctas in (1, 2, 7):
+            assert np.abs(outs[n_ctas][b] - outs[0][b]).max() <= 2e-5 * scale
+
+
+# --------------------------------------------------------------------------- T6: append then decode, end to end
+@pytest.mark.parametrize("name", ["tiny", "qwen"])
+def test_append_then_decode_end_to_end(name, request):
+    case = request.getfixturevalue(name)
+    lens0 = np.array([700, 129, 64], np.int32)
+    cache = _cache(case, lens0, capacity=lens0 + 2)
+    # prefill with the GPU encoder
+    toks, seqs, poss = [], [], []
+    for b, n in enumerate(lens0):
+        k, v, _ = case.draw(500 + b, int(n), 1)
+        toks.append((k, v)); seqs.append(np.full(n, b, np.int32)); poss.append(np.arange(n, dtype=np.int32))
+    k = np.concatenate([t[0] for t in toks]); v = np.concatenate([t[1] for t in toks])
+    cache.seq_lens.zero_()
+    cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(np.concatenate(seqs)), _dev(np.concatenate(poss)))
+    # one decode step: append one token per sequence, then attend (the new token is visible)
+    k1, v1, q = case.draw(510, len(lens0), len(lens0))
+    cache.append(0, _dev(k1, torch.bfloat16), _dev(v1, torch.bfloat16), _dev(np.arange(len(lens0), dtype=np.int32)),
+                 _dev(lens0.astype(np.int32)))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens0 + 1)
+    for b, n in enumerate(lens0):
+        kb = np.concatenate([toks[b][0], k1[b:b + 1]]).astype(np.float64)
+        vb = np.concatenate([toks[b][1], v1[b:b + 1]]).astype(np.float64)
+        enc = case.oracle.encode(kb, vb)
+        gk, gv = cache.load_logical(b, 0, int(n) + 1)
+        check_indices(gk, enc, "k"); check_indices(gv, enc, "v")
+        # decode parity on the GPU's own indices (identical to the oracle's unless a near-tie flipped one)
+        check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
+        check_output(out[b], case.oracle.decode(q[b].astype(np.float64), enc["kidx"], enc["vidx"]))
+
+
+# --------------------------------------------------------------------------- output modes, host step
+def test_bf16_output_and_custom_scale(qwen):
+    case = qwen
+    lens = np.array([513, 2000], np.int32)
+    cache = _cache(case, lens)
+    encs = _fill_with_oracle(case, cache, lens, 600)
+    _, _, q = case.draw(601, 1, 2)
+    qd = _dev(q, torch.bfloat16)
+    o32 = cache.decode(0, qd, sm_scale=0.05)
+    o16 = torch.empty_like(o32, dtype=torch.bfloat16)
+    cache.decode(0, qd, out=o16, sm_scale=0.05)
+    assert torch.equal(o16, o32.to(torch.bfloat16))
+    for b in range(2):
+        ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], sm_scale=0.05)
+        check_output(o32[b].cpu().numpy(), ref)
+
+
+def test_step_host_equals_device_calls(qwen):
+    case = qwen
+    lens0 = np.array([300, 65], np.int32)
+    caches = [_cache(case, lens0, capacity=lens0 + 1, seed=9) for _ in range(2)]
+    for c in caches:
+        _fill_with_oracle(case, c, lens0, 700)
+    k1, v1, q = case.draw(701, 2, 2)
+    seq = np.arange(2, dtype=np.int32); pos = lens0.copy()
+    # device path
+    caches[0].append(0, _dev(k1, torch.bfloat16), _dev(v1, torch.bfloat16), _dev(seq), _dev(pos))
+    ref = caches[0].decode(0, _dev(q, torch.bfloat16)).cpu()
+    # host path
+    c = caches[1]
+    pin = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(dt) if dt else torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+    out_h = torch.empty((2, case.ctx.n_q_heads, case.ctx.head_dim), dtype=torch.float32).pin_memory()
+    staging = torch.empty(case.ctx.novakv_step_staging_bytes(2, 2), dtype=torch.uint8, device="cuda")
+    case.ctx.novakv_step_host(0, pin(k1, torch.bfloat16), pin(v1, torch.bfloat16), pin(seq), pin(pos),
+                              pin(q, torch.bfloat16), c.k_pages, c.v_pages, c.page_table, c.seq_lens, out_h,
+                              staging, c.workspace)
+    assert torch.equal(out_h, ref)
+    assert torch.equal(caches[0].k_pages, c.k_pages) and torch.equal(caches[0].v_pages, c.v_pages)
+
+
+# --------------------------------------------------------------------------- T7: host-injected faults
+def test_faults_are_reported_not_trapped(qwen):
+    from paper_2608_04074_b200.binding import Context, NovaKVError
+    case = qwen
+    lens = np.array([200, 100], np.int32)
+    cache = _cache(case, lens)
+    _fill_with_oracle(case, cache, lens, 800)
+    _, _, q = case.draw(801, 1, 2)
+    qd = _dev(q, torch.bfloat16)
+    good = cache.decode(0, qd).clone()
+    # a page id outside the pool: reported in the device status word, the kernel stays in bounds
+    saved = cache.page_table.clone()
+    cache.page_table[0, 1] = cache.n_pages + 5
+    cache.decode(0, qd)
+    torch.cuda.synchronize()
+    assert case.ctx.novakv_last_device_status() & 1
+    cache.page_table.copy_(saved)
+    # a length beyond the page table: clamped and reported
+    cache.seq_lens[1] = 64 * cache.page_table.shape[1] + 7
+    cache.decode(0, qd)
+    assert case.ctx.novakv_last_device_status() & 2
+    cache.seq_lens.copy_(torch.from_numpy(lens).cuda())
+    assert torch.equal(cache.decode(0, qd), good)          # the context is still usable
+    assert case.ctx.novakv_last_device_status() == 0
+    # an appended token that names a sequence slot out of range
+    k1, v1, _ = case.draw(802, 1, 1)
+    cache.append(0, _dev(k1, torch.bfloat16), _dev(v1, torch.bfloat16), _dev(np.array([7], np.int32)),
+                 _dev(np.array([0], np.int32)))
+    assert case.ctx.novakv_last_device_status() & 8
+    # host-side validation
+    with pytest.raises(NovaKVError, match="workspace"):
+        case.ctx.novakv_decode_attention(0, qd, cache.k_pages, cache.v_pages, cache.page_table, cache.seq_lens,
+                                         good, cache.workspace[:256])
+    fresh = Context(32, 8, 128, n_layers=2)
+    fresh.novakv_load_calibration(0, case.cal)
+    with pytest.raises(NovaKVError, match="no calibration"):
+        fresh.novakv_decode_attention(1, qd, cache.k_pages, cache.v_pages, cache.page_table, cache.seq_lens,
+                                      good, cache.workspace)
+    bad = type("C", (), {})()
+    for n in ("rk", "rk_inv_t", "rv", "k_mean", "v_mean", "cb_k", "cb_v"):
+        setattr(bad, n, getattr(case.cal, n))
+    bad.cb_v = case.cal.cb_v + np.float32(1e-4)             # no longer binary16-representable
+    with pytest.raises(NovaKVError, match="unsupported calibration"):
+        fresh.novakv_load_calibration(1, bad)
+    with pytest.raises(NovaKVError, match="unsupported shape"):
+        Context(64, 8, 128)                                  # d = 128 with 8 query heads per KV head
+    fresh.close()
+
+
+# --------------------------------------------------------------------------- full bench configuration, sampled
+def test_bench_configuration_sampled():
+    """Qwen3-8B shape, B = 8, S = 16384, in the launch configuration bench.py times: the cache is
+    filled by the GPU encoder; indices are checked on sampled tokens, outputs on sampled sequences."""
+    wl = workloads.qwen3_8b(batch=8, seq_len=16384, calib_tokens=4096, lloyd_iters=6)
+    case = Case(wl)
+    from paper_2608_04074_b200.runtime import PagedCache
+    cache = PagedCache(case.ctx, wl.seq_lens, seed=11)
+    S = 16384
+    cache.seq_lens.zero_()
+    host_tokens = {}
+    for b in range(wl.batch):
+        k, v, _ = case.draw(900 + b, S, 1)
+        host_tokens[b] = (k, v)
+        cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16),
+                     _dev(np.full(S, b, np.int32)), _dev(np.arange(S, dtype=np.int32)))
+    _, _, q = case.draw(950, 1, wl.batch)
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), wl.seq_lens)
+    gen = synth.rng(77)
+    for b in (0, 5):
+        k, v = host_tokens[b]
+        gk, gv = cache.load_logical(b, 0, S)
+        pick = np.sort(gen.choice(S, size=1024, replace=False))
+        enc = case.oracle.encode(k[pick].astype(np.float64), v[pick].astype(np.float64))
+        dk, _ = check_indices(gk[pick], enc, "k")
+        dv, _ = check_indices(gv[pick], enc, "v")
+        ratio = check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
+        print(f"[bench cfg seq {b}] sampled index mismatches K {dk} V {dv}; max|delta|/||o||inf {ratio:.3e}")
