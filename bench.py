@@ -1,0 +1,459 @@
+#!/usr/bin/env python
+"""Benchmark of the NOVA-KV hot path on B200: one step = append one new token per sequence to
+the 2-bit VQ cache (transform + nearest-codeword encode) and one decode-attention pass over it.
+
+Default workload: Qwen3-8B-shaped layer (32 query / 8 KV heads, d = 128), batch 8, S = 16384,
+synthetic inputs.  Metric: decode-attention HBM GB/s at 2 bits/element = algorithmic bytes the
+decode step must read (packed indices + codebooks + transforms + q/out) / time of the whole step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-sweep]
+
+N > 1 is launched under torchrun, one rank per GPU; every rank runs its own batch (weak scaling,
+no collective on the data path), time is the max over ranks.  `--impl reference` times the CPU
+oracle on the host cores on a bounded sample of the same workload.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attention_hbm_gbps_at_2bit"
+UNIT = "GB/s"
+NOMINAL_HBM_GBPS = 8000.0
+FALLBACK_PEAK_GBPS = 6650.0
+
+
+def env_rank():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_PEAK_GBPS, "fallback"
+
+
+def ncu_traffic_per_launch(name):
+    """dram bytes per launch of the scan kernel from the committed ncu summary, if there is one."""
+    p = os.path.join(ROOT, "profiles", name)
+    try:
+        for line in open(p):
+            if line.startswith("dram_bytes_per_launch:"):
+                return float(line.split(":")[1].split()[0])
+    except OSError:
+        pass
+    return None
+
+
+class ClockSampler:
+    """Samples SM clock, power and clock-event reasons through NVML in a thread while the timed
+    region runs (read-only queries; no GPU setting is touched)."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, cuda_index, period_s=0.0005):
+        import threading
+        self.samples, self.mask, self.max_mhz, self.err = [], 0, None, None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            p = torch.cuda.get_device_properties(cuda_index)
+            try:
+                bus = "%08x:%02x:%02x.0" % (p.pci_domain_id, p.pci_bus_id, p.pci_device_id)
+                self.h = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.nv = pynvml
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:          # noqa: BLE001
+            self.err = f"nvml unavailable: {e}"
+            return
+
+        def loop():
+            nv = self.nv
+            while not self._stop.is_set():
+                try:
+                    mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                    pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                    try:
+                        m = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    except Exception:
+                        m = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                    self.samples.append((float(mhz), pw))
+                    self.mask |= int(m)
+                except Exception as e:   # noqa: BLE001
+                    self.err = str(e)
+                    return
+                self._stop.wait(period_s)
+
+        self._thread = threading.Thread(target=loop, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "samples": 0, "reasons": [self.err or "no samples"]}
+        mhz = sorted(s[0] for s in self.samples)
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_min_mhz": mhz[0], "sm_max_mhz": self.max_mhz,
+                "power_w_max": round(max(s[1] for s in self.samples), 1), "samples": len(mhz),
+                "reasons": sorted(name for bit, name in self.REASONS.items() if self.mask & bit)}
+
+
+# ------------------------------------------------------------------------------------------------
+def algorithmic_decode_bytes(wl, n_tables_heads=None):
+    """Bytes the decode step must move: indices + codebooks (fp32 keys, fp16 values) + the two
+    transforms it applies + queries (bf16) + outputs (fp32) + page table and lengths."""
+    s = wl.shape
+    d, L = s.head_dim, s.head_dim // 4
+    idx = wl.decode_index_bytes()
+    cb = s.n_kv_heads * L * 256 * 4 * (4 + 2)
+    tr = s.n_kv_heads * 2 * d * d * 4
+    qo = wl.batch * s.n_q_heads * d * (2 + 4)
+    pt = int(np.sum((wl.seq_lens.astype(np.int64) + 63) // 64)) * 4 + wl.batch * 4
+    return idx + cb + tr + qo + pt, idx
+
+
+def fill_cache_gpu(case_ctx, cache, laws, seq_lens, seed, share_content=False):
+    """Fill the paged cache with the GPU encoder (the path under test elsewhere)."""
+    import torch
+    from paper_2608_04074_b200 import synth
+    from paper_2608_04074_b200.runtime import bf16_tensor
+    cache.seq_lens.zero_()
+    CH = 8192
+    if not share_content:
+        for b, n in enumerate(seq_lens):
+            n = int(n)
+            for t0 in range(0, n, CH):
+                m = min(CH, n - t0)
+                k, v = synth.draw_kv(laws, seed + 131 * b + t0 // CH, m)
+                cache.append(0, bf16_tensor(k), bf16_tensor(v),
+                             torch.full((m,), b, dtype=torch.int32, device="cuda"),
+                             torch.arange(t0, t0 + m, dtype=torch.int32, device="cuda"))
+        return
+    # one drawn sequence, encoded once, its pages copied to every other sequence (distinct physical pages)
+    nmax = int(max(seq_lens))
+    b0 = int(np.argmax(seq_lens))
+    for t0 in range(0, nmax, CH):
+        m = min(CH, nmax - t0)
+        k, v = synth.draw_kv(laws, seed + t0 // CH, m)
+        cache.append(0, bf16_tensor(k), bf16_tensor(v), torch.full((m,), b0, dtype=torch.int32, device="cuda"),
+                     torch.arange(t0, t0 + m, dtype=torch.int32, device="cuda"))
+    src = cache.page_table[b0].long()
+    for b, n in enumerate(seq_lens):
+        if b == b0:
+            continue
+        npg = (int(n) + 63) // 64
+        dst = cache.page_table[b, :npg].long()
+        cache.k_pages[dst] = cache.k_pages[src[:npg]]
+        cache.v_pages[dst] = cache.v_pages[src[:npg]]
+    cache.seq_lens.copy_(torch.from_numpy(np.asarray(seq_lens, np.int32)).cuda())
+
+
+def time_steps(fn, steps, warmup, flush, after_warmup=None):
+    """Per-step CUDA-event timing on the current stream; the L2 flush sits outside the events."""
+    import torch
+    for _ in range(warmup):
+        flush(); fn()
+    torch.cuda.synchronize()
+    if after_warmup is not None:
+        after_warmup()
+    evs = []
+    for _ in range(steps):
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_04074_b200 import synth, workloads
+    from paper_2608_04074_b200.binding import Context
+    from paper_2608_04074_b200.runtime import PagedCache, bf16_tensor
+
+    rank, local_rank, world = env_rank()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+
+    wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len)
+    laws = wl.laws()
+    cal = wl.calibration(laws)
+    s = wl.shape
+    ctx = Context(s.n_q_heads, s.n_kv_heads, s.head_dim, device=local_rank)
+    ctx.novakv_load_calibration(0, cal)
+    B, S = wl.batch, args.seq_len
+    cache = PagedCache(ctx, wl.seq_lens, capacity_tokens=wl.seq_lens + 64, seed=17 + rank, device=dev)
+    fill_cache_gpu(ctx, cache, laws, wl.seq_lens, seed=5000 + 100000 * rank)
+
+    # step inputs: one new token per sequence at position S, one query per sequence
+    k1, v1 = synth.draw_kv(laws, 7001 + rank, B)
+    q = synth.draw_q(laws, 7002 + rank, B)
+    k1d, v1d, qd = bf16_tensor(k1, dev), bf16_tensor(v1, dev), bf16_tensor(q, dev)
+    tok_seq = torch.arange(B, dtype=torch.int32, device=dev)
+    tok_pos = torch.full((B,), S, dtype=torch.int32, device=dev)
+    out = torch.empty((B, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # > 126 MB L2
+
+    def flush():
+        flush_buf.zero_()
+
+    def step():
+        cache.append(0, k1d, v1d, tok_seq, tok_pos)
+        cache.decode(0, qd, out=out)
+
+    wl_after = workloads.qwen3_8b(batch=B, seq_len=S + 1)
+    alg_bytes, idx_bytes = algorithmic_decode_bytes(wl_after)
+
+    # ---- device-resident timing -------------------------------------------------------------
+    ctx.novakv_profile_enable(False)
+    for _ in range(2):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ctx.novakv_profile_enable(True)
+    mark = {}
+
+    def after_warmup():
+        ctx.novakv_profile_read(0); ctx.novakv_profile_read(1)
+        mark["launches0"] = ctx.novakv_launch_count()
+
+    times = time_steps(step, args.steps, args.warmup, flush, after_warmup)
+    s1_ms, s1_n = ctx.novakv_profile_read(0)
+    enc_ms, enc_n = ctx.novakv_profile_read(1)
+    ctx.novakv_profile_enable(False)
+    launches = ctx.novakv_launch_count() - mark["launches0"]
+    clocks = sampler.stop() if sampler else None
+    status = ctx.novakv_last_device_status()
+    ms_step = sum(times) / len(times)
+    if world > 1:
+        t = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+
+    # ---- decode only / encode only (explanatory numbers) ------------------------------------
+    dec_times = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, flush)
+    dec_ms = statistics.median(dec_times)
+    nowarm = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, lambda: None)
+    dec_ms_warm_l2 = statistics.median(nowarm)
+
+    # ---- end to end from pinned host buffers through the C ABI --------------------------------
+    pin = lambda t: t.cpu().pin_memory()
+    k1h, v1h, qh, seqh, posh = pin(k1d), pin(v1d), pin(qd), pin(tok_seq), pin(tok_pos)
+    out_h = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    staging = torch.empty(ctx.novakv_step_staging_bytes(B, B), dtype=torch.uint8, device=dev)
+
+    def step_host():
+        ctx.novakv_step_host(0, k1h, v1h, seqh, posh, qh, cache.k_pages, cache.v_pages, cache.page_table,
+                             cache.seq_lens, out_h, staging, cache.workspace)
+
+    e2e_times = time_steps(step_host, args.steps, 3, flush)
+    e2e_ms = sum(e2e_times) / len(e2e_times)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = int(k1h.numel() * 2 + v1h.numel() * 2 + qh.numel() * 2 + seqh.numel() * 4 + posh.numel() * 4)
+    d2h = int(out_h.numel() * 4)
+
+    result = None
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        s1_avg_ms = s1_ms / max(s1_n, 1)
+        s1_bytes = alg_bytes            # the scan kernel and its two small neighbours move all of it
+        achieved = s1_bytes / (s1_avg_ms * 1e-3) / 1e9
+        value = alg_bytes * world / (ms_step * 1e-3) / 1e9
+        result = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"qwen3_8b_shape decode step: Hq=32 Hkv=8 d=128 B={B} S={S}+1 per GPU, "
+                                   "2-bit VQ K and V (g=4, 256-entry codebooks), bf16 q, 64-token pages; "
+                                   "step = encode_append of B tokens + decode_attention",
+                       "batch_per_gpu": B, "seq_len": S, "l2": "flushed between timed steps (256 MB write)",
+                       "parallelism": f"replicas x{world}, no data-path collective"},
+            "pct_of_8TBps": round(100 * value / world / NOMINAL_HBM_GBPS, 2),
+            "algorithmic_bytes_per_step": alg_bytes, "index_bytes_per_step": idx_bytes,
+            "clocks": clocks,
+            "e2e": {"value": round(alg_bytes * world / (e2e_ms * 1e-3) / 1e9, 2), "unit": UNIT,
+                    "ms_per_step": round(e2e_ms, 5), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "roofline": {"kernel": "novakv_decode_stage1_kernel<128,4>", "bound": "hbm",
+                         "achieved": round(achieved, 1), "peak": peak, "peak_kind": f"of {peak_kind}",
+                         "unit": "GB/s", "frac": round(achieved / peak, 4),
+                         "avg_launch_ms": round(s1_avg_ms, 5), "launches_timed": s1_n,
+                         "traffic": ncu_traffic_per_launch("decode_stage1_qwen3_8b_B8_S16384.md")},
+            "decode_only": {"ms": round(dec_ms, 5), "gbps": round(alg_bytes / (dec_ms * 1e-3) / 1e9, 1),
+                            "pct_of_8TBps": round(100 * alg_bytes / (dec_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
+                            "ms_l2_not_flushed": round(dec_ms_warm_l2, 5)},
+            "encode_append": {"tokens": B, "avg_kernel_ms": round(enc_ms / max(enc_n, 1), 5)},
+            "device_status": status,
+        }
+
+    # ---- sweep: long-context bandwidth configs and prefill encode (rank 0 of a 1-GPU run only) ----
+    if rank == 0 and world == 1 and not args.no_sweep:
+        sweep = []
+        del cache
+        torch.cuda.empty_cache()
+        for (b2, s2) in ((64, 32768), (64, 65536)):
+            wl2 = workloads.qwen3_8b(batch=b2, seq_len=s2)
+            c2 = PagedCache(ctx, wl2.seq_lens, seed=23, device=dev)
+            fill_cache_gpu(ctx, c2, laws, wl2.seq_lens, seed=9000, share_content=True)
+            q2 = bf16_tensor(synth.draw_q(laws, 7100, b2), dev)
+            o2 = torch.empty((b2, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
+            ctx.novakv_profile_enable(True); ctx.novakv_profile_read(0)
+            tt = time_steps(lambda: c2.decode(0, q2, out=o2), max(5, args.steps // 2), 3, lambda: None)
+            k_ms, k_n = ctx.novakv_profile_read(0)
+            ctx.novakv_profile_enable(False)
+            ab, ib = algorithmic_decode_bytes(wl2)
+            ms = statistics.median(tt)
+            sweep.append({"workload": f"qwen3_8b_shape B={b2} S={s2} decode only, inputs larger than L2",
+                          "ms": round(ms, 4), "gbps": round(ab / (ms * 1e-3) / 1e9, 1),
+                          "pct_of_8TBps": round(100 * ab / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
+                          "scan_kernel_ms": round(k_ms / max(k_n, 1), 4),
+                          "scan_kernel_frac_of_measured_peak": round(ab / (k_ms / max(k_n, 1) * 1e-3) / 1e9 / measured_peak()[0], 4),
+                          "algorithmic_bytes": ab})
+            del c2, q2, o2
+            torch.cuda.empty_cache()
+        # prefill encode: 32768 tokens x 8 KV heads x d=128, K and V
+        T = 32768
+        wl3 = workloads.qwen3_8b(batch=1, seq_len=T)
+        c3 = PagedCache(ctx, wl3.seq_lens, seed=29, device=dev)
+        kk, vv = synth.draw_kv(laws, 7200, T)
+        kd, vd = bf16_tensor(kk, dev), bf16_tensor(vv, dev)
+        ts = torch.zeros(T, dtype=torch.int32, device=dev)
+        tp = torch.arange(T, dtype=torch.int32, device=dev)
+        tt = time_steps(lambda: c3.append(0, kd, vd, ts, tp), 5, 2, lambda: None)
+        ms = statistics.median(tt)
+        sweep.append({"workload": f"prefill encode {T} tokens x 8 KV heads x d=128 (K and V)", "ms": round(ms, 4),
+                      "tokens_per_s": round(T / (ms * 1e-3), 1)})
+        result["sweep"] = sweep
+
+    if rank == 0:
+        result["cpu_baseline"] = cpu_baseline_sample(wl, laws, cal, args)
+        print(json.dumps(result))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_inputs(wl, laws, cal, n_seq):
+    """A bounded sample of the workload for the CPU oracle: n_seq sequences of the full length whose
+    indices are 2048 oracle-encoded tokens tiled along the sequence (content does not change timing)."""
+    from oracle import novakv_oracle as O
+    from paper_2608_04074_b200 import synth
+    orc = O.Oracle.from_calibration(cal)
+    S = int(wl.seq_lens[0])
+    k, v = synth.draw_kv(laws, 8101, 2048)
+    k, v = synth.to_bf16_representable(k), synth.to_bf16_representable(v)
+    enc = orc.encode(k.astype(np.float64), v.astype(np.float64), with_gaps=False)
+    reps = (S + 2047) // 2048
+    kidx = np.tile(enc["kidx"], (reps, 1, 1))[:S]
+    vidx = np.tile(enc["vidx"], (reps, 1, 1))[:S]
+    q = synth.to_bf16_representable(synth.draw_q(laws, 8102, n_seq))
+    k1, v1 = synth.draw_kv(laws, 8103, n_seq)
+    return orc, kidx, vidx, q, synth.to_bf16_representable(k1), synth.to_bf16_representable(v1)
+
+
+def oracle_step(orc, kidx, vidx, q, k1, v1):
+    """One oracle step on the sample: encode the new tokens, then decode every sampled sequence."""
+    orc.encode(k1.astype(np.float64), v1.astype(np.float64), with_gaps=False)
+    for b in range(q.shape[0]):
+        orc.decode(q[b].astype(np.float64), kidx, vidx)
+
+
+def cpu_baseline_sample(wl, laws, cal, args):
+    from oracle import novakv_oracle as O
+    n_seq = 2
+    orc, kidx, vidx, q, k1, v1 = oracle_sample_inputs(wl, laws, cal, n_seq)
+    t0 = time.perf_counter()
+    oracle_step(orc, kidx, vidx, q, k1, v1)
+    dt = time.perf_counter() - t0
+    s = wl.shape
+    sample_bytes = n_seq * int(wl.seq_lens[0]) * s.n_kv_heads * 2 * (s.head_dim // 4)
+    return {"value": round(sample_bytes / dt / 1e9, 6), "unit": UNIT, "cores": O.cpu_threads(), "kind": "oracle",
+            "seconds": round(dt, 3),
+            "sample": f"{n_seq} of {wl.batch} sequences (S={int(wl.seq_lens[0])}, all heads): oracle encode of "
+                      f"{n_seq} new tokens + explicit-dequantise decode; index bytes of the sample / wall time"}
+
+
+def run_reference(args):
+    rank, _, world = env_rank()
+    if rank != 0:
+        return
+    from oracle import novakv_oracle as O
+    from paper_2608_04074_b200 import workloads
+    wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len)
+    laws = wl.laws()
+    cal = wl.calibration(laws)
+    n_seq = 1
+    orc, kidx, vidx, q, k1, v1 = oracle_sample_inputs(wl, laws, cal, n_seq)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(orc, kidx, vidx, q, k1, v1)
+    steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(orc, kidx, vidx, q, k1, v1)
+    dt = (time.perf_counter() - t0) / steps
+    s = wl.shape
+    sample_bytes = n_seq * int(wl.seq_lens[0]) * s.n_kv_heads * 2 * (s.head_dim // 4)
+    val = round(sample_bytes / dt / 1e9, 6)
+    sample = (f"each step: {n_seq} of {wl.batch} sequences (S={int(wl.seq_lens[0])}, all heads), oracle encode + "
+              f"decode; {steps} steps timed")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"qwen3_8b_shape decode step: Hq=32 Hkv=8 d=128 B={args.batch} S={args.seq_len}, "
+                               "CPU oracle on a bounded sample"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": O.cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=8)
+    ap.add_argument("--seq-len", type=int, default=16384)
+    ap.add_argument("--no-sweep", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -45,7 +45,8 @@ def load_library(path=None):
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = str(path or _build.LIB_CUDA)
+    import os
+    p = str(path or os.environ.get("NOVAKV_LIB") or _build.LIB_CUDA)
     try:
         lib = ctypes.CDLL(p)
     except OSError as e:

@@ -23,7 +23,10 @@
 
 namespace {
 
-constexpr int NCW = 8;                        // consumer warps
+#ifndef NOVAKV_NCW
+#define NOVAKV_NCW 8
+#endif
+constexpr int NCW = NOVAKV_NCW;               // consumer warps
 constexpr int S1_THREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int LUT_PLANE_BYTES = 256 * 256;    // 256 codes x 16 entries x 16 bytes
 constexpr int VCB_BYTES = 256 * 256;          // 256 codes x 32 group slots x 4 halves
@@ -37,11 +40,18 @@ struct S1 {
     static constexpr int HSETS = HG <= 4 ? 1 : 2;             // table entries are 4 heads wide
     static constexpr int HPAD = HSETS * 4;
     static constexpr int CHUNK = NOVAKV_PAGE_TOKENS * L;      // bytes of one page of one head, K or V
-    static constexpr int NST = D == 128 ? 6 : 8;              // ring stages
     static constexpr int LUT_BYTES = HSETS * PLANES * LUT_PLANE_BYTES;
-    static constexpr int RING_BYTES = NST * 2 * CHUNK;
     static constexpr int P_WARP_BYTES = 32 * HPAD * 8;        // 32 tokens x HPAD heads x (p, p)
     static constexpr int P_BYTES = NCW * P_WARP_BYTES;
+    // Ring stages (each = one page of K and of V).  A consumer warp takes every (NCW/2)-th page; the
+    // stage count is a multiple of that stride, so that the page a warp waits for reuses the stage of
+    // a page the same warp has already consumed: a waiter is then never more than one mbarrier phase
+    // ahead, which the parity test of a phase wait requires.
+    static constexpr int STRIDE = NCW / 2;
+    static constexpr int NST_FIT = (232448 - 256 - LUT_BYTES - VCB_BYTES - P_BYTES) / (2 * CHUNK);
+    static constexpr int NST = (NST_FIT / STRIDE >= 2 ? 2 : 1) * STRIDE;
+    static_assert(NCW % 2 == 0 && NST <= NST_FIT, "ring does not fit in shared memory");
+    static constexpr int RING_BYTES = NST * 2 * CHUNK;
     static constexpr int OFF_LUT = 0;
     static constexpr int OFF_VCB = OFF_LUT + LUT_BYTES;
     static constexpr int OFF_RING = OFF_VCB + VCB_BYTES;
@@ -274,7 +284,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     const long gp = gp_base + i;
                     const int st = (int)(gp % NST);
                     const uint32_t par = (uint32_t)((gp / NST) & 1);
-                    if (!mbar_wait_bounded(bar_empty(st), par ^ 1u)) {
+                    if (!mbar_wait_bounded(bar_empty(st), par ^ 1u, abort_flag)) {
                         atomicOr(dev_status, NOVAKV_DEV_WAIT_TIMEOUT);
                         *abort_flag = 1;
                         break;
@@ -290,7 +300,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         } else {
             // ---- score table: LUT[hs][plane][code][e] (4 heads per entry) ----------------------
             {
-                const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;      // 256 threads: 16 codes x 16 entries
+                constexpr int CPI = NCW * 2;                                   // codes per iteration (16 entries each)
+                const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
                 const int sigma = e & 7, mpar = e >> 3;
                 const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)sg.kvh * C::PLANES * 256 * 16;
                 const float* qs = reinterpret_cast<const float*>(smem + C::OFF_P);
@@ -301,8 +312,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 #pragma unroll
                     for (int h = 0; h < HPAD; ++h) qseg[h] = *reinterpret_cast<const float4*>(qs + h * D + l * 4);
 #pragma unroll 4
-                    for (int it = 0; it < 16; ++it) {
-                        const int code = code0 + it * 16;
+                    for (int it = 0; it < (256 + CPI - 1) / CPI; ++it) {
+                        const int code = code0 + it * CPI;
+                        if (code >= 256) break;
                         const float4 cw = cbk[((size_t)pl * 256 + code) * 16 + e];
 #pragma unroll
                         for (int hs = 0; hs < HSETS; ++hs) {
@@ -319,7 +331,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             // consumer-only barrier: table complete, q' staging no longer needed
             asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
             if (need_vcb) {
-                if (!mbar_wait_bounded(bar_vcb, vcb_phase)) {
+                if (!mbar_wait_bounded(bar_vcb, vcb_phase, abort_flag)) {
                     atomicOr(dev_status, NOVAKV_DEV_WAIT_TIMEOUT);
                     *abort_flag = 1;
                 }
@@ -334,7 +346,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 const long gp = gp_base + pgi;
                 const int st = (int)(gp % NST);
                 const uint32_t par = (uint32_t)((gp / NST) & 1);
-                if (!mbar_wait_bounded(bar_full(st), par)) {
+                if (!mbar_wait_bounded(bar_full(st), par, abort_flag)) {
                     atomicOr(dev_status, NOVAKV_DEV_WAIT_TIMEOUT);
                     *abort_flag = 1;
                     break;
@@ -509,8 +521,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     // fault path only: let copies that were issued but never consumed land before the CTA retires
     if (*abort_flag && threadIdx.x == NCW * 32) {
         for (int st = 0; st < NST; ++st) {
-            mbar_wait_bounded(bar_full(st), 0, 1u << 16);
-            mbar_wait_bounded(bar_full(st), 1, 1u << 16);
+            mbar_wait_bounded(bar_full(st), 0, nullptr, 1ll << 22);
+            mbar_wait_bounded(bar_full(st), 1, nullptr, 1ll << 22);
         }
     }
 }

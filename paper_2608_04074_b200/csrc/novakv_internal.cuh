@@ -107,12 +107,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls and reports false (the caller records the fault).
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = (1u << 24)) {
-    for (uint32_t it = 0; it < limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: polls until the phase completes, another thread of the CTA has raised `abort`, or
+// about `limit_cycles` SM clocks (default 2^29, a quarter of a second) have passed; false means
+// "gave up" and the caller records the fault.  A healthy wait lasts microseconds.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort = nullptr,
+                                                  long long limit_cycles = (1ll << 29)) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 32; ++it)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (abort != nullptr && *abort) return false;
+        if (clock64() - t0 > limit_cycles) return false;
     }
-    return false;
 }
 // 1-D bulk asynchronous copy global -> shared of this CTA, completion on an mbarrier.
 // Both addresses 16-byte aligned, size a multiple of 16 bytes.
