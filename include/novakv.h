@@ -145,6 +145,29 @@ novakv_status novakv_decode_attention(novakv_ctx* ctx, int layer, const void* q,
     float sm_scale, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
     novakv_stream stream);
 
+/*
+ * The same decode step for callers that cannot supply a workspace and cannot allocate one: an
+ * engine that gave all device memory to its own pool, a plug-in inside it, a serving loop that must
+ * never call cudaMalloc (the call synchronises the device).  (The paper has no counterpart; this is
+ * a property of the library, not of the method.)  The scratch that novakv_decode_attention takes as
+ * `workspace` is a fixed array of NOVAKV_NOALLOC_SCRATCH_BYTES inside the library's device image:
+ * every GPU that loads the library holds it until the process exits.
+ *   - Arguments and results are those of novakv_decode_attention without workspace/workspace_bytes.
+ *   - Returns NOVAKV_EWORKSPACE when novakv_decode_workspace_bytes(ctx, batch) exceeds
+ *     NOVAKV_NOALLOC_SCRATCH_BYTES (for the Qwen3-8B shape that is a batch of about 100 sequences).
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine, and records no timing events.
+ *   - All calls on a device share the array: calls that overlap on the GPU (other streams, other
+ *     contexts) race; calls on one stream are ordered and safe.  Every scratch word is written
+ *     before it is read within a call, so nothing needs clearing between calls.
+ *   - The first call on each device queries the array's device address (a synchronous runtime
+ *     call); issue that first call before any stream capture begins.
+ */
+#define NOVAKV_NOALLOC_SCRATCH_BYTES (4u << 20)
+novakv_status novakv_decode_attention_noalloc(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch,
+    float sm_scale, void* out, int out_is_fp32, novakv_stream stream);
+
 /* Synchronises `stream`, returns the device status word in *word and clears it. */
 novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word);
 

@@ -20,7 +20,7 @@ EXPORTED = [
     "novakv_decode_attention", "novakv_last_device_status", "novakv_step_staging_bytes",
     "novakv_step_host", "novakv_search_coefficients", "novakv_bf16_workspace_bytes",
     "novakv_bf16_decode_attention", "novakv_profile_enable", "novakv_profile_read",
-    "novakv_launch_count", "novakv_debug_set_scan_ctas",
+    "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc",
 ]
 
 
@@ -65,6 +65,8 @@ def load_library(path=None):
     lib.novakv_decode_attention.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                             c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p,
                                             c_size_t, c_void_p]
+    lib.novakv_decode_attention_noalloc.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+                                                    c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p]
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
     lib.novakv_step_staging_bytes.argtypes = [c_void_p, c_int, c_int]
     lib.novakv_step_staging_bytes.restype = c_size_t
@@ -163,6 +165,15 @@ class Context:
             int(page_table.shape[1]), _ptr(seq_lens), batch, scale, _ptr(out),
             1 if out.dtype == torch.float32 else 0, _ptr(workspace),
             int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention")
+
+    def novakv_decode_attention_noalloc(self, layer, q, k_pages, v_pages, page_table, seq_lens, out, sm_scale=None):
+        """Decode step whose scratch is the library's fixed device array (no workspace argument)."""
+        import torch
+        scale = float(self.head_dim) ** -0.5 if sm_scale is None else float(sm_scale)
+        _check(self.lib, self.lib.novakv_decode_attention_noalloc(
+            self.handle, layer, _ptr(q), _ptr(k_pages), _ptr(v_pages), int(k_pages.shape[0]), _ptr(page_table),
+            int(page_table.shape[1]), _ptr(seq_lens), int(q.shape[0]), scale, _ptr(out),
+            1 if out.dtype == torch.float32 else 0, _stream()), "novakv_decode_attention_noalloc")
 
     def novakv_last_device_status(self):
         word = c_uint32(0)

@@ -15,7 +15,8 @@ INCLUDE = PKG_DIR.parent / "include"
 LIB_CUDA = PKG_DIR / "libnovakv.so"
 LIB_CALIB = PKG_DIR / "libnovakv_calib.so"
 
-CUDA_SOURCES = ["novakv_api.cu", "novakv_encode.cu", "novakv_decode.cu", "novakv_bf16_decode.cu"]
+CUDA_SOURCES = ["novakv_api.cu", "novakv_encode.cu", "novakv_decode.cu", "novakv_bf16_decode.cu",
+                "novakv_noalloc.cu"]
 
 
 def _newer(target: Path, sources: list[Path]) -> bool:
