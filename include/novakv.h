@@ -10,7 +10,8 @@
  * codeword indices for the key and L for the value: 8/g = 2 bits per cached element, no
  * per-token metadata.  Pages hold 64 tokens.  Two caller-owned device pools of equal geometry:
  *     key pool    uint8 [n_pages][Hkv][64][L]        token-major
- *     value pool  uint8 [n_pages][Hkv][4][L][16]     four 16-token blocks, group-major in a block
+ *     value pool  uint8 [n_pages][Hkv][4][L][16]     four 16-token blocks; in a block one 16-byte row per
+ *                                                    group, group g in row (g % 8) * (L / 8) + g / 8
  * page_table[seq][i] (int32, row length max_pages_per_seq) names the page of tokens 64i..64i+63.
  *
  * Ownership: the context owns device copies of the calibration tables and one device status
@@ -227,6 +228,13 @@ novakv_status novakv_profile_read(novakv_ctx* ctx, int kind, double* total_ms, l
  * rounding, because the split over the sequence is merged exactly (App. B, two-stage split-KV).
  */
 novakv_status novakv_debug_set_scan_ctas(novakv_ctx* ctx, int n_ctas);
+
+/*
+ * Value-accumulation variant of the decode scan kernel: 1 (default) runs sum_j p_j * codeword_j on
+ * tensor cores (fp16 weights and codewords, fp32 accumulation); 0 keeps it on CUDA cores in fp32.
+ * Both are held to the same output tolerance; the benchmark reports both.
+ */
+novakv_status novakv_debug_set_value_path(novakv_ctx* ctx, int path);
 
 /* Kernels this library launched since the context was created (all kinds). */
 long novakv_launch_count(const novakv_ctx* ctx);

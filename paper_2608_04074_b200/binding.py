@@ -20,7 +20,7 @@ EXPORTED = [
     "novakv_decode_attention", "novakv_last_device_status", "novakv_step_staging_bytes",
     "novakv_step_host", "novakv_search_coefficients", "novakv_bf16_workspace_bytes",
     "novakv_bf16_decode_attention", "novakv_profile_enable", "novakv_profile_read",
-    "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc",
+    "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc", "novakv_debug_set_value_path",
 ]
 
 
@@ -83,6 +83,7 @@ def load_library(path=None):
     lib.novakv_profile_read.argtypes = [c_void_p, c_int, POINTER(c_double), POINTER(c_long)]
     lib.novakv_launch_count.argtypes = [c_void_p]
     lib.novakv_debug_set_scan_ctas.argtypes = [c_void_p, c_int]
+    lib.novakv_debug_set_value_path.argtypes = [c_void_p, c_int]
     lib.novakv_launch_count.restype = c_long
     if path is None:
         _lib = lib
@@ -227,6 +228,9 @@ class Context:
 
     def novakv_debug_set_scan_ctas(self, n_ctas):
         _check(self.lib, self.lib.novakv_debug_set_scan_ctas(self.handle, int(n_ctas)), "novakv_debug_set_scan_ctas")
+
+    def novakv_debug_set_value_path(self, path):
+        _check(self.lib, self.lib.novakv_debug_set_value_path(self.handle, int(path)), "novakv_debug_set_value_path")
 
     def novakv_launch_count(self):
         return int(self.lib.novakv_launch_count(self.handle))

@@ -7,8 +7,9 @@ side, i.e. exactly 8/g = 2 bits per cached element.
 Physical layout of a page (64 tokens), identical for every KV head:
 
 * key pool    ``uint8 [n_pages][Hkv][64][L]``           token-major;
-* value pool  ``uint8 [n_pages][Hkv][4][L][16]``        four 16-token blocks, group-major
-  inside a block (the 16 bytes of one group and 16 consecutive tokens are contiguous).
+* value pool  ``uint8 [n_pages][Hkv][4][L][16]``        four 16-token blocks; inside a block one
+  16-byte row per group (16 consecutive tokens), group ``g`` in row ``(g % 8) * (L // 8) + g // 8``
+  (the decode kernel's tensor-core lanes then read their rows from distinct shared-memory banks).
 
 ``page_table[seq][i]`` names the physical page that holds tokens ``64 i .. 64 i + 63``.
 The functions below only permute bytes; they hold no arithmetic of the method.
@@ -25,6 +26,12 @@ CODEBOOK_SIZE = 256
 
 def n_groups(head_dim: int) -> int:
     return head_dim // GROUP_SIZE
+
+
+def value_row_of_group(n_groups_: int) -> np.ndarray:
+    """Row of each group inside a 16-token block of the value pool."""
+    g = np.arange(n_groups_)
+    return (g % 8) * (n_groups_ // 8) + g // 8
 
 
 def index_bytes_per_token_per_kv_head(head_dim: int) -> int:
@@ -68,7 +75,7 @@ def write_tokens(k_pool: np.ndarray, v_pool: np.ndarray, page_table_row: np.ndar
     t = pos % PAGE_TOKENS
     for h in range(hkv):
         kp[page, h, t, :] = kidx[:, h, :]
-        vp[page, h, t // V_BLOCK, :, t % V_BLOCK] = vidx[:, h, :]
+        vp[page[:, None], h, (t // V_BLOCK)[:, None], value_row_of_group(l)[None, :], (t % V_BLOCK)[:, None]] = vidx[:, h, :]
 
 
 def read_tokens(k_pool: np.ndarray, v_pool: np.ndarray, page_table_row: np.ndarray, n_kv_heads: int,
@@ -84,5 +91,5 @@ def read_tokens(k_pool: np.ndarray, v_pool: np.ndarray, page_table_row: np.ndarr
     vidx = np.empty((n, n_kv_heads, l), np.uint8)
     for h in range(n_kv_heads):
         kidx[:, h, :] = kp[page, h, t, :]
-        vidx[:, h, :] = vp[page, h, t // V_BLOCK, :, t % V_BLOCK]
+        vidx[:, h, :] = vp[page[:, None], h, (t // V_BLOCK)[:, None], value_row_of_group(l)[None, :], (t % V_BLOCK)[:, None]]
     return kidx, vidx

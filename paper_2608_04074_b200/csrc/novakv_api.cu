@@ -64,7 +64,7 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
 static void free_layer(novakv_layer& ly) {
     cudaFree(ly.rk_d); cudaFree(ly.rv_d); cudaFree(ly.k_mean_d); cudaFree(ly.v_mean_d);
     cudaFree(ly.cb_k); cudaFree(ly.cb_v); cudaFree(ly.rk_inv_t); cudaFree(ly.rv_t);
-    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_half);
+    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_half); cudaFree(ly.cb_v_mma);
     ly = novakv_layer();
 }
 
@@ -95,7 +95,10 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
     const size_t n_mat = (size_t)H * d * d, n_vec = (size_t)H * d, n_cb = (size_t)H * L * C * g;
 
     // value codewords must survive the binary16 round trip exactly
+    // cbv_grp: slot = group (scratch);  cbv_half: slot = index row of the group (CUDA-core value side)
+    std::vector<__half> cbv_grp((size_t)H * C * 32 * g, __float2half(0.f));
     std::vector<__half> cbv_half((size_t)H * C * 32 * g, __float2half(0.f));
+    std::vector<__half> cbv_mma((size_t)H * C * 32 * g, __float2half(0.f));
     for (int hh = 0; hh < H; ++hh)
         for (int l = 0; l < L; ++l)
             for (int c = 0; c < C; ++c)
@@ -103,8 +106,20 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
                     float x = h->cb_v[(((size_t)hh * L + l) * C + c) * g + i];
                     __half hx = __float2half_rn(x);
                     if (!(__half2float(hx) == x)) return NOVAKV_EUNSUPPORTED;
-                    cbv_half[(((size_t)hh * C + c) * 32 + l) * g + i] = hx;
+                    cbv_grp[(((size_t)hh * C + c) * 32 + l) * g + i] = hx;
+                    cbv_half[(((size_t)hh * C + c) * 32 + ((l & 7) * (L / 8) + (l >> 3))) * g + i] = hx;
                 }
+    // tensor-core value side: slot pos = 16*rho + 4*xb + r' holds group 8*(xb mod NGB) + 4*rho + r'
+    // (NGB = L/8 group blocks; for L = 16 every group appears twice).  The four lanes of an MMA quad
+    // then read four different 8-byte bank pairs whatever codes their tokens carry.
+    for (int hh = 0; hh < H; ++hh)
+        for (int c = 0; c < C; ++c)
+            for (int pos = 0; pos < 32; ++pos) {
+                const int rho = pos >> 4, xb = (pos >> 2) & 3, rp = pos & 3;
+                const int l = 8 * (xb % (L / 8)) + 4 * rho + rp;
+                for (int i = 0; i < g; ++i)
+                    cbv_mma[(((size_t)hh * C + c) * 32 + pos) * g + i] = cbv_grp[(((size_t)hh * C + c) * 32 + l) * g + i];
+            }
 
     std::vector<double> rk_d(n_mat), rv_d(n_mat), km_d(n_vec, 0.0), vm_d(n_vec, 0.0);
     std::vector<float> vm_f(n_vec, 0.f);
@@ -140,7 +155,7 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
               upload(&ly.cb_k, cbk) == cudaSuccess && upload(&ly.cb_v, cbv) == cudaSuccess &&
               upload(&ly.rk_inv_t, rkinv) == cudaSuccess && upload(&ly.rv_t, rvt) == cudaSuccess &&
               upload(&ly.v_mean, vm_f) == cudaSuccess && upload(&ly.cb_k_lut, cbk_lut) == cudaSuccess &&
-              upload(&ly.cb_v_half, cbv_half) == cudaSuccess;
+              upload(&ly.cb_v_half, cbv_half) == cudaSuccess && upload(&ly.cb_v_mma, cbv_mma) == cudaSuccess;
     if (!ok) { free_layer(ly); return NOVAKV_ECUDA; }
     ly.loaded = true;
     return NOVAKV_OK;
@@ -346,6 +361,12 @@ extern "C" novakv_status novakv_profile_read(novakv_ctx* ctx, int kind, double* 
 extern "C" novakv_status novakv_debug_set_scan_ctas(novakv_ctx* ctx, int n_ctas) {
     if (!ctx || n_ctas < 0) return NOVAKV_EINVAL;
     ctx->scan_ctas = n_ctas;
+    return NOVAKV_OK;
+}
+
+extern "C" novakv_status novakv_debug_set_value_path(novakv_ctx* ctx, int path) {
+    if (!ctx || (path != 0 && path != 1)) return NOVAKV_EINVAL;
+    ctx->value_path = path;
     return NOVAKV_OK;
 }
 

@@ -9,8 +9,10 @@
 //                - a producer warp streams 64-token index chunks into a shared-memory ring with
 //                  1-D bulk asynchronous copies (mbarrier completion),
 //                - consumer warps: lane <-> token, 32 table lookups summed in registers (no cross
-//                  lane reduction), online softmax per 32-token tile, then lane <-> group value
-//                  accumulation of p * value-codeword in the value-transform domain,
+//                  lane reduction), online softmax per 32-token tile, then accumulation of
+//                  p * value-codeword in the value-transform domain: a dense [heads x tokens] x
+//                  [tokens x d] contraction, run on tensor cores (mma.sync, fp16 operands, fp32
+//                  accumulators) or, as the selectable alternative, on CUDA cores in fp32,
 //                - the warps' partial (m, l, acc) are merged and written once per segment.
 //   merge    : exact log-sum-exp merge of the partials of every (sequence, KV head), then the inverse
 //              value transform o = o' rv^T + v_mean, once per head.
@@ -26,23 +28,36 @@ namespace {
 #ifndef NOVAKV_NCW
 #define NOVAKV_NCW 8
 #endif
+// 1: the producer prefetches the pages of its next batch of 32 page ids into L2; 0: no prefetch
+#ifndef NOVAKV_L2_PREFETCH_PAGES
+#define NOVAKV_L2_PREFETCH_PAGES 0
+#endif
+#ifndef NOVAKV_PRODUCER_PAGES
+#define NOVAKV_PRODUCER_PAGES 4              // pages issued per producer instruction group (2 lanes per page)
+#endif
 constexpr int NCW = NOVAKV_NCW;               // consumer warps
 constexpr int S1_THREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int LUT_PLANE_BYTES = 256 * 256;    // 256 codes x 16 entries x 16 bytes
-constexpr int VCB_BYTES = 256 * 256;          // 256 codes x 32 group slots x 4 halves
+constexpr int VCB_BYTES = 256 * 256;          // 256 codes x 32 slots x 4 halves
 constexpr float M_INIT = -1.0e30f;
 
-template <int D, int HG>
+// VM selects the value side: false = CUDA cores (fp32 FMA, weights broadcast from shared memory),
+// true = tensor cores (mma.sync m16n8k16, fp16 weights and codewords, fp32 accumulators).
+template <int D, int HG, bool VM>
 struct S1 {
     static constexpr int L = D / NOVAKV_G;
     static constexpr int GPS = L / 8;                         // groups per slot: 4 (d=128) or 2 (d=64)
     static constexpr int PLANES = GPS / 2;
+    static constexpr int NGB = L / 8;                         // group blocks of 8 groups (value side, MMA rows)
     static constexpr int HSETS = HG <= 4 ? 1 : 2;             // table entries are 4 heads wide
     static constexpr int HPAD = HSETS * 4;
     static constexpr int CHUNK = NOVAKV_PAGE_TOKENS * L;      // bytes of one page of one head, K or V
     static constexpr int LUT_BYTES = HSETS * PLANES * LUT_PLANE_BYTES;
-    static constexpr int P_WARP_BYTES = 32 * HPAD * 8;        // 32 tokens x HPAD heads x (p, p)
-    static constexpr int P_BYTES = NCW * P_WARP_BYTES;
+    // per-warp staging of the softmax weights of one 32-token tile
+    //   VM: fp16 [HPAD][4 k-slot pairs][8 tokens]        otherwise: fp32 pairs [32 tokens][HPAD][2]
+    static constexpr int P_WARP_BYTES = VM ? HPAD * 64 : 32 * HPAD * 8;
+    static constexpr int Q_BYTES = HPAD * D * 4;              // q' staging during the table build
+    static constexpr int P_BYTES = NCW * P_WARP_BYTES > Q_BYTES ? NCW * P_WARP_BYTES : Q_BYTES;
     // Ring stages (each = one page of K and of V).  A consumer warp takes every (NCW/2)-th page; the
     // stage count is a multiple of that stride, so that the page a warp waits for reuses the stage of
     // a page the same warp has already consumed: a waiter is then never more than one mbarrier phase
@@ -61,7 +76,6 @@ struct S1 {
     // merge buffer (aliases the table once a segment's scan is done)
     static constexpr int MERGE_ACC_BYTES = NCW * HPAD * D * 4;
     static_assert(MERGE_ACC_BYTES + NCW * HPAD * 8 <= LUT_BYTES, "merge buffer must fit in the table");
-    static_assert(HPAD * D * 4 <= P_BYTES, "q' staging must fit in the P area");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
@@ -210,17 +224,18 @@ __device__ __forceinline__ Segment locate(const int32_t* __restrict__ page_prefi
 // ------------------------------------------------------------------------------------------------
 // stage 1: persistent index scan
 // ------------------------------------------------------------------------------------------------
-template <int D, int HG>
+template <int D, int HG, bool VM>
 __global__ void __launch_bounds__(S1_THREADS, 1)
 novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restrict__ cb_k_lut,
-                            const __half* __restrict__ cb_v_half, const uint8_t* __restrict__ k_pages,
+                            const __half* __restrict__ cb_v_img, const uint8_t* __restrict__ k_pages,
                             const uint8_t* __restrict__ v_pages, int n_pages,
                             const int32_t* __restrict__ page_table, int max_pages_per_seq,
                             const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ page_prefix,
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
                             float* __restrict__ part_acc, uint32_t* __restrict__ dev_status) {
-    using C = S1<D, HG>;
+    using C = S1<D, HG, VM>;
     constexpr int L = C::L, GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, NST = C::NST, CHUNK = C::CHUNK;
+    constexpr int NGB = C::NGB;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t s_base = smem_u32(smem);
     const uint32_t s_lut = s_base + C::OFF_LUT, s_vcb = s_base + C::OFF_VCB, s_ring = s_base + C::OFF_RING;
@@ -237,7 +252,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     if (u_begin >= u_end) return;
 
     if (threadIdx.x == 0) {
-        for (int st = 0; st < NST; ++st) { mbar_init(bar_full(st), 1); mbar_init(bar_empty(st), 2); }
+        for (int st = 0; st < NST; ++st) { mbar_init(bar_full(st), 2); mbar_init(bar_empty(st), 2); }
         mbar_init(bar_vcb, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -246,9 +261,23 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
     // per-warp running state (consumer warps)
     float m_run[HPAD], l_run[HPAD];
-    uint64_t acc[HPAD][2];                       // lane <-> group: 4 value coefficients x HPAD heads
+    uint64_t acc[HPAD][2];                       // !VM: lane <-> group, 4 value coefficients x HPAD heads
+    float macc[HSETS][NGB][4];                   //  VM: lane (r, c): head 4*hs + c, group 8*gb + r, 4 coefficients
 #pragma unroll
     for (int h = 0; h < HPAD; ++h) { m_run[h] = M_INIT; l_run[h] = 0.f; acc[h][0] = 0ull; acc[h][1] = 0ull; }
+#pragma unroll
+    for (int hs = 0; hs < HSETS; ++hs)
+#pragma unroll
+        for (int gb = 0; gb < NGB; ++gb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) macc[hs][gb][i] = 0.f;
+
+    // lane roles of the tensor-core value side (MMA fragment coordinates)
+    const int fr = lane >> 2, fc = lane & 3;
+    // byte selector that moves byte fc of an index word to bits 8..15 over a slot offset in bits 0..7
+    const uint32_t sel_c = 0x5504u | ((uint32_t)fc << 4);
+    // B fragments carry a weight in the low or high half depending on the column parity (fr & 1)
+    const uint32_t sel_b0 = (fr & 1) ? 0x1044u : 0x4410u, sel_b1 = (fr & 1) ? 0x3244u : 0x4432u;
 
     int vcb_head = -1;       // KV head whose value codebook is resident
     uint32_t vcb_phase = 0;
@@ -271,30 +300,73 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             if (need_vcb) {
                 fence_proxy_async();
                 mbar_arrive_expect_tx(bar_vcb, VCB_BYTES);
-                bulk_g2s(s_vcb, cb_v_half + (size_t)sg.kvh * (VCB_BYTES / 2), VCB_BYTES, bar_vcb);
+                bulk_g2s(s_vcb, cb_v_img + (size_t)sg.kvh * (VCB_BYTES / 2), VCB_BYTES, bar_vcb);
             }
         }
         __syncthreads();
 
         if (warp == NCW) {
-            // ---- producer: stream the segment's pages through the ring ------------------------
-            if (lane == 0) {
-                for (int i = 0; i < sg.npg; ++i) {
-                    if (*abort_flag) break;
-                    const long gp = gp_base + i;
-                    const int st = (int)(gp % NST);
-                    const uint32_t par = (uint32_t)((gp / NST) & 1);
-                    if (!mbar_wait_bounded(bar_empty(st), par ^ 1u, abort_flag)) {
-                        atomicOr(dev_status, NOVAKV_DEV_WAIT_TIMEOUT);
-                        *abort_flag = 1;
-                        break;
+            // ---- producer warp: stream the segment's pages through the ring --------------------
+            // Page ids are fetched 32 at a time (one coalesced load per batch, the next batch in flight
+            // while the current one is issued), so that no global-memory latency sits between two bulk
+            // copies.
+            {
+                const int32_t* pt = page_table + (size_t)sg.b * max_pages_per_seq + sg.pg0;
+                auto load_ids = [&](int i0) {
+                    int page = 0;
+                    if (i0 + lane < sg.npg) {
+                        page = pt[i0 + lane];
+                        if (page < 0 || page >= n_pages) { atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE); page = 0; }
                     }
-                    int page = page_table[(size_t)sg.b * max_pages_per_seq + sg.pg0 + i];
-                    if (page < 0 || page >= n_pages) { atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE); page = 0; }
-                    const size_t off = ((size_t)page * n_kv_heads + sg.kvh) * CHUNK;
-                    mbar_arrive_expect_tx(bar_full(st), 2 * CHUNK);
-                    bulk_g2s(s_ring + st * 2 * CHUNK, k_pages + off, CHUNK, bar_full(st));
-                    bulk_g2s(s_ring + st * 2 * CHUNK + CHUNK, v_pages + off, CHUNK, bar_full(st));
+                    return page;
+                };
+                int ids_next = load_ids(0);
+                bool stop = false;
+                // One thread can start a bulk copy only every few hundred clocks, while several lanes of
+                // a warp issuing in the same instruction cost little more than one: 2*PG lanes each
+                // issue one chunk (K or V) of PG consecutive pages.
+                constexpr int PG = NOVAKV_PRODUCER_PAGES;
+                const int side = lane & 1;
+                for (int i0 = 0; i0 < sg.npg && !stop; i0 += 32) {
+                    const int ids = ids_next;
+                    ids_next = load_ids(i0 + 32);
+                    const int nb = min(32, sg.npg - i0);
+                    for (int j = 0; j < nb; j += PG) {
+                        const int pj = j + (lane >> 1);
+                        const int page = __shfl_sync(0xffffffffu, ids, pj & 31);
+                        if (NOVAKV_L2_PREFETCH_PAGES > 0) {
+                            // line prefetches into L2, NOVAKV_L2_PREFETCH_PAGES pages ahead of the ring:
+                            // one instruction of the warp covers the K and V chunk of one page
+                            for (int q = 0; q < PG; ++q) {
+                                const int jj = j + q + NOVAKV_L2_PREFETCH_PAGES;
+                                const int pf_page = __shfl_sync(0xffffffffu, jj < 32 ? ids : ids_next, jj & 31);
+                                if (i0 + jj < sg.npg) {
+                                    constexpr int LINES = CHUNK / 128;        // 128-byte lines per chunk: 16 or 8
+                                    const size_t off = ((size_t)pf_page * n_kv_heads + sg.kvh) * CHUNK;
+                                    const uint8_t* src = (lane < LINES ? k_pages : v_pages) + off + (size_t)(lane % LINES) * 128;
+                                    if (lane < 2 * LINES) asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
+                                }
+                            }
+                        }
+                        int ok = 1;
+                        if (lane < 2 * PG && pj < nb) {
+                            const long gp = gp_base + i0 + pj;
+                            const int st = (int)(gp % NST);
+                            const uint32_t par = (uint32_t)((gp / NST) & 1);
+                            if (*abort_flag) {
+                                ok = 0;
+                            } else if (!mbar_wait_bounded(bar_empty(st), par ^ 1u, abort_flag)) {
+                                atomicOr(dev_status, NOVAKV_DEV_WAIT_TIMEOUT);
+                                *abort_flag = 1;
+                                ok = 0;
+                            } else {
+                                const size_t off = ((size_t)page * n_kv_heads + sg.kvh) * CHUNK;
+                                mbar_arrive_expect_tx(bar_full(st), CHUNK);
+                                bulk_g2s(s_ring + st * 2 * CHUNK + side * CHUNK, (side ? v_pages : k_pages) + off, CHUNK, bar_full(st));
+                            }
+                        }
+                        if (!__all_sync(0xffffffffu, ok)) { stop = true; break; }
+                    }
                 }
             }
         } else {
@@ -352,7 +424,10 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     break;
                 }
                 const int tok0 = (sg.pg0 + pgi) * NOVAKV_PAGE_TOKENS + half * 32;
-                const int nvalid = min(32, sg.len - tok0);
+                int nvalid = min(32, sg.len - tok0);
+#ifdef NOVAKV_EXPERIMENT_SKIP_COMPUTE
+                nvalid = 0;     // measurement only: stream the ring without consuming it
+#endif
                 if (nvalid > 0) {
                     const uint32_t s_k = s_ring + st * 2 * CHUNK + half * 32 * L;
                     const uint32_t s_v = s_ring + st * 2 * CHUNK + CHUNK + half * 2 * (L * NOVAKV_VBLOCK);
@@ -385,6 +460,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     for (int h = 0; h < HPAD / 2; ++h) unpack2(z[h], zf[2 * h], zf[2 * h + 1]);
                     bool rescale = false;
                     float alpha[HPAD];
+                    __half ph[HPAD];
 #pragma unroll
                     for (int h = 0; h < HPAD; ++h) {
                         if (lane >= nvalid) zf[h] = -CUDART_INF_F;
@@ -394,58 +470,41 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                         rescale |= (m_new != m_run[h]);
                         m_run[h] = m_new;
                         zf[h] = ex2(zf[h] - m_new);                 // p
+                        if (VM) {
+                            // the weight that multiplies the value and the one summed into the normaliser are
+                            // the same fp16-rounded number, so the result is an exact softmax of perturbed logits
+                            ph[h] = __float2half_rn(zf[h]);
+                            zf[h] = __half2float(ph[h]);
+                        }
                         l_run[h] = fmaf(l_run[h], alpha[h], zf[h]);
                     }
-                    if (rescale) {
-#pragma unroll
-                        for (int h = 0; h < HPAD; ++h) {
-                            const uint64_t a2 = pack2(alpha[h], alpha[h]);
-                            fmul2(acc[h][0], a2);
-                            fmul2(acc[h][1], a2);
-                        }
-                    }
-                    __syncwarp();      // previous tile's readers of the P area are done
-#pragma unroll
-                    for (int h = 0; h < HPAD; h += 2)
-                        sts_2x64(s_pw + lane * (HPAD * 8) + h * 8, pack2(zf[h], zf[h]), pack2(zf[h + 1], zf[h + 1]));
-                    __syncwarp();
 
-                    // ---- value side: lane <-> group, p * codeword in the transform domain ------
-                    if (D == 128) {
-                        const uint32_t l8 = lane * 8;
+                    if (!VM) {
+                        if (rescale) {
 #pragma unroll
-                        for (int blk = 0; blk < 2; ++blk) {
-                            const uint4 vb = lds_u128(s_v + blk * (L * NOVAKV_VBLOCK) + lane * 16);
-                            const uint32_t vw[4] = {vb.x, vb.y, vb.z, vb.w};
-#pragma unroll
-                            for (int t = 0; t < 16; ++t) {
-                                const uint32_t a = __byte_perm(vw[t >> 2], l8, 0x5504 | ((t & 3) << 4)) + s_vcb;
-                                const uint2 cw = lds_u64(a);
-                                const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&cw.x));
-                                const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&cw.y));
-                                const uint64_t v01 = pack2(f01.x, f01.y), v23 = pack2(f23.x, f23.y);
-                                const uint32_t pa = s_pw + (blk * 16 + t) * (HPAD * 8);
-#pragma unroll
-                                for (int h = 0; h < HPAD; h += 2) {
-                                    uint64_t p0, p1;
-                                    lds_2x64(pa + h * 8, p0, p1);
-                                    ffma2(acc[h][0], v01, p0);
-                                    ffma2(acc[h][1], v23, p0);
-                                    ffma2(acc[h + 1][0], v01, p1);
-                                    ffma2(acc[h + 1][1], v23, p1);
-                                }
+                            for (int h = 0; h < HPAD; ++h) {
+                                const uint64_t a2 = pack2(alpha[h], alpha[h]);
+                                fmul2(acc[h][0], a2);
+                                fmul2(acc[h][1], a2);
                             }
                         }
-                    } else {
-                        // d = 64: 16 groups; the two half warps split each 16-token block 8 / 8
-                        const int hf = lane >> 4, l = lane & 15;
-                        const uint32_t l8 = l * 8;
+                        __syncwarp();      // previous tile's readers of the P area are done
+#pragma unroll
+                        for (int h = 0; h < HPAD; h += 2)
+                            sts_2x64(s_pw + lane * (HPAD * 8) + h * 8, pack2(zf[h], zf[h]), pack2(zf[h + 1], zf[h + 1]));
+                        __syncwarp();
+
+                        // ---- value side on CUDA cores: lane <-> index row (group 8 (row % NGB) + row / NGB) ----
+                        constexpr int TPB = D == 128 ? 16 : 8;         // tokens of a 16-token block one lane handles
+                        const int hf = D == 128 ? 0 : (lane >> 4), lg = D == 128 ? lane : (lane & 15);
+                        const uint32_t l8 = lg * 8;
 #pragma unroll
                         for (int blk = 0; blk < 2; ++blk) {
-                            const uint4 vb = lds_u128(s_v + blk * (L * NOVAKV_VBLOCK) + l * 16);
-                            const uint32_t vw[2] = {hf ? vb.z : vb.x, hf ? vb.w : vb.y};
+                            const uint4 vb = lds_u128(s_v + blk * (L * NOVAKV_VBLOCK) + lg * 16);
+                            uint32_t vw[4] = {vb.x, vb.y, vb.z, vb.w};
+                            if (D == 64) { vw[0] = hf ? vb.z : vb.x; vw[1] = hf ? vb.w : vb.y; }
 #pragma unroll
-                            for (int t = 0; t < 8; ++t) {
+                            for (int t = 0; t < TPB; ++t) {
                                 const uint32_t a = __byte_perm(vw[t >> 2], l8, 0x5504 | ((t & 3) << 4)) + s_vcb;
                                 const uint2 cw = lds_u64(a);
                                 const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&cw.x));
@@ -460,6 +519,105 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                                     ffma2(acc[h][1], v23, p0);
                                     ffma2(acc[h + 1][0], v01, p1);
                                     ffma2(acc[h + 1][1], v23, p1);
+                                }
+                            }
+                        }
+                    } else {
+                        // ---- value side on tensor cores ---------------------------------------------
+                        // D[m][n] += sum_k A[m][k] B[k][n], m16 n8 k16, per 8-token sub-tile and group block gb:
+                        //   k = (token j of the sub-tile, sub-coefficient i in {0,1}),
+                        //   A[m][(j,i)] = codeword(token j, group 8gb + (m & 7))[2 (m >> 3) + i]      fp16
+                        //   B[(j,i)][(h,i')] = p_h(token j) * [i == i']                                fp16
+                        //   D[m][(h,i')] = partial of head h, group 8gb + (m & 7), coefficient 2 (m >> 3) + i'
+                        if (rescale) {
+#pragma unroll
+                            for (int hs = 0; hs < HSETS; ++hs) {
+                                const float a01 = fc & 1 ? alpha[hs * 4 + 1] : alpha[hs * 4 + 0];
+                                const float a23 = fc & 1 ? alpha[hs * 4 + 3] : alpha[hs * 4 + 2];
+                                const float al = fc & 2 ? a23 : a01;
+#pragma unroll
+                                for (int gb = 0; gb < NGB; ++gb)
+#pragma unroll
+                                    for (int i = 0; i < 4; ++i) macc[hs][gb][i] *= al;
+                            }
+                        }
+                        // weights -> shared memory as fp16, [head][k-slot pair = token & 3][token >> 3, (token >> 2) & 1]
+                        __syncwarp();      // previous tile's readers of the P area are done
+                        {
+                            const uint32_t wa = s_pw + (lane & 3) * 16 + ((lane >> 3) * 2 + ((lane >> 2) & 1)) * 2;
+#pragma unroll
+                            for (int h = 0; h < HPAD; ++h)
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + h * 64), "h"(__half_as_ushort(ph[h])) : "memory");
+                        }
+                        __syncwarp();
+                        // B-fragment sources: 8 weights of head (4 hs + fr/2) for the tokens with (token & 3) == fc
+                        uint4 pw[HSETS];
+#pragma unroll
+                        for (int hs = 0; hs < HSETS; ++hs) pw[hs] = lds_u128(s_pw + (hs * 4 + (fr >> 1)) * 64 + fc * 16);
+
+                        // slot of this lane's codeword in the value-codebook row for load x (see the image layout)
+                        constexpr int NX = NGB;                      // loads per (sub-tile, token slot): one per group block
+#pragma unroll
+                        for (int blk = 0; blk < 2; ++blk) {
+                            // index rows of this lane's groups for the 16 tokens of the block
+                            uint32_t vw[NX][4];
+                            uint32_t pos8[NX];
+#pragma unroll
+                            for (int x = 0; x < NX; ++x) {
+                                const int xb4 = (x + fc) & 3;                       // rotated so that a quad hits 4 different slots
+                                const int row = fr * NGB + (xb4 % NGB);               // row of group 8 (xb4 % NGB) + fr
+                                const uint4 vb = lds_u128(s_v + blk * (L * NOVAKV_VBLOCK) + row * 16);
+                                vw[x][0] = vb.x; vw[x][1] = vb.y; vw[x][2] = vb.z; vw[x][3] = vb.w;
+                                pos8[x] = (16 * (fr >> 2) + 4 * xb4 + (fr & 3)) * 8;
+                            }
+#pragma unroll
+                            for (int ts = 0; ts < 2; ++ts) {                       // 8-token sub-tiles of the block
+                                // gather: X[x][u] = codeword (token 8ts + 4u + fc, group of load x), 2 registers each
+                                uint32_t X[NX][2][2];
+#pragma unroll
+                                for (int x = 0; x < NX; ++x)
+#pragma unroll
+                                    for (int uu = 0; uu < 2; ++uu) {
+                                        const uint32_t a = __byte_perm(vw[x][2 * ts + uu], pos8[x], sel_c) + s_vcb;
+                                        const uint2 cw = lds_u64(a);
+                                        X[x][uu][0] = cw.x; X[x][uu][1] = cw.y;
+                                    }
+                                // un-rotate: Y[gb] = X[(gb - fc) mod NX]
+                                uint32_t Y[NX][2][2];
+                                if (NX == 4) {
+                                    uint32_t T[4][2][2];
+#pragma unroll
+                                    for (int gb = 0; gb < 4; ++gb)
+#pragma unroll
+                                        for (int uu = 0; uu < 2; ++uu)
+#pragma unroll
+                                            for (int i = 0; i < 2; ++i) T[gb][uu][i] = (fc & 1) ? X[(gb + 3) & 3][uu][i] : X[gb][uu][i];
+#pragma unroll
+                                    for (int gb = 0; gb < 4; ++gb)
+#pragma unroll
+                                        for (int uu = 0; uu < 2; ++uu)
+#pragma unroll
+                                            for (int i = 0; i < 2; ++i) Y[gb][uu][i] = (fc & 2) ? T[(gb + 2) & 3][uu][i] : T[gb][uu][i];
+                                } else {
+#pragma unroll
+                                    for (int gb = 0; gb < NX; ++gb)
+#pragma unroll
+                                        for (int uu = 0; uu < 2; ++uu)
+#pragma unroll
+                                            for (int i = 0; i < 2; ++i) Y[gb][uu][i] = (fc & 1) ? X[(gb + 1) & 1][uu][i] : X[gb][uu][i];
+                                }
+                                const int t = blk * 2 + ts;                         // sub-tile index within the 32-token tile
+#pragma unroll
+                                for (int hs = 0; hs < HSETS; ++hs) {
+                                    const uint32_t w = t == 0 ? pw[hs].x : (t == 1 ? pw[hs].y : (t == 2 ? pw[hs].z : pw[hs].w));
+                                    const uint32_t b0 = __byte_perm(w, 0u, sel_b0), b1 = __byte_perm(w, 0u, sel_b1);
+#pragma unroll
+                                    for (int gb = 0; gb < NGB; ++gb) {
+                                        asm volatile(
+                                            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                            : "+f"(macc[hs][gb][0]), "+f"(macc[hs][gb][1]), "+f"(macc[hs][gb][2]), "+f"(macc[hs][gb][3])
+                                            : "r"(Y[gb][0][0]), "r"(Y[gb][0][1]), "r"(Y[gb][1][0]), "r"(Y[gb][1][1]), "r"(b0), "r"(b1));
+                                    }
                                 }
                             }
                         }
@@ -478,20 +636,36 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         if (warp < NCW) {
 #pragma unroll
             for (int h = 0; h < HPAD; ++h) {
-                float a0, a1, a2, a3;
-                unpack2(acc[h][0], a0, a1);
-                unpack2(acc[h][1], a2, a3);
-                if (D == 64) {
-                    a0 += __shfl_xor_sync(0xffffffffu, a0, 16);
-                    a1 += __shfl_xor_sync(0xffffffffu, a1, 16);
-                    a2 += __shfl_xor_sync(0xffffffffu, a2, 16);
-                    a3 += __shfl_xor_sync(0xffffffffu, a3, 16);
-                }
                 const float lsum = warp_sum(l_run[h]);
-                if (lane < L)
-                    *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + h) * D + lane * 4) = make_float4(a0, a1, a2, a3);
                 if (lane == 0) { m_ml[(warp * HPAD + h) * 2] = m_run[h]; m_ml[(warp * HPAD + h) * 2 + 1] = lsum; }
-                m_run[h] = M_INIT; l_run[h] = 0.f; acc[h][0] = 0ull; acc[h][1] = 0ull;
+                if (!VM) {
+                    float a0, a1, a2, a3;
+                    unpack2(acc[h][0], a0, a1);
+                    unpack2(acc[h][1], a2, a3);
+                    if (D == 64) {
+                        a0 += __shfl_xor_sync(0xffffffffu, a0, 16);
+                        a1 += __shfl_xor_sync(0xffffffffu, a1, 16);
+                        a2 += __shfl_xor_sync(0xffffffffu, a2, 16);
+                        a3 += __shfl_xor_sync(0xffffffffu, a3, 16);
+                    }
+                    if (lane < L) {
+                        const int g = 8 * (lane % NGB) + lane / NGB;          // group of index row `lane`
+                        *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + h) * D + g * 4) = make_float4(a0, a1, a2, a3);
+                    }
+                    acc[h][0] = 0ull; acc[h][1] = 0ull;
+                }
+                m_run[h] = M_INIT; l_run[h] = 0.f;
+            }
+            if (VM) {
+#pragma unroll
+                for (int hs = 0; hs < HSETS; ++hs)
+#pragma unroll
+                    for (int gb = 0; gb < NGB; ++gb) {
+                        *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + hs * 4 + fc) * D + (8 * gb + fr) * 4) =
+                            make_float4(macc[hs][gb][0], macc[hs][gb][1], macc[hs][gb][2], macc[hs][gb][3]);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) macc[hs][gb][i] = 0.f;
+                    }
             }
         }
         __syncthreads();
@@ -602,13 +776,13 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     return w;
 }
 
-template <int D, int HG>
+template <int D, int HG, bool VM>
 novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
                               const uint8_t* k_pages, const uint8_t* v_pages, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens,
                               int batch, float sm_scale, void* out, int out_is_fp32, void* workspace,
                               cudaStream_t stream) {
-    using C = S1<D, HG>;
+    using C = S1<D, HG, VM>;
     const WsLayout w = ws_layout(ctx, batch);
     char* ws = (char*)workspace;
     float* qp = (float*)(ws + w.qp);
@@ -621,12 +795,12 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status);
     ctx->launches++;
 
-    auto kern = novakv_decode_stage1_kernel<D, HG>;
+    auto kern = novakv_decode_stage1_kernel<D, HG, VM>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
     const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
     {
         novakv_prof_scope ps(ctx, 0, stream);
-        kern<<<grid, S1_THREADS, C::SMEM, stream>>>(qp, ly.cb_k_lut, ly.cb_v_half, k_pages, v_pages, n_pages,
+        kern<<<grid, S1_THREADS, C::SMEM, stream>>>(qp, ly.cb_k_lut, VM ? ly.cb_v_mma : ly.cb_v_half, k_pages, v_pages, n_pages,
             page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc, ctx->dev_status);
         ps.end();
         ctx->launches++;
@@ -648,9 +822,15 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
     (void)workspace_bytes;
     const int d = ctx->cfg.head_dim, hg = ctx->hg;
 #define NOVAKV_DISPATCH(DD, HH)                                                                             \
-    if (d == DD && hg == HH)                                                                                \
-        return launch_decode_t<DD, HH>(ctx, ly, q, k_pages, v_pages, n_pages, page_table, max_pages_per_seq, \
-                                       seq_lens, batch, sm_scale, out, out_is_fp32, workspace, stream);
+    if (d == DD && hg == HH) {                                                                                   \
+        if (ctx->value_path == 0)                                                                                \
+            return launch_decode_t<DD, HH, false>(ctx, ly, q, k_pages, v_pages, n_pages, page_table,             \
+                                                  max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
+                                                  workspace, stream);                                            \
+        return launch_decode_t<DD, HH, true>(ctx, ly, q, k_pages, v_pages, n_pages, page_table,                  \
+                                             max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,     \
+                                             workspace, stream);                                                 \
+    }
     NOVAKV_DISPATCH(128, 1)
     NOVAKV_DISPATCH(128, 2)
     NOVAKV_DISPATCH(128, 4)

@@ -163,7 +163,8 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
             if (side == 0) {
                 k_pages[base + (size_t)slot * L + l] = idx_s[i];
             } else {
-                v_pages[base + ((size_t)(slot / NOVAKV_VBLOCK) * L + l) * NOVAKV_VBLOCK + (slot % NOVAKV_VBLOCK)] = idx_s[i];
+                const int row = (l & 7) * (L / 8) + (l >> 3);       // row of group l inside a 16-token block
+                v_pages[base + ((size_t)(slot / NOVAKV_VBLOCK) * L + row) * NOVAKV_VBLOCK + (slot % NOVAKV_VBLOCK)] = idx_s[i];
             }
         }
     }

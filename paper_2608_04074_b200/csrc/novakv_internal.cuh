@@ -29,7 +29,8 @@ struct novakv_layer {
     float* rv_t = nullptr;        // [Hkv][d][d]  transposed R_V: rv_t[c][r] = R_V[r][c]
     float* v_mean = nullptr;      // [Hkv][d]
     float* cb_k_lut = nullptr;    // [Hkv][plane][256][16][4]  the order the score table is built in
-    __half* cb_v_half = nullptr;  // [Hkv][256][32][4]         row of 256 bytes per code (padded for L=16)
+    __half* cb_v_half = nullptr;  // [Hkv][256][32][4]         row of 256 bytes per code, slot = group (CUDA-core value side)
+    __half* cb_v_mma = nullptr;   // [Hkv][256][32][4]         same codewords, slots permuted for the tensor-core value side
 };
 
 struct novakv_event_pair {
@@ -46,6 +47,7 @@ struct novakv_ctx {
     std::vector<novakv_event_pair> prof_free;
     long launches = 0;
     int scan_ctas = 0;            // 0 = one per SM
+    int value_path = 1;           // 1 = tensor cores, 0 = CUDA cores
 };
 
 // RAII-free helper: brackets a launch with events when profiling is on.
@@ -127,6 +129,10 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Asynchronous prefetch of a global range into L2 (no destination, no completion to wait for).
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

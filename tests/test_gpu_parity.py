@@ -112,16 +112,19 @@ def test_decode_matches_oracle(name, lens, request):
     cache = _cache(case, lens)
     encs = _fill_with_oracle(case, cache, lens, 300)
     _, _, q = case.draw(301, 1, len(lens))
-    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
-    assert case.ctx.novakv_last_device_status() == 0
-    worst = 0.0
-    for b, n in enumerate(lens):
-        ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
-        if n == 0:
-            assert not out[b].any()
-            continue
-        worst = max(worst, check_output(out[b], ref))
-    print(f"[{name} {lens.tolist()}] max|delta|/||o||inf = {worst:.3e}")
+    refs = [case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"]) for b in range(len(lens))]
+    for path, label in ((1, "tensor-core value side"), (0, "CUDA-core value side")):
+        case.ctx.novakv_debug_set_value_path(path)
+        out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+        assert case.ctx.novakv_last_device_status() == 0
+        worst = 0.0
+        for b, n in enumerate(lens):
+            if n == 0:
+                assert not out[b].any()
+                continue
+            worst = max(worst, check_output(out[b], refs[b]))
+        print(f"[{name} {lens.tolist()} {label}] max|delta|/||o||inf = {worst:.3e}")
+    case.ctx.novakv_debug_set_value_path(1)
 
 
 # --------------------------------------------------------------------------- T4: split invariance, determinism
@@ -144,8 +147,10 @@ def test_split_count_invariance_and_determinism(qwen):
         for n_ctas, o in outs.items():
             check_output(o[b], ref)
         scale = np.abs(ref).max()
+        # different splits see different running maxima, hence round the fp16 softmax weights of the
+        # tensor-core value side differently (2^-12 relative per weight): invariance holds to ~1e-4
         for n_ctas in (1, 2, 7):
-            assert np.abs(outs[n_ctas][b] - outs[0][b]).max() <= 2e-5 * scale
+            assert np.abs(outs[n_ctas][b] - outs[0][b]).max() <= 2e-4 * scale
 
 
 # --------------------------------------------------------------------------- T6: append then decode, end to end
@@ -287,6 +292,9 @@ def test_bench_configuration_sampled():
                      _dev(np.full(S, b, np.int32)), _dev(np.arange(S, dtype=np.int32)))
     _, _, q = case.draw(950, 1, wl.batch)
     out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    case.ctx.novakv_debug_set_value_path(0)
+    out_cc = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    case.ctx.novakv_debug_set_value_path(1)
     assert case.ctx.novakv_last_device_status() == 0
     assert np.array_equal(cache.seq_lens.cpu().numpy(), wl.seq_lens)
     gen = synth.rng(77)
@@ -297,5 +305,8 @@ def test_bench_configuration_sampled():
         enc = case.oracle.encode(k[pick].astype(np.float64), v[pick].astype(np.float64))
         dk, _ = check_indices(gk[pick], enc, "k")
         dv, _ = check_indices(gv[pick], enc, "v")
-        ratio = check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
-        print(f"[bench cfg seq {b}] sampled index mismatches K {dk} V {dv}; max|delta|/||o||inf {ratio:.3e}")
+        ref = case.oracle.decode(q[b].astype(np.float64), gk, gv)
+        ratio = check_output(out[b], ref)
+        ratio_cc = check_output(out_cc[b], ref)
+        print(f"[bench cfg seq {b}] sampled index mismatches K {dk} V {dv}; max|delta|/||o||inf "
+              f"{ratio:.3e} (tensor-core value side) {ratio_cc:.3e} (CUDA-core value side)")

@@ -59,12 +59,13 @@ def test_cache_layout_round_trip_and_positions():
     for b, n in enumerate(lens):
         k, v = cache_format.read_tokens(kp, vp, table[b], hkv, d, 0, int(n))
         assert np.array_equal(k, ref[b][0]) and np.array_equal(v, ref[b][1])
-    # documented byte positions: key token-major, value 16-token blocks group-major
+    # documented byte positions: key token-major; value 16-token blocks, one row per group, rows permuted
     b, pos, h, l = 0, 77, 1, 9
     page = table[b][pos // 64]
     t = pos % 64
     assert kp[page, h, t * L + l] == ref[b][0][pos, h, l]
-    assert vp[page, h, ((t // 16) * L + l) * 16 + t % 16] == ref[b][1][pos, h, l]
+    row = (l % 8) * (L // 8) + l // 8
+    assert vp[page, h, ((t // 16) * L + row) * 16 + t % 16] == ref[b][1][pos, h, l]
 
 
 def test_workloads_have_the_stated_shapes():
