@@ -8,10 +8,14 @@
  *
  * Cache format (Sec. 2.2 "Quantization", Sec. 5 "Bit rate"): per token and KV head, L uint8
  * codeword indices for the key and L for the value: 8/g = 2 bits per cached element, no
- * per-token metadata.  Pages hold 64 tokens.  Two caller-owned device pools of equal geometry:
- *     key pool    uint8 [n_pages][Hkv][64][L]        token-major
- *     value pool  uint8 [n_pages][Hkv][4][L][16]     four 16-token blocks; in a block one 16-byte row per
- *                                                    group, group g in row (g % 8) * (L / 8) + g / 8
+ * per-token metadata.  Pages hold 64 tokens.  Two caller-owned device pools of equal geometry,
+ * uint8 [n_pages][Hkv][64*L] each: one contiguous chunk of 64*L bytes per (page, KV head) for keys
+ * and one for values.  Inside a chunk (t = token slot in the page, l = group):
+ *     keys    [tile = t/32][plane][t%32][16 bytes]: a token's L bytes are 8 "slots" of L/8 consecutive
+ *             groups, stored rotated: position j holds slot (j + t%8 + (t/8)%4) % 8; plane = byte / 16.
+ *     values  [block = t/16][fr = l%8][fc = t%4][x][b = (t%16)/4],  x = (l/8 - fc) mod (L/8).
+ * Both orders make every lane of a decode warp load exactly the bytes it consumes with coalesced
+ * 128-bit loads, and keep its shared-memory table gathers free of bank conflicts.
  * page_table[seq][i] (int32, row length max_pages_per_seq) names the page of tokens 64i..64i+63.
  *
  * Ownership: the context owns device copies of the calibration tables and one device status

@@ -4,12 +4,19 @@ One uint8 codeword index per group of g = 4 transform coefficients, per token, p
 for keys and for values (Sec. 2.2 "Quantization"; Sec. 5 "Bit rate"): L = d/4 bytes per
 side, i.e. exactly 8/g = 2 bits per cached element.
 
-Physical layout of a page (64 tokens), identical for every KV head:
+Physical layout: a page holds 64 tokens; per (page, KV head) one contiguous chunk of 64*L bytes
+in the key pool and one in the value pool (``uint8 [n_pages][Hkv][64*L]`` each).  Inside a chunk
+the bytes are ordered so that each lane of a decode warp loads, with one or two coalesced 128-bit
+loads, exactly the bytes it consumes:
 
-* key pool    ``uint8 [n_pages][Hkv][64][L]``           token-major;
-* value pool  ``uint8 [n_pages][Hkv][4][L][16]``        four 16-token blocks; inside a block one
-  16-byte row per group (16 consecutive tokens), group ``g`` in row ``(g % 8) * (L // 8) + g // 8``
-  (the decode kernel's tensor-core lanes then read their rows from distinct shared-memory banks).
+* keys:   ``[tile = t // 32][plane][t % 32][16 bytes]``.  A token's L bytes are split into 8
+  "slots" of L/8 consecutive groups; they are stored rotated, position j holding slot
+  ``(j + t % 8 + (t // 8) % 4) % 8`` (the lanes of a quarter warp then read 8 different banks of
+  the score table at every step); plane = byte position // 16.
+* values: ``[block = t // 16][fr = l % 8][fc = t % 4][x][b = (t % 16) // 4]`` with
+  ``x = (l // 8 - fc) mod (L // 8)``: the 16 (or 8) bytes of MMA lane (fr, fc) are contiguous.
+
+(t = token slot in the page, l = group.)
 
 ``page_table[seq][i]`` names the physical page that holds tokens ``64 i .. 64 i + 63``.
 The functions below only permute bytes; they hold no arithmetic of the method.
@@ -28,10 +35,22 @@ def n_groups(head_dim: int) -> int:
     return head_dim // GROUP_SIZE
 
 
-def value_row_of_group(n_groups_: int) -> np.ndarray:
-    """Row of each group inside a 16-token block of the value pool."""
-    g = np.arange(n_groups_)
-    return (g % 8) * (n_groups_ // 8) + g // 8
+def key_offset(t, l, n_groups_: int):
+    """Byte offset of (token slot t, group l) inside a key chunk (numpy arrays broadcast)."""
+    gps, kpl = n_groups_ // 8, n_groups_ // 16
+    sigma, m = l // gps, l % gps
+    rot = ((t & 7) + ((t >> 3) & 3)) & 7
+    bytepos = ((sigma - rot) & 7) * gps + m
+    return (((t >> 5) * kpl + (bytepos >> 4)) * 32 + (t & 31)) * 16 + (bytepos & 15)
+
+
+def value_offset(t, l, n_groups_: int):
+    """Byte offset of (token slot t, group l) inside a value chunk (numpy arrays broadcast)."""
+    ngb = n_groups_ // 8
+    tb = t & 15
+    fc, b, fr = tb & 3, tb >> 2, l & 7
+    x = ((l >> 3) - fc) & (ngb - 1)
+    return (t >> 4) * (n_groups_ * 16) + (fr * 4 + fc) * (ngb * 4) + x * 4 + b
 
 
 def index_bytes_per_token_per_kv_head(head_dim: int) -> int:
@@ -66,30 +85,31 @@ def alloc_pools(n_pages: int, n_kv_heads: int, head_dim: int) -> tuple[np.ndarra
 
 def write_tokens(k_pool: np.ndarray, v_pool: np.ndarray, page_table_row: np.ndarray, pos0: int,
                  kidx: np.ndarray, vidx: np.ndarray) -> None:
-    """Store logical indices [n][Hkv][L] of one sequence at positions pos0.. into the pools."""
+    """Store logical indices [n][Hkv][L] of one sequence at positions pos0.. into the pools
+    (pools shaped [n_pages][Hkv][64*L])."""
     n, hkv, l = kidx.shape
-    kp = k_pool.reshape(k_pool.shape[0], hkv, PAGE_TOKENS, l)
-    vp = v_pool.reshape(v_pool.shape[0], hkv, PAGE_TOKENS // V_BLOCK, l, V_BLOCK)
     pos = pos0 + np.arange(n)
-    page = page_table_row[pos // PAGE_TOKENS]
-    t = pos % PAGE_TOKENS
+    page = page_table_row[pos // PAGE_TOKENS][:, None]
+    t = (pos % PAGE_TOKENS)[:, None]
+    g = np.arange(l)[None, :]
+    ko, vo = key_offset(t, g, l), value_offset(t, g, l)
     for h in range(hkv):
-        kp[page, h, t, :] = kidx[:, h, :]
-        vp[page[:, None], h, (t // V_BLOCK)[:, None], value_row_of_group(l)[None, :], (t % V_BLOCK)[:, None]] = vidx[:, h, :]
+        k_pool[page, h, ko] = kidx[:, h, :]
+        v_pool[page, h, vo] = vidx[:, h, :]
 
 
 def read_tokens(k_pool: np.ndarray, v_pool: np.ndarray, page_table_row: np.ndarray, n_kv_heads: int,
                 head_dim: int, pos0: int, n: int) -> tuple[np.ndarray, np.ndarray]:
     """Logical indices [n][Hkv][L] of positions pos0 .. pos0+n-1 of one sequence."""
     l = n_groups(head_dim)
-    kp = k_pool.reshape(k_pool.shape[0], n_kv_heads, PAGE_TOKENS, l)
-    vp = v_pool.reshape(v_pool.shape[0], n_kv_heads, PAGE_TOKENS // V_BLOCK, l, V_BLOCK)
     pos = pos0 + np.arange(n)
-    page = page_table_row[pos // PAGE_TOKENS]
-    t = pos % PAGE_TOKENS
+    page = page_table_row[pos // PAGE_TOKENS][:, None]
+    t = (pos % PAGE_TOKENS)[:, None]
+    g = np.arange(l)[None, :]
+    ko, vo = key_offset(t, g, l), value_offset(t, g, l)
     kidx = np.empty((n, n_kv_heads, l), np.uint8)
     vidx = np.empty((n, n_kv_heads, l), np.uint8)
     for h in range(n_kv_heads):
-        kidx[:, h, :] = kp[page, h, t, :]
-        vidx[:, h, :] = vp[page[:, None], h, (t // V_BLOCK)[:, None], value_row_of_group(l)[None, :], (t % V_BLOCK)[:, None]]
+        kidx[:, h, :] = k_pool[page, h, ko]
+        vidx[:, h, :] = v_pool[page, h, vo]
     return kidx, vidx

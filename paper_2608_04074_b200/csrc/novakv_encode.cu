@@ -161,10 +161,9 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
             const int slot = slot_s[t];
             const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
             if (side == 0) {
-                k_pages[base + (size_t)slot * L + l] = idx_s[i];
+                k_pages[base + novakv_k_offset<L>(slot, l)] = idx_s[i];
             } else {
-                const int row = (l & 7) * (L / 8) + (l >> 3);       // row of group l inside a 16-token block
-                v_pages[base + ((size_t)(slot / NOVAKV_VBLOCK) * L + row) * NOVAKV_VBLOCK + (slot % NOVAKV_VBLOCK)] = idx_s[i];
+                v_pages[base + novakv_v_offset<L>(slot, l)] = idx_s[i];
             }
         }
     }

@@ -87,6 +87,27 @@ novakv_status novakv_launch_bf16_decode(novakv_ctx* ctx, const __nv_bfloat16* q,
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 
+// Byte offsets inside the 64*L-byte chunk of one (page, KV head); t = token slot in the page
+// (0..63), l = group.  These define the cache format (see the public header).
+//   keys:   [tile = t/32][plane][token t%32][16 bytes]; a token's L bytes are its 8 "slots" of L/8
+//           groups each, stored rotated: position j holds slot (j + t%8 + (t/8)%4) % 8.
+//   values: [block = t/16][fr = l%8][fc = t%4][x][b = (t%16)/4], x = (l/8 - fc) mod (L/8).
+template <int L>
+__host__ __device__ __forceinline__ int novakv_k_offset(int t, int l) {
+    constexpr int GPS = L / 8, KPL = L / 16;
+    const int sigma = l / GPS, m = l % GPS;
+    const int rot = ((t & 7) + ((t >> 3) & 3)) & 7;
+    const int bytepos = ((sigma - rot) & 7) * GPS + m;
+    return (((t >> 5) * KPL + (bytepos >> 4)) * 32 + (t & 31)) * 16 + (bytepos & 15);
+}
+template <int L>
+__host__ __device__ __forceinline__ int novakv_v_offset(int t, int l) {
+    constexpr int NGB = L / 8;
+    const int tb = t & 15, fc = tb & 3, b = tb >> 2, fr = l & 7;
+    const int x = ((l >> 3) - fc) & (NGB - 1);
+    return (t >> 4) * (L * 16) + (fr * 4 + fc) * (NGB * 4) + x * 4 + b;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

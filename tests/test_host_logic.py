@@ -59,13 +59,24 @@ def test_cache_layout_round_trip_and_positions():
     for b, n in enumerate(lens):
         k, v = cache_format.read_tokens(kp, vp, table[b], hkv, d, 0, int(n))
         assert np.array_equal(k, ref[b][0]) and np.array_equal(v, ref[b][1])
-    # documented byte positions: key token-major; value 16-token blocks, one row per group, rows permuted
+    # documented byte positions of the chunk layouts (d = 64: L = 16, 2 groups per slot, 2 group blocks)
     b, pos, h, l = 0, 77, 1, 9
     page = table[b][pos // 64]
-    t = pos % 64
-    assert kp[page, h, t * L + l] == ref[b][0][pos, h, l]
-    row = (l % 8) * (L // 8) + l // 8
-    assert vp[page, h, ((t // 16) * L + row) * 16 + t % 16] == ref[b][1][pos, h, l]
+    t = pos % 64                                       # 13
+    rot = (t % 8 + (t // 8) % 4) % 8                   # slot rotation of this token
+    bytepos = ((l // 2 - rot) % 8) * 2 + l % 2
+    k_off = (((t // 32) * 1 + bytepos // 16) * 32 + t % 32) * 16 + bytepos % 16
+    assert kp[page, h, k_off] == ref[b][0][pos, h, l]
+    fc, bb, fr = (t % 16) % 4, (t % 16) // 4, l % 8
+    x = (l // 8 - fc) % 2
+    v_off = (t // 16) * (L * 16) + (fr * 4 + fc) * 8 + x * 4 + bb
+    assert vp[page, h, v_off] == ref[b][1][pos, h, l]
+    # every byte of a chunk is hit exactly once
+    tt, ll = np.meshgrid(np.arange(64), np.arange(L), indexing="ij")
+    for LL in (16, 32):
+        tt, ll = np.meshgrid(np.arange(64), np.arange(LL), indexing="ij")
+        assert sorted(cache_format.key_offset(tt, ll, LL).ravel().tolist()) == list(range(64 * LL))
+        assert sorted(cache_format.value_offset(tt, ll, LL).ravel().tolist()) == list(range(64 * LL))
 
 
 def test_workloads_have_the_stated_shapes():
