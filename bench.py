@@ -66,7 +66,7 @@ class ClockSampler:
 
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, cuda_index, period_s=0.0005):
+    def __init__(self, cuda_index, period_s=0.0):
         import threading
         self.samples, self.mask, self.max_mhz, self.err = [], 0, None, None
         self._stop = threading.Event()
@@ -102,7 +102,8 @@ class ClockSampler:
                 except Exception as e:   # noqa: BLE001
                     self.err = str(e)
                     return
-                self._stop.wait(period_s)
+                if period_s > 0:
+                    self._stop.wait(period_s)
 
         self._thread = threading.Thread(target=loop, daemon=True)
         self._thread.start()
@@ -167,6 +168,27 @@ def fill_cache_gpu(case_ctx, cache, laws, seq_lens, seed, share_content=False):
         cache.k_pages[dst] = cache.k_pages[src[:npg]]
         cache.v_pages[dst] = cache.v_pages[src[:npg]]
     cache.seq_lens.copy_(torch.from_numpy(np.asarray(seq_lens, np.int32)).cuda())
+
+
+def time_bf16_comparator(ctx, wl, dev, steps, flush):
+    """The in-house uncompressed bf16 decode kernel on the same shape (random bf16 cache content)."""
+    import torch
+    from paper_2608_04074_b200 import synth
+    s = wl.shape
+    table, n_pages = synth.shuffled_page_table(31, np.maximum(wl.seq_lens, 1), 64)
+    kp = torch.empty((n_pages, s.n_kv_heads, 64, s.head_dim), dtype=torch.bfloat16, device=dev).normal_()
+    vp = torch.empty((n_pages, s.n_kv_heads, 64, s.head_dim), dtype=torch.bfloat16, device=dev).normal_()
+    pt = torch.from_numpy(np.where(table < 0, 0, table).astype(np.int32)).to(dev)
+    sl = torch.from_numpy(wl.seq_lens.astype(np.int32)).to(dev)
+    q = torch.empty((wl.batch, s.n_q_heads, s.head_dim), dtype=torch.bfloat16, device=dev).normal_()
+    out = torch.empty((wl.batch, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
+    ws = torch.empty(ctx.novakv_bf16_workspace_bytes(wl.batch, table.shape[1]), dtype=torch.uint8, device=dev)
+    tt = time_steps(lambda: ctx.novakv_bf16_decode_attention(q, kp, vp, pt, sl, out, ws), steps, 3, flush)
+    ms = statistics.median(tt)
+    kv_bytes = int(np.sum(wl.seq_lens.astype(np.int64))) * s.n_kv_heads * 2 * s.head_dim * 2
+    del kp, vp
+    torch.cuda.empty_cache()
+    return {"ms": round(ms, 4), "kv_bytes": kv_bytes, "gbps": round(kv_bytes / (ms * 1e-3) / 1e9, 1)}
 
 
 def time_steps(fn, steps, warmup, flush, after_warmup=None):
@@ -249,7 +271,6 @@ def run_ours(args):
     enc_ms, enc_n = ctx.novakv_profile_read(1)
     ctx.novakv_profile_enable(False)
     launches = ctx.novakv_launch_count() - mark["launches0"]
-    clocks = sampler.stop() if sampler else None
     status = ctx.novakv_last_device_status()
     ms_step = sum(times) / len(times)
     if world > 1:
@@ -262,6 +283,13 @@ def run_ours(args):
     dec_ms = statistics.median(dec_times)
     nowarm = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, lambda: None)
     dec_ms_warm_l2 = statistics.median(nowarm)
+
+    # ---- the CUDA-core value-side variant and the uncompressed bf16 comparator, same shape ------
+    ctx.novakv_debug_set_value_path(0)
+    cc_times = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, flush)
+    ctx.novakv_debug_set_value_path(1)
+    cc_ms = statistics.median(cc_times)
+    bf16 = time_bf16_comparator(ctx, wl_after, dev, max(5, args.steps // 2), flush)
 
     # ---- end to end from pinned host buffers through the C ABI --------------------------------
     pin = lambda t: t.cpu().pin_memory()
@@ -279,6 +307,9 @@ def run_ours(args):
         t = torch.tensor([e2e_ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
+    # the sampler ran from before the warm-up through every timed loop above (NVML queries take
+    # milliseconds, so the few-ms headline loop alone would give one sample)
+    clocks = sampler.stop() if sampler else None
     h2d = int(k1h.numel() * 2 + v1h.numel() * 2 + qh.numel() * 2 + seqh.numel() * 4 + posh.numel() * 4)
     d2h = int(out_h.numel() * 4)
 
@@ -312,6 +343,9 @@ def run_ours(args):
             "decode_only": {"ms": round(dec_ms, 5), "gbps": round(alg_bytes / (dec_ms * 1e-3) / 1e9, 1),
                             "pct_of_8TBps": round(100 * alg_bytes / (dec_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
                             "ms_l2_not_flushed": round(dec_ms_warm_l2, 5)},
+            "decode_only_cuda_core_value_side": {"ms": round(cc_ms, 5),
+                                                 "gbps": round(alg_bytes / (cc_ms * 1e-3) / 1e9, 1)},
+            "bf16_comparator": dict(bf16, speedup_of_2bit_decode=round(bf16["ms"] / dec_ms, 2)),
             "encode_append": {"tokens": B, "avg_kernel_ms": round(enc_ms / max(enc_n, 1), 5)},
             "device_status": status,
         }
@@ -333,13 +367,17 @@ def run_ours(args):
             ctx.novakv_profile_enable(False)
             ab, ib = algorithmic_decode_bytes(wl2)
             ms = statistics.median(tt)
+            del c2
+            torch.cuda.empty_cache()
+            bf = time_bf16_comparator(ctx, wl2, dev, 5, lambda: None)
             sweep.append({"workload": f"qwen3_8b_shape B={b2} S={s2} decode only, inputs larger than L2",
                           "ms": round(ms, 4), "gbps": round(ab / (ms * 1e-3) / 1e9, 1),
                           "pct_of_8TBps": round(100 * ab / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
                           "scan_kernel_ms": round(k_ms / max(k_n, 1), 4),
                           "scan_kernel_frac_of_measured_peak": round(ab / (k_ms / max(k_n, 1) * 1e-3) / 1e9 / measured_peak()[0], 4),
-                          "algorithmic_bytes": ab})
-            del c2, q2, o2
+                          "algorithmic_bytes": ab,
+                          "bf16_comparator": dict(bf, speedup_of_2bit_decode=round(bf["ms"] / ms, 2))})
+            del q2, o2
             torch.cuda.empty_cache()
         # prefill encode: 32768 tokens x 8 KV heads x d=128, K and V
         T = 32768
@@ -439,6 +477,7 @@ def run_reference(args):
 
 
 def main():
+    sys.setswitchinterval(1e-4)          # let the clock-sampling thread run between short GPU calls
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)

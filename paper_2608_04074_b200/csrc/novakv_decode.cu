@@ -29,11 +29,7 @@
 namespace {
 
 #ifndef NOVAKV_NCW
-#define NOVAKV_NCW 8
-#endif
-// L2 line prefetch distance, in 32-token tiles of the same warp (0 = off)
-#ifndef NOVAKV_L2_PREFETCH_TILES
-#define NOVAKV_L2_PREFETCH_TILES 0
+#define NOVAKV_NCW 12
 #endif
 constexpr int NCW = NOVAKV_NCW;               // warps of the scan kernel
 constexpr int S1_THREADS = NCW * 32;
@@ -80,14 +76,16 @@ __device__ __forceinline__ int clamp_len(int len, int max_pages) {
 // ------------------------------------------------------------------------------------------------
 // prepare: query transform + page prefix
 // ------------------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(D)
+// One block per (sequence, KV head): the Hg queries of the head share every load of rk_inv_t.
+// 512 threads = D columns x (512/D) row parts; each thread's loads are independent and all in flight.
+template <int D, int HG>
+__global__ void __launch_bounds__(512)
 novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict__ rk_inv_t,
                       const int32_t* __restrict__ seq_lens, int batch, int n_q_heads, int n_kv_heads,
                       int max_pages_per_seq, float scale_log2, float* __restrict__ qp,
                       int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status) {
     const int blk = blockIdx.x;
-    if (blk == batch * n_q_heads) {
+    if (blk == batch * n_kv_heads) {
         // exclusive prefix over sequences of (pages * Hkv); small, done by one warp
         if (threadIdx.x < 32) {
             int carry = 0;
@@ -113,16 +111,35 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         }
         return;
     }
-    __shared__ float q_s[D];
-    const int b = blk / n_q_heads, h = blk - b * n_q_heads;
-    const int kvh = h / (n_q_heads / n_kv_heads);
-    q_s[threadIdx.x] = __bfloat162float(q[((size_t)b * n_q_heads + h) * D + threadIdx.x]);
+    constexpr int PARTS = 512 / D, ROWS = D / PARTS;
+    __shared__ float q_s[HG][D];
+    __shared__ float red_s[PARTS][HG][D];
+    const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
+    for (int i = threadIdx.x; i < HG * D; i += 512)
+        q_s[i / D][i % D] = __bfloat162float(q[((size_t)b * n_q_heads + kvh * HG) * D + i]);
     __syncthreads();
-    const float* R = rk_inv_t + (size_t)kvh * D * D;
-    float acc = 0.f;
-#pragma unroll 8
-    for (int r = 0; r < D; ++r) acc = fmaf(q_s[r], R[(size_t)r * D + threadIdx.x], acc);
-    qp[((size_t)b * n_q_heads + h) * D + threadIdx.x] = acc * scale_log2;
+    const int c = threadIdx.x % D, part = threadIdx.x / D;
+    const float* R = rk_inv_t + (size_t)kvh * D * D + (size_t)part * ROWS * D + c;
+    float rv[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) rv[r] = R[(size_t)r * D];
+    float acc[HG];
+#pragma unroll
+    for (int h = 0; h < HG; ++h) acc[h] = 0.f;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+        for (int h = 0; h < HG; ++h) acc[h] = fmaf(q_s[h][part * ROWS + r], rv[r], acc[h]);
+#pragma unroll
+    for (int h = 0; h < HG; ++h) red_s[part][h][c] = acc[h];
+    __syncthreads();
+    for (int i = threadIdx.x; i < HG * D; i += 512) {
+        const int h = i / D, cc = i % D;
+        float v = 0.f;
+#pragma unroll
+        for (int p = 0; p < PARTS; ++p) v += red_s[p][h][cc];
+        qp[((size_t)b * n_q_heads + kvh * HG + h) * D + cc] = v * scale_log2;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -392,16 +409,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             const TileRegs<L> cur = nxt;
             if (((it + 1) & 31) == 0) { ids_cur = ids_next; ids_next = load_ids(((it + 1) >> 5) + 1); }
             if (it + 1 < n_it) load_tile(it + 1, nxt);
-            if (NOVAKV_L2_PREFETCH_TILES > 0 && it + NOVAKV_L2_PREFETCH_TILES < n_it) {
-                // one instruction: 2 * TILE_BYTES / 128 lanes each prefetch a line of a later tile into L2
-                const int pit = it + NOVAKV_L2_PREFETCH_TILES;
-                const int pbatch = pit >> 5, cbatch = (it + 1) >> 5;
-                const int page = __shfl_sync(0xffffffffu, pbatch == cbatch ? ids_cur : ids_next, pit & 31);
-                constexpr int LINES = TILE_BYTES / 128;
-                const size_t off = ((size_t)page * n_kv_heads + sg.kvh) * PAGE_BYTES + ((warp + NCW * pit) & 1) * TILE_BYTES;
-                const uint8_t* src = (lane < LINES ? k_pages : v_pages) + off + (size_t)(lane % LINES) * 128;
-                if (lane < 2 * LINES && pbatch <= cbatch + 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
-            }
             const int hp = warp + NCW * it;
             const int tok0 = (sg.pg0 + (hp >> 1)) * NOVAKV_PAGE_TOKENS + (hp & 1) * 32;
             const int nvalid = min(32, sg.len - tok0);
@@ -688,15 +695,36 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         o_s[i] = val;
     }
     __syncthreads();
+    // o_h = o'_h rv^T + v_mean: threads = D outputs x PARTS column parts, all HG heads share each load
+    constexpr int NT = HG * D > 512 ? 512 : HG * D;
+    constexpr int PARTS = NT / D, COLS = D / PARTS;
+    __shared__ float red_s[PARTS][HG][D];
+    {
+        const int r = threadIdx.x % D, part = threadIdx.x / D;
+        float acc[HG];
+#pragma unroll
+        for (int h = 0; h < HG; ++h) acc[h] = 0.f;
+        if (pages_b > 0) {
+            const float* R = rv_t + (size_t)kvh * D * D + (size_t)part * COLS * D + r;     // rv_t[c][r] = R_V[r][c]
+            float rv[COLS];
+#pragma unroll
+            for (int c = 0; c < COLS; ++c) rv[c] = R[(size_t)c * D];
+#pragma unroll
+            for (int c = 0; c < COLS; ++c)
+#pragma unroll
+                for (int h = 0; h < HG; ++h) acc[h] = fmaf(o_s[h * D + part * COLS + c], rv[c], acc[h]);
+        }
+#pragma unroll
+        for (int h = 0; h < HG; ++h) red_s[part][h][r] = acc[h];
+    }
+    __syncthreads();
     for (int i = threadIdx.x; i < HG * D; i += blockDim.x) {
         const int h = i / D, r = i - h * D;
         float o = 0.f;
         if (pages_b > 0) {
-            const float* R = rv_t + (size_t)kvh * D * D;     // rv_t[c][r] = R_V[r][c]
-            float acc = 0.f;
-#pragma unroll 8
-            for (int c = 0; c < D; ++c) acc = fmaf(o_s[h * D + c], R[(size_t)c * D + r], acc);
-            o = acc + v_mean[(size_t)kvh * D + r];
+#pragma unroll
+            for (int p = 0; p < PARTS; ++p) o += red_s[p][h][r];
+            o += v_mean[(size_t)kvh * D + r];
         }
         const size_t oi = ((size_t)b * n_q_heads + kvh * HG + h) * D + r;
         if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
@@ -736,7 +764,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     float* part_acc = (float*)(ws + w.acc);
     const int hq = ctx->cfg.n_q_heads, hkv = ctx->cfg.n_kv_heads;
 
-    novakv_prepare_kernel<D><<<batch * hq + 1, D, 0, stream>>>(q, ly.rk_inv_t, seq_lens, batch, hq, hkv,
+    novakv_prepare_kernel<D, HG><<<batch * hkv + 1, 512, 0, stream>>>(q, ly.rk_inv_t, seq_lens, batch, hq, hkv,
         max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status);
     ctx->launches++;
 

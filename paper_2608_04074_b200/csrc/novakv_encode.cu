@@ -10,6 +10,9 @@ namespace {
 constexpr int ENC_THREADS = 256;
 constexpr int ENC_TILE = 64;   // tokens per tile (search granularity)
 constexpr int ENC_XT = 32;     // tokens per transform pass (bounds the binary64 staging buffer)
+#ifndef NOVAKV_SMALL_APPEND_TOKENS
+#define NOVAKV_SMALL_APPEND_TOKENS 256   // batches up to this size take the per-group append kernel
+#endif
 
 template <int D>
 struct EncSmem {
@@ -169,6 +172,90 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     }
 }
 
+// Append-sized batches (a decode step appends one token per sequence): the tiled kernel above would
+// pad every (head, side) to a 64-token tile and fill a 128 KB codebook per CTA.  Here one warp owns one
+// group of one (head, side): lanes are tokens, the warp stages only its 4 columns of the transform
+// (4 KB of binary64) and its group's codebook (4 KB), so the work spreads over L/4 * Hkv * 2 CTAs.
+// Arithmetic is identical to the tiled kernel (binary64 accumulation in index order, dist4 search).
+template <int D>
+__global__ void __launch_bounds__(128)
+novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
+                           const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
+                           const double* __restrict__ rk_d, const double* __restrict__ rv_d,
+                           const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
+                           const float* __restrict__ cb_k, const float* __restrict__ cb_v,
+                           uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages, int n_pages,
+                           const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
+                           int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
+    constexpr int L = D / NOVAKV_G;
+    __shared__ double R_s[4][D][4];
+    __shared__ float4 cb_s[4][NOVAKV_C];
+    __shared__ double mean_s[D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int l = blockIdx.x * 4 + warp, kvh = blockIdx.y, side = blockIdx.z;
+    const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
+    const double* R = (side == 0 ? rk_d : rv_d) + (size_t)kvh * D * D;
+    const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
+    const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + ((size_t)kvh * L + l) * NOVAKV_C * NOVAKV_G);
+    for (int i = lane; i < D; i += 32) {
+        const double2 a = *reinterpret_cast<const double2*>(R + (size_t)i * D + l * 4);
+        const double2 b = *reinterpret_cast<const double2*>(R + (size_t)i * D + l * 4 + 2);
+        R_s[warp][i][0] = a.x; R_s[warp][i][1] = a.y; R_s[warp][i][2] = b.x; R_s[warp][i][3] = b.y;
+    }
+    for (int c = lane; c < NOVAKV_C; c += 32) cb_s[warp][c] = cb_g[c];
+    for (int i = threadIdx.x; i < D; i += 128) mean_s[i] = mean[i];
+    __syncthreads();
+
+    for (int t0 = 0; t0 < n_tokens; t0 += 32) {
+        const int tkn = t0 + lane;
+        int page = -1, slot = 0;
+        if (tkn < n_tokens) {
+            const int s = tok_seq[tkn], pos = tok_pos[tkn];
+            if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
+                if (blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0) atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
+            } else {
+                page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
+                slot = pos % NOVAKV_PAGE_TOKENS;
+                if (page < 0 || page >= n_pages) {
+                    if (blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0) atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
+                    page = -1;
+                } else if (blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0) {
+                    atomicMax(&seq_lens[s], pos + 1);
+                }
+            }
+        }
+        if (page < 0) continue;
+        // coefficients of group l: binary64 accumulation over the input dimension in index order
+        double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
+        const uint4* xrow = reinterpret_cast<const uint4*>(x_new + ((size_t)tkn * n_kv_heads + kvh) * D);
+#pragma unroll 2
+        for (int i8 = 0; i8 < D / 8; ++i8) {
+            const uint4 raw = xrow[i8];
+            const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&raw);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = i8 * 8 + j;
+                const double xc = (double)__bfloat162float(xb[j]) - mean_s[i];
+                acc0 = fma(xc, R_s[warp][i][0], acc0);
+                acc1 = fma(xc, R_s[warp][i][1], acc1);
+                acc2 = fma(xc, R_s[warp][i][2], acc2);
+                acc3 = fma(xc, R_s[warp][i][3], acc3);
+            }
+        }
+        const float4 r = make_float4((float)acc0, (float)acc1, (float)acc2, (float)acc3);
+        float best = dist4(r, cb_s[warp][0]);
+        int bi = 0;
+#pragma unroll 8
+        for (int c = 1; c < NOVAKV_C; ++c) {
+            const float dd = dist4(r, cb_s[warp][c]);
+            if (dd < best) { best = dd; bi = c; }
+        }
+        const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
+        if (side == 0) k_pages[base + novakv_k_offset<L>(slot, l)] = (uint8_t)bi;
+        else v_pages[base + novakv_v_offset<L>(slot, l)] = (uint8_t)bi;
+    }
+}
+
 // Search only, from given binary32 coefficients [n][Hkv][D]; logical indices out [n][Hkv][L].
 template <int D>
 __global__ void __launch_bounds__(ENC_THREADS, 1)
@@ -208,6 +295,16 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                               int n_tokens, uint8_t* k_pages, uint8_t* v_pages, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
                               cudaStream_t stream) {
+    if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS) {
+        dim3 grid(D / NOVAKV_G / 4, ctx->cfg.n_kv_heads, 2);
+        novakv_prof_scope ps(ctx, 1, stream);
+        novakv_encode_small_kernel<D><<<grid, 128, 0, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d,
+            ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages, page_table,
+            max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads, ctx->dev_status);
+        ps.end();
+        ctx->launches++;
+        return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
+    }
     auto kern = novakv_encode_kernel<D>;
     const size_t smem = EncSmem<D>::total;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;

@@ -310,3 +310,41 @@ def test_bench_configuration_sampled():
         ratio_cc = check_output(out_cc[b], ref)
         print(f"[bench cfg seq {b}] sampled index mismatches K {dk} V {dv}; max|delta|/||o||inf "
               f"{ratio:.3e} (tensor-core value side) {ratio_cc:.3e} (CUDA-core value side)")
+
+
+# --------------------------------------------------------------------------- uncompressed comparator
+@pytest.mark.parametrize("name,window", [("qwen", 0), ("qwen", 128), ("gptoss", 0), ("gptoss", 128)])
+def test_bf16_comparator_matches_textbook_attention(name, window, request):
+    """The in-house bf16 decode kernel (used for the compression speed-up and for sliding-window
+    layers) against textbook attention on the same bf16 keys and values."""
+    from oracle import novakv_oracle as O
+    case = request.getfixturevalue(name)
+    ctx = case.ctx
+    lens = np.array([1, 200, 1025, 0, 3000], np.int32)
+    table, n_pages = synth.shuffled_page_table(7, np.maximum(lens, 1), 64)
+    hkv, d = ctx.n_kv_heads, ctx.head_dim
+    gen = synth.rng(123)
+    kp = np.zeros((n_pages, hkv, 64, d), np.float32)
+    vp = np.zeros((n_pages, hkv, 64, d), np.float32)
+    ks, vs = [], []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(1400 + b, max(int(n), 1), 1)
+        ks.append(k[:n]); vs.append(v[:n])
+        pos = np.arange(n)
+        kp[table[b][pos // 64], :, pos % 64, :] = k[:n]
+        vp[table[b][pos // 64], :, pos % 64, :] = v[:n]
+    _, _, q = case.draw(1450, 1, len(lens))
+    kd, vd = _dev(kp, torch.bfloat16), _dev(vp, torch.bfloat16)
+    pt = _dev(np.where(table < 0, 0, table).astype(np.int32))
+    sl = _dev(lens)
+    ws = torch.empty(ctx.novakv_bf16_workspace_bytes(len(lens), table.shape[1]), dtype=torch.uint8, device="cuda")
+    out = torch.empty((len(lens), ctx.n_q_heads, d), dtype=torch.float32, device="cuda")
+    ctx.novakv_bf16_decode_attention(_dev(q, torch.bfloat16), kd, vd, pt, sl, out, ws, window=window)
+    got = out.cpu().numpy()
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert not got[b].any()
+            continue
+        s0 = max(0, int(n) - window) if window > 0 else 0
+        ref = O.attention(q[b].astype(np.float64), ks[b][s0:].astype(np.float64), vs[b][s0:].astype(np.float64))
+        check_output(got[b], ref)
