@@ -3,11 +3,13 @@
 //
 // The search is ALU-bound (256 distance evaluations per group, per token, per side); the codebook
 // of the CTA's head and side stays in shared memory and every warp reads codewords as broadcasts.
+#include <math_constants.h>
+
 #include "novakv_internal.cuh"
 
 namespace {
 
-constexpr int ENC_THREADS = 256;
+constexpr int ENC_THREADS = 512;
 constexpr int ENC_TILE = 64;   // tokens per tile (search granularity)
 constexpr int ENC_XT = 32;     // tokens per transform pass (bounds the binary64 staging buffer)
 #ifndef NOVAKV_SMALL_APPEND_TOKENS
@@ -32,9 +34,47 @@ __device__ __forceinline__ float dist4(const float4 r, const float4 c) {
     return __fmaf_rn(e3, e3, __fmaf_rn(e2, e2, __fmaf_rn(e1, e1, __fmul_rn(e0, e0))));
 }
 
-// Search of the tile's coefficients (r_s, [ENC_TILE][RSTRIDE] float) against cb_s ([L][256] float4).
-// Warp w owns groups w, w+8, ...; lane t owns tokens t and t+32.  Ascending codeword index with a
-// strict '<' keeps the first minimum.
+// Packed binary32 pairs: two IEEE operations per instruction (same roundings as the scalar forms).
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// Distances of one coefficient vector (each component duplicated into a pair) to two codewords at once:
+// cw[i] = (codeword c, component i ; codeword c+1, component i).  Same chain as dist4, per half.
+__device__ __forceinline__ void dist4x2(const uint64_t (&r2)[4], const uint64_t (&cw)[4], float& d0, float& d1) {
+    const uint64_t e0 = sub2(r2[0], cw[0]), e1 = sub2(r2[1], cw[1]), e2 = sub2(r2[2], cw[2]), e3 = sub2(r2[3], cw[3]);
+    const uint64_t d = fma2(e3, e3, fma2(e2, e2, fma2(e1, e1, mul2(e0, e0))));
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+}
+
+// Shared-memory image of a (head, side) codebook for the search: [L][128 codeword pairs][4 components][2].
+__device__ __forceinline__ void fill_codebook_pairs(float* cb_s, const float4* __restrict__ cb_g, int n_groups) {
+    for (int i = threadIdx.x; i < n_groups * NOVAKV_C; i += ENC_THREADS) {
+        const float4 v = cb_g[i];
+        float* dst = cb_s + (size_t)(i >> 1) * 8 + (i & 1);
+        dst[0] = v.x; dst[2] = v.y; dst[4] = v.z; dst[6] = v.w;
+    }
+}
+
+// Search of the tile's coefficients (r_s, [ENC_TILE][RSTRIDE] float) against the paired codebook image.
+// Warp w owns groups w, w+16, ...; lane t owns tokens t and t+32.  Codewords are visited in ascending
+// index with a strict '<', which keeps the first minimum.
 template <int D>
 __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s, uint8_t* idx_s, int n_valid) {
     constexpr int L = D / NOVAKV_G;
@@ -43,20 +83,22 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
     for (int l = warp; l < L; l += ENC_THREADS / 32) {
         const float4 ra = *reinterpret_cast<const float4*>(r_s + (size_t)lane * RS + l * 4);
         const float4 rb = *reinterpret_cast<const float4*>(r_s + (size_t)(lane + 32) * RS + l * 4);
-        float best_a = 0.f, best_b = 0.f;
+        const uint64_t ra2[4] = {pk2(ra.x, ra.x), pk2(ra.y, ra.y), pk2(ra.z, ra.z), pk2(ra.w, ra.w)};
+        const uint64_t rb2[4] = {pk2(rb.x, rb.x), pk2(rb.y, rb.y), pk2(rb.z, rb.z), pk2(rb.w, rb.w)};
+        float best_a = CUDART_INF_F, best_b = CUDART_INF_F;
         int ia = 0, ib = 0;
-        const float4* cb = cb_s + (size_t)l * NOVAKV_C;
-        {
-            const float4 c0 = cb[0];
-            best_a = dist4(ra, c0);
-            best_b = dist4(rb, c0);
-        }
+        const ulonglong2* cb = reinterpret_cast<const ulonglong2*>(cb_s) + (size_t)l * NOVAKV_C;   // 2 x 16 B per pair
 #pragma unroll 4
-        for (int c = 1; c < NOVAKV_C; ++c) {
-            const float4 cw = cb[c];
-            const float da = dist4(ra, cw), db = dist4(rb, cw);
-            if (da < best_a) { best_a = da; ia = c; }
-            if (db < best_b) { best_b = db; ib = c; }
+        for (int p = 0; p < NOVAKV_C / 2; ++p) {
+            const ulonglong2 q0 = cb[2 * p], q1 = cb[2 * p + 1];
+            const uint64_t cw[4] = {q0.x, q0.y, q1.x, q1.y};
+            float a0, a1, b0, b1;
+            dist4x2(ra2, cw, a0, a1);
+            dist4x2(rb2, cw, b0, b1);
+            if (a0 < best_a) { best_a = a0; ia = 2 * p; }
+            if (a1 < best_a) { best_a = a1; ia = 2 * p + 1; }
+            if (b0 < best_b) { best_b = b0; ib = 2 * p; }
+            if (b1 < best_b) { best_b = b1; ib = 2 * p + 1; }
         }
         if (lane < n_valid) idx_s[lane * L + l] = (uint8_t)ia;
         if (lane + 32 < n_valid) idx_s[(lane + 32) * L + l] = (uint8_t)ib;
@@ -91,7 +133,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
 
     // codebook of this (head, side) -> shared memory, once per CTA
-    for (int i = threadIdx.x; i < L * NOVAKV_C; i += ENC_THREADS) cb_s[i] = cb_g[i];
+    fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);
 
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
     const int tile0 = blockIdx.x * tiles_per_cta;
@@ -137,12 +179,13 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
             __syncthreads();
             // transform: r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA, rounded once to binary32.
             // thread -> column c = tid % D, token subset tid / D (stride ENC_THREADS / D).
-            constexpr int TSUB = ENC_THREADS / D;           // 2 (D=128) or 4 (D=64)
-            constexpr int TPT = ENC_XT / TSUB;              // tokens per thread: 16 or 8
+            constexpr int TSUB = ENC_THREADS / D;           // 4 (D=128) or 8 (D=64)
+            constexpr int TPT = ENC_XT / TSUB;              // tokens per thread: 8 or 4
             const int c = threadIdx.x % D, sub = threadIdx.x / D;
             double acc[TPT];
 #pragma unroll
             for (int j = 0; j < TPT; ++j) acc[j] = 0.0;
+#pragma unroll 8
             for (int i = 0; i < D; ++i) {
                 const double rv = R[(size_t)i * D + c];
 #pragma unroll
@@ -269,7 +312,7 @@ novakv_search_kernel(const float* __restrict__ coef, int n, const float* __restr
     uint8_t* idx_s = smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes + EncSmem<D>::r_bytes;
     const int kvh = blockIdx.y;
     const float4* cb_g = reinterpret_cast<const float4*>(cb_all + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
-    for (int i = threadIdx.x; i < L * NOVAKV_C; i += ENC_THREADS) cb_s[i] = cb_g[i];
+    fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);
     const int n_tiles = (n + ENC_TILE - 1) / ENC_TILE;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int t0 = tile * ENC_TILE;
@@ -311,9 +354,18 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
     const int hs = ctx->cfg.n_kv_heads * 2;
     // enough CTAs per (head, side) to fill the machine about twice, each amortising its codebook fill
-    int ctas_x = max(1, min(n_tiles, (2 * ctx->n_sm + hs - 1) / hs));
-    const int tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
-    ctas_x = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    // CTAs per (head, side): whole waves of the machine, each CTA amortising its 128 KB codebook fill
+    // (counted as 1.5 tiles) over several tiles
+    int ctas_x = 1, tiles_per_cta = n_tiles;
+    double best = 1e30;
+    for (int w = 1; w <= 8; ++w) {
+        int cx = min(n_tiles, max(1, (w * ctx->n_sm) / hs));
+        const int tp = (n_tiles + cx - 1) / cx;
+        cx = (n_tiles + tp - 1) / tp;
+        const int waves = (cx * hs + ctx->n_sm - 1) / ctx->n_sm;
+        const double cost = waves * (tp + 1.5);
+        if (cost < best) { best = cost; ctas_x = cx; tiles_per_cta = tp; }
+    }
     dim3 grid(ctas_x, ctx->cfg.n_kv_heads, 2);
     novakv_prof_scope ps(ctx, 1, stream);
     kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d, ly.rv_d,
