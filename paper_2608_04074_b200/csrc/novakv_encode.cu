@@ -177,22 +177,34 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                 xc_s[i] = x;
             }
             __syncthreads();
-            // transform: r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA, rounded once to binary32.
-            // thread -> column c = tid % D, token subset tid / D (stride ENC_THREADS / D).
-            constexpr int TSUB = ENC_THREADS / D;           // 4 (D=128) or 8 (D=64)
-            constexpr int TPT = ENC_XT / TSUB;              // tokens per thread: 8 or 4
-            const int c = threadIdx.x % D, sub = threadIdx.x / D;
-            double acc[TPT];
+            // transform: r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA in index order, rounded once to
+            // binary32.  Each thread owns 2 columns (c, c + D/2) x TM tokens and walks i two at a time, so
+            // that one 128-bit broadcast load of xc feeds 4 FMAs (the loop is shared-memory bound otherwise).
+            constexpr int HALF = D / 2;
+            constexpr int TSUB = ENC_THREADS / HALF;        // 8 (D=128) or 16 (D=64) token subsets
+            constexpr int TM = ENC_XT / TSUB;               // tokens per thread: 4 or 2
+            const int c = threadIdx.x % HALF, sub = threadIdx.x / HALF;
+            double acc0[TM], acc1[TM];
 #pragma unroll
-            for (int j = 0; j < TPT; ++j) acc[j] = 0.0;
-#pragma unroll 8
-            for (int i = 0; i < D; ++i) {
-                const double rv = R[(size_t)i * D + c];
+            for (int j = 0; j < TM; ++j) { acc0[j] = 0.0; acc1[j] = 0.0; }
+#pragma unroll 4
+            for (int i = 0; i < D; i += 2) {
+                const double ra0 = R[(size_t)i * D + c], rb0 = R[(size_t)i * D + c + HALF];
+                const double ra1 = R[(size_t)(i + 1) * D + c], rb1 = R[(size_t)(i + 1) * D + c + HALF];
 #pragma unroll
-                for (int j = 0; j < TPT; ++j) acc[j] = fma(xc_s[(size_t)(sub + j * TSUB) * D + i], rv, acc[j]);
+                for (int j = 0; j < TM; ++j) {
+                    const double2 x = *reinterpret_cast<const double2*>(xc_s + (size_t)(sub + j * TSUB) * D + i);
+                    acc0[j] = fma(x.x, ra0, acc0[j]);
+                    acc1[j] = fma(x.x, rb0, acc1[j]);
+                    acc0[j] = fma(x.y, ra1, acc0[j]);
+                    acc1[j] = fma(x.y, rb1, acc1[j]);
+                }
             }
 #pragma unroll
-            for (int j = 0; j < TPT; ++j) r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc[j];
+            for (int j = 0; j < TM; ++j) {
+                r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc0[j];
+                r_s[(size_t)(tb + sub + j * TSUB) * RS + c + HALF] = (float)acc1[j];
+            }
         }
         __syncthreads();
 
@@ -384,7 +396,8 @@ novakv_status launch_search_t(novakv_ctx* ctx, const novakv_layer& ly, int which
     const size_t smem = EncSmem<D>::total;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;
     const int n_tiles = (n + ENC_TILE - 1) / ENC_TILE;
-    dim3 grid(max(1, min(n_tiles, 2 * ctx->n_sm / ctx->cfg.n_kv_heads + 1)), ctx->cfg.n_kv_heads);
+    // CTAs per head: about two whole waves of the machine
+    dim3 grid(max(1, min(n_tiles, (2 * ctx->n_sm) / ctx->cfg.n_kv_heads)), ctx->cfg.n_kv_heads);
     kern<<<grid, ENC_THREADS, smem, stream>>>(coef, n, which == 0 ? ly.cb_k : ly.cb_v, ctx->cfg.n_kv_heads, idx_out);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
