@@ -247,6 +247,72 @@ __device__ __forceinline__ uint2 ldg_stream_64(const void* p) {
     return v;
 }
 
+// Segment prologue pieces, kept out of line so that their register-hungry load batches do not
+// disturb the register allocation of the scan loop.
+template <int D, int HG, bool VM>
+__device__ __noinline__ void load_value_codebook(unsigned char* smem, const __half* __restrict__ cb_v_img, int kvh) {
+    using C = S1<D, HG, VM>;
+    const uint4* src = reinterpret_cast<const uint4*>(cb_v_img + (size_t)kvh * (VCB_BYTES / 2));
+    uint4* dst = reinterpret_cast<uint4*>(smem + C::OFF_VCB);
+    // all loads of a thread in flight before the first store (one L2 latency for the whole copy)
+    constexpr int NV4 = (VCB_BYTES / 16 + S1_THREADS - 1) / S1_THREADS;
+    uint4 tmp[NV4];
+#pragma unroll
+    for (int k = 0; k < NV4; ++k) {
+        const int i = threadIdx.x + k * S1_THREADS;
+        if (i < VCB_BYTES / 16) tmp[k] = src[i];
+    }
+#pragma unroll
+    for (int k = 0; k < NV4; ++k) {
+        const int i = threadIdx.x + k * S1_THREADS;
+        if (i < VCB_BYTES / 16) dst[i] = tmp[k];
+    }
+}
+
+// LUT[hs][plane][code][e] = <q'_h segment of group l(e, plane), key codeword> for 4 heads per entry.
+template <int D, int HG, bool VM>
+__device__ __noinline__ void build_score_table(unsigned char* smem, const float* __restrict__ cb_k_lut, int kvh) {
+    using C = S1<D, HG, VM>;
+    constexpr int GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS;
+        {
+    constexpr int CPI = NCW * 2;                                   // codes per iteration (16 entries each)
+    const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
+    const int sigma = e & 7, mpar = e >> 3;
+    const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)kvh * C::PLANES * 256 * 16;
+    const float* qs = reinterpret_cast<const float*>(smem + C::OFF_P);
+#pragma unroll
+    for (int pl = 0; pl < C::PLANES; ++pl) {
+        const int l = sigma * GPS + pl * 2 + mpar;
+        float4 qseg[HPAD];
+#pragma unroll
+        for (int h = 0; h < HPAD; ++h) qseg[h] = *reinterpret_cast<const float4*>(qs + h * D + l * 4);
+        // all codeword loads of the plane in flight before the first use
+        constexpr int NIT = (256 + CPI - 1) / CPI;
+        float4 cwv[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int code = code0 + it * CPI;
+            if (code < 256) cwv[it] = cbk[((size_t)pl * 256 + code) * 16 + e];
+        }
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int code = code0 + it * CPI;
+            if (code >= 256) break;
+            const float4 cw = cwv[it];
+#pragma unroll
+            for (int hs = 0; hs < HSETS; ++hs) {
+                float4 o;
+                o.x = fmaf(qseg[hs * 4 + 0].w, cw.w, fmaf(qseg[hs * 4 + 0].z, cw.z, fmaf(qseg[hs * 4 + 0].y, cw.y, qseg[hs * 4 + 0].x * cw.x)));
+                o.y = fmaf(qseg[hs * 4 + 1].w, cw.w, fmaf(qseg[hs * 4 + 1].z, cw.z, fmaf(qseg[hs * 4 + 1].y, cw.y, qseg[hs * 4 + 1].x * cw.x)));
+                o.z = fmaf(qseg[hs * 4 + 2].w, cw.w, fmaf(qseg[hs * 4 + 2].z, cw.z, fmaf(qseg[hs * 4 + 2].y, cw.y, qseg[hs * 4 + 2].x * cw.x)));
+                o.w = fmaf(qseg[hs * 4 + 3].w, cw.w, fmaf(qseg[hs * 4 + 3].z, cw.z, fmaf(qseg[hs * 4 + 3].y, cw.y, qseg[hs * 4 + 3].x * cw.x)));
+                *reinterpret_cast<float4*>(smem + C::OFF_LUT + (hs * C::PLANES + pl) * LUT_PLANE_BYTES + code * 256 + e * 16) = o;
+            }
+        }
+    }
+}
+}
+
 // Index bytes of one 32-token tile as one lane holds them.
 //   kw: this lane's token (lane = token within the tile), L bytes in rotated slot order: position j
 //       holds slot (j + lane%8 + lane/8) % 8, so that step j of every lane reads a different slot.
@@ -323,11 +389,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             reinterpret_cast<float*>(smem + C::OFF_P)[i] = v;
         }
         if (vcb_head != sg.kvh) {
-            // value codebook of this KV head (binary16 image, 64 KB) -> shared memory
-            const uint4* src = reinterpret_cast<const uint4*>(cb_v_img + (size_t)sg.kvh * (VCB_BYTES / 2));
-            uint4* dst = reinterpret_cast<uint4*>(smem + C::OFF_VCB);
-#pragma unroll 4
-            for (int i = threadIdx.x; i < VCB_BYTES / 16; i += S1_THREADS) dst[i] = src[i];
+            load_value_codebook<D, HG, VM>(smem, cb_v_img, sg.kvh);
             vcb_head = sg.kvh;
         }
         __syncthreads();
@@ -373,35 +435,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         // (the first tile's loads are issued before, so that they fly during the table build)
         TileRegs<L> nxt;
         if (n_it > 0) load_tile(0, nxt);
-        {
-            constexpr int CPI = NCW * 2;                                   // codes per iteration (16 entries each)
-            const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
-            const int sigma = e & 7, mpar = e >> 3;
-            const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)sg.kvh * C::PLANES * 256 * 16;
-            const float* qs = reinterpret_cast<const float*>(smem + C::OFF_P);
-#pragma unroll
-            for (int pl = 0; pl < C::PLANES; ++pl) {
-                const int l = sigma * GPS + pl * 2 + mpar;
-                float4 qseg[HPAD];
-#pragma unroll
-                for (int h = 0; h < HPAD; ++h) qseg[h] = *reinterpret_cast<const float4*>(qs + h * D + l * 4);
-#pragma unroll 4
-                for (int it = 0; it < (256 + CPI - 1) / CPI; ++it) {
-                    const int code = code0 + it * CPI;
-                    if (code >= 256) break;
-                    const float4 cw = cbk[((size_t)pl * 256 + code) * 16 + e];
-#pragma unroll
-                    for (int hs = 0; hs < HSETS; ++hs) {
-                        float4 o;
-                        o.x = fmaf(qseg[hs * 4 + 0].w, cw.w, fmaf(qseg[hs * 4 + 0].z, cw.z, fmaf(qseg[hs * 4 + 0].y, cw.y, qseg[hs * 4 + 0].x * cw.x)));
-                        o.y = fmaf(qseg[hs * 4 + 1].w, cw.w, fmaf(qseg[hs * 4 + 1].z, cw.z, fmaf(qseg[hs * 4 + 1].y, cw.y, qseg[hs * 4 + 1].x * cw.x)));
-                        o.z = fmaf(qseg[hs * 4 + 2].w, cw.w, fmaf(qseg[hs * 4 + 2].z, cw.z, fmaf(qseg[hs * 4 + 2].y, cw.y, qseg[hs * 4 + 2].x * cw.x)));
-                        o.w = fmaf(qseg[hs * 4 + 3].w, cw.w, fmaf(qseg[hs * 4 + 3].z, cw.z, fmaf(qseg[hs * 4 + 3].y, cw.y, qseg[hs * 4 + 3].x * cw.x)));
-                        *reinterpret_cast<float4*>(smem + C::OFF_LUT + (hs * C::PLANES + pl) * LUT_PLANE_BYTES + code * 256 + e * 16) = o;
-                    }
-                }
-            }
-        }
+        build_score_table<D, HG, VM>(smem, cb_k_lut, sg.kvh);
         __syncthreads();     // table and value codebook complete; q' staging no longer needed
 
         // ---- scan: 32-token tiles, loads of the next tile in flight while this one is consumed ------
