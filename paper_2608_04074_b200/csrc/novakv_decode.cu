@@ -84,9 +84,10 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                       const int32_t* __restrict__ seq_lens, int batch, int n_q_heads, int n_kv_heads,
                       int max_pages_per_seq, float scale_log2, float* __restrict__ qp,
                       int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status) {
+    novakv_grid_dependency_wait();
     const int blk = blockIdx.x;
     if (blk == batch * n_kv_heads) {
-        // exclusive prefix over sequences of (pages * Hkv); small, done by one warp
+        // exclusive prefix over sequences of their page counts; small, done by one warp
         if (threadIdx.x < 32) {
             int carry = 0;
             for (int b0 = 0; b0 < batch; b0 += 32) {
@@ -96,7 +97,7 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                     const int raw = seq_lens[b];
                     const int len = clamp_len(raw, max_pages_per_seq);
                     if (raw != len) atomicOr(dev_status, NOVAKV_DEV_BAD_LENGTH);
-                    v = ((len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS) * n_kv_heads;
+                    v = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
                 }
                 int incl = v;
 #pragma unroll
@@ -211,21 +212,25 @@ struct Segment {
     int b, kvh, pg0, npg, len;
 };
 
-// Locate the (sequence, KV head, page) of global page unit u.  page_prefix is exclusive, length batch+1.
+// Locate the (KV head, sequence, page) of global page unit u.  Units are ordered KV-head-major:
+// u = kvh * P + page_prefix[b] + page, with P = page_prefix[batch] the pages of all sequences, so that
+// consecutive segments of a CTA share the KV head (and its value codebook).  page_prefix is exclusive,
+// length batch + 1.
 __device__ __forceinline__ Segment locate(const int32_t* __restrict__ page_prefix, const int32_t* __restrict__ seq_lens,
-                                          int batch, int n_kv_heads, int max_pages, long u, long u_end) {
-    int lo = 0, hi = batch;                    // find b: prefix[b] <= u < prefix[b+1]
+                                          int batch, int max_pages, long u, long u_end) {
+    const long P = page_prefix[batch];
+    Segment s;
+    s.kvh = (int)(u / P);
+    const long r = u - (long)s.kvh * P;
+    int lo = 0, hi = batch;                    // find b: prefix[b] <= r < prefix[b+1]
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if ((long)page_prefix[mid] <= u) lo = mid; else hi = mid;
+        if ((long)page_prefix[mid] <= r) lo = mid; else hi = mid;
     }
-    Segment s;
     s.b = lo;
     s.len = clamp_len(seq_lens[lo], max_pages);
     const int pages_b = (s.len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
-    const int rel = (int)(u - page_prefix[lo]);
-    s.kvh = rel / pages_b;
-    s.pg0 = rel - s.kvh * pages_b;
+    s.pg0 = (int)(r - page_prefix[lo]);
     const long left = u_end - u;
     s.npg = (int)(left < (long)(pages_b - s.pg0) ? left : (long)(pages_b - s.pg0));
     return s;
@@ -338,11 +343,12 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     constexpr int L = C::L, GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, NGB = C::NGB, KPL = C::KPL;
     constexpr int TILE_BYTES = C::TILE_BYTES, PAGE_BYTES = 2 * TILE_BYTES;
     extern __shared__ __align__(1024) unsigned char smem[];
+    novakv_grid_dependency_wait();
     const uint32_t s_base = smem_u32(smem);
     const uint32_t s_lut = s_base + C::OFF_LUT, s_vcb = s_base + C::OFF_VCB, s_p = s_base + C::OFF_P;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long U = page_prefix[batch];
+    const long U = (long)page_prefix[batch] * n_kv_heads;
     const long u_begin = ((long)blockIdx.x * U) / gridDim.x, u_end = ((long)(blockIdx.x + 1) * U) / gridDim.x;
     if (u_begin >= u_end) return;
 
@@ -377,8 +383,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     int vcb_head = -1;       // KV head whose value codebook is resident
     long u = u_begin;
     while (u < u_end) {
-        const Segment sg = locate(page_prefix, seq_lens, batch, n_kv_heads, max_pages_per_seq, u, u_end);
-        const int pair = sg.b * n_kv_heads + sg.kvh;
+        const Segment sg = locate(page_prefix, seq_lens, batch, max_pages_per_seq, u, u_end);
+        const int pair = sg.kvh * batch + sg.b;            // grows along the walk
 
         // ---- segment prologue -----------------------------------------------------------------
         // q' of this segment's heads -> P area (fp32 [HPAD][D]); heads beyond HG are zero
@@ -698,28 +704,30 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
                            const float* __restrict__ rv_t, const float* __restrict__ v_mean,
                            void* __restrict__ out, int out_is_fp32) {
     __shared__ float o_s[HG * D];
+    novakv_grid_dependency_wait();
     const int pair = blockIdx.x;
     const int b = pair / n_kv_heads, kvh = pair - b * n_kv_heads;
     const int len = clamp_len(seq_lens[b], max_pages_per_seq);
     const int pages_b = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
-    const long U = page_prefix[batch];
+    const long P = page_prefix[batch], U = P * n_kv_heads;
+    const int slot0 = kvh * batch + b;                     // the scan kernel's pair index (walk order)
     for (int i = threadIdx.x; i < HG * D; i += blockDim.x) {
         const int h = i / D, c = i - h * D;
         float val = 0.f;
         if (pages_b > 0) {
-            const long u0 = (long)page_prefix[b] + (long)kvh * pages_b, u1 = u0 + pages_b;
+            const long u0 = (long)kvh * P + page_prefix[b], u1 = u0 + pages_b;
             // CTA of unit u: the largest c with floor(c*U/G) <= u
             const int c_first = (int)(((u0 + 1) * grid_s1 - 1) / U), c_last = (int)((u1 * grid_s1 - 1) / U);
             // CTAs in between whose own range is empty wrote nothing: skip them
             float M = M_INIT;
             for (int cta = c_first; cta <= c_last; ++cta) {
                 if (((long)cta * U) / grid_s1 >= ((long)(cta + 1) * U) / grid_s1) continue;
-                M = fmaxf(M, part_ml[(((size_t)pair + cta) * HG + h) * 2]);
+                M = fmaxf(M, part_ml[(((size_t)slot0 + cta) * HG + h) * 2]);
             }
             float a = 0.f, lsum = 0.f;
             for (int cta = c_first; cta <= c_last; ++cta) {
                 if (((long)cta * U) / grid_s1 >= ((long)(cta + 1) * U) / grid_s1) continue;
-                const size_t pidx = (size_t)pair + cta;
+                const size_t pidx = (size_t)slot0 + cta;
                 const float sc = ex2(part_ml[(pidx * HG + h) * 2] - M);
                 a = fmaf(sc, part_acc[(pidx * HG + h) * D + c], a);
                 lsum = fmaf(sc, part_ml[(pidx * HG + h) * 2 + 1], lsum);
@@ -798,22 +806,28 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     float* part_acc = (float*)(ws + w.acc);
     const int hq = ctx->cfg.n_q_heads, hkv = ctx->cfg.n_kv_heads;
 
-    novakv_prepare_kernel<D, HG><<<batch * hkv + 1, 512, 0, stream>>>(q, ly.rk_inv_t, seq_lens, batch, hq, hkv,
-        max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status);
+    novakv_launch_pdl(novakv_prepare_kernel<D, HG>, dim3(batch * hkv + 1), dim3(512), 0, stream, q, ly.rk_inv_t, seq_lens,
+                      batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status);
     ctx->launches++;
 
     auto kern = novakv_decode_stage1_kernel<D, HG, VM>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
+    static bool smem_opt_in = false;      // per template instantiation; the attribute is sticky
+    if (!smem_opt_in) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
+        smem_opt_in = true;
+    }
     const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
     {
         novakv_prof_scope ps(ctx, 0, stream);
-        kern<<<grid, S1_THREADS, C::SMEM, stream>>>(qp, ly.cb_k_lut, ly.cb_v_mma, k_pages, v_pages, n_pages,
-            page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc, ctx->dev_status);
+        novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut, ly.cb_v_mma, k_pages, v_pages,
+                          n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
+                          ctx->dev_status);
         ps.end();
         ctx->launches++;
     }
-    novakv_decode_merge_kernel<D, HG><<<batch * hkv, (HG * D > 512 ? 512 : HG * D), 0, stream>>>(part_ml, part_acc,
-        prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out, out_is_fp32);
+    novakv_launch_pdl(novakv_decode_merge_kernel<D, HG>, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
+                      part_ml, part_acc, prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out,
+                      out_is_fp32);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
 }

@@ -246,6 +246,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
     __shared__ double R_s[4][D][4];
     __shared__ float4 cb_s[4][NOVAKV_C];
     __shared__ double mean_s[D];
+    novakv_grid_dependency_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int l = blockIdx.x * 4 + warp, kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
@@ -353,9 +354,9 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS) {
         dim3 grid(D / NOVAKV_G / 4, ctx->cfg.n_kv_heads, 2);
         novakv_prof_scope ps(ctx, 1, stream);
-        novakv_encode_small_kernel<D><<<grid, 128, 0, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d,
-            ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages, page_table,
-            max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads, ctx->dev_status);
+        novakv_launch_pdl(novakv_encode_small_kernel<D>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos, n_tokens,
+                          ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
+                          page_table, max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads, ctx->dev_status);
         ps.end();
         ctx->launches++;
         return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;

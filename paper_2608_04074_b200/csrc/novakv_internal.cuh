@@ -87,6 +87,32 @@ novakv_status novakv_launch_bf16_decode(novakv_ctx* ctx, const __nv_bfloat16* q,
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 
+// Programmatic dependent launch: a kernel launched with novakv_launch_pdl may be scheduled while its
+// predecessor in the stream is still running; it must call novakv_grid_dependency_wait() before it
+// touches anything the predecessor reads or writes (every kernel here does so first thing), which
+// blocks until the predecessor grid has completed and its writes are visible.  Only the launch latency
+// is hidden; there is no unbounded wait in user code.
+__device__ __forceinline__ void novakv_grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t novakv_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Byte offsets inside the 64*L-byte chunk of one (page, KV head); t = token slot in the page
 // (0..63), l = group.  These define the cache format (see the public header).
 //   keys:   [tile = t/32][plane][token t%32][16 bytes]; a token's L bytes are its 8 "slots" of L/8
