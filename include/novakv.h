@@ -24,9 +24,11 @@
  * unless stated.  A context is used from one host thread at a time.
  *
  * Errors: every entry point validates its arguments on the host and returns a status; nothing
- * aborts.  Faults only the device can see (page id out of range, length beyond the page table, a
- * pipeline wait that ran out) set bits in the device status word, skip the offending work and
- * never trap; read them with novakv_last_device_status.
+ * aborts.  Faults only the device can see (page id out of range, length beyond the page table, an
+ * appended token that names no valid slot) set bits in the device status word and never trap: a bad
+ * page id is replaced by page 0 (every access stays in bounds, the affected sequence's output is
+ * unspecified), a bad length is clamped, a bad token is skipped.  Read the word with
+ * novakv_last_device_status.  The kernels contain no spin wait.
  *
  * Determinism: for fixed inputs, shapes and device, outputs are bitwise reproducible.
  */
@@ -57,7 +59,7 @@ typedef enum {
 /* Bits of the device status word. */
 #define NOVAKV_DEV_BAD_PAGE      1u   /* a page id was outside [0, n_pages) */
 #define NOVAKV_DEV_BAD_LENGTH    2u   /* a sequence length exceeded 64 * max_pages_per_seq */
-#define NOVAKV_DEV_WAIT_TIMEOUT  4u   /* an in-kernel pipeline wait hit its iteration limit */
+#define NOVAKV_DEV_WAIT_TIMEOUT  4u   /* reserved: no kernel of this build waits on another thread or copy */
 #define NOVAKV_DEV_BAD_TOKEN     8u   /* an appended token named a sequence slot or position out of range */
 
 typedef struct {

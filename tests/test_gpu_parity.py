@@ -348,3 +348,38 @@ def test_bf16_comparator_matches_textbook_attention(name, window, request):
         s0 = max(0, int(n) - window) if window > 0 else 0
         ref = O.attention(q[b].astype(np.float64), ks[b][s0:].astype(np.float64), vs[b][s0:].astype(np.float64))
         check_output(got[b], ref)
+
+
+# --------------------------------------------------------------------------- ragged serving mix, sampled
+def test_paged_mix_append_then_decode_sampled(qwen):
+    """Serving-mix structure at a size the oracle can follow: 40 ragged sequences (lognormal lengths),
+    shuffled 64-token pages, prefill by the GPU encoder, then one step = append one token per sequence
+    + decode; indices and outputs of sampled sequences are checked against the oracle."""
+    case = qwen
+    lens0 = synth.lognormal_lengths(4242, 40, median=900, sigma=1.0, lo=1, hi=6000)
+    from paper_2608_04074_b200.runtime import PagedCache
+    cache = PagedCache(case.ctx, lens0, capacity_tokens=lens0 + 1, seed=77)
+    cache.seq_lens.zero_()
+    toks = {}
+    ks, vs, seqs, poss = [], [], [], []
+    for b, n in enumerate(lens0):
+        k, v, _ = case.draw(2000 + b, int(n), 1)
+        toks[b] = (k, v)
+        ks.append(k); vs.append(v); seqs.append(np.full(n, b, np.int32)); poss.append(np.arange(n, dtype=np.int32))
+    cache.append(0, _dev(np.concatenate(ks), torch.bfloat16), _dev(np.concatenate(vs), torch.bfloat16),
+                 _dev(np.concatenate(seqs)), _dev(np.concatenate(poss)))
+    k1, v1, q = case.draw(2100, len(lens0), len(lens0))
+    cache.append(0, _dev(k1, torch.bfloat16), _dev(v1, torch.bfloat16), _dev(np.arange(len(lens0), dtype=np.int32)),
+                 _dev(lens0.astype(np.int32)))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens0 + 1)
+    order = np.argsort(lens0)
+    for b in (int(order[0]), int(order[len(order) // 2]), int(order[-1]), 7):
+        n = int(lens0[b]) + 1
+        kb = np.concatenate([toks[b][0], k1[b:b + 1]]).astype(np.float64)
+        vb = np.concatenate([toks[b][1], v1[b:b + 1]]).astype(np.float64)
+        enc = case.oracle.encode(kb, vb)
+        gk, gv = cache.load_logical(b, 0, n)
+        check_indices(gk, enc, "k"); check_indices(gv, enc, "v")
+        check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
