@@ -53,8 +53,7 @@ struct S1 {
     // per-warp staging of the softmax weights of one 32-token tile
     //   VM: fp16 [HPAD][4 k-slot pairs][8 tokens]        otherwise: fp32 [32 tokens][HPAD]
     static constexpr int P_WARP_BYTES = VM ? HPAD * 64 : 32 * HPAD * 4;
-    static constexpr int Q_BYTES = HPAD * D * 4;              // q' staging during the table build
-    static constexpr int P_BYTES = NCW * P_WARP_BYTES > Q_BYTES ? NCW * P_WARP_BYTES : Q_BYTES;
+    static constexpr int P_BYTES = NCW * P_WARP_BYTES;
     static constexpr int OFF_LUT = 0;
     static constexpr int OFF_VCB = OFF_LUT + LUT_BYTES;
     static constexpr int OFF_P = OFF_VCB + VCB_BYTES;
@@ -202,22 +201,23 @@ struct Segment {
 // Locate the (KV head, sequence, page) of global page unit u.  Units are ordered KV-head-major:
 // u = kvh * P + page_prefix[b] + page, with P = page_prefix[batch] the pages of all sequences, so that
 // consecutive segments of a CTA share the KV head (and its value codebook).  page_prefix is exclusive,
-// length batch + 1.
+// length batch + 1.  Cooperative: every thread tests one sequence (all loads independent, one memory
+// latency), the owner publishes (b, length) through shared memory.  Contains a __syncthreads().
 __device__ __forceinline__ Segment locate(const int32_t* __restrict__ page_prefix, const int32_t* __restrict__ seq_lens,
-                                          int batch, int max_pages, long u, long u_end) {
+                                          int batch, int max_pages, long u, long u_end, int* s_found) {
     const long P = page_prefix[batch];
     Segment s;
     s.kvh = (int)(u / P);
     const long r = u - (long)s.kvh * P;
-    int lo = 0, hi = batch;                    // find b: prefix[b] <= r < prefix[b+1]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if ((long)page_prefix[mid] <= r) lo = mid; else hi = mid;
+    for (int t = threadIdx.x; t < batch; t += S1_THREADS) {
+        const int lo = page_prefix[t], hi = page_prefix[t + 1], len = seq_lens[t];
+        if ((long)lo <= r && r < (long)hi) { s_found[0] = t; s_found[1] = clamp_len(len, max_pages); s_found[2] = lo; }
     }
-    s.b = lo;
-    s.len = clamp_len(seq_lens[lo], max_pages);
+    __syncthreads();
+    s.b = s_found[0];
+    s.len = s_found[1];
     const int pages_b = (s.len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
-    s.pg0 = (int)(r - page_prefix[lo]);
+    s.pg0 = (int)(r - s_found[2]);
     const long left = u_end - u;
     s.npg = (int)(left < (long)(pages_b - s.pg0) ? left : (long)(pages_b - s.pg0));
     return s;
@@ -263,7 +263,8 @@ __device__ __noinline__ void load_value_codebook(unsigned char* smem, const __ha
 
 // LUT[hs][plane][code][e] = <q'_h segment of group l(e, plane), key codeword> for 4 heads per entry.
 template <int D, int HG, bool VM>
-__device__ __noinline__ void build_score_table(unsigned char* smem, const float* __restrict__ cb_k_lut, int kvh) {
+__device__ __noinline__ void build_score_table(unsigned char* smem, const float* __restrict__ cb_k_lut, int kvh,
+                                               const float* __restrict__ q_pair /* q' of the pair's heads, [HG][D] */) {
     using C = S1<D, HG, VM>;
     constexpr int GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS;
         {
@@ -271,13 +272,13 @@ __device__ __noinline__ void build_score_table(unsigned char* smem, const float*
     const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
     const int sigma = e & 7, mpar = e >> 3;
     const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)kvh * C::PLANES * 256 * 16;
-    const float* qs = reinterpret_cast<const float*>(smem + C::OFF_P);
 #pragma unroll
     for (int pl = 0; pl < C::PLANES; ++pl) {
         const int l = sigma * GPS + pl * 2 + mpar;
-        float4 qseg[HPAD];
+        float4 qseg[HPAD];                        // heads beyond HG are zero
 #pragma unroll
-        for (int h = 0; h < HPAD; ++h) qseg[h] = *reinterpret_cast<const float4*>(qs + h * D + l * 4);
+        for (int h = 0; h < HPAD; ++h)
+            qseg[h] = h < HG ? *reinterpret_cast<const float4*>(q_pair + h * D + l * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
         // all codeword loads of the plane in flight before the first use
         constexpr int NIT = (256 + CPI - 1) / CPI;
         float4 cwv[NIT];
@@ -330,6 +331,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     constexpr int L = C::L, GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, NGB = C::NGB, KPL = C::KPL;
     constexpr int TILE_BYTES = C::TILE_BYTES, PAGE_BYTES = 2 * TILE_BYTES;
     extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ int s_found[4];
     novakv_grid_dependency_wait();
     const uint32_t s_base = smem_u32(smem);
     const uint32_t s_lut = s_base + C::OFF_LUT, s_vcb = s_base + C::OFF_VCB, s_p = s_base + C::OFF_P;
@@ -370,22 +372,14 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     int vcb_head = -1;       // KV head whose value codebook is resident
     long u = u_begin;
     while (u < u_end) {
-        const Segment sg = locate(page_prefix, seq_lens, batch, max_pages_per_seq, u, u_end);
+        const Segment sg = locate(page_prefix, seq_lens, batch, max_pages_per_seq, u, u_end, s_found);
         const int pair = sg.kvh * batch + sg.b;            // grows along the walk
 
         // ---- segment prologue -----------------------------------------------------------------
-        // q' of this segment's heads -> P area (fp32 [HPAD][D]); heads beyond HG are zero
-        for (int i = threadIdx.x; i < HPAD * D; i += S1_THREADS) {
-            const int h = i / D, c = i - h * D;
-            float v = 0.f;
-            if (h < HG) v = qp[((size_t)sg.b * n_q_heads + sg.kvh * HG + h) * D + c];
-            reinterpret_cast<float*>(smem + C::OFF_P)[i] = v;
-        }
         if (vcb_head != sg.kvh) {
             load_value_codebook<D, HG, VM>(smem, cb_v_img, sg.kvh);
             vcb_head = sg.kvh;
         }
-        __syncthreads();
 
         // this warp's tiles of the segment: half pages hp = warp, warp + NCW, ...
         const int n_it = (2 * sg.npg > warp) ? (2 * sg.npg - warp + NCW - 1) / NCW : 0;
@@ -428,8 +422,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         // (the first tile's loads are issued before, so that they fly during the table build)
         TileRegs<L> nxt;
         if (n_it > 0) load_tile(0, nxt);
-        build_score_table<D, HG, VM>(smem, cb_k_lut, sg.kvh);
-        __syncthreads();     // table and value codebook complete; q' staging no longer needed
+        build_score_table<D, HG, VM>(smem, cb_k_lut, sg.kvh, qp + ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D);
+        __syncthreads();     // table and value codebook complete
 
         // ---- scan: 32-token tiles, loads of the next tile in flight while this one is consumed ------
         for (int it = 0; it < n_it; ++it) {
