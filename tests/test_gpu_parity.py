@@ -383,3 +383,32 @@ def test_paged_mix_append_then_decode_sampled(qwen):
         gk, gv = cache.load_logical(b, 0, n)
         check_indices(gk, enc, "k"); check_indices(gv, enc, "v")
         check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
+
+
+# --------------------------------------------------------------------------- other head-group sizes
+@pytest.mark.parametrize("hq,hkv,d", [(2, 2, 128), (4, 2, 128), (3, 3, 64), (4, 2, 64)])
+def test_small_head_groups(hq, hkv, d):
+    """Hq/Hkv of 1 and 2 (padded to a 4-wide table entry inside the kernel), both head dims, both value paths."""
+    wl = workloads.Workload(f"hg{hq // hkv}_d{d}", synth.LayerShape(hq, hkv, d), np.array([700, 65], np.int32), seed=9,
+                            calib_tokens=2048, calib_queries_for_values=512, lloyd_iters=3)
+    case = Case(wl)
+    lens = wl.seq_lens
+    cache = _cache(case, lens, capacity=lens + 1)
+    cache.seq_lens.zero_()
+    toks = []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(2300 + b, int(n), 1)
+        toks.append((k, v))
+        cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(np.full(n, b, np.int32)),
+                     _dev(np.arange(n, dtype=np.int32)))
+    _, _, q = case.draw(2350, 1, len(lens))
+    for path in (1, 0):
+        case.ctx.novakv_debug_set_value_path(path)
+        out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+        assert case.ctx.novakv_last_device_status() == 0
+        for b, n in enumerate(lens):
+            enc = case.oracle.encode(toks[b][0].astype(np.float64), toks[b][1].astype(np.float64))
+            gk, gv = cache.load_logical(b, 0, int(n))
+            check_indices(gk, enc, "k"); check_indices(gv, enc, "v")
+            check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
+    case.ctx.close()
