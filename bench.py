@@ -499,7 +499,7 @@ def oracle_step(orc, kidx, vidx, q, k1, v1):
 
 def cpu_baseline_sample(wl, laws, cal, args):
     from oracle import novakv_oracle as O
-    n_seq = 2
+    n_seq = min(wl.batch, 8)          # about 20 core-seconds of oracle work on the benchmark shape
     orc, kidx, vidx, q, k1, v1 = oracle_sample_inputs(wl, laws, cal, n_seq)
     t0 = time.perf_counter()
     oracle_step(orc, kidx, vidx, q, k1, v1)
