@@ -266,44 +266,47 @@ template <int D, int HG, bool VM>
 __device__ __noinline__ void build_score_table(unsigned char* smem, const float* __restrict__ cb_k_lut, int kvh,
                                                const float* __restrict__ q_pair /* q' of the pair's heads, [HG][D] */) {
     using C = S1<D, HG, VM>;
-    constexpr int GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS;
-        {
+    constexpr int GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, PLANES = C::PLANES;
     constexpr int CPI = NCW * 2;                                   // codes per iteration (16 entries each)
+    constexpr int NIT = (256 + CPI - 1) / CPI;
     const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
     const int sigma = e & 7, mpar = e >> 3;
-    const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)kvh * C::PLANES * 256 * 16;
+    const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)kvh * PLANES * 256 * 16;
+    // every load of the thread (query segments and codewords of all planes) is issued before the first
+    // use: one memory latency for the whole table
+    float4 qseg[PLANES][HPAD];                    // heads beyond HG are zero
+    float4 cwv[PLANES][NIT];
 #pragma unroll
-    for (int pl = 0; pl < C::PLANES; ++pl) {
+    for (int pl = 0; pl < PLANES; ++pl) {
         const int l = sigma * GPS + pl * 2 + mpar;
-        float4 qseg[HPAD];                        // heads beyond HG are zero
 #pragma unroll
         for (int h = 0; h < HPAD; ++h)
-            qseg[h] = h < HG ? *reinterpret_cast<const float4*>(q_pair + h * D + l * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        // all codeword loads of the plane in flight before the first use
-        constexpr int NIT = (256 + CPI - 1) / CPI;
-        float4 cwv[NIT];
+            qseg[pl][h] = h < HG ? *reinterpret_cast<const float4*>(q_pair + h * D + l * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int it = 0; it < NIT; ++it) {
             const int code = code0 + it * CPI;
-            if (code < 256) cwv[it] = cbk[((size_t)pl * 256 + code) * 16 + e];
-        }
-#pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int code = code0 + it * CPI;
-            if (code >= 256) break;
-            const float4 cw = cwv[it];
-#pragma unroll
-            for (int hs = 0; hs < HSETS; ++hs) {
-                float4 o;
-                o.x = fmaf(qseg[hs * 4 + 0].w, cw.w, fmaf(qseg[hs * 4 + 0].z, cw.z, fmaf(qseg[hs * 4 + 0].y, cw.y, qseg[hs * 4 + 0].x * cw.x)));
-                o.y = fmaf(qseg[hs * 4 + 1].w, cw.w, fmaf(qseg[hs * 4 + 1].z, cw.z, fmaf(qseg[hs * 4 + 1].y, cw.y, qseg[hs * 4 + 1].x * cw.x)));
-                o.z = fmaf(qseg[hs * 4 + 2].w, cw.w, fmaf(qseg[hs * 4 + 2].z, cw.z, fmaf(qseg[hs * 4 + 2].y, cw.y, qseg[hs * 4 + 2].x * cw.x)));
-                o.w = fmaf(qseg[hs * 4 + 3].w, cw.w, fmaf(qseg[hs * 4 + 3].z, cw.z, fmaf(qseg[hs * 4 + 3].y, cw.y, qseg[hs * 4 + 3].x * cw.x)));
-                *reinterpret_cast<float4*>(smem + C::OFF_LUT + (hs * C::PLANES + pl) * LUT_PLANE_BYTES + code * 256 + e * 16) = o;
-            }
+            if (code < 256) cwv[pl][it] = cbk[((size_t)pl * 256 + code) * 16 + e];
         }
     }
-}
+#pragma unroll
+    for (int pl = 0; pl < PLANES; ++pl)
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int code = code0 + it * CPI;
+            if (code < 256) {
+                const float4 cw = cwv[pl][it];
+#pragma unroll
+                for (int hs = 0; hs < HSETS; ++hs) {
+                    const float4* q = &qseg[pl][hs * 4];
+                    float4 o;
+                    o.x = fmaf(q[0].w, cw.w, fmaf(q[0].z, cw.z, fmaf(q[0].y, cw.y, q[0].x * cw.x)));
+                    o.y = fmaf(q[1].w, cw.w, fmaf(q[1].z, cw.z, fmaf(q[1].y, cw.y, q[1].x * cw.x)));
+                    o.z = fmaf(q[2].w, cw.w, fmaf(q[2].z, cw.z, fmaf(q[2].y, cw.y, q[2].x * cw.x)));
+                    o.w = fmaf(q[3].w, cw.w, fmaf(q[3].z, cw.z, fmaf(q[3].y, cw.y, q[3].x * cw.x)));
+                    *reinterpret_cast<float4*>(smem + C::OFF_LUT + (hs * PLANES + pl) * LUT_PLANE_BYTES + code * 256 + e * 16) = o;
+                }
+            }
+        }
 }
 
 // Index bytes of one 32-token tile as one lane holds them.
