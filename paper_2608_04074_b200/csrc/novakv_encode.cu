@@ -73,14 +73,15 @@ __device__ __forceinline__ void fill_codebook_pairs(float* cb_s, const float4* _
 }
 
 // Search of the tile's coefficients (r_s, [ENC_TILE][RSTRIDE] float) against the paired codebook image.
-// Warp w owns groups w, w+16, ...; lane t owns tokens t and t+32.  Codewords are visited in ascending
+// Warp w of n_warps owns groups w, w+n_warps, ...; lane t owns tokens t and t+32.  Codewords are visited in ascending
 // index with a strict '<', which keeps the first minimum.
 template <int D>
-__device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s, uint8_t* idx_s, int n_valid) {
+__device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s, uint8_t* idx_s, int n_valid,
+                                            int warp, int n_warps) {
     constexpr int L = D / NOVAKV_G;
     constexpr int RS = EncSmem<D>::RSTRIDE;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int l = warp; l < L; l += ENC_THREADS / 32) {
+    const int lane = threadIdx.x & 31;
+    for (int l = warp; l < L; l += n_warps) {
         const float4 ra = *reinterpret_cast<const float4*>(r_s + (size_t)lane * RS + l * 4);
         const float4 rb = *reinterpret_cast<const float4*>(r_s + (size_t)(lane + 32) * RS + l * 4);
         const uint64_t ra2[4] = {pk2(ra.x, ra.x), pk2(ra.y, ra.y), pk2(ra.z, ra.z), pk2(ra.w, ra.w)};
@@ -105,6 +106,36 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
     }
 }
 
+// Named barriers of the tiled encode kernel (hardware barriers; bar.arrive does not block).
+__device__ __forceinline__ void nbar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ void nbar_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+constexpr int BAR_T = 1, BAR_S = 2, BAR_FULL = 3 /* +buf */, BAR_EMPTY = 5 /* +buf */;
+constexpr int ENC_HALF_THREADS = ENC_THREADS / 2;
+
+// Shared-memory plan of the pipelined encode kernel.
+template <int D>
+struct EncPipe {
+    static constexpr int L = D / NOVAKV_G;
+    static constexpr int RS = D + 4;
+    static constexpr int XT = 16;                              // tokens per transform pass
+    static constexpr size_t cb_bytes = (size_t)L * NOVAKV_C * NOVAKV_G * sizeof(float);
+    static constexpr size_t r_bytes = (size_t)ENC_TILE * RS * sizeof(float);       // one buffer
+    static constexpr size_t xc_bytes = (size_t)XT * D * sizeof(double);
+    static constexpr size_t idx_bytes = (size_t)ENC_TILE * L;
+    static constexpr size_t off_r = cb_bytes;
+    static constexpr size_t off_xc = off_r + 2 * r_bytes;
+    static constexpr size_t off_idx = off_xc + xc_bytes;
+    static constexpr size_t off_pos = off_idx + idx_bytes;                          // [2][2][ENC_TILE] ints
+    static constexpr size_t off_mean = off_pos + 4 * ENC_TILE * sizeof(int);        // [D] doubles
+    static constexpr size_t total = off_mean + D * sizeof(double);
+    static_assert(total <= 232448, "shared memory budget");
+};
+
+// Tiled (prefill) encode, one CTA per (run of 64-token tiles, KV head, side), the codebook of the
+// (head, side) resident in shared memory.  The two phases of a tile use different units of the SM:
+// the binary64 transform runs on the fp64 pipe and the load/store unit, the 256-way search on the FMA
+// pipe.  Half of the warps therefore transform tile i+1 while the other half searches tile i
+// (coefficients double-buffered in shared memory, hand-over by named hardware barriers).
 template <int D>
 __global__ void __launch_bounds__(ENC_THREADS, 1)
 novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
@@ -116,15 +147,14 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                      const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                      int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
                      uint32_t* __restrict__ dev_status) {
-    constexpr int L = D / NOVAKV_G;
-    constexpr int RS = EncSmem<D>::RSTRIDE;
+    using P = EncPipe<D>;
+    constexpr int L = D / NOVAKV_G, RS = P::RS, XT = P::XT, NT = ENC_HALF_THREADS;
     extern __shared__ __align__(16) unsigned char smem[];
     float4* cb_s = reinterpret_cast<float4*>(smem);
-    double* xc_s = reinterpret_cast<double*>(smem + EncSmem<D>::cb_bytes);
-    float* r_s = reinterpret_cast<float*>(smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes);
-    uint8_t* idx_s = smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes + EncSmem<D>::r_bytes;
-    int* page_s = reinterpret_cast<int*>(idx_s + EncSmem<D>::idx_bytes);   // [ENC_TILE] page id or -1
-    int* slot_s = page_s + ENC_TILE;                                       // [ENC_TILE] slot in page
+    double* xc_s = reinterpret_cast<double*>(smem + P::off_xc);
+    uint8_t* idx_s = smem + P::off_idx;
+    int* pos_s = reinterpret_cast<int*>(smem + P::off_pos);                // [buf][page|slot][ENC_TILE]
+    double* mean_s = reinterpret_cast<double*>(smem + P::off_mean);
 
     const int kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
@@ -134,95 +164,124 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 
     // codebook of this (head, side) -> shared memory, once per CTA
     fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);
+    for (int i = threadIdx.x; i < D; i += ENC_THREADS) mean_s[i] = mean[i];
+    __syncthreads();
 
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
     const int tile0 = blockIdx.x * tiles_per_cta;
-    for (int tile = tile0; tile < min(n_tiles, tile0 + tiles_per_cta); ++tile) {
-        const int t0 = tile * ENC_TILE;
-        const int n_valid = min(ENC_TILE, n_tokens - t0);
-        __syncthreads();   // previous tile's readers are done (also orders the codebook fill)
+    const int n_local = max(0, min(n_tiles, tile0 + tiles_per_cta) - tile0);
+    const bool is_transform = threadIdx.x < NT;
+    const int tid = is_transform ? threadIdx.x : threadIdx.x - NT;
 
-        // destination of each token (validated once)
-        if (threadIdx.x < ENC_TILE) {
-            const int t = threadIdx.x;
-            int page = -1, slot = 0;
-            if (t < n_valid) {
-                const int s = tok_seq[t0 + t], pos = tok_pos[t0 + t];
-                if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
-                    atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
-                } else {
-                    page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
-                    slot = pos % NOVAKV_PAGE_TOKENS;
-                    if (page < 0 || page >= n_pages) {
-                        atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
-                        page = -1;
-                    } else if (kvh == 0 && side == 0) {
-                        atomicMax(&seq_lens[s], pos + 1);
+    if (is_transform) {
+        // ---------------- transform warps: fill r_s[buf] and the destinations of tile i ----------------
+        for (int i = 0; i < n_local; ++i) {
+            const int buf = i & 1;
+            const int t0 = (tile0 + i) * ENC_TILE;
+            const int n_valid = min(ENC_TILE, n_tokens - t0);
+            float* r_s = reinterpret_cast<float*>(smem + P::off_r + buf * P::r_bytes);
+            if (i >= 2) nbar_sync(BAR_EMPTY + buf, ENC_THREADS);          // the search of tile i-2 has released the buffer
+            if (tid < ENC_TILE) {                                          // destination of each token (validated once)
+                const int t = tid;
+                int page = -1, slot = 0;
+                if (t < n_valid) {
+                    const int s = tok_seq[t0 + t], pos = tok_pos[t0 + t];
+                    if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
+                        atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
+                    } else {
+                        page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
+                        slot = pos % NOVAKV_PAGE_TOKENS;
+                        if (page < 0 || page >= n_pages) {
+                            atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
+                            page = -1;
+                        } else if (kvh == 0 && side == 0) {
+                            atomicMax(&seq_lens[s], pos + 1);
+                        }
                     }
                 }
+                pos_s[(buf * 2 + 0) * ENC_TILE + t] = page;
+                pos_s[(buf * 2 + 1) * ENC_TILE + t] = slot;
             }
-            page_s[t] = page;
-            slot_s[t] = slot;
-        }
-
-        for (int half = 0; half < ENC_TILE / ENC_XT; ++half) {
-            const int tb = half * ENC_XT;
-            if (half > 0) __syncthreads();   // the previous pass no longer reads xc_s
-            // centred inputs in binary64: xc[t][i] = x[t][i] - mean[i]   (exact)
-            for (int i = threadIdx.x; i < ENC_XT * D; i += ENC_THREADS) {
-                const int t = i / D, c = i - t * D;
-                double x = 0.0;
-                if (tb + t < n_valid)
-                    x = (double)__bfloat162float(x_new[((size_t)(t0 + tb + t) * n_kv_heads + kvh) * D + c]) - mean[c];
-                xc_s[i] = x;
-            }
-            __syncthreads();
-            // transform: r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA in index order, rounded once to
-            // binary32.  Each thread owns 2 columns (c, c + D/2) x TM tokens and walks i two at a time, so
-            // that one 128-bit broadcast load of xc feeds 4 FMAs (the loop is shared-memory bound otherwise).
-            constexpr int HALF = D / 2;
-            constexpr int TSUB = ENC_THREADS / HALF;        // 8 (D=128) or 16 (D=64) token subsets
-            constexpr int TM = ENC_XT / TSUB;               // tokens per thread: 4 or 2
-            const int c = threadIdx.x % HALF, sub = threadIdx.x / HALF;
-            double acc0[TM], acc1[TM];
+            for (int pass = 0; pass < ENC_TILE / XT; ++pass) {
+                const int tb = pass * XT;
+                // centred inputs in binary64: xc[t][i] = x[t][i] - mean[i]   (exact); 8 bf16 per 128-bit load
+                for (int e = tid; e < XT * D / 8; e += NT) {
+                    const int t = e / (D / 8), c8 = (e - t * (D / 8)) * 8;
+                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                    const bool valid = tb + t < n_valid;
+                    if (valid) raw = *reinterpret_cast<const uint4*>(x_new + ((size_t)(t0 + tb + t) * n_kv_heads + kvh) * D + c8);
+                    const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&raw);
 #pragma unroll
-            for (int j = 0; j < TM; ++j) { acc0[j] = 0.0; acc1[j] = 0.0; }
-#pragma unroll 4
-            for (int i = 0; i < D; i += 2) {
-                const double ra0 = R[(size_t)i * D + c], rb0 = R[(size_t)i * D + c + HALF];
-                const double ra1 = R[(size_t)(i + 1) * D + c], rb1 = R[(size_t)(i + 1) * D + c + HALF];
+                    for (int j = 0; j < 8; j += 2) {
+                        double2 v;
+                        v.x = valid ? (double)__bfloat162float(xb[j]) - mean_s[c8 + j] : 0.0;
+                        v.y = valid ? (double)__bfloat162float(xb[j + 1]) - mean_s[c8 + j + 1] : 0.0;
+                        *reinterpret_cast<double2*>(xc_s + (size_t)t * D + c8 + j) = v;
+                    }
+                }
+                nbar_sync(BAR_T, NT);
+                // r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA in index order, rounded once to binary32.
+                // Each thread owns 2 columns (c, c + D/2) x TM tokens and walks i two at a time, so that one
+                // 128-bit broadcast load of xc feeds 4 FMAs.
+                constexpr int HALF = D / 2;
+                constexpr int TSUB = NT / HALF;                 // 4 (D=128) or 8 (D=64) token subsets
+                constexpr int TM = XT / TSUB;                   // tokens per thread: 4 or 2
+                const int c = tid % HALF, sub = tid / HALF;
+                double acc0[TM], acc1[TM];
+#pragma unroll
+                for (int j = 0; j < TM; ++j) { acc0[j] = 0.0; acc1[j] = 0.0; }
+                constexpr int KB = 8;                            // rows of R fetched per batch (16 loads in flight)
+#pragma unroll 1
+                for (int k0 = 0; k0 < D; k0 += KB) {
+                    double ra[KB], rb[KB];
+#pragma unroll
+                    for (int kk = 0; kk < KB; ++kk) {
+                        ra[kk] = R[(size_t)(k0 + kk) * D + c];
+                        rb[kk] = R[(size_t)(k0 + kk) * D + c + HALF];
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < KB; kk += 2) {
+#pragma unroll
+                        for (int j = 0; j < TM; ++j) {
+                            const double2 x = *reinterpret_cast<const double2*>(xc_s + (size_t)(sub + j * TSUB) * D + k0 + kk);
+                            acc0[j] = fma(x.x, ra[kk], acc0[j]);
+                            acc1[j] = fma(x.x, rb[kk], acc1[j]);
+                            acc0[j] = fma(x.y, ra[kk + 1], acc0[j]);
+                            acc1[j] = fma(x.y, rb[kk + 1], acc1[j]);
+                        }
+                    }
+                }
 #pragma unroll
                 for (int j = 0; j < TM; ++j) {
-                    const double2 x = *reinterpret_cast<const double2*>(xc_s + (size_t)(sub + j * TSUB) * D + i);
-                    acc0[j] = fma(x.x, ra0, acc0[j]);
-                    acc1[j] = fma(x.x, rb0, acc1[j]);
-                    acc0[j] = fma(x.y, ra1, acc0[j]);
-                    acc1[j] = fma(x.y, rb1, acc1[j]);
+                    r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc0[j];
+                    r_s[(size_t)(tb + sub + j * TSUB) * RS + c + HALF] = (float)acc1[j];
                 }
+                nbar_sync(BAR_T, NT);                            // xc_s may be refilled
             }
-#pragma unroll
-            for (int j = 0; j < TM; ++j) {
-                r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc0[j];
-                r_s[(size_t)(tb + sub + j * TSUB) * RS + c + HALF] = (float)acc1[j];
-            }
+            __threadfence_block();
+            nbar_arrive(BAR_FULL + buf, ENC_THREADS);            // hand tile i to the search warps
         }
-        __syncthreads();
-
-        search_tile<D>(r_s, cb_s, idx_s, n_valid);
-        __syncthreads();
-
-        // paged store
-        for (int i = threadIdx.x; i < n_valid * L; i += ENC_THREADS) {
-            const int t = i / L, l = i - t * L;
-            const int page = page_s[t];
-            if (page < 0) continue;
-            const int slot = slot_s[t];
-            const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
-            if (side == 0) {
-                k_pages[base + novakv_k_offset<L>(slot, l)] = idx_s[i];
-            } else {
-                v_pages[base + novakv_v_offset<L>(slot, l)] = idx_s[i];
+    } else {
+        // ---------------- search warps: nearest codewords of tile i, paged store ------------------------
+        for (int i = 0; i < n_local; ++i) {
+            const int buf = i & 1;
+            const int t0 = (tile0 + i) * ENC_TILE;
+            const int n_valid = min(ENC_TILE, n_tokens - t0);
+            const float* r_s = reinterpret_cast<const float*>(smem + P::off_r + buf * P::r_bytes);
+            nbar_sync(BAR_FULL + buf, ENC_THREADS);
+            search_tile<D>(r_s, cb_s, idx_s, n_valid, tid >> 5, NT / 32);
+            nbar_sync(BAR_S, NT);
+            for (int e = tid; e < n_valid * L; e += NT) {
+                const int t = e / L, l = e - t * L;
+                const int page = pos_s[(buf * 2 + 0) * ENC_TILE + t];
+                if (page < 0) continue;
+                const int slot = pos_s[(buf * 2 + 1) * ENC_TILE + t];
+                const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
+                if (side == 0) k_pages[base + novakv_k_offset<L>(slot, l)] = idx_s[e];
+                else v_pages[base + novakv_v_offset<L>(slot, l)] = idx_s[e];
             }
+            nbar_sync(BAR_S, NT);                                // idx_s and the buffer are free again
+            if (i + 2 < n_local) nbar_arrive(BAR_EMPTY + buf, ENC_THREADS);
         }
     }
 }
@@ -336,7 +395,7 @@ novakv_search_kernel(const float* __restrict__ coef, int n, const float* __restr
             r_s[(size_t)t * RS + c] = t < n_valid ? coef[((size_t)(t0 + t) * n_kv_heads + kvh) * D + c] : 0.f;
         }
         __syncthreads();
-        search_tile<D>(r_s, cb_s, idx_s, n_valid);
+        search_tile<D>(r_s, cb_s, idx_s, n_valid, threadIdx.x >> 5, ENC_THREADS / 32);
         __syncthreads();
         for (int i = threadIdx.x; i < n_valid * L; i += ENC_THREADS) {
             const int t = i / L, l = i - t * L;
@@ -362,7 +421,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
     }
     auto kern = novakv_encode_kernel<D>;
-    const size_t smem = EncSmem<D>::total;
+    const size_t smem = EncPipe<D>::total;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
     const int hs = ctx->cfg.n_kv_heads * 2;
