@@ -117,10 +117,10 @@ template <int D>
 struct EncPipe {
     static constexpr int L = D / NOVAKV_G;
     static constexpr int RS = D + 4;
-    static constexpr int XT = 16;                              // tokens per transform pass
+    static constexpr int XT = 32;                              // tokens per transform pass
     static constexpr size_t cb_bytes = (size_t)L * NOVAKV_C * NOVAKV_G * sizeof(float);
     static constexpr size_t r_bytes = (size_t)ENC_TILE * RS * sizeof(float);       // one buffer
-    static constexpr size_t xc_bytes = (size_t)XT * D * sizeof(double);
+    static constexpr size_t xc_bytes = (size_t)XT * (D / 2) * sizeof(double);   // half of the input dimension at a time
     static constexpr size_t idx_bytes = (size_t)ENC_TILE * L;
     static constexpr size_t off_r = cb_bytes;
     static constexpr size_t off_xc = off_r + 2 * r_bytes;
@@ -202,61 +202,65 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                 pos_s[(buf * 2 + 0) * ENC_TILE + t] = page;
                 pos_s[(buf * 2 + 1) * ENC_TILE + t] = slot;
             }
+            // r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA in index order, rounded once to binary32.
+            // A pass covers XT tokens; each thread owns 2 columns (c, c + D/2) x TM tokens and keeps their
+            // accumulators in registers while the input dimension is walked in two halves (the staging buffer
+            // holds XT x D/2 centred inputs), so the transform matrix is fetched once per XT tokens.
+            constexpr int HALF = D / 2;
+            constexpr int TSUB = NT / HALF;                 // 4 (D=128) or 8 (D=64) token subsets
+            constexpr int TM = XT / TSUB;                   // tokens per thread: 8 or 4
+            constexpr int KB = 4;                           // rows of R fetched per batch
+            const int c = tid % HALF, sub = tid / HALF;
             for (int pass = 0; pass < ENC_TILE / XT; ++pass) {
                 const int tb = pass * XT;
-                // centred inputs in binary64: xc[t][i] = x[t][i] - mean[i]   (exact); 8 bf16 per 128-bit load
-                for (int e = tid; e < XT * D / 8; e += NT) {
-                    const int t = e / (D / 8), c8 = (e - t * (D / 8)) * 8;
-                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-                    const bool valid = tb + t < n_valid;
-                    if (valid) raw = *reinterpret_cast<const uint4*>(x_new + ((size_t)(t0 + tb + t) * n_kv_heads + kvh) * D + c8);
-                    const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&raw);
-#pragma unroll
-                    for (int j = 0; j < 8; j += 2) {
-                        double2 v;
-                        v.x = valid ? (double)__bfloat162float(xb[j]) - mean_s[c8 + j] : 0.0;
-                        v.y = valid ? (double)__bfloat162float(xb[j + 1]) - mean_s[c8 + j + 1] : 0.0;
-                        *reinterpret_cast<double2*>(xc_s + (size_t)t * D + c8 + j) = v;
-                    }
-                }
-                nbar_sync(BAR_T, NT);
-                // r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA in index order, rounded once to binary32.
-                // Each thread owns 2 columns (c, c + D/2) x TM tokens and walks i two at a time, so that one
-                // 128-bit broadcast load of xc feeds 4 FMAs.
-                constexpr int HALF = D / 2;
-                constexpr int TSUB = NT / HALF;                 // 4 (D=128) or 8 (D=64) token subsets
-                constexpr int TM = XT / TSUB;                   // tokens per thread: 4 or 2
-                const int c = tid % HALF, sub = tid / HALF;
                 double acc0[TM], acc1[TM];
 #pragma unroll
                 for (int j = 0; j < TM; ++j) { acc0[j] = 0.0; acc1[j] = 0.0; }
-                constexpr int KB = 8;                            // rows of R fetched per batch (16 loads in flight)
 #pragma unroll 1
-                for (int k0 = 0; k0 < D; k0 += KB) {
-                    double ra[KB], rb[KB];
+                for (int kh = 0; kh < D; kh += HALF) {
+                    // centred inputs in binary64: xc[t][i - kh] = x[t][i] - mean[i]   (exact); 8 bf16 per 128-bit load
+                    for (int e = tid; e < XT * HALF / 8; e += NT) {
+                        const int t = e / (HALF / 8), c8 = (e - t * (HALF / 8)) * 8;
+                        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                        const bool valid = tb + t < n_valid;
+                        if (valid) raw = *reinterpret_cast<const uint4*>(x_new + ((size_t)(t0 + tb + t) * n_kv_heads + kvh) * D + kh + c8);
+                        const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&raw);
 #pragma unroll
-                    for (int kk = 0; kk < KB; ++kk) {
-                        ra[kk] = R[(size_t)(k0 + kk) * D + c];
-                        rb[kk] = R[(size_t)(k0 + kk) * D + c + HALF];
-                    }
-#pragma unroll
-                    for (int kk = 0; kk < KB; kk += 2) {
-#pragma unroll
-                        for (int j = 0; j < TM; ++j) {
-                            const double2 x = *reinterpret_cast<const double2*>(xc_s + (size_t)(sub + j * TSUB) * D + k0 + kk);
-                            acc0[j] = fma(x.x, ra[kk], acc0[j]);
-                            acc1[j] = fma(x.x, rb[kk], acc1[j]);
-                            acc0[j] = fma(x.y, ra[kk + 1], acc0[j]);
-                            acc1[j] = fma(x.y, rb[kk + 1], acc1[j]);
+                        for (int j = 0; j < 8; j += 2) {
+                            double2 v;
+                            v.x = valid ? (double)__bfloat162float(xb[j]) - mean_s[kh + c8 + j] : 0.0;
+                            v.y = valid ? (double)__bfloat162float(xb[j + 1]) - mean_s[kh + c8 + j + 1] : 0.0;
+                            *reinterpret_cast<double2*>(xc_s + (size_t)t * HALF + c8 + j) = v;
                         }
                     }
+                    nbar_sync(BAR_T, NT);
+#pragma unroll 1
+                    for (int k0 = 0; k0 < HALF; k0 += KB) {
+                        double ra[KB], rb[KB];
+#pragma unroll
+                        for (int kk = 0; kk < KB; ++kk) {
+                            ra[kk] = R[(size_t)(kh + k0 + kk) * D + c];
+                            rb[kk] = R[(size_t)(kh + k0 + kk) * D + c + HALF];
+                        }
+#pragma unroll
+                        for (int kk = 0; kk < KB; kk += 2) {
+#pragma unroll
+                            for (int j = 0; j < TM; ++j) {
+                                const double2 x = *reinterpret_cast<const double2*>(xc_s + (size_t)(sub + j * TSUB) * HALF + k0 + kk);
+                                acc0[j] = fma(x.x, ra[kk], acc0[j]);
+                                acc1[j] = fma(x.x, rb[kk], acc1[j]);
+                                acc0[j] = fma(x.y, ra[kk + 1], acc0[j]);
+                                acc1[j] = fma(x.y, rb[kk + 1], acc1[j]);
+                            }
+                        }
+                    }
+                    nbar_sync(BAR_T, NT);                        // xc_s may be refilled
                 }
 #pragma unroll
                 for (int j = 0; j < TM; ++j) {
                     r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc0[j];
                     r_s[(size_t)(tb + sub + j * TSUB) * RS + c + HALF] = (float)acc1[j];
                 }
-                nbar_sync(BAR_T, NT);                            // xc_s may be refilled
             }
             __threadfence_block();
             nbar_arrive(BAR_FULL + buf, ENC_THREADS);            // hand tile i to the search warps
