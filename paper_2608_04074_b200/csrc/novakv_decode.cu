@@ -83,8 +83,19 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                       const int32_t* __restrict__ seq_lens, int batch, int n_q_heads, int n_kv_heads,
                       int max_pages_per_seq, float scale_log2, float* __restrict__ qp,
                       int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status) {
-    novakv_grid_dependency_wait();
     const int blk = blockIdx.x;
+    constexpr int PARTS = 512 / D, ROWS = D / PARTS;
+    const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
+    const int c = threadIdx.x % D, part = threadIdx.x / D;
+    // this thread's slice of the (constant) transform is fetched before the grid-dependency wait, so the
+    // loads overlap the tail of the preceding kernel in the stream
+    float rv[ROWS];
+    if (blk < batch * n_kv_heads) {
+        const float* R = rk_inv_t + (size_t)kvh * D * D + (size_t)part * ROWS * D + c;
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) rv[r] = R[(size_t)r * D];
+    }
+    novakv_grid_dependency_wait();
     if (blk == batch * n_kv_heads) {
         // exclusive prefix over sequences of their page counts; small, done by one warp
         if (threadIdx.x < 32) {
@@ -111,18 +122,11 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         }
         return;
     }
-    constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     __shared__ float q_s[HG][D];
     __shared__ float red_s[PARTS][HG][D];
-    const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
     for (int i = threadIdx.x; i < HG * D; i += 512)
         q_s[i / D][i % D] = __bfloat162float(q[((size_t)b * n_q_heads + kvh * HG) * D + i]);
     __syncthreads();
-    const int c = threadIdx.x % D, part = threadIdx.x / D;
-    const float* R = rk_inv_t + (size_t)kvh * D * D + (size_t)part * ROWS * D + c;
-    float rv[ROWS];
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) rv[r] = R[(size_t)r * D];
     float acc[HG];
 #pragma unroll
     for (int h = 0; h < HG; ++h) acc[h] = 0.f;
@@ -241,11 +245,10 @@ __device__ __forceinline__ uint2 ldg_stream_64(const void* p) {
 
 // Segment prologue pieces, kept out of line so that their register-hungry load batches do not
 // disturb the register allocation of the scan loop.
-template <int D, int HG, bool VM>
-__device__ __noinline__ void load_value_codebook(unsigned char* smem, const __half* __restrict__ cb_v_img, int kvh) {
-    using C = S1<D, HG, VM>;
-    const uint4* src = reinterpret_cast<const uint4*>(cb_v_img + (size_t)kvh * (VCB_BYTES / 2));
-    uint4* dst = reinterpret_cast<uint4*>(smem + C::OFF_VCB);
+// 64 KB image (value codebook of a KV head, or one plane of its key codebook) -> shared memory.
+__device__ __noinline__ void stage_image_64k(unsigned char* dst_smem, const void* __restrict__ src_g) {
+    const uint4* src = reinterpret_cast<const uint4*>(src_g);
+    uint4* dst = reinterpret_cast<uint4*>(dst_smem);
     // all loads of a thread in flight before the first store (one L2 latency for the whole copy)
     constexpr int NV4 = (VCB_BYTES / 16 + S1_THREADS - 1) / S1_THREADS;
     uint4 tmp[NV4];
@@ -263,7 +266,8 @@ __device__ __noinline__ void load_value_codebook(unsigned char* smem, const __ha
 
 // LUT[hs][plane][code][e] = <q'_h segment of group l(e, plane), key codeword> for 4 heads per entry.
 template <int D, int HG, bool VM>
-__device__ __noinline__ void build_score_table(unsigned char* smem, const float* __restrict__ cb_k_lut, int kvh,
+__device__ __noinline__ void build_score_table(unsigned char* smem,
+                                               const float* __restrict__ cb_k_planes /* key codewords of the KV head, table order */,
                                                const float* __restrict__ q_pair /* q' of the pair's heads, [HG][D] */) {
     using C = S1<D, HG, VM>;
     constexpr int GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, PLANES = C::PLANES;
@@ -271,7 +275,7 @@ __device__ __noinline__ void build_score_table(unsigned char* smem, const float*
     constexpr int NIT = (256 + CPI - 1) / CPI;
     const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
     const int sigma = e & 7, mpar = e >> 3;
-    const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + (size_t)kvh * PLANES * 256 * 16;
+    const float4* cbk = reinterpret_cast<const float4*>(cb_k_planes);
     // every load of the thread (query segments and codewords of all planes) is issued before the first
     // use: one memory latency for the whole table
     float4 qseg[PLANES][HPAD];                    // heads beyond HG are zero
@@ -380,7 +384,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
         // ---- segment prologue -----------------------------------------------------------------
         if (vcb_head != sg.kvh) {
-            load_value_codebook<D, HG, VM>(smem, cb_v_img, sg.kvh);
+            stage_image_64k(smem + C::OFF_VCB, cb_v_img + (size_t)sg.kvh * (VCB_BYTES / 2));
             vcb_head = sg.kvh;
         }
 
@@ -425,7 +429,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         // (the first tile's loads are issued before, so that they fly during the table build)
         TileRegs<L> nxt;
         if (n_it > 0) load_tile(0, nxt);
-        build_score_table<D, HG, VM>(smem, cb_k_lut, sg.kvh, qp + ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D);
+        build_score_table<D, HG, VM>(smem, cb_k_lut + (size_t)sg.kvh * C::PLANES * (LUT_PLANE_BYTES / 4),
+                                     qp + ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D);
         __syncthreads();     // table and value codebook complete
 
         // ---- scan: 32-token tiles, loads of the next tile in flight while this one is consumed ------
@@ -680,17 +685,32 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 // ------------------------------------------------------------------------------------------------
 // merge + inverse value transform
 // ------------------------------------------------------------------------------------------------
-template <int D, int HG>
-__global__ void __launch_bounds__(HG * D > 512 ? 512 : HG * D)
+// MINB = resident blocks per SM the register budget allows for: 1 keeps the prefetched constants in
+// registers (lowest latency, small batches), 2 trades a few spills for occupancy (many pairs).
+template <int D, int HG, int MINB>
+__global__ void __launch_bounds__(HG * D > 512 ? 512 : HG * D, MINB)
 novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __restrict__ part_acc,
                            const int32_t* __restrict__ page_prefix, const int32_t* __restrict__ seq_lens,
                            int batch, int n_q_heads, int n_kv_heads, int max_pages_per_seq, int grid_s1,
                            const float* __restrict__ rv_t, const float* __restrict__ v_mean,
                            void* __restrict__ out, int out_is_fp32) {
     __shared__ float o_s[HG * D];
-    novakv_grid_dependency_wait();
+    constexpr int NT = HG * D > 512 ? 512 : HG * D;
+    constexpr int PARTS = NT / D, COLS = D / PARTS;
     const int pair = blockIdx.x;
     const int b = pair / n_kv_heads, kvh = pair - b * n_kv_heads;
+    // constants of the inverse transform are fetched before the grid-dependency wait (they overlap the
+    // tail of the scan kernel): this thread's slice of rv_t and the mean of its output coordinates
+    float rv[COLS];
+    {
+        const float* R = rv_t + (size_t)kvh * D * D + (size_t)(threadIdx.x / D) * COLS * D + threadIdx.x % D;   // rv_t[c][r] = R_V[r][c]
+#pragma unroll
+        for (int c = 0; c < COLS; ++c) rv[c] = R[(size_t)c * D];
+    }
+    float vm[(HG * D + NT - 1) / NT];
+#pragma unroll
+    for (int k = 0; k < (HG * D + NT - 1) / NT; ++k) vm[k] = v_mean[(size_t)kvh * D + (threadIdx.x + k * NT) % D];
+    novakv_grid_dependency_wait();
     const int len = clamp_len(seq_lens[b], max_pages_per_seq);
     const int pages_b = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
     const long P = page_prefix[batch], U = P * n_kv_heads;
@@ -722,8 +742,6 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
     }
     __syncthreads();
     // o_h = o'_h rv^T + v_mean: threads = D outputs x PARTS column parts, all HG heads share each load
-    constexpr int NT = HG * D > 512 ? 512 : HG * D;
-    constexpr int PARTS = NT / D, COLS = D / PARTS;
     __shared__ float red_s[PARTS][HG][D];
     {
         const int r = threadIdx.x % D, part = threadIdx.x / D;
@@ -731,10 +749,6 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
 #pragma unroll
         for (int h = 0; h < HG; ++h) acc[h] = 0.f;
         if (pages_b > 0) {
-            const float* R = rv_t + (size_t)kvh * D * D + (size_t)part * COLS * D + r;     // rv_t[c][r] = R_V[r][c]
-            float rv[COLS];
-#pragma unroll
-            for (int c = 0; c < COLS; ++c) rv[c] = R[(size_t)c * D];
 #pragma unroll
             for (int c = 0; c < COLS; ++c)
 #pragma unroll
@@ -744,13 +758,16 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         for (int h = 0; h < HG; ++h) red_s[part][h][r] = acc[h];
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < HG * D; i += blockDim.x) {
+#pragma unroll
+    for (int k = 0; k < (HG * D + NT - 1) / NT; ++k) {
+        const int i = threadIdx.x + k * NT;
+        if (i >= HG * D) break;
         const int h = i / D, r = i - h * D;
         float o = 0.f;
         if (pages_b > 0) {
 #pragma unroll
             for (int p = 0; p < PARTS; ++p) o += red_s[p][h][r];
-            o += v_mean[(size_t)kvh * D + r];
+            o += vm[k];
         }
         const size_t oi = ((size_t)b * n_q_heads + kvh * HG + h) * D + r;
         if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
@@ -809,7 +826,8 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         ps.end();
         ctx->launches++;
     }
-    novakv_launch_pdl(novakv_decode_merge_kernel<D, HG>, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
+    auto merge = batch * hkv > 2 * ctx->n_sm ? novakv_decode_merge_kernel<D, HG, 2> : novakv_decode_merge_kernel<D, HG, 1>;
+    novakv_launch_pdl(merge, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
                       part_ml, part_acc, prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out,
                       out_is_fp32);
     ctx->launches++;

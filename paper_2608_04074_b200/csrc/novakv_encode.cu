@@ -292,13 +292,19 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 
 // Append-sized batches (a decode step appends one token per sequence): the tiled kernel above would
 // pad every (head, side) to a 64-token tile and fill a 128 KB codebook per CTA.  Here one warp owns one
-// group of one (head, side): lanes are tokens, the warp stages only its 4 columns of the transform
-// (4 KB of binary64) and its group's codebook (4 KB), so the work spreads over L/4 * Hkv * 2 CTAs.
+// group of one (head, side) and stages only its 4 columns of the transform (4 KB of binary64) and its
+// group's codebook (4 KB), so the work spreads over L/4 * Hkv * 2 CTAs.  A pass covers tp tokens
+// (tp = 1, 2, ... 32, the smallest power of two that holds the batch, at most 32): lane = grp * tp + token.
+// The 32 / tp lane groups of a token compute the same coefficients (redundantly) and search disjoint
+// ranges of the codebook; their minima are merged with the lowest index winning ties.
+// Everything that depends only on the calibration is staged before the grid-dependency wait, so it
+// overlaps the tail of the preceding kernel in the stream.
 // Arithmetic is identical to the tiled kernel (binary64 accumulation in index order, dist4 search).
 template <int D>
 __global__ void __launch_bounds__(128)
 novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                            const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
+                           int tp_log2,
                            const double* __restrict__ rk_d, const double* __restrict__ rv_d,
                            const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
                            const float* __restrict__ cb_k, const float* __restrict__ cb_v,
@@ -306,72 +312,106 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                            const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                            int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
     constexpr int L = D / NOVAKV_G;
-    __shared__ double R_s[4][D][4];
+    __shared__ __align__(16) double R_s[4][D][4];
     __shared__ float4 cb_s[4][NOVAKV_C];
     __shared__ double mean_s[D];
-    novakv_grid_dependency_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int l = blockIdx.x * 4 + warp, kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
     const double* R = (side == 0 ? rk_d : rv_d) + (size_t)kvh * D * D;
     const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + ((size_t)kvh * L + l) * NOVAKV_C * NOVAKV_G);
-    for (int i = lane; i < D; i += 32) {
-        const double2 a = *reinterpret_cast<const double2*>(R + (size_t)i * D + l * 4);
-        const double2 b = *reinterpret_cast<const double2*>(R + (size_t)i * D + l * 4 + 2);
-        R_s[warp][i][0] = a.x; R_s[warp][i][1] = a.y; R_s[warp][i][2] = b.x; R_s[warp][i][3] = b.y;
+    {
+        // calibration constants -> shared memory; every load is issued before the first store
+        double2 ra[D / 32], rb[D / 32];
+        float4 cw[NOVAKV_C / 32];
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k) {
+            ra[k] = *reinterpret_cast<const double2*>(R + (size_t)(lane + 32 * k) * D + l * 4);
+            rb[k] = *reinterpret_cast<const double2*>(R + (size_t)(lane + 32 * k) * D + l * 4 + 2);
+        }
+#pragma unroll
+        for (int k = 0; k < NOVAKV_C / 32; ++k) cw[k] = cb_g[lane + 32 * k];
+        const double mv = threadIdx.x < D ? mean[threadIdx.x] : 0.0;
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k) {
+            *reinterpret_cast<double2*>(&R_s[warp][lane + 32 * k][0]) = ra[k];
+            *reinterpret_cast<double2*>(&R_s[warp][lane + 32 * k][2]) = rb[k];
+        }
+#pragma unroll
+        for (int k = 0; k < NOVAKV_C / 32; ++k) cb_s[warp][lane + 32 * k] = cw[k];
+        if (threadIdx.x < D) mean_s[threadIdx.x] = mv;
     }
-    for (int c = lane; c < NOVAKV_C; c += 32) cb_s[warp][c] = cb_g[c];
-    for (int i = threadIdx.x; i < D; i += 128) mean_s[i] = mean[i];
     __syncthreads();
+    novakv_grid_dependency_wait();           // inputs and the cache may be written by preceding kernels
 
-    for (int t0 = 0; t0 < n_tokens; t0 += 32) {
-        const int tkn = t0 + lane;
+    const int tp = 1 << tp_log2;
+    const int tok_in_pass = lane & (tp - 1), grp = lane >> tp_log2;
+    const int codes_per_grp = NOVAKV_C >> (5 - tp_log2);
+    const int c0 = grp * codes_per_grp;
+    const bool reporter = blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0 && grp == 0;
+
+    for (int t0 = 0; t0 < n_tokens; t0 += tp) {
+        const int tkn = t0 + tok_in_pass;
+        const bool in_range = tkn < n_tokens;
+        // this lane's token row (all loads in flight together with the destination lookup)
+        uint4 xr[D / 8];
+        const uint4* xrow = reinterpret_cast<const uint4*>(x_new + ((size_t)(in_range ? tkn : 0) * n_kv_heads + kvh) * D);
+#pragma unroll
+        for (int i8 = 0; i8 < D / 8; ++i8) xr[i8] = xrow[i8];
         int page = -1, slot = 0;
-        if (tkn < n_tokens) {
+        if (in_range) {
             const int s = tok_seq[tkn], pos = tok_pos[tkn];
             if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
-                if (blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0) atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
+                if (reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
             } else {
                 page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
                 slot = pos % NOVAKV_PAGE_TOKENS;
                 if (page < 0 || page >= n_pages) {
-                    if (blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0) atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
+                    if (reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
                     page = -1;
-                } else if (blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0) {
+                } else if (reporter) {
                     atomicMax(&seq_lens[s], pos + 1);
                 }
             }
         }
-        if (page < 0) continue;
         // coefficients of group l: binary64 accumulation over the input dimension in index order
         double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
-        const uint4* xrow = reinterpret_cast<const uint4*>(x_new + ((size_t)tkn * n_kv_heads + kvh) * D);
-#pragma unroll 2
+#pragma unroll
         for (int i8 = 0; i8 < D / 8; ++i8) {
-            const uint4 raw = xrow[i8];
-            const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&raw);
+            const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&xr[i8]);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int i = i8 * 8 + j;
                 const double xc = (double)__bfloat162float(xb[j]) - mean_s[i];
-                acc0 = fma(xc, R_s[warp][i][0], acc0);
-                acc1 = fma(xc, R_s[warp][i][1], acc1);
-                acc2 = fma(xc, R_s[warp][i][2], acc2);
-                acc3 = fma(xc, R_s[warp][i][3], acc3);
+                const double2 r01 = *reinterpret_cast<const double2*>(&R_s[warp][i][0]);
+                const double2 r23 = *reinterpret_cast<const double2*>(&R_s[warp][i][2]);
+                acc0 = fma(xc, r01.x, acc0);
+                acc1 = fma(xc, r01.y, acc1);
+                acc2 = fma(xc, r23.x, acc2);
+                acc3 = fma(xc, r23.y, acc3);
             }
         }
         const float4 r = make_float4((float)acc0, (float)acc1, (float)acc2, (float)acc3);
-        float best = dist4(r, cb_s[warp][0]);
-        int bi = 0;
+        // this lane group's range of the codebook, ascending with a strict '<' (first minimum)
+        float best = dist4(r, cb_s[warp][c0]);
+        int bi = c0;
 #pragma unroll 8
-        for (int c = 1; c < NOVAKV_C; ++c) {
-            const float dd = dist4(r, cb_s[warp][c]);
-            if (dd < best) { best = dd; bi = c; }
+        for (int c = 1; c < codes_per_grp; ++c) {
+            const float dd = dist4(r, cb_s[warp][c0 + c]);
+            if (dd < best) { best = dd; bi = c0 + c; }
         }
-        const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
-        if (side == 0) k_pages[base + novakv_k_offset<L>(slot, l)] = (uint8_t)bi;
-        else v_pages[base + novakv_v_offset<L>(slot, l)] = (uint8_t)bi;
+        // merge the groups of a token: smaller distance wins, equal distances keep the lower index
+        for (int off = tp; off < 32; off <<= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        }
+        if (grp == 0 && page >= 0) {
+            const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
+            if (side == 0) k_pages[base + novakv_k_offset<L>(slot, l)] = (uint8_t)bi;
+            else v_pages[base + novakv_v_offset<L>(slot, l)] = (uint8_t)bi;
+        }
     }
 }
 
@@ -417,8 +457,10 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS) {
         dim3 grid(D / NOVAKV_G / 4, ctx->cfg.n_kv_heads, 2);
         novakv_prof_scope ps(ctx, 1, stream);
+        int tp_log2 = 0;
+        while ((1 << tp_log2) < n_tokens && tp_log2 < 5) ++tp_log2;
         novakv_launch_pdl(novakv_encode_small_kernel<D>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos, n_tokens,
-                          ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
+                          tp_log2, ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
                           page_table, max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads, ctx->dev_status);
         ps.end();
         ctx->launches++;

@@ -89,9 +89,11 @@ novakv_status novakv_launch_bf16_decode(novakv_ctx* ctx, const __nv_bfloat16* q,
 
 // Programmatic dependent launch: a kernel launched with novakv_launch_pdl may be scheduled while its
 // predecessor in the stream is still running; it must call novakv_grid_dependency_wait() before it
-// touches anything the predecessor reads or writes (every kernel here does so first thing), which
-// blocks until the predecessor grid has completed and its writes are visible.  Only the launch latency
-// is hidden; there is no unbounded wait in user code.
+// touches anything a preceding kernel may write, which blocks until the predecessor grid has completed
+// and its writes are visible.  Before the wait a kernel only reads calibration constants (uploaded
+// synchronously by novakv_load_calibration, never written by a kernel) into registers or its own shared
+// memory, so the launch latency and that staging overlap the predecessor's tail.  There is no unbounded
+// wait in user code.
 __device__ __forceinline__ void novakv_grid_dependency_wait() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
