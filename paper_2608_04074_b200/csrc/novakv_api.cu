@@ -63,6 +63,7 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
 
 static void free_layer(novakv_layer& ly) {
     cudaFree(ly.rk_d); cudaFree(ly.rv_d); cudaFree(ly.k_mean_d); cudaFree(ly.v_mean_d);
+    cudaFree(ly.rk_d_mma); cudaFree(ly.rv_d_mma);
     cudaFree(ly.cb_k); cudaFree(ly.cb_v); cudaFree(ly.rk_inv_t); cudaFree(ly.rv_t);
     cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_half); cudaFree(ly.cb_v_mma);
     ly = novakv_layer();
@@ -124,6 +125,15 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
     std::vector<double> rk_d(n_mat), rv_d(n_mat), km_d(n_vec, 0.0), vm_d(n_vec, 0.0);
     std::vector<float> vm_f(n_vec, 0.f);
     for (size_t i = 0; i < n_mat; ++i) { rk_d[i] = (double)h->rk[i]; rv_d[i] = (double)h->rv[i]; }
+    // the same matrices with the input dimension blocked by 4: img[h][k/4][c][k%4] = R[h][k][c]
+    std::vector<double> rk_mma(n_mat), rv_mma(n_mat);
+    for (int hh = 0; hh < H; ++hh)
+        for (int k = 0; k < d; ++k)
+            for (int c = 0; c < d; ++c) {
+                const size_t dst = (((size_t)hh * (d / 4) + k / 4) * d + c) * 4 + k % 4, src = ((size_t)hh * d + k) * d + c;
+                rk_mma[dst] = rk_d[src];
+                rv_mma[dst] = rv_d[src];
+            }
     if (h->k_mean) for (size_t i = 0; i < n_vec; ++i) km_d[i] = (double)h->k_mean[i];
     if (h->v_mean) for (size_t i = 0; i < n_vec; ++i) { vm_d[i] = (double)h->v_mean[i]; vm_f[i] = h->v_mean[i]; }
 
@@ -151,6 +161,7 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
         for (int r = 0; r < d; ++r)
             for (int c = 0; c < d; ++c) rvt[((size_t)hh * d + c) * d + r] = h->rv[((size_t)hh * d + r) * d + c];
     bool ok = upload(&ly.rk_d, rk_d) == cudaSuccess && upload(&ly.rv_d, rv_d) == cudaSuccess &&
+              upload(&ly.rk_d_mma, rk_mma) == cudaSuccess && upload(&ly.rv_d_mma, rv_mma) == cudaSuccess &&
               upload(&ly.k_mean_d, km_d) == cudaSuccess && upload(&ly.v_mean_d, vm_d) == cudaSuccess &&
               upload(&ly.cb_k, cbk) == cudaSuccess && upload(&ly.cb_v, cbv) == cudaSuccess &&
               upload(&ly.rk_inv_t, rkinv) == cudaSuccess && upload(&ly.rv_t, rvt) == cudaSuccess &&

@@ -58,9 +58,20 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
 // Distances of one coefficient vector (each component duplicated into a pair) to two codewords at once:
 // cw[i] = (codeword c, component i ; codeword c+1, component i).  Same chain as dist4, per half.
 __device__ __forceinline__ void dist4x2(const uint64_t (&r2)[4], const uint64_t (&cw)[4], float& d0, float& d1) {
+#ifdef NOVAKV_SCALAR_SEARCH
+    float r[4], lo[4], hi[4], dummy;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        asm("mov.b64 {%0,%1}, %2;" : "=f"(r[i]), "=f"(dummy) : "l"(r2[i]));
+        asm("mov.b64 {%0,%1}, %2;" : "=f"(lo[i]), "=f"(hi[i]) : "l"(cw[i]));
+    }
+    d0 = dist4(make_float4(r[0], r[1], r[2], r[3]), make_float4(lo[0], lo[1], lo[2], lo[3]));
+    d1 = dist4(make_float4(r[0], r[1], r[2], r[3]), make_float4(hi[0], hi[1], hi[2], hi[3]));
+#else
     const uint64_t e0 = sub2(r2[0], cw[0]), e1 = sub2(r2[1], cw[1]), e2 = sub2(r2[2], cw[2]), e3 = sub2(r2[3], cw[3]);
     const uint64_t d = fma2(e3, e3, fma2(e2, e2, fma2(e1, e1, mul2(e0, e0))));
     asm("mov.b64 {%0,%1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+#endif
 }
 
 // Shared-memory image of a (head, side) codebook for the search: [L][128 codeword pairs][4 components][2].
@@ -72,9 +83,20 @@ __device__ __forceinline__ void fill_codebook_pairs(float* cb_s, const float4* _
     }
 }
 
+__device__ __forceinline__ float fmin3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Search of the tile's coefficients (r_s, [ENC_TILE][RSTRIDE] float) against the paired codebook image.
-// Warp w of n_warps owns groups w, w+n_warps, ...; lane t owns tokens t and t+32.  Codewords are visited in ascending
-// index with a strict '<', which keeps the first minimum.
+// Warp w of n_warps owns groups w, w+n_warps, ...; lane t owns tokens t and t+32.
+// The result is the first minimum in ascending codeword order (what a scan with a strict '<' keeps), found in
+// two steps that need far fewer compare/select instructions than a per-codeword running argmin:
+//   1. blocks of 8 codewords: the block minimum (a tree of 3-input minima) updates the running minimum with a
+//      strict '<', which keeps the first block that attains the overall minimum;
+//   2. the 8 distances of that block are recomputed (same instructions, same bits) and the first one equal to
+//      the minimum gives the index.
 template <int D>
 __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s, uint8_t* idx_s, int n_valid,
                                             int warp, int n_warps) {
@@ -87,19 +109,41 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
         const uint64_t ra2[4] = {pk2(ra.x, ra.x), pk2(ra.y, ra.y), pk2(ra.z, ra.z), pk2(ra.w, ra.w)};
         const uint64_t rb2[4] = {pk2(rb.x, rb.x), pk2(rb.y, rb.y), pk2(rb.z, rb.z), pk2(rb.w, rb.w)};
         float best_a = CUDART_INF_F, best_b = CUDART_INF_F;
-        int ia = 0, ib = 0;
+        int blk_a = 0, blk_b = 0;
         const ulonglong2* cb = reinterpret_cast<const ulonglong2*>(cb_s) + (size_t)l * NOVAKV_C;   // 2 x 16 B per pair
-#pragma unroll 4
-        for (int p = 0; p < NOVAKV_C / 2; ++p) {
-            const ulonglong2 q0 = cb[2 * p], q1 = cb[2 * p + 1];
-            const uint64_t cw[4] = {q0.x, q0.y, q1.x, q1.y};
-            float a0, a1, b0, b1;
-            dist4x2(ra2, cw, a0, a1);
-            dist4x2(rb2, cw, b0, b1);
-            if (a0 < best_a) { best_a = a0; ia = 2 * p; }
-            if (a1 < best_a) { best_a = a1; ia = 2 * p + 1; }
-            if (b0 < best_b) { best_b = b0; ib = 2 * p; }
-            if (b1 < best_b) { best_b = b1; ib = 2 * p + 1; }
+#pragma unroll 2
+        for (int blk = 0; blk < NOVAKV_C / 8; ++blk) {
+            float da[8], db[8];
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                const ulonglong2 q0 = cb[8 * blk + 2 * p], q1 = cb[8 * blk + 2 * p + 1];
+                const uint64_t cw[4] = {q0.x, q0.y, q1.x, q1.y};
+                dist4x2(ra2, cw, da[2 * p], da[2 * p + 1]);
+                dist4x2(rb2, cw, db[2 * p], db[2 * p + 1]);
+            }
+            const float ma = fmin3(fmin3(da[0], da[1], da[2]), fmin3(da[3], da[4], da[5]), fminf(da[6], da[7]));
+            const float mb = fmin3(fmin3(db[0], db[1], db[2]), fmin3(db[3], db[4], db[5]), fminf(db[6], db[7]));
+            if (ma < best_a) { best_a = ma; blk_a = blk; }
+            if (mb < best_b) { best_b = mb; blk_b = blk; }
+        }
+        // the winning blocks again: first codeword whose distance equals the minimum
+        int ia = 8 * blk_a, ib = 8 * blk_b;
+        {
+            float da[8], db[8];
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                const ulonglong2 qa0 = cb[8 * blk_a + 2 * p], qa1 = cb[8 * blk_a + 2 * p + 1];
+                const uint64_t cwa[4] = {qa0.x, qa0.y, qa1.x, qa1.y};
+                dist4x2(ra2, cwa, da[2 * p], da[2 * p + 1]);
+                const ulonglong2 qb0 = cb[8 * blk_b + 2 * p], qb1 = cb[8 * blk_b + 2 * p + 1];
+                const uint64_t cwb[4] = {qb0.x, qb0.y, qb1.x, qb1.y};
+                dist4x2(rb2, cwb, db[2 * p], db[2 * p + 1]);
+            }
+#pragma unroll
+            for (int k = 7; k >= 0; --k) {
+                if (da[k] == best_a) ia = 8 * blk_a + k;
+                if (db[k] == best_b) ib = 8 * blk_b + k;
+            }
         }
         if (lane < n_valid) idx_s[lane * L + l] = (uint8_t)ia;
         if (lane + 32 < n_valid) idx_s[(lane + 32) * L + l] = (uint8_t)ib;
@@ -117,14 +161,16 @@ template <int D>
 struct EncPipe {
     static constexpr int L = D / NOVAKV_G;
     static constexpr int RS = D + 4;
-    static constexpr int XT = 32;                              // tokens per transform pass
+    static constexpr int KS = 8;                               // rows of the transform matrix per slab
     static constexpr size_t cb_bytes = (size_t)L * NOVAKV_C * NOVAKV_G * sizeof(float);
     static constexpr size_t r_bytes = (size_t)ENC_TILE * RS * sizeof(float);       // one buffer
-    static constexpr size_t xc_bytes = (size_t)XT * (D / 2) * sizeof(double);   // half of the input dimension at a time
+    static constexpr size_t slab_x_bytes = (size_t)ENC_TILE * KS * sizeof(double);  // centred inputs [64][KS]
+    static constexpr size_t slab_r_bytes = (size_t)KS * D * sizeof(double);         // KS rows of R
+    static constexpr size_t slab_bytes = slab_x_bytes + slab_r_bytes;
     static constexpr size_t idx_bytes = (size_t)ENC_TILE * L;
     static constexpr size_t off_r = cb_bytes;
-    static constexpr size_t off_xc = off_r + 2 * r_bytes;
-    static constexpr size_t off_idx = off_xc + xc_bytes;
+    static constexpr size_t off_slab = off_r + 2 * r_bytes;                         // 2 slab buffers
+    static constexpr size_t off_idx = off_slab + 2 * slab_bytes;
     static constexpr size_t off_pos = off_idx + idx_bytes;                          // [2][2][ENC_TILE] ints
     static constexpr size_t off_mean = off_pos + 4 * ENC_TILE * sizeof(int);        // [D] doubles
     static constexpr size_t total = off_mean + D * sizeof(double);
@@ -148,17 +194,16 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                      int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
                      uint32_t* __restrict__ dev_status) {
     using P = EncPipe<D>;
-    constexpr int L = D / NOVAKV_G, RS = P::RS, XT = P::XT, NT = ENC_HALF_THREADS;
+    constexpr int L = D / NOVAKV_G, RS = P::RS, NT = ENC_HALF_THREADS;
     extern __shared__ __align__(16) unsigned char smem[];
     float4* cb_s = reinterpret_cast<float4*>(smem);
-    double* xc_s = reinterpret_cast<double*>(smem + P::off_xc);
     uint8_t* idx_s = smem + P::off_idx;
     int* pos_s = reinterpret_cast<int*>(smem + P::off_pos);                // [buf][page|slot][ENC_TILE]
     double* mean_s = reinterpret_cast<double*>(smem + P::off_mean);
 
     const int kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
-    const double* R = (side == 0 ? rk_d : rv_d) + (size_t)kvh * D * D;
+    const double* R = (side == 0 ? rk_d : rv_d) + (size_t)kvh * D * D;      // fragment order [d/4][d][4]
     const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
 
@@ -175,93 +220,108 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 
     if (is_transform) {
         // ---------------- transform warps: fill r_s[buf] and the destinations of tile i ----------------
+        // r[t][c] = sum_i xc[t][i] R[i][c] in binary64 on the tensor cores (mma.sync m8n8k4, f64): exact
+        // products, binary64 accumulation in blocks of 4 input dimensions taken in index order, one rounding
+        // to binary32 at the end.  Warp w owns the 16 columns 16w .. 16w+15 of all 64 tokens: 8 x 2 fragments
+        // of 8 tokens x 8 columns, 2 accumulator registers each.  The input dimension is walked in slabs of
+        // KS rows: a slab is KS rows of R in fragment order (one contiguous block, asynchronous copy) and the
+        // centred inputs xc[64][KS]; slabs are double buffered and slab s + 1 is fetched while slab s is
+        // consumed, one barrier of the transform warps per slab.
+        constexpr int KS = P::KS, NSLAB = D / KS;
+        constexpr int NWT = NT / 32;                    // transform warps
+        constexpr int NTILE_N = D / 8 / NWT;            // column fragments per warp: 2 (D=128) or 1 (D=64)
+        constexpr int NTILE_M = ENC_TILE / 8;           // token fragments: 8
+        static_assert(NSLAB % 2 == 0 && ENC_TILE * KS / 2 == NT && NTILE_N >= 1, "slab mapping");
+        const int wt = tid >> 5, lane = tid & 31, fr = lane >> 2, fk = lane & 3;
+        const int xt = tid / (KS / 2), xk = (tid % (KS / 2)) * 2;      // this thread's two inputs of a slab
+        uint32_t xraw = 0u;
+        auto slab_issue = [&](int tile_t0, int tile_valid, int sl) {
+            unsigned char* buf_b = smem + P::off_slab + (sl & 1) * P::slab_bytes;
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(buf_b + P::slab_x_bytes);
+            const char* src = reinterpret_cast<const char*>(R + (size_t)sl * KS * D);
+#pragma unroll
+            for (int q = 0; q < (int)(P::slab_r_bytes / 16 / NT); ++q)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (tid + q * NT) * 16),
+                             "l"(src + (size_t)(tid + q * NT) * 16) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            xraw = 0u;
+            if (xt < tile_valid)
+                xraw = *reinterpret_cast<const uint32_t*>(x_new + ((size_t)(tile_t0 + xt) * n_kv_heads + kvh) * D + sl * KS + xk);
+        };
+        if (n_local > 0) slab_issue(tile0 * ENC_TILE, min(ENC_TILE, n_tokens - tile0 * ENC_TILE), 0);
         for (int i = 0; i < n_local; ++i) {
             const int buf = i & 1;
             const int t0 = (tile0 + i) * ENC_TILE;
             const int n_valid = min(ENC_TILE, n_tokens - t0);
             float* r_s = reinterpret_cast<float*>(smem + P::off_r + buf * P::r_bytes);
+            // destination of each token (validated once); written to shared memory when the buffer is free
+            int page = -1, slot = 0;
+            if (tid < n_valid) {
+                const int sq = tok_seq[t0 + tid], pos = tok_pos[t0 + tid];
+                if (sq < 0 || sq >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
+                    atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
+                } else {
+                    page = page_table[(size_t)sq * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
+                    slot = pos % NOVAKV_PAGE_TOKENS;
+                    if (page < 0 || page >= n_pages) {
+                        atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
+                        page = -1;
+                    } else if (kvh == 0 && side == 0) {
+                        atomicMax(&seq_lens[sq], pos + 1);
+                    }
+                }
+            }
+            double acc[NTILE_M][NTILE_N][2];
+#pragma unroll
+            for (int mt = 0; mt < NTILE_M; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NTILE_N; ++nt) { acc[mt][nt][0] = 0.0; acc[mt][nt][1] = 0.0; }
+#pragma unroll 1
+            for (int sl = 0; sl < NSLAB; ++sl) {
+                unsigned char* buf_b = smem + P::off_slab + (sl & 1) * P::slab_bytes;
+                double* xs = reinterpret_cast<double*>(buf_b);
+                const double* Rs = reinterpret_cast<const double*>(buf_b + P::slab_x_bytes);
+                // slab sl: its rows of R have landed, its inputs are centred in binary64 (exact) and stored
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                {
+                    const __nv_bfloat162 xb = *reinterpret_cast<const __nv_bfloat162*>(&xraw);
+                    const bool valid = xt < n_valid;
+                    double2 v;
+                    v.x = valid ? (double)__bfloat162float(xb.x) - mean_s[sl * KS + xk] : 0.0;
+                    v.y = valid ? (double)__bfloat162float(xb.y) - mean_s[sl * KS + xk + 1] : 0.0;
+                    *reinterpret_cast<double2*>(xs + ((size_t)(xk >> 2) * ENC_TILE + xt) * 4 + (xk & 3)) = v;   // [k/4][t][k%4]
+                }
+                nbar_sync(BAR_T, NT);       // slab sl visible; everyone is done with slab sl - 1 (the other buffer)
+                if (sl + 1 < NSLAB) slab_issue(t0, n_valid, sl + 1);
+                else if (i + 1 < n_local) slab_issue(t0 + ENC_TILE, min(ENC_TILE, n_tokens - t0 - ENC_TILE), 0);
+#pragma unroll
+                for (int kq = 0; kq < KS / 4; ++kq) {
+                    // B fragments: R[4 kq + fk][column 16 wt + 8 nt + fr]; A fragments: xc[token 8 mt + fr][4 kq + fk]
+                    double bf[NTILE_N];
+#pragma unroll
+                    for (int nt = 0; nt < NTILE_N; ++nt) bf[nt] = Rs[((size_t)kq * D + (wt * NTILE_N + nt) * 8 + fr) * 4 + fk];
+#pragma unroll
+                    for (int mt = 0; mt < NTILE_M; ++mt) {
+                        const double af = xs[((size_t)kq * ENC_TILE + mt * 8 + fr) * 4 + fk];
+#pragma unroll
+                        for (int nt = 0; nt < NTILE_N; ++nt)
+                            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                         : "+d"(acc[mt][nt][0]), "+d"(acc[mt][nt][1]) : "d"(af), "d"(bf[nt]));
+                    }
+                }
+            }
             if (i >= 2) nbar_sync(BAR_EMPTY + buf, ENC_THREADS);          // the search of tile i-2 has released the buffer
-            if (tid < ENC_TILE) {                                          // destination of each token (validated once)
-                const int t = tid;
-                int page = -1, slot = 0;
-                if (t < n_valid) {
-                    const int s = tok_seq[t0 + t], pos = tok_pos[t0 + t];
-                    if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
-                        atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
-                    } else {
-                        page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
-                        slot = pos % NOVAKV_PAGE_TOKENS;
-                        if (page < 0 || page >= n_pages) {
-                            atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
-                            page = -1;
-                        } else if (kvh == 0 && side == 0) {
-                            atomicMax(&seq_lens[s], pos + 1);
-                        }
-                    }
-                }
-                pos_s[(buf * 2 + 0) * ENC_TILE + t] = page;
-                pos_s[(buf * 2 + 1) * ENC_TILE + t] = slot;
+            if (tid < ENC_TILE) {
+                pos_s[(buf * 2 + 0) * ENC_TILE + tid] = page;
+                pos_s[(buf * 2 + 1) * ENC_TILE + tid] = slot;
             }
-            // r[t][c] = sum_i xc[t][i] R[i][c], binary64 FMA in index order, rounded once to binary32.
-            // A pass covers XT tokens; each thread owns 2 columns (c, c + D/2) x TM tokens and keeps their
-            // accumulators in registers while the input dimension is walked in two halves (the staging buffer
-            // holds XT x D/2 centred inputs), so the transform matrix is fetched once per XT tokens.
-            constexpr int HALF = D / 2;
-            constexpr int TSUB = NT / HALF;                 // 4 (D=128) or 8 (D=64) token subsets
-            constexpr int TM = XT / TSUB;                   // tokens per thread: 8 or 4
-            constexpr int KB = 4;                           // rows of R fetched per batch
-            const int c = tid % HALF, sub = tid / HALF;
-            for (int pass = 0; pass < ENC_TILE / XT; ++pass) {
-                const int tb = pass * XT;
-                double acc0[TM], acc1[TM];
+            // accumulator fragment: token 8 mt + fr, columns 16 wt + 8 nt + 2 fk, + 1
 #pragma unroll
-                for (int j = 0; j < TM; ++j) { acc0[j] = 0.0; acc1[j] = 0.0; }
-#pragma unroll 1
-                for (int kh = 0; kh < D; kh += HALF) {
-                    // centred inputs in binary64: xc[t][i - kh] = x[t][i] - mean[i]   (exact); 8 bf16 per 128-bit load
-                    for (int e = tid; e < XT * HALF / 8; e += NT) {
-                        const int t = e / (HALF / 8), c8 = (e - t * (HALF / 8)) * 8;
-                        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-                        const bool valid = tb + t < n_valid;
-                        if (valid) raw = *reinterpret_cast<const uint4*>(x_new + ((size_t)(t0 + tb + t) * n_kv_heads + kvh) * D + kh + c8);
-                        const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&raw);
+            for (int mt = 0; mt < NTILE_M; ++mt)
 #pragma unroll
-                        for (int j = 0; j < 8; j += 2) {
-                            double2 v;
-                            v.x = valid ? (double)__bfloat162float(xb[j]) - mean_s[kh + c8 + j] : 0.0;
-                            v.y = valid ? (double)__bfloat162float(xb[j + 1]) - mean_s[kh + c8 + j + 1] : 0.0;
-                            *reinterpret_cast<double2*>(xc_s + (size_t)t * HALF + c8 + j) = v;
-                        }
-                    }
-                    nbar_sync(BAR_T, NT);
-#pragma unroll 1
-                    for (int k0 = 0; k0 < HALF; k0 += KB) {
-                        double ra[KB], rb[KB];
-#pragma unroll
-                        for (int kk = 0; kk < KB; ++kk) {
-                            ra[kk] = R[(size_t)(kh + k0 + kk) * D + c];
-                            rb[kk] = R[(size_t)(kh + k0 + kk) * D + c + HALF];
-                        }
-#pragma unroll
-                        for (int kk = 0; kk < KB; kk += 2) {
-#pragma unroll
-                            for (int j = 0; j < TM; ++j) {
-                                const double2 x = *reinterpret_cast<const double2*>(xc_s + (size_t)(sub + j * TSUB) * HALF + k0 + kk);
-                                acc0[j] = fma(x.x, ra[kk], acc0[j]);
-                                acc1[j] = fma(x.x, rb[kk], acc1[j]);
-                                acc0[j] = fma(x.y, ra[kk + 1], acc0[j]);
-                                acc1[j] = fma(x.y, rb[kk + 1], acc1[j]);
-                            }
-                        }
-                    }
-                    nbar_sync(BAR_T, NT);                        // xc_s may be refilled
-                }
-#pragma unroll
-                for (int j = 0; j < TM; ++j) {
-                    r_s[(size_t)(tb + sub + j * TSUB) * RS + c] = (float)acc0[j];
-                    r_s[(size_t)(tb + sub + j * TSUB) * RS + c + HALF] = (float)acc1[j];
-                }
-            }
+                for (int nt = 0; nt < NTILE_N; ++nt)
+                    *reinterpret_cast<float2*>(r_s + (size_t)(mt * 8 + fr) * RS + (wt * NTILE_N + nt) * 8 + 2 * fk) =
+                        make_float2((float)acc[mt][nt][0], (float)acc[mt][nt][1]);
             __threadfence_block();
             nbar_arrive(BAR_FULL + buf, ENC_THREADS);            // hand tile i to the search warps
         }
@@ -486,7 +546,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     }
     dim3 grid(ctas_x, ctx->cfg.n_kv_heads, 2);
     novakv_prof_scope ps(ctx, 1, stream);
-    kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d, ly.rv_d,
+    kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d_mma, ly.rv_d_mma,
                                                ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
                                                page_table, max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads,
                                                tiles_per_cta, ctx->dev_status);

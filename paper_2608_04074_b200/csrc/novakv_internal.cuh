@@ -20,6 +20,8 @@ struct novakv_layer {
     // write path (binary64 transforms, see the encode entry of the public header)
     double* rk_d = nullptr;       // [Hkv][d][d]
     double* rv_d = nullptr;       // [Hkv][d][d]
+    double* rk_d_mma = nullptr;   // [Hkv][d/4][d][4]: rk_d with the input dimension blocked by 4 (tensor-core fragments)
+    double* rv_d_mma = nullptr;   // same for rv_d
     double* k_mean_d = nullptr;   // [Hkv][d]
     double* v_mean_d = nullptr;   // [Hkv][d]
     float* cb_k = nullptr;        // [Hkv][L][256][4]  search layout
