@@ -28,8 +28,11 @@
  * Pins (tests/test_oracle_pins.py): exact invariance of the attention products when the
  * quantiser is the identity, generalised Parseval relation (Prop. 1), Lemma S1, one-token
  * and equal-logit caches, brute force against an independently written search, hand-built
- * tie cases, split invariance, planted needle.  No end-to-end numeric value is printed in
- * the paper, so the numeric end-to-end parity is pinned by those identities only.
+ * tie cases, split invariance, planted needle; for the scaled key format: power-of-two
+ * equivariance, unit RMS of the normalised coefficients, reduction to the unscaled encoder at
+ * rho = 1, linearity of the reconstruction in rho, the paper's bit-rate arithmetic.  No
+ * end-to-end numeric value is printed in the paper, so the numeric end-to-end parity is pinned
+ * by those identities only.
  */
 #include <math.h>
 #include <stdint.h>
@@ -253,6 +256,124 @@ void oracle_decode(const oracle_tables* t, const double* q, const uint8_t* kidx,
     double* k_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
     double* v_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
     oracle_reconstruct(t, kidx, vidx, S, k_hat, v_hat);
+    oracle_attention(q, k_hat, v_hat, S, Hq, H, d, sm_scale, out);
+    free(k_hat);
+    free(v_hat);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Key format with a per-token scale (Algorithm "Codebook training", the "Normalize" step; App. B
+ * "Decoding kernel and read path": the kernel "applies the per-token scale rho_j recovered from
+ * metadata (one multiply)"; Sec. 5 "Bit rate": a BF16 scale per token, 16/128 = 0.125 bit/elem).
+ *
+ *   rho_j = ||r_j||_2 / sqrt(d),   r_j <- r_j / rho_j   before the codebook search,
+ *   k^_j  = rho_j * Q(r_j / rho_j) R_K^{-1} + kbar       on the read side.
+ *
+ * Where floating point decides stored bits the arithmetic is the one the library boundary
+ * documents: r is the binary32-rounded coefficient vector; the sum of squares is accumulated
+ * in binary64; rho = sqrt(sum / d) in binary64, rounded to binary32 and then to bfloat16
+ * (round to nearest even both times); a scale that is not a positive finite number is replaced
+ * by 1; the normalised coefficient is the binary32 quotient r_i / rho.
+ * ---------------------------------------------------------------------------------------------- */
+static float bf16_round(float x)
+{
+    uint32_t u;
+    memcpy(&u, &x, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return x;          /* inf / nan unchanged */
+    u += 0x7fffu + ((u >> 16) & 1u);                          /* round to nearest, ties to even */
+    u &= 0xffff0000u;
+    memcpy(&x, &u, 4);
+    return x;
+}
+
+/* coef: d float64 coefficients.  Returns rho (a bfloat16 value held in a float) and writes the
+ * normalised coefficients (binary32 values held in float64) to out. */
+float oracle_key_scale(const double* coef, int d, double* out)
+{
+    double ss = 0.0;
+    for (int i = 0; i < d; ++i) {
+        const double r = (double)(float)coef[i];
+        ss += r * r;
+    }
+    float rho = bf16_round((float)sqrt(ss / (double)d));
+    if (!(rho > 0.f) || !isfinite(rho)) rho = 1.f;
+    for (int i = 0; i < d; ++i) out[i] = (double)((float)coef[i] / rho);
+    return rho;
+}
+
+/* Write path with the key scale: as oracle_encode, plus kscale [n][Hkv] (bfloat16 values as float). */
+void oracle_encode_scaled(const oracle_tables* t, const double* k, const double* v, long n,
+                          uint8_t* kidx, uint8_t* vidx, float* kscale, uint8_t* kidx64, uint8_t* vidx64,
+                          double* kgap, double* vgap)
+{
+    const int d = t->head_dim, g = t->group_size, C = t->codebook_size, H = t->n_kv_heads;
+    const int L = d / g;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long j = 0; j < n; ++j) {
+        for (int h = 0; h < H; ++h) {
+            double* coef = (double*)malloc(sizeof(double) * d);
+            double* nrm = (double*)malloc(sizeof(double) * d);
+            long o = (j * H + h);
+            oracle_coefficients(k + o * d, t->k_mean + (long)h * d, t->rk + (long)h * d * d, d, coef);
+            kscale[o] = oracle_key_scale(coef, d, nrm);
+            for (int l = 0; l < L; ++l) {
+                int i64; double gp;
+                int i32 = search_group(nrm + l * g, t->cb_k + ((long)h * L + l) * C * g, g, C, &i64, &gp);
+                kidx[o * L + l] = (uint8_t)i32;
+                if (kidx64) kidx64[o * L + l] = (uint8_t)i64;
+                if (kgap) kgap[o * L + l] = gp;
+            }
+            oracle_coefficients(v + o * d, t->v_mean + (long)h * d, t->rv + (long)h * d * d, d, coef);
+            for (int l = 0; l < L; ++l) {
+                int i64; double gp;
+                int i32 = search_group(coef + l * g, t->cb_v + ((long)h * L + l) * C * g, g, C, &i64, &gp);
+                vidx[o * L + l] = (uint8_t)i32;
+                if (vidx64) vidx64[o * L + l] = (uint8_t)i64;
+                if (vgap) vgap[o * L + l] = gp;
+            }
+            free(coef);
+            free(nrm);
+        }
+    }
+}
+
+/* Dequantise one scaled key: r^ = rho * concat_l cb_k[l][idx[l]];  k^ = r^ R_K^{-1} + kbar. */
+static void reconstruct_key_scaled(const oracle_tables* t, int h, const uint8_t* idx, double rho, double* out)
+{
+    const int d = t->head_dim, g = t->group_size, C = t->codebook_size, L = d / g;
+    double* r = (double*)malloc(sizeof(double) * d);
+    for (int l = 0; l < L; ++l)
+        for (int i = 0; i < g; ++i)
+            r[l * g + i] = rho * t->cb_k[(((long)h * L + l) * C + idx[l]) * g + i];
+    rowvec_mat_t(r, t->rk_inv_t + (long)h * d * d, d, out);
+    for (int i = 0; i < d; ++i) out[i] += t->k_mean[(long)h * d + i];
+    free(r);
+}
+
+/* kidx, vidx: [S][Hkv][L], kscale [S][Hkv] -> k_hat, v_hat: [S][Hkv][d] */
+void oracle_reconstruct_scaled(const oracle_tables* t, const uint8_t* kidx, const uint8_t* vidx,
+                               const float* kscale, long S, double* k_hat, double* v_hat)
+{
+    const int d = t->head_dim, H = t->n_kv_heads, L = d / t->group_size;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long j = 0; j < S; ++j)
+        for (int h = 0; h < H; ++h) {
+            long o = j * H + h;
+            if (k_hat) reconstruct_key_scaled(t, h, kidx + o * L, (double)kscale[o], k_hat + o * d);
+            if (v_hat) reconstruct_value(t, h, vidx + o * L, v_hat + o * d);
+        }
+}
+
+/* Decode step of one sequence on the scaled-key cache: explicit dequantisation, textbook attention. */
+void oracle_decode_scaled(const oracle_tables* t, const double* q, const uint8_t* kidx,
+                          const uint8_t* vidx, const float* kscale, long S, int Hq, double sm_scale,
+                          double* out)
+{
+    const int d = t->head_dim, H = t->n_kv_heads;
+    if (S <= 0) { memset(out, 0, sizeof(double) * (size_t)Hq * d); return; }
+    double* k_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
+    double* v_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
+    oracle_reconstruct_scaled(t, kidx, vidx, kscale, S, k_hat, v_hat);
     oracle_attention(q, k_hat, v_hat, S, Hq, H, d, sm_scale, out);
     free(k_hat);
     free(v_hat);

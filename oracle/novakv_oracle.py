@@ -140,6 +140,68 @@ class Oracle:
                               p("kidx64"), p("vidx64"), p("kgap"), p("vgap"))
         return res
 
+    def key_scale(self, coef):
+        """Per-token scale of coefficient vectors [n][d] (Algorithm "Codebook training", Normalize):
+        returns (rho [n] float32 holding bfloat16 values, normalised coefficients [n][d])."""
+        coef = _f64(coef)
+        n, d = coef.shape
+        rho = np.empty(n, np.float32)
+        out = np.empty_like(coef)
+        lib = _load()
+        lib.oracle_key_scale.restype = ctypes.c_float
+        for j in range(n):
+            rho[j] = lib.oracle_key_scale(ctypes.c_void_p(coef[j].ctypes.data), d,
+                                          ctypes.c_void_p(out[j].ctypes.data))
+        return rho, out
+
+    def encode_scaled(self, k, v, with_gaps: bool = True):
+        """Write path of the scaled key format: as encode(), plus kscale [n][Hkv] (float32 holding
+        bfloat16 values)."""
+        k, v = _f64(k), _f64(v)
+        n = k.shape[0]
+        shp = (n, self.n_kv_heads, self.n_groups)
+        res = dict(kidx=np.empty(shp, np.uint8), vidx=np.empty(shp, np.uint8),
+                   kscale=np.empty((n, self.n_kv_heads), np.float32))
+        if with_gaps:
+            res.update(kidx64=np.empty(shp, np.uint8), vidx64=np.empty(shp, np.uint8),
+                       kgap=np.empty(shp, np.float64), vgap=np.empty(shp, np.float64))
+
+        def p(name):
+            return ctypes.c_void_p(res[name].ctypes.data) if name in res else ctypes.c_void_p(0)
+
+        _load().oracle_encode_scaled(ctypes.byref(self._t), ctypes.c_void_p(k.ctypes.data),
+                                     ctypes.c_void_p(v.ctypes.data), ctypes.c_long(n), p("kidx"), p("vidx"),
+                                     p("kscale"), p("kidx64"), p("vidx64"), p("kgap"), p("vgap"))
+        return res
+
+    def reconstruct_scaled(self, kidx, vidx, kscale):
+        """Explicit dequantisation of the scaled key format: k_hat = rho * Q(.) R_K^{-1} + k_mean."""
+        kidx, vidx = _u8(kidx), _u8(vidx)
+        kscale = np.ascontiguousarray(kscale, np.float32)
+        s = kidx.shape[0]
+        k_hat = np.empty((s, self.n_kv_heads, self.d))
+        v_hat = np.empty((s, self.n_kv_heads, self.d))
+        _load().oracle_reconstruct_scaled(ctypes.byref(self._t), ctypes.c_void_p(kidx.ctypes.data),
+                                          ctypes.c_void_p(vidx.ctypes.data), ctypes.c_void_p(kscale.ctypes.data),
+                                          ctypes.c_long(s), ctypes.c_void_p(k_hat.ctypes.data),
+                                          ctypes.c_void_p(v_hat.ctypes.data))
+        return k_hat, v_hat
+
+    def decode_scaled(self, q, kidx, vidx, kscale, sm_scale: float | None = None):
+        """One decode step of one sequence on the scaled key format."""
+        q = _f64(q)
+        kidx, vidx = _u8(kidx), _u8(vidx)
+        kscale = np.ascontiguousarray(kscale, np.float32)
+        hq = q.shape[0]
+        s = kidx.shape[0]
+        scale = 1.0 / np.sqrt(self.d) if sm_scale is None else float(sm_scale)
+        out = np.empty((hq, self.d))
+        _load().oracle_decode_scaled(ctypes.byref(self._t), ctypes.c_void_p(q.ctypes.data),
+                                     ctypes.c_void_p(kidx.ctypes.data), ctypes.c_void_p(vidx.ctypes.data),
+                                     ctypes.c_void_p(kscale.ctypes.data), ctypes.c_long(s), hq,
+                                     ctypes.c_double(scale), ctypes.c_void_p(out.ctypes.data))
+        return out
+
     # -- read path --------------------------------------------------------------------
     def reconstruct(self, kidx, vidx):
         """Explicit dequantisation: indices [S][Hkv][L] -> (k_hat, v_hat) [S][Hkv][d]."""

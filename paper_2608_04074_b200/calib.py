@@ -170,11 +170,13 @@ def train_codebooks(coef: np.ndarray, n_groups: int, codebook_size: int, iters: 
 def calibrate(q_cal: np.ndarray, k_cal: np.ndarray, v_cal: np.ndarray, *, n_kv_heads: int,
               group_size: int = 4, codebook_size: int = 256, lloyd_iters: int = 25,
               seed: int = 0, n_q_for_values: int | None = None,
-              snap_value_codebook_fp16: bool = True) -> Calibration:
+              snap_value_codebook_fp16: bool = True, key_scale: bool = False) -> Calibration:
     """Run the whole offline calibration for one layer.
 
     q_cal: [N][Hq][d], k_cal / v_cal: [M][Hkv][d] (float64).
     n_q_for_values bounds how many calibration queries per head form M_o (cost is N*M*d).
+    key_scale: train the key codebooks on RMS-normalised coefficients r / rho, rho = ||r|| / sqrt(d)
+    (Algorithm 3, "Normalize"), for the key format that stores a per-token scale.
     """
     n, hq, d = q_cal.shape
     hg = hq // n_kv_heads
@@ -194,6 +196,9 @@ def calibrate(q_cal: np.ndarray, k_cal: np.ndarray, v_cal: np.ndarray, *, n_kv_h
         order = equalizing_order(var_k, n_groups)
         rk, rk_inv_t = rk[:, order], rk_inv_t[:, order]
         coef = coef[:, order]
+        if key_scale:
+            rho = np.sqrt((coef * coef).mean(axis=1, keepdims=True))
+            coef = coef / np.where(rho > 0, rho, 1.0)
         cb_k, dist_k = train_codebooks(coef, n_groups, codebook_size, lloyd_iters, gen)
         # ---- values (Corollary 1)
         nq = n if n_q_for_values is None else min(n, n_q_for_values)

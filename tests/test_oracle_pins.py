@@ -401,3 +401,87 @@ def test_gqa_head_mapping():
     for h in range(4):
         ref = np_attention(q[h], k[:, h // 2], v[:, h // 2], 1 / np.sqrt(8))
         assert np.abs(out[h] - ref).max() < 1e-13
+
+
+# ---- key format with a per-token scale (Algorithm 3 "Normalize"; App. B read path; Sec. 5 "Bit rate") ----
+def _bf16_values(x):
+    """float32 array -> nearest bfloat16 values (ties to even), by integer arithmetic on the bits."""
+    u = np.ascontiguousarray(x, np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32)
+
+
+def test_key_scale_is_rms_in_bf16_and_normalised_coefficients_have_unit_rms(tiny_case):
+    o = tiny_case["oracle"]
+    coef = o.coefficients(tiny_case["k"][:64], "k")[:, 0, :]
+    rho, nrm = o.key_scale(coef)
+    r32 = coef.astype(np.float32).astype(np.float64)
+    rms = np.sqrt((r32 * r32).sum(axis=1) / o.d)            # ||r||_2 / sqrt(d), not / d
+    np.testing.assert_array_equal(rho, _bf16_values(rms.astype(np.float32)))
+    # quotient in binary32
+    np.testing.assert_array_equal(nrm, (coef.astype(np.float32) / rho[:, None]).astype(np.float64))
+    # unit RMS up to the bfloat16 rounding of rho (relative 2^-8)
+    assert np.abs(np.sqrt((nrm * nrm).mean(axis=1)) - 1.0).max() < 2.0 ** -8 + 1e-6
+    # a zero vector keeps scale 1 and zero coefficients
+    rho0, nrm0 = o.key_scale(np.zeros((1, o.d)))
+    assert rho0[0] == 1.0 and not nrm0.any()
+
+
+def test_key_scale_power_of_two_equivariance(tiny_case):
+    o = tiny_case["oracle"]
+    k, v = tiny_case["k"][:48], tiny_case["v"][:48]
+    a = o.encode_scaled(k, v, with_gaps=False)
+    k4 = o.k_mean[None] + 4.0 * (k - o.k_mean[None])          # exact in binary64
+    b = o.encode_scaled(k4, v, with_gaps=False)
+    np.testing.assert_array_equal(a["kidx"], b["kidx"])
+    np.testing.assert_array_equal(4.0 * a["kscale"], b["kscale"])
+    np.testing.assert_array_equal(a["vidx"], b["vidx"])      # values carry no scale
+
+
+def test_key_scale_one_reduces_to_unscaled_encoder():
+    # identity transform, zero mean, keys with entries +-1: r = k, rho = 1 exactly
+    d, g, c = 64, 4, 256
+    gen = np.random.Generator(np.random.PCG64(5))
+    eye = np.eye(d)[None]
+    cb = gen.standard_normal((1, d // g, c, g)).astype(np.float32)
+    o = O.Oracle(eye, eye, eye, np.zeros((1, d)), np.zeros((1, d)), cb, cb)
+    k = gen.choice([-1.0, 1.0], size=(32, 1, d))
+    v = gen.standard_normal((32, 1, d))
+    a, b = o.encode(k, v, with_gaps=False), o.encode_scaled(k, v, with_gaps=False)
+    assert (b["kscale"] == 1.0).all()
+    np.testing.assert_array_equal(a["kidx"], b["kidx"])
+    np.testing.assert_array_equal(a["vidx"], b["vidx"])
+
+
+def test_scaled_reconstruction_is_linear_in_rho_and_logits_follow(tiny_case):
+    o = tiny_case["oracle"]
+    k, v, q = tiny_case["k"][:40], tiny_case["v"][:40], tiny_case["q"]
+    e = o.encode_scaled(k, v, with_gaps=False)
+    k1, v1 = o.reconstruct(e["kidx"], e["vidx"])              # scale ignored
+    ks, vs = o.reconstruct_scaled(e["kidx"], e["vidx"], e["kscale"])
+    np.testing.assert_array_equal(v1, vs)
+    lin = o.k_mean[None] + e["kscale"][:, :, None].astype(np.float64) * (k1 - o.k_mean[None])
+    np.testing.assert_allclose(ks, lin, rtol=0, atol=1e-12 * np.abs(lin).max())
+    # read-path identity: q k^ = rho * <q R_K^{-T}, codewords> + q kbar   (one multiply per token)
+    qf = q[0] @ o.rk_inv_t[0]
+    cw = np.stack([o.cb_k[0, np.arange(o.n_groups), e["kidx"][j, 0]].reshape(-1) for j in range(40)])
+    lhs = ks[:, 0, :] @ q[0]
+    rhs = e["kscale"][:, 0] * (cw @ qf) + q[0] @ o.k_mean[0]
+    np.testing.assert_allclose(lhs, rhs, rtol=0, atol=1e-9 * np.abs(lhs).max())
+    # decode on the scaled format = textbook attention on the explicit reconstruction
+    out = o.decode_scaled(q, e["kidx"], e["vidx"], e["kscale"])
+    hg = q.shape[0] // o.n_kv_heads
+    ref = np.stack([np_attention(q[h], ks[:, h // hg, :], vs[:, h // hg, :], 1.0 / np.sqrt(o.d)) for h in range(q.shape[0])])
+    np.testing.assert_allclose(out, ref, rtol=0, atol=1e-12)
+
+
+def test_scaled_key_rate_matches_paper_arithmetic():
+    gold = {}
+    for line in (Path(__file__).parent / "golden" / "paper_arithmetic.txt").read_text().splitlines():
+        if line.strip() and not line.startswith("#"):
+            name, val = line.split("#")[0].split()
+            gold[name] = float(val)
+    kb, vb = cache_format.bits_per_element(128, key_scale_bits=16, value_meta_bits=32)
+    assert kb == gold["bpe_keys_deployed"] and vb == gold["bpe_values_deployed"]
+    assert (kb + vb) / 2 == gold["bpe_mean_deployed"]
+    assert cache_format.bits_per_element(128, key_scale_bits=16)[0] - cache_format.bits_per_element(128)[0] == 16 / 128
