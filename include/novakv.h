@@ -153,6 +153,35 @@ novakv_status novakv_decode_attention(novakv_ctx* ctx, int layer, const void* q,
     novakv_stream stream);
 
 /*
+ * Key format with a per-token scale (Algorithm 3, the "Normalize" step; App. B "Decoding kernel and
+ * read path": the kernel "applies the per-token scale rho_j recovered from metadata (one multiply)";
+ * Sec. 5 "Bit rate": one BF16 scale per token and KV head, 16/d extra bits per key element, 2.125 at
+ * d = 128).  The key codebooks of the layer must have been trained on normalised coefficients.
+ *   write:  r as in novakv_encode_append (binary32 coefficients);
+ *           rho = bf16( float( sqrt( sum_i r_i^2 / d ) ) ), the sum and the root in binary64, both
+ *           roundings to nearest even (the order of the binary64 sum is not specified); a rho that is
+ *           not positive and finite is replaced by 1;  n_i = r_i / rho in binary32 (IEEE division);
+ *           the codeword search runs on n as in novakv_encode_append.  Values are not scaled.
+ *   read:   z_hj = rho_j * sm_scale * sum_l < q'_h[4l..4l+3], cb_k[l][kidx_j[l]] >, the rest as in
+ *           novakv_decode_attention.
+ *   k_scales  device, bf16 [n_pages][Hkv][64]: the scale of the token in slot s of page p, KV head h,
+ *             at (p * Hkv + h) * 64 + s; novakv_scale_page_bytes() = Hkv * 64 * 2 bytes per page.
+ * Other arguments, ownership and errors are those of the unscaled calls; NOVAKV_EUNSUPPORTED if the
+ * CUDA-core value path was selected with novakv_debug_set_value_path.
+ */
+size_t novakv_scale_page_bytes(const novakv_ctx* ctx);
+novakv_status novakv_encode_append_scaled(novakv_ctx* ctx, int layer,
+    const void* k_new, const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos,
+    int n_tokens, uint8_t* k_pages, uint8_t* v_pages, void* k_scales, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
+    novakv_stream stream);
+novakv_status novakv_decode_attention_scaled(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch,
+    float sm_scale, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
+    novakv_stream stream);
+
+/*
  * The same decode step for callers that cannot supply a workspace and cannot allocate one: an
  * engine that gave all device memory to its own pool, a plug-in inside it, a serving loop that must
  * never call cudaMalloc (the call synchronises the device).  (The paper has no counterpart; this is

@@ -21,6 +21,7 @@ EXPORTED = [
     "novakv_step_host", "novakv_search_coefficients", "novakv_bf16_workspace_bytes",
     "novakv_bf16_decode_attention", "novakv_profile_enable", "novakv_profile_read",
     "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc", "novakv_debug_set_value_path",
+    "novakv_scale_page_bytes", "novakv_encode_append_scaled", "novakv_decode_attention_scaled",
 ]
 
 
@@ -65,6 +66,14 @@ def load_library(path=None):
     lib.novakv_decode_attention.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                             c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p,
                                             c_size_t, c_void_p]
+    lib.novakv_scale_page_bytes.argtypes = [c_void_p]
+    lib.novakv_scale_page_bytes.restype = c_size_t
+    lib.novakv_encode_append_scaled.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
+                                                c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int,
+                                                c_void_p, c_void_p]
+    lib.novakv_decode_attention_scaled.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
+                                                   c_void_p, c_int, c_void_p, c_int, c_float, c_void_p, c_int,
+                                                   c_void_p, c_size_t, c_void_p]
     lib.novakv_decode_attention_noalloc.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                                     c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p]
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
@@ -166,6 +175,29 @@ class Context:
             int(page_table.shape[1]), _ptr(seq_lens), batch, scale, _ptr(out),
             1 if out.dtype == torch.float32 else 0, _ptr(workspace),
             int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention")
+
+    def novakv_scale_page_bytes(self):
+        return int(self.lib.novakv_scale_page_bytes(self.handle))
+
+    def novakv_encode_append_scaled(self, layer, k_new, v_new, tok_seq, tok_pos, k_pages, v_pages, k_scales,
+                                    page_table, seq_lens):
+        n_tokens = int(k_new.shape[0]) if k_new is not None else 0
+        _check(self.lib, self.lib.novakv_encode_append_scaled(
+            self.handle, layer, _ptr(k_new), _ptr(v_new), _ptr(tok_seq), _ptr(tok_pos), n_tokens,
+            _ptr(k_pages), _ptr(v_pages), _ptr(k_scales), int(k_pages.shape[0]), _ptr(page_table),
+            int(page_table.shape[1]), int(page_table.shape[0]), _ptr(seq_lens), _stream()),
+            "novakv_encode_append_scaled")
+
+    def novakv_decode_attention_scaled(self, layer, q, k_pages, v_pages, k_scales, page_table, seq_lens, out,
+                                       workspace, sm_scale=None):
+        import torch
+        batch = int(q.shape[0])
+        scale = float(self.head_dim) ** -0.5 if sm_scale is None else float(sm_scale)
+        _check(self.lib, self.lib.novakv_decode_attention_scaled(
+            self.handle, layer, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(k_scales), int(k_pages.shape[0]),
+            _ptr(page_table), int(page_table.shape[1]), _ptr(seq_lens), batch, scale, _ptr(out),
+            1 if out.dtype == torch.float32 else 0, _ptr(workspace),
+            int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_scaled")
 
     def novakv_decode_attention_noalloc(self, layer, q, k_pages, v_pages, page_table, seq_lens, out, sm_scale=None):
         """Decode step whose scratch is the library's fixed device array (no workspace argument)."""

@@ -224,6 +224,46 @@ extern "C" novakv_status novakv_decode_attention(novakv_ctx* ctx, int layer, con
                                 workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
+extern "C" size_t novakv_scale_page_bytes(const novakv_ctx* ctx) {
+    return ctx ? (size_t)ctx->cfg.n_kv_heads * NOVAKV_PAGE_TOKENS * 2 : 0;
+}
+
+extern "C" novakv_status novakv_encode_append_scaled(novakv_ctx* ctx, int layer, const void* k_new,
+    const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens, uint8_t* k_pages,
+    uint8_t* v_pages, void* k_scales, int n_pages, const int32_t* page_table, int max_pages_per_seq, int n_seq,
+    int32_t* seq_lens, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (n_tokens < 0) return NOVAKV_EINVAL;
+    if (n_tokens == 0) return NOVAKV_OK;
+    if (!k_new || !v_new || !tok_seq || !tok_pos || !k_pages || !v_pages || !k_scales || !page_table || !seq_lens) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0 || n_seq <= 0) return NOVAKV_EPAGE;
+    if ((uintptr_t)k_scales & 1) return NOVAKV_EINVAL;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_encode(ctx, ctx->layers[layer], (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new,
+                                tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages, page_table,
+                                max_pages_per_seq, n_seq, seq_lens, (cudaStream_t)stream, (__nv_bfloat16*)k_scales);
+}
+
+extern "C" novakv_status novakv_decode_attention_scaled(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out, int out_is_fp32,
+    void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!q || !k_pages || !v_pages || !k_scales || !page_table || !seq_lens || !out) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_pages & 15) || ((uintptr_t)v_pages & 15) || ((uintptr_t)k_scales & 1)) return NOVAKV_EINVAL;
+    if (!(sm_scale == sm_scale)) return NOVAKV_EINVAL;
+    if (!workspace || workspace_bytes < novakv_decode_ws_bytes(ctx, batch) || ((uintptr_t)workspace & 255)) return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_decode(ctx, ctx->layers[layer], (const __nv_bfloat16*)q, k_pages, v_pages, n_pages,
+                                page_table, max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,
+                                workspace, workspace_bytes, (cudaStream_t)stream, (const __nv_bfloat16*)k_scales);
+}
+
 extern "C" novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word) {
     if (!ctx || !word) return NOVAKV_EINVAL;
     cudaStream_t s = (cudaStream_t)stream;

@@ -323,13 +323,16 @@ template <int L>
 struct TileRegs {
     uint32_t kw[L / 4];
     uint32_t vw[2][L / 8];
+    uint32_t ks;          // this lane's token: bfloat16 key scale in the high half (a binary32 bit pattern), if used
 };
 
-template <int D, int HG, bool VM>
+// KSC: the key format carries a per-token bfloat16 scale (k_scales [n_pages][Hkv][64]); the logits of a
+// token are multiplied by it once, after the table lookups are summed.
+template <int D, int HG, bool VM, bool KSC>
 __global__ void __launch_bounds__(S1_THREADS, 1)
 novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restrict__ cb_k_lut,
                             const __half* __restrict__ cb_v_img, const uint8_t* __restrict__ k_pages,
-                            const uint8_t* __restrict__ v_pages, int n_pages,
+                            const uint8_t* __restrict__ v_pages, const __nv_bfloat16* __restrict__ k_scales, int n_pages,
                             const int32_t* __restrict__ page_table, int max_pages_per_seq,
                             const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ page_prefix,
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
@@ -406,6 +409,11 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             const int page = __shfl_sync(0xffffffffu, ids_cur, it & 31);
             const int half = (warp + NCW * it) & 1;
             const size_t off = ((size_t)page * n_kv_heads + sg.kvh) * PAGE_BYTES + half * TILE_BYTES;
+            if (KSC) {
+                const unsigned short raw = __ldg(reinterpret_cast<const unsigned short*>(k_scales) +
+                                                 ((size_t)page * n_kv_heads + sg.kvh) * NOVAKV_PAGE_TOKENS + half * 32 + lane);
+                t.ks = (uint32_t)raw << 16;
+            }
             const uint8_t* kp = k_pages + off + lane * 16;
             const uint8_t* vp = v_pages + off + lane * (NGB * 4);
 #pragma unroll
@@ -469,6 +477,11 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             float zf[HPAD];
 #pragma unroll
             for (int h = 0; h < HPAD / 2; ++h) unpack2(z[h], zf[2 * h], zf[2 * h + 1]);
+            if (KSC) {
+                const float rho = __uint_as_float(cur.ks);
+#pragma unroll
+                for (int h = 0; h < HPAD; ++h) zf[h] *= rho;
+            }
             bool rescale = false;
             float alpha[HPAD];
             __half ph[HPAD];
@@ -792,9 +805,9 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     return w;
 }
 
-template <int D, int HG, bool VM>
+template <int D, int HG, bool VM, bool KSC>
 novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
-                              const uint8_t* k_pages, const uint8_t* v_pages, int n_pages,
+                              const uint8_t* k_pages, const uint8_t* v_pages, const __nv_bfloat16* k_scales, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens,
                               int batch, float sm_scale, void* out, int out_is_fp32, void* workspace,
                               cudaStream_t stream) {
@@ -811,7 +824,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                       batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status);
     ctx->launches++;
 
-    auto kern = novakv_decode_stage1_kernel<D, HG, VM>;
+    auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC>;
     static bool smem_opt_in = false;      // per template instantiation; the attribute is sticky
     if (!smem_opt_in) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
@@ -821,7 +834,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     {
         novakv_prof_scope ps(ctx, 0, stream);
         novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut, ly.cb_v_mma, k_pages, v_pages,
-                          n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
+                          k_scales, n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
                           ctx->dev_status);
         ps.end();
         ctx->launches++;
@@ -841,16 +854,21 @@ size_t novakv_decode_ws_bytes(const novakv_ctx* ctx, int batch) { return ws_layo
 novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
-    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream, const __nv_bfloat16* k_scales) {
     (void)workspace_bytes;
     const int d = ctx->cfg.head_dim, hg = ctx->hg;
+    if (k_scales != nullptr && ctx->value_path == 0) return NOVAKV_EUNSUPPORTED;   // scaled keys: tensor-core value side only
 #define NOVAKV_DISPATCH(DD, HH)                                                                             \
     if (d == DD && hg == HH) {                                                                                   \
-        if (ctx->value_path == 0)                                                                                \
-            return launch_decode_t<DD, HH, false>(ctx, ly, q, k_pages, v_pages, n_pages, page_table,             \
+        if (k_scales != nullptr)                                                                                 \
+            return launch_decode_t<DD, HH, true, true>(ctx, ly, q, k_pages, v_pages, k_scales, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
                                                   workspace, stream);                                            \
-        return launch_decode_t<DD, HH, true>(ctx, ly, q, k_pages, v_pages, n_pages, page_table,                  \
+        if (ctx->value_path == 0)                                                                                \
+            return launch_decode_t<DD, HH, false, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table, \
+                                                  max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
+                                                  workspace, stream);                                            \
+        return launch_decode_t<DD, HH, true, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table,  \
                                              max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,     \
                                              workspace, stream);                                                 \
     }

@@ -173,7 +173,8 @@ struct EncPipe {
     static constexpr size_t off_idx = off_slab + 2 * slab_bytes;
     static constexpr size_t off_pos = off_idx + idx_bytes;                          // [2][2][ENC_TILE] ints
     static constexpr size_t off_mean = off_pos + 4 * ENC_TILE * sizeof(int);        // [D] doubles
-    static constexpr size_t total = off_mean + D * sizeof(double);
+    static constexpr size_t off_rho = off_mean + D * sizeof(double);                // [2][ENC_TILE] floats (key scales)
+    static constexpr size_t total = off_rho + 2 * ENC_TILE * sizeof(float);
     static_assert(total <= 232448, "shared memory budget");
 };
 
@@ -182,14 +183,20 @@ struct EncPipe {
 // the binary64 transform runs on the fp64 pipe and the load/store unit, the 256-way search on the FMA
 // pipe.  Half of the warps therefore transform tile i+1 while the other half searches tile i
 // (coefficients double-buffered in shared memory, hand-over by named hardware barriers).
-template <int D>
+// KSC (key format with a per-token scale, Algorithm 3 "Normalize"): after the key transform of a tile
+// the transform warps compute rho = ||r||_2 / sqrt(d) of each token's binary32 coefficients (sum of squares
+// in binary64), round it to binary32 and then to bfloat16 (a scale that is not positive and finite becomes
+// 1), divide the coefficients by it in binary32 (IEEE division) and hand rho to the search warps, which
+// store it beside the indices (k_scales [n_pages][Hkv][64]).  Values are not scaled.
+template <int D, bool KSC>
 __global__ void __launch_bounds__(ENC_THREADS, 1)
 novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                      const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
                      const double* __restrict__ rk_d, const double* __restrict__ rv_d,
                      const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
                      const float* __restrict__ cb_k, const float* __restrict__ cb_v,
-                     uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages, int n_pages,
+                     uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages,
+                     __nv_bfloat16* __restrict__ k_scales, int n_pages,
                      const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                      int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
                      uint32_t* __restrict__ dev_status) {
@@ -200,6 +207,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     uint8_t* idx_s = smem + P::off_idx;
     int* pos_s = reinterpret_cast<int*>(smem + P::off_pos);                // [buf][page|slot][ENC_TILE]
     double* mean_s = reinterpret_cast<double*>(smem + P::off_mean);
+    float* rho_s = reinterpret_cast<float*>(smem + P::off_rho);            // [buf][ENC_TILE]
 
     const int kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
@@ -322,6 +330,25 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                 for (int nt = 0; nt < NTILE_N; ++nt)
                     *reinterpret_cast<float2*>(r_s + (size_t)(mt * 8 + fr) * RS + (wt * NTILE_N + nt) * 8 + 2 * fk) =
                         make_float2((float)acc[mt][nt][0], (float)acc[mt][nt][1]);
+            if (KSC && side == 0) {
+                // 4 threads per token, thread `part` takes the columns = part (mod 4): conflict-free rows
+                nbar_sync(BAR_T, NT);
+                const int t = tid >> 2, part = tid & 3;
+                float* row = r_s + (size_t)t * RS + part;
+                double ss = 0.0;
+#pragma unroll 8
+                for (int i = 0; i < D / 4; ++i) {
+                    const double r = (double)row[4 * i];
+                    ss = fma(r, r, ss);
+                }
+                ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                float rho = __bfloat162float(__float2bfloat16_rn((float)sqrt(ss / (double)D)));
+                if (!(rho > 0.f) || !isfinite(rho)) rho = 1.f;
+#pragma unroll 8
+                for (int i = 0; i < D / 4; ++i) row[4 * i] = __fdiv_rn(row[4 * i], rho);
+                if (part == 0) rho_s[buf * ENC_TILE + t] = rho;
+            }
             __threadfence_block();
             nbar_arrive(BAR_FULL + buf, ENC_THREADS);            // hand tile i to the search warps
         }
@@ -343,6 +370,12 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                 const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
                 if (side == 0) k_pages[base + novakv_k_offset<L>(slot, l)] = idx_s[e];
                 else v_pages[base + novakv_v_offset<L>(slot, l)] = idx_s[e];
+            }
+            if (KSC && side == 0 && tid < n_valid) {
+                const int page = pos_s[(buf * 2 + 0) * ENC_TILE + tid];
+                if (page >= 0)
+                    k_scales[((size_t)page * n_kv_heads + kvh) * NOVAKV_PAGE_TOKENS + pos_s[(buf * 2 + 1) * ENC_TILE + tid]] =
+                        __float2bfloat16_rn(rho_s[buf * ENC_TILE + tid]);
             }
             nbar_sync(BAR_S, NT);                                // idx_s and the buffer are free again
             if (i + 2 < n_local) nbar_arrive(BAR_EMPTY + buf, ENC_THREADS);
@@ -513,8 +546,9 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                               const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos,
                               int n_tokens, uint8_t* k_pages, uint8_t* v_pages, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
-                              cudaStream_t stream) {
-    if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS) {
+                              cudaStream_t stream, __nv_bfloat16* k_scales) {
+    // (the scaled key format needs all coefficients of a token in one CTA: it always takes the tiled kernel)
+    if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS && k_scales == nullptr) {
         dim3 grid(D / NOVAKV_G / 4, ctx->cfg.n_kv_heads, 2);
         novakv_prof_scope ps(ctx, 1, stream);
         int tp_log2 = 0;
@@ -526,7 +560,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         ctx->launches++;
         return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
     }
-    auto kern = novakv_encode_kernel<D>;
+    auto kern = k_scales ? novakv_encode_kernel<D, true> : novakv_encode_kernel<D, false>;
     const size_t smem = EncPipe<D>::total;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
@@ -547,9 +581,9 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     dim3 grid(ctas_x, ctx->cfg.n_kv_heads, 2);
     novakv_prof_scope ps(ctx, 1, stream);
     kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d_mma, ly.rv_d_mma,
-                                               ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
-                                               page_table, max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads,
-                                               tiles_per_cta, ctx->dev_status);
+                                               ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, k_scales,
+                                               n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
+                                               ctx->cfg.n_kv_heads, tiles_per_cta, ctx->dev_status);
     ps.end();
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
@@ -574,12 +608,12 @@ novakv_status launch_search_t(novakv_ctx* ctx, const novakv_layer& ly, int which
 novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* k_new,
     const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens,
     uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
-    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream) {
+    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream, __nv_bfloat16* k_scales) {
     if (ctx->cfg.head_dim == 128)
         return launch_encode_t<128>(ctx, ly, k_new, v_new, tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages,
-                                    page_table, max_pages_per_seq, n_seq, seq_lens, stream);
+                                    page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales);
     return launch_encode_t<64>(ctx, ly, k_new, v_new, tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages,
-                               page_table, max_pages_per_seq, n_seq, seq_lens, stream);
+                               page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales);
 }
 
 novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef,

@@ -67,7 +67,8 @@ struct novakv_prof_scope {
 novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* k_new,
     const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens,
     uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
-    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream);
+    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream,
+    __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */);
 novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef,
     int n, uint8_t* idx_out, cudaStream_t stream);
 
@@ -76,7 +77,8 @@ size_t novakv_decode_ws_bytes(const novakv_ctx* ctx, int batch);
 novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
-    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream,
+    const __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */);
 
 // bf16 comparator
 size_t novakv_bf16_ws_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq);

@@ -15,8 +15,10 @@ from .binding import Context
 class PagedCache:
     """Key/value index pools plus page table and lengths for a batch of sequences."""
 
-    def __init__(self, ctx: Context, seq_lens, capacity_tokens=None, seed: int = 0, device="cuda:0"):
+    def __init__(self, ctx: Context, seq_lens, capacity_tokens=None, seed: int = 0, device="cuda:0",
+                 key_scale: bool = False):
         self.ctx = ctx
+        self.key_scale = key_scale
         self.device = torch.device(device)
         seq_lens = np.asarray(seq_lens, dtype=np.int32)
         cap = seq_lens if capacity_tokens is None else np.maximum(np.asarray(capacity_tokens, np.int32), seq_lens)
@@ -27,6 +29,9 @@ class PagedCache:
         self.page_bytes = ctx.novakv_page_bytes()
         self.k_pages = torch.zeros((self.n_pages, self.page_bytes), dtype=torch.uint8, device=self.device)
         self.v_pages = torch.zeros((self.n_pages, self.page_bytes), dtype=torch.uint8, device=self.device)
+        # scaled key format: one bf16 scale per token and KV head, [n_pages][Hkv][64]
+        self.k_scales = (torch.ones((self.n_pages, ctx.n_kv_heads, cache_format.PAGE_TOKENS), dtype=torch.bfloat16,
+                                    device=self.device) if key_scale else None)
         # unused table entries point at page 0 so that a wrong read stays in bounds
         self.page_table = torch.from_numpy(np.where(table < 0, 0, table).astype(np.int32)).to(self.device)
         self.seq_lens = torch.from_numpy(seq_lens.copy()).to(self.device)
@@ -57,8 +62,24 @@ class PagedCache:
         return cache_format.read_tokens(kp, vp, self.page_table_host[seq], self.ctx.n_kv_heads,
                                         self.ctx.head_dim, pos0, n)
 
+    def store_scales(self, seq: int, pos0: int, kscale: np.ndarray):
+        """kscale [n][Hkv] (bf16-representable float32) -> scale pool, positions pos0.. of one sequence."""
+        sp = self.k_scales.float().cpu().numpy()
+        pos = pos0 + np.arange(kscale.shape[0])
+        sp[self.page_table_host[seq][pos // cache_format.PAGE_TOKENS], :, pos % cache_format.PAGE_TOKENS] = kscale
+        self.k_scales.copy_(torch.from_numpy(sp).to(torch.bfloat16))
+
+    def load_scales(self, seq: int, pos0: int, n: int) -> np.ndarray:
+        sp = self.k_scales.float().cpu().numpy()
+        pos = pos0 + np.arange(n)
+        return sp[self.page_table_host[seq][pos // cache_format.PAGE_TOKENS], :, pos % cache_format.PAGE_TOKENS]
+
     # ---- hot path calls
     def append(self, layer, k_new, v_new, tok_seq, tok_pos):
+        if self.key_scale:
+            self.ctx.novakv_encode_append_scaled(layer, k_new, v_new, tok_seq, tok_pos, self.k_pages, self.v_pages,
+                                                 self.k_scales, self.page_table, self.seq_lens)
+            return
         self.ctx.novakv_encode_append(layer, k_new, v_new, tok_seq, tok_pos, self.k_pages, self.v_pages,
                                       self.page_table, self.seq_lens)
 
@@ -66,6 +87,10 @@ class PagedCache:
         if out is None:
             out = torch.empty((self.batch, self.ctx.n_q_heads, self.ctx.head_dim), dtype=torch.float32,
                               device=self.device)
+        if self.key_scale:
+            self.ctx.novakv_decode_attention_scaled(layer, q, self.k_pages, self.v_pages, self.k_scales,
+                                                    self.page_table, self.seq_lens, out, self.workspace, sm_scale)
+            return out
         self.ctx.novakv_decode_attention(layer, q, self.k_pages, self.v_pages, self.page_table, self.seq_lens,
                                          out, self.workspace, sm_scale)
         return out

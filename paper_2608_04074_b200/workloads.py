@@ -48,12 +48,14 @@ class Workload:
         return synth.draw_layer_laws(self.shape, 1000 * self.seed + 1, n_outlier=self.n_outlier,
                                      heavy_fraction=self.heavy_fraction, logit_std=self.logit_std)
 
-    def calibration(self, laws: synth.LayerLaws | None = None) -> Calibration:
+    def calibration(self, laws: synth.LayerLaws | None = None, key_scale: bool = False) -> Calibration:
+        """key_scale: key codebooks trained on RMS-normalised coefficients (per-token scale format)."""
         laws = laws or self.laws()
         k, v = synth.draw_kv(laws, 1000 * self.seed + 2, self.calib_tokens)
         q = synth.draw_q(laws, 1000 * self.seed + 3, self.calib_tokens)
         return calibrate(q, k, v, n_kv_heads=self.shape.n_kv_heads, lloyd_iters=self.lloyd_iters,
-                         seed=1000 * self.seed + 4, n_q_for_values=self.calib_queries_for_values)
+                         seed=1000 * self.seed + 4, n_q_for_values=self.calib_queries_for_values,
+                         key_scale=key_scale)
 
 
 def tiny(seq_len: int = 1024, seed: int = 1) -> Workload:

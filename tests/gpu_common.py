@@ -13,11 +13,12 @@ NEAR_TIE = 1e-6         # index mismatches are allowed only where the oracle's f
 class Case:
     """Calibration + context + oracle for one layer shape."""
 
-    def __init__(self, wl, n_layers=1):
+    def __init__(self, wl, n_layers=1, key_scale=False):
         from paper_2608_04074_b200.binding import Context
         self.wl = wl
+        self.key_scale = key_scale
         self.laws = wl.laws()
-        self.cal = wl.calibration(self.laws)
+        self.cal = wl.calibration(self.laws, key_scale=key_scale)
         self.oracle = O.Oracle.from_calibration(self.cal)
         s = wl.shape
         self.ctx = Context(s.n_q_heads, s.n_kv_heads, s.head_dim, n_layers=n_layers)

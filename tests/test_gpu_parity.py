@@ -412,3 +412,109 @@ def test_small_head_groups(hq, hkv, d):
             check_indices(gk, enc, "k"); check_indices(gv, enc, "v")
             check_output(out[b], case.oracle.decode(q[b].astype(np.float64), gk, gv))
     case.ctx.close()
+
+
+# --------------------------------------------------------------------------- key format with a per-token scale
+@pytest.fixture(scope="module")
+def qwen_scaled():
+    return Case(workloads.qwen3_8b(batch=4, seq_len=4096, calib_tokens=4096, lloyd_iters=6), key_scale=True)
+
+
+@pytest.fixture(scope="module")
+def gptoss_scaled():
+    return Case(workloads.gpt_oss_20b(batch=2, seq_len=2048, calib_tokens=4096, lloyd_iters=6), key_scale=True)
+
+
+@pytest.mark.parametrize("name", ["qwen_scaled", "gptoss_scaled"])
+def test_scaled_encode_matches_oracle_indices_and_scales(name, request):
+    """Append (tiled kernel: a long run, a ragged tail, a single token) on the scaled key format:
+    indices as in the unscaled test, scales bit for bit (bfloat16)."""
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = request.getfixturevalue(name)
+    lens0 = np.array([0, 5, 63, 130], np.int32)
+    add = np.array([200, 64, 1, 130], np.int32)
+    cache = PagedCache(case.ctx, lens0, capacity_tokens=lens0 + add, seed=3, key_scale=True)
+    n = int(add.sum())
+    k, v, _ = case.draw(210, n, 1)
+    # a wide range of key norms, so that the scale matters: every token scaled by a power of two
+    k = synth.to_bf16_representable(k * (2.0 ** synth.rng(6).integers(-3, 4, size=(n, 1, 1))))
+    tok_seq = np.concatenate([np.full(a, b, np.int32) for b, a in enumerate(add)])
+    tok_pos = np.concatenate([lens0[b] + np.arange(a, dtype=np.int32) for b, a in enumerate(add)])
+    perm = synth.rng(7).permutation(n)
+    k, v, tok_seq, tok_pos = k[perm], v[perm], tok_seq[perm], tok_pos[perm]
+    cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(tok_seq), _dev(tok_pos))
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens0 + add)
+    enc = case.oracle.encode_scaled(k.astype(np.float64), v.astype(np.float64))
+    got_k = np.empty_like(enc["kidx"]); got_v = np.empty_like(enc["vidx"])
+    got_s = np.empty_like(enc["kscale"])
+    for t in range(n):
+        kk, vv = cache.load_logical(int(tok_seq[t]), int(tok_pos[t]), 1)
+        got_k[t], got_v[t] = kk[0], vv[0]
+        got_s[t] = cache.load_scales(int(tok_seq[t]), int(tok_pos[t]), 1)[0]
+    assert np.array_equal(got_s, enc["kscale"]), f"{int((got_s != enc['kscale']).sum())} scales differ"
+    assert len(np.unique(enc["kscale"])) > 8
+    dk, nk = check_indices(got_k, enc, "k")
+    dv, nv = check_indices(got_v, enc, "v")
+    print(f"[{name}] scaled format: index mismatches K {dk} V {dv}; near-ties K {nk} V {nv} of {got_k.size}")
+
+
+@pytest.mark.parametrize("name,lens", [("qwen_scaled", [1, 63, 64, 65, 1000, 0, 3001]), ("gptoss_scaled", [2048, 77, 640])])
+def test_scaled_decode_matches_oracle(name, lens, request):
+    """Decode on the oracle's scaled encoding (indices + scales) against explicit dequantisation."""
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = request.getfixturevalue(name)
+    lens = np.array(lens, np.int32)
+    cache = PagedCache(case.ctx, lens, seed=3, key_scale=True)
+    encs = []
+    for b, n in enumerate(lens):
+        if n == 0:
+            encs.append(None)
+            continue
+        k, v, _ = case.draw(320 + b, int(n), 1)
+        k = synth.to_bf16_representable(k * (2.0 ** synth.rng(8 + b).integers(-2, 3, size=(int(n), 1, 1))))
+        e = case.oracle.encode_scaled(k.astype(np.float64), v.astype(np.float64), with_gaps=False)
+        cache.store_logical(b, 0, e["kidx"], e["vidx"])
+        cache.store_scales(b, 0, e["kscale"])
+        encs.append(e)
+    _, _, q = case.draw(321, 1, len(lens))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    worst = 0.0
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert not out[b].any()
+            continue
+        ref = case.oracle.decode_scaled(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], encs[b]["kscale"])
+        worst = max(worst, check_output(out[b], ref))
+        # the scale is not a no-op on this input: ignoring it moves the output by far more than the tolerance
+        if n >= 64:
+            no_scale = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
+            assert np.abs(no_scale - ref).max() > 10 * 2e-3 * np.abs(ref).max()
+    print(f"[{name} {lens.tolist()}] scaled format: max|delta|/||o||inf = {worst:.3e}")
+
+
+def test_scaled_append_then_decode_end_to_end(qwen_scaled):
+    """Whole path on the scaled format: prefill append, one decode-sized append, decode."""
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = qwen_scaled
+    lens = np.array([300, 65, 1], np.int32)
+    cache = PagedCache(case.ctx, np.zeros(3, np.int32), capacity_tokens=lens + 1, seed=4, key_scale=True)
+    ks, vs = [], []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(400 + b, int(n) + 1, 1)
+        ks.append(k); vs.append(v)
+        cache.append(0, _dev(k[:n], torch.bfloat16), _dev(v[:n], torch.bfloat16),
+                     _dev(np.full(int(n), b, np.int32)), _dev(np.arange(int(n), dtype=np.int32)))
+    # decode-sized append: one token per sequence
+    cache.append(0, _dev(np.stack([ks[b][lens[b]] for b in range(3)]), torch.bfloat16),
+                 _dev(np.stack([vs[b][lens[b]] for b in range(3)]), torch.bfloat16),
+                 _dev(np.arange(3, dtype=np.int32)), _dev(lens.astype(np.int32)))
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens + 1)
+    _, _, q = case.draw(401, 1, 3)
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    for b in range(3):
+        e = case.oracle.encode_scaled(ks[b].astype(np.float64), vs[b].astype(np.float64), with_gaps=False)
+        ref = case.oracle.decode_scaled(q[b].astype(np.float64), e["kidx"], e["vidx"], e["kscale"])
+        check_output(out[b], ref)
