@@ -167,6 +167,8 @@ def fill_cache_gpu(case_ctx, cache, laws, seq_lens, seed, share_content=False):
         dst = cache.page_table[b, :npg].long()
         cache.k_pages[dst] = cache.k_pages[src[:npg]]
         cache.v_pages[dst] = cache.v_pages[src[:npg]]
+        if getattr(cache, "k_scales", None) is not None:
+            cache.k_scales[dst] = cache.k_scales[src[:npg]]
     cache.seq_lens.copy_(torch.from_numpy(np.asarray(seq_lens, np.int32)).cuda())
 
 
@@ -428,6 +430,37 @@ def run_ours(args):
         ms = statistics.median(tt)
         sweep.append({"workload": f"prefill encode {T} tokens x 8 KV heads x d=128 (K and V)", "ms": round(ms, 4),
                       "tokens_per_s": round(T / (ms * 1e-3), 1)})
+        # key format with a per-token bf16 scale (2.125 bits per key element): prefill encode, append, decode
+        c3s = PagedCache(ctx, wl3.seq_lens, seed=29, device=dev, key_scale=True)
+        tt = time_steps(lambda: c3s.append(0, kd, vd, ts, tp), 5, 2, lambda: None)
+        ms_enc_s = statistics.median(tt)
+        del c3s, c3
+        torch.cuda.empty_cache()
+        b6, s6 = 64, 32768
+        wl6 = workloads.qwen3_8b(batch=b6, seq_len=s6)
+        c6 = PagedCache(ctx, wl6.seq_lens, capacity_tokens=wl6.seq_lens + 64, seed=41, device=dev, key_scale=True)
+        fill_cache_gpu(ctx, c6, laws, wl6.seq_lens, seed=9200, share_content=True)
+        q6 = bf16_tensor(synth.draw_q(laws, 7400, b6), dev)
+        o6 = torch.empty((b6, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
+        td6 = time_steps(lambda: c6.decode(0, q6, out=o6), max(5, args.steps // 2), 3, lambda: None)
+        k6, v6 = synth.draw_kv(laws, 7401, b6)
+        k6d, v6d = bf16_tensor(k6, dev), bf16_tensor(v6, dev)
+        seq6 = torch.arange(b6, dtype=torch.int32, device=dev)
+        pos6 = torch.from_numpy(wl6.seq_lens.astype(np.int32)).to(dev)
+        ta6 = time_steps(lambda: c6.append(0, k6d, v6d, seq6, pos6), max(5, args.steps // 2), 3, lambda: None)
+        ab6, ib6 = algorithmic_decode_bytes(wl6)
+        ab6 += int(wl6.seq_lens.astype(np.int64).sum()) * s.n_kv_heads * 2          # the scales are read too
+        ms6 = statistics.median(td6)
+        sweep.append({"workload": f"scaled key format (bf16 scale per token and KV head, 2.125 bit per key element), qwen3_8b_shape "
+                                  f"B={b6} S={s6}: decode only; append of {b6} tokens; prefill encode of {T} tokens "
+                                  "(timing only: the codebooks loaded are those of the unscaled format)",
+                      "ms": round(ms6, 4), "gbps": round(ab6 / (ms6 * 1e-3) / 1e9, 1),
+                      "pct_of_8TBps": round(100 * ab6 / (ms6 * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
+                      "algorithmic_bytes": ab6, "append_ms": round(statistics.median(ta6), 4),
+                      "prefill_encode_ms": round(ms_enc_s, 4), "prefill_tokens_per_s": round(T / (ms_enc_s * 1e-3), 1),
+                      "device_status": ctx.novakv_last_device_status()})
+        del c6, q6, o6
+        torch.cuda.empty_cache()
         # GPT-OSS-20B-shaped hybrid pair: full-attention layer on the 2-bit cache + sliding-window (128) layer in bf16
         wl4 = workloads.gpt_oss_20b(batch=16, seq_len=65536)
         laws4 = wl4.laws()
