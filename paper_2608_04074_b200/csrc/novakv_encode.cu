@@ -111,7 +111,7 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
         float best_a = CUDART_INF_F, best_b = CUDART_INF_F;
         int blk_a = 0, blk_b = 0;
         const ulonglong2* cb = reinterpret_cast<const ulonglong2*>(cb_s) + (size_t)l * NOVAKV_C;   // 2 x 16 B per pair
-#pragma unroll 2
+#pragma unroll 4
         for (int blk = 0; blk < NOVAKV_C / 8; ++blk) {
             float da[8], db[8];
 #pragma unroll
