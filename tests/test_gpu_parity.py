@@ -518,3 +518,42 @@ def test_scaled_append_then_decode_end_to_end(qwen_scaled):
         e = case.oracle.encode_scaled(ks[b].astype(np.float64), vs[b].astype(np.float64), with_gaps=False)
         ref = case.oracle.decode_scaled(q[b].astype(np.float64), e["kidx"], e["vidx"], e["kscale"])
         check_output(out[b], ref)
+
+
+# --------------------------------------------------------------------------- many pairs / one long sequence
+def test_many_short_sequences_more_pairs_than_ctas(qwen):
+    """320 (sequence, KV head) pairs on 148 scan CTAs: many segments per CTA, CTAs spanning several pairs,
+    empty sequences in between, and the high-occupancy variant of the merge kernel."""
+    case = qwen
+    gen = synth.rng(77)
+    lens = gen.integers(1, 200, size=40).astype(np.int32)
+    lens[[3, 17, 39]] = 0
+    lens[5], lens[6] = 64, 65
+    assert len(lens) * case.ctx.n_kv_heads > 2 * 148
+    cache = _cache(case, lens, seed=9)
+    encs = _fill_with_oracle(case, cache, lens, 700)
+    _, _, q = case.draw(701, 1, len(lens))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    worst = 0.0
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert not out[b].any()
+            continue
+        ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
+        worst = max(worst, check_output(out[b], ref))
+    print(f"[40 short sequences] max|delta|/||o||inf = {worst:.3e}")
+
+
+def test_one_long_sequence_all_ctas_share_each_pair(qwen):
+    """One sequence of 20000 tokens (313 pages, ragged last page): every (sequence, KV head) pair is split
+    over ~18 scan CTAs, so the merge combines many partials per pair."""
+    case = qwen
+    lens = np.array([20000], np.int32)
+    cache = _cache(case, lens, seed=10)
+    encs = _fill_with_oracle(case, cache, lens, 800)
+    _, _, q = case.draw(801, 1, 1)
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    ref = case.oracle.decode(q[0].astype(np.float64), encs[0]["kidx"], encs[0]["vidx"])
+    print(f"[one 20000-token sequence] max|delta|/||o||inf = {check_output(out[0], ref):.3e}")
