@@ -378,3 +378,54 @@ void oracle_decode_scaled(const oracle_tables* t, const double* q, const uint8_t
     free(k_hat);
     free(v_hat);
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Learned attention sink (App. "Attention sinks in the quantized serving path"): an extra logit
+ * s_h per query head that enters the softmax normaliser but has no value vector,
+ *     p_j = exp(z_j) / ( sum_i exp(z_i) + exp(s_h) ),   o = sum_j p_j v_j,
+ * with z_j the full logits q.k_j * sm_scale (the oracle dequantises keys explicitly, mean included,
+ * so the offset correction the GPU applies to the sink logit has no counterpart here).
+ * sink: [Hq] natural-log units.  S == 0 gives zeros (all the mass sits on the sink).
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_attention_sink(const double* q, const double* k, const double* v, long S, int Hq, int Hkv,
+                           int d, double sm_scale, const double* sink, double* out)
+{
+    const int hg = Hq / Hkv;
+#pragma omp parallel for schedule(static)
+    for (int h = 0; h < Hq; ++h) {
+        const int kv = h / hg;
+        double* z = (double*)malloc(sizeof(double) * (S > 0 ? S : 1));
+        double zmax = sink[h];
+        for (long j = 0; j < S; ++j) {
+            const double* kj = k + (j * Hkv + kv) * d;
+            double s = 0.0;
+            for (int i = 0; i < d; ++i) s += q[(long)h * d + i] * kj[i];
+            z[j] = s * sm_scale;
+            if (z[j] > zmax) zmax = z[j];
+        }
+        double den = exp(sink[h] - zmax);
+        for (long j = 0; j < S; ++j) { z[j] = exp(z[j] - zmax); den += z[j]; }
+        for (int i = 0; i < d; ++i) out[(long)h * d + i] = 0.0;
+        for (long j = 0; j < S; ++j) {
+            const double p = z[j] / den;
+            const double* vj = v + (j * Hkv + kv) * d;
+            for (int i = 0; i < d; ++i) out[(long)h * d + i] += p * vj[i];
+        }
+        free(z);
+    }
+}
+
+/* Decode step with a sink: explicit dequantisation (kscale may be NULL: unscaled key format). */
+void oracle_decode_sink(const oracle_tables* t, const double* q, const uint8_t* kidx, const uint8_t* vidx,
+                        const float* kscale, long S, int Hq, double sm_scale, const double* sink, double* out)
+{
+    const int d = t->head_dim, H = t->n_kv_heads;
+    if (S <= 0) { memset(out, 0, sizeof(double) * (size_t)Hq * d); return; }
+    double* k_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
+    double* v_hat = (double*)malloc(sizeof(double) * (size_t)S * H * d);
+    if (kscale) oracle_reconstruct_scaled(t, kidx, vidx, kscale, S, k_hat, v_hat);
+    else oracle_reconstruct(t, kidx, vidx, S, k_hat, v_hat);
+    oracle_attention_sink(q, k_hat, v_hat, S, Hq, H, d, sm_scale, sink, out);
+    free(k_hat);
+    free(v_hat);
+}

@@ -228,6 +228,37 @@ class Oracle:
                               ctypes.c_void_p(out.ctypes.data))
         return out
 
+    def decode_sink(self, q, kidx, vidx, sink, kscale=None, sm_scale: float | None = None):
+        """Decode step with a learned sink logit per query head (sink [Hq], natural-log units)."""
+        q = _f64(q)
+        kidx, vidx = _u8(kidx), _u8(vidx)
+        sink = _f64(sink)
+        ks = None if kscale is None else np.ascontiguousarray(kscale, np.float32)
+        hq = q.shape[0]
+        s = kidx.shape[0]
+        scale = 1.0 / np.sqrt(self.d) if sm_scale is None else float(sm_scale)
+        out = np.empty((hq, self.d))
+        _load().oracle_decode_sink(ctypes.byref(self._t), ctypes.c_void_p(q.ctypes.data),
+                                   ctypes.c_void_p(kidx.ctypes.data), ctypes.c_void_p(vidx.ctypes.data),
+                                   ctypes.c_void_p(ks.ctypes.data if ks is not None else 0), ctypes.c_long(s), hq,
+                                   ctypes.c_double(scale), ctypes.c_void_p(sink.ctypes.data),
+                                   ctypes.c_void_p(out.ctypes.data))
+        return out
+
+
+def attention_sink(q, k, v, sink, sm_scale: float | None = None):
+    """Textbook attention with an extra value-less logit per head: q [Hq][d], k/v [S][Hkv][d], sink [Hq]."""
+    q, k, v, sink = _f64(q), _f64(k), _f64(v), _f64(sink)
+    hq, d = q.shape
+    s, hkv, _ = k.shape
+    scale = 1.0 / np.sqrt(d) if sm_scale is None else float(sm_scale)
+    out = np.empty((hq, d))
+    _load().oracle_attention_sink(ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(k.ctypes.data),
+                                  ctypes.c_void_p(v.ctypes.data), ctypes.c_long(s), hq, hkv, d,
+                                  ctypes.c_double(scale), ctypes.c_void_p(sink.ctypes.data),
+                                  ctypes.c_void_p(out.ctypes.data))
+    return out
+
 
 def attention(q, k, v, sm_scale: float | None = None):
     """Textbook attention on explicit float64 keys/values: q [Hq][d], k/v [S][Hkv][d]."""

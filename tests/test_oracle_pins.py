@@ -485,3 +485,56 @@ def test_scaled_key_rate_matches_paper_arithmetic():
     assert kb == gold["bpe_keys_deployed"] and vb == gold["bpe_values_deployed"]
     assert (kb + vb) / 2 == gold["bpe_mean_deployed"]
     assert cache_format.bits_per_element(128, key_scale_bits=16)[0] - cache_format.bits_per_element(128)[0] == 16 / 128
+
+
+# ---- learned attention sink (App. "Attention sinks in the quantized serving path") ----
+def test_sink_closed_forms(tiny_case):
+    o = tiny_case["oracle"]
+    k, v, q = tiny_case["k"][:50], tiny_case["v"][:50], tiny_case["q"]
+    e = o.encode(k, v, with_gaps=False)
+    k_hat, v_hat = o.reconstruct(e["kidx"], e["vidx"])
+    hq = q.shape[0]
+    hg = hq // o.n_kv_heads
+    scale = 1.0 / np.sqrt(o.d)
+    plain = o.decode(q, e["kidx"], e["vidx"])
+    # (a) a sink at -inf is no sink
+    np.testing.assert_allclose(o.decode_sink(q, e["kidx"], e["vidx"], np.full(hq, -1e300)), plain, rtol=0, atol=1e-13)
+    # (b) the sink only rescales: o_sink = o_plain * L / (L + exp(s)),  L = sum_j exp(z_j)
+    sink = np.linspace(-2.0, 3.0, hq)
+    got = o.decode_sink(q, e["kidx"], e["vidx"], sink)
+    for h in range(hq):
+        z = (k_hat[:, h // hg, :] @ q[h]) * scale
+        big = np.exp(z).sum()
+        np.testing.assert_allclose(got[h], plain[h] * big / (big + np.exp(sink[h])), rtol=0, atol=1e-12)
+    # (c) one token: p = 1 / (1 + exp(s - z))
+    one = o.decode_sink(q, e["kidx"][:1], e["vidx"][:1], sink)
+    for h in range(hq):
+        z = (k_hat[0, h // hg, :] @ q[h]) * scale
+        np.testing.assert_allclose(one[h], v_hat[0, h // hg, :] / (1.0 + np.exp(sink[h] - z)), rtol=0, atol=1e-12)
+    # (d) empty cache: all the mass on the sink
+    assert not o.decode_sink(q, e["kidx"][:0], e["vidx"][:0], sink).any()
+    # (e) independent numpy restatement on explicit keys/values
+    ref = np.empty_like(got)
+    for h in range(hq):
+        z = np.concatenate([(k_hat[:, h // hg, :] @ q[h]) * scale, [sink[h]]])
+        p = np.exp(z - z.max()); p /= p.sum()
+        ref[h] = p[:-1] @ v_hat[:, h // hg, :]
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(O.attention_sink(q, k_hat, v_hat, sink), ref, rtol=0, atol=1e-12)
+
+
+def test_sink_breaks_key_offset_invariance(tiny_case):
+    """With a sink Lemma S1 no longer holds: moving the key mean changes the output unless the sink logit
+    moves by q.kbar * scale with it (the correction the read path applies)."""
+    o = tiny_case["oracle"]
+    k, v, q = tiny_case["k"][:40], tiny_case["v"][:40], tiny_case["q"]
+    e = o.encode(k, v, with_gaps=False)
+    hq = q.shape[0]
+    sink = np.zeros(hq)
+    base = o.decode_sink(q, e["kidx"], e["vidx"], sink)
+    shift = np.full((1, o.d), 1.0)
+    o2 = O.Oracle(o.rk, o.rk_inv_t, o.rv, o.k_mean + shift, o.v_mean, o.cb_k, o.cb_v)
+    moved = o2.decode_sink(q, e["kidx"], e["vidx"], sink)
+    assert np.abs(moved - base).max() > 1e-3 * np.abs(base).max()
+    fixed = o2.decode_sink(q, e["kidx"], e["vidx"], sink + (q @ shift[0]) / np.sqrt(o.d))
+    np.testing.assert_allclose(fixed, base, rtol=0, atol=1e-12)
