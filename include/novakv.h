@@ -182,6 +182,25 @@ novakv_status novakv_decode_attention_scaled(novakv_ctx* ctx, int layer, const v
     novakv_stream stream);
 
 /*
+ * Decode step with a learned attention sink (App. "Attention sinks in the quantized serving path"):
+ * an extra logit sink_logits[h] per query head that enters the softmax normaliser and has no value,
+ *     p_hj = exp(z_hj) / ( sum_i exp(z_hi) + exp(sink_h) ),   o_h = sum_j p_hj v^_j.
+ * The sink term is added exactly once, after the cross-split merge.  Because the read path drops the
+ * constant q_h . k_mean * sm_scale from every token logit (Lemma S1 no longer applies with a sink),
+ * the kernel shifts the sink logit by the same constant (one d-dimensional dot product per head and
+ * step), and v_mean enters with the token mass sum_j p_hj instead of 1.
+ *   sink_logits  device, float32 [Hq], natural-log units (the units of q.k * sm_scale)
+ *   k_scales     NULL for the 2-bit key format, else the scale pool of novakv_encode_append_scaled
+ * Other arguments, results and errors are those of novakv_decode_attention; a sequence of length 0
+ * yields zeros.
+ */
+novakv_status novakv_decode_attention_sink(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, const float* sink_logits,
+    int n_pages, const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch,
+    float sm_scale, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
+    novakv_stream stream);
+
+/*
  * The same decode step for callers that cannot supply a workspace and cannot allocate one: an
  * engine that gave all device memory to its own pool, a plug-in inside it, a serving loop that must
  * never call cudaMalloc (the call synchronises the device).  (The paper has no counterpart; this is

@@ -22,6 +22,7 @@ EXPORTED = [
     "novakv_bf16_decode_attention", "novakv_profile_enable", "novakv_profile_read",
     "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc", "novakv_debug_set_value_path",
     "novakv_scale_page_bytes", "novakv_encode_append_scaled", "novakv_decode_attention_scaled",
+    "novakv_decode_attention_sink",
 ]
 
 
@@ -74,6 +75,9 @@ def load_library(path=None):
     lib.novakv_decode_attention_scaled.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
                                                    c_void_p, c_int, c_void_p, c_int, c_float, c_void_p, c_int,
                                                    c_void_p, c_size_t, c_void_p]
+    lib.novakv_decode_attention_sink.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                                 c_int, c_void_p, c_int, c_void_p, c_int, c_float, c_void_p, c_int,
+                                                 c_void_p, c_size_t, c_void_p]
     lib.novakv_decode_attention_noalloc.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                                     c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p]
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
@@ -198,6 +202,18 @@ class Context:
             _ptr(page_table), int(page_table.shape[1]), _ptr(seq_lens), batch, scale, _ptr(out),
             1 if out.dtype == torch.float32 else 0, _ptr(workspace),
             int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_scaled")
+
+    def novakv_decode_attention_sink(self, layer, q, k_pages, v_pages, k_scales, sink_logits, page_table, seq_lens,
+                                     out, workspace, sm_scale=None):
+        """Decode step with a learned sink logit per query head (k_scales may be None)."""
+        import torch
+        batch = int(q.shape[0])
+        scale = float(self.head_dim) ** -0.5 if sm_scale is None else float(sm_scale)
+        _check(self.lib, self.lib.novakv_decode_attention_sink(
+            self.handle, layer, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(k_scales) if k_scales is not None else None,
+            _ptr(sink_logits), int(k_pages.shape[0]), _ptr(page_table), int(page_table.shape[1]), _ptr(seq_lens),
+            batch, scale, _ptr(out), 1 if out.dtype == torch.float32 else 0, _ptr(workspace),
+            int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_sink")
 
     def novakv_decode_attention_noalloc(self, layer, q, k_pages, v_pages, page_table, seq_lens, out, sm_scale=None):
         """Decode step whose scratch is the library's fixed device array (no workspace argument)."""

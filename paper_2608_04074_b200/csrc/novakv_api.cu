@@ -63,7 +63,7 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
 
 static void free_layer(novakv_layer& ly) {
     cudaFree(ly.rk_d); cudaFree(ly.rv_d); cudaFree(ly.k_mean_d); cudaFree(ly.v_mean_d);
-    cudaFree(ly.rk_d_mma); cudaFree(ly.rv_d_mma);
+    cudaFree(ly.rk_d_mma); cudaFree(ly.rv_d_mma); cudaFree(ly.k_mean);
     cudaFree(ly.cb_k); cudaFree(ly.cb_v); cudaFree(ly.rk_inv_t); cudaFree(ly.rv_t);
     cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_half); cudaFree(ly.cb_v_mma);
     ly = novakv_layer();
@@ -123,7 +123,7 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
             }
 
     std::vector<double> rk_d(n_mat), rv_d(n_mat), km_d(n_vec, 0.0), vm_d(n_vec, 0.0);
-    std::vector<float> vm_f(n_vec, 0.f);
+    std::vector<float> vm_f(n_vec, 0.f), km_f(n_vec, 0.f);
     for (size_t i = 0; i < n_mat; ++i) { rk_d[i] = (double)h->rk[i]; rv_d[i] = (double)h->rv[i]; }
     // the same matrices with the input dimension blocked by 4: img[h][k/4][c][k%4] = R[h][k][c]
     std::vector<double> rk_mma(n_mat), rv_mma(n_mat);
@@ -134,7 +134,7 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
                 rk_mma[dst] = rk_d[src];
                 rv_mma[dst] = rv_d[src];
             }
-    if (h->k_mean) for (size_t i = 0; i < n_vec; ++i) km_d[i] = (double)h->k_mean[i];
+    if (h->k_mean) for (size_t i = 0; i < n_vec; ++i) { km_d[i] = (double)h->k_mean[i]; km_f[i] = h->k_mean[i]; }
     if (h->v_mean) for (size_t i = 0; i < n_vec; ++i) { vm_d[i] = (double)h->v_mean[i]; vm_f[i] = h->v_mean[i]; }
 
     // key codebook in score-table order: [Hkv][plane][code][e = (m%2)*8 + sigma][4],
@@ -165,7 +165,7 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
               upload(&ly.k_mean_d, km_d) == cudaSuccess && upload(&ly.v_mean_d, vm_d) == cudaSuccess &&
               upload(&ly.cb_k, cbk) == cudaSuccess && upload(&ly.cb_v, cbv) == cudaSuccess &&
               upload(&ly.rk_inv_t, rkinv) == cudaSuccess && upload(&ly.rv_t, rvt) == cudaSuccess &&
-              upload(&ly.v_mean, vm_f) == cudaSuccess && upload(&ly.cb_k_lut, cbk_lut) == cudaSuccess &&
+              upload(&ly.v_mean, vm_f) == cudaSuccess && upload(&ly.k_mean, km_f) == cudaSuccess && upload(&ly.cb_k_lut, cbk_lut) == cudaSuccess &&
               upload(&ly.cb_v_half, cbv_half) == cudaSuccess && upload(&ly.cb_v_mma, cbv_mma) == cudaSuccess;
     if (!ok) { free_layer(ly); return NOVAKV_ECUDA; }
     ly.loaded = true;
@@ -262,6 +262,26 @@ extern "C" novakv_status novakv_decode_attention_scaled(novakv_ctx* ctx, int lay
     return novakv_launch_decode(ctx, ctx->layers[layer], (const __nv_bfloat16*)q, k_pages, v_pages, n_pages,
                                 page_table, max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,
                                 workspace, workspace_bytes, (cudaStream_t)stream, (const __nv_bfloat16*)k_scales);
+}
+
+extern "C" novakv_status novakv_decode_attention_sink(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, const float* sink_logits, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
+    int out_is_fp32, void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!q || !k_pages || !v_pages || !sink_logits || !page_table || !seq_lens || !out) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_pages & 15) || ((uintptr_t)v_pages & 15) || ((uintptr_t)k_scales & 1) || ((uintptr_t)sink_logits & 3)) return NOVAKV_EINVAL;
+    if (!(sm_scale == sm_scale)) return NOVAKV_EINVAL;
+    if (!workspace || workspace_bytes < novakv_decode_ws_bytes(ctx, batch) || ((uintptr_t)workspace & 255)) return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_decode(ctx, ctx->layers[layer], (const __nv_bfloat16*)q, k_pages, v_pages, n_pages,
+                                page_table, max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,
+                                workspace, workspace_bytes, (cudaStream_t)stream, (const __nv_bfloat16*)k_scales,
+                                sink_logits);
 }
 
 extern "C" novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word) {

@@ -67,6 +67,11 @@ struct S1 {
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
 __device__ __forceinline__ int clamp_len(int len, int max_pages) {
     const int cap = max_pages * NOVAKV_PAGE_TOKENS;
     return len < 0 ? 0 : (len > cap ? cap : len);
@@ -82,7 +87,8 @@ __global__ void __launch_bounds__(512)
 novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restrict__ rk_inv_t,
                       const int32_t* __restrict__ seq_lens, int batch, int n_q_heads, int n_kv_heads,
                       int max_pages_per_seq, float scale_log2, float* __restrict__ qp,
-                      int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status) {
+                      int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status,
+                      const float* __restrict__ k_mean /* [Hkv][D] */, float* __restrict__ qk_off /* [batch][Hq] or null */) {
     const int blk = blockIdx.x;
     constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
@@ -143,6 +149,15 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
 #pragma unroll
         for (int p = 0; p < PARTS; ++p) v += red_s[p][h][cc];
         qp[((size_t)b * n_q_heads + kvh * HG + h) * D + cc] = v * scale_log2;
+    }
+    // the constant the read path drops from every logit of a query, q . k_mean * sm_scale (base-2 units):
+    // only a learned sink logit needs it (it must be shifted by the same amount)
+    if (qk_off != nullptr && (threadIdx.x >> 5) < HG) {
+        const int h = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        float acc = 0.f;
+        for (int i = lane; i < D; i += 32) acc = fmaf(q_s[h][i], k_mean[(size_t)kvh * D + i], acc);
+        acc = warp_sum_f(acc);
+        if (lane == 0) qk_off[(size_t)b * n_q_heads + kvh * HG + h] = acc * scale_log2;
     }
 }
 
@@ -706,8 +721,11 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
                            const int32_t* __restrict__ page_prefix, const int32_t* __restrict__ seq_lens,
                            int batch, int n_q_heads, int n_kv_heads, int max_pages_per_seq, int grid_s1,
                            const float* __restrict__ rv_t, const float* __restrict__ v_mean,
-                           void* __restrict__ out, int out_is_fp32) {
+                           void* __restrict__ out, int out_is_fp32,
+                           const float* __restrict__ sink_logits /* [Hq] natural-log units, or null */,
+                           const float* __restrict__ qk_off /* [batch][Hq], base-2 units */) {
     __shared__ float o_s[HG * D];
+    __shared__ float frac_s[HG];      // share of the softmax mass that sits on tokens (1 without a sink)
     constexpr int NT = HG * D > 512 ? 512 : HG * D;
     constexpr int PARTS = NT / D, COLS = D / PARTS;
     const int pair = blockIdx.x;
@@ -749,7 +767,21 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
                 a = fmaf(sc, part_acc[(pidx * HG + h) * D + c], a);
                 lsum = fmaf(sc, part_ml[(pidx * HG + h) * 2 + 1], lsum);
             }
+            float frac = 1.f;
+            if (sink_logits != nullptr) {
+                // learned sink: an extra logit in the normaliser, added exactly once, after the cross-split
+                // combine; it is shifted by the per-query constant the token logits dropped (q . k_mean)
+                const int hq = kvh * HG + h;
+                const float s2 = sink_logits[hq] * 1.4426950408889634f - qk_off[(size_t)b * n_q_heads + hq];
+                const float M2 = fmaxf(M, s2);
+                const float w = ex2(M - M2);
+                const float ltok = lsum * w;
+                lsum = ltok + ex2(s2 - M2);
+                a *= w;
+                frac = ltok / lsum;
+            }
             val = a / lsum;
+            if (c == 0) frac_s[h] = frac;
         }
         o_s[i] = val;
     }
@@ -780,7 +812,7 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         if (pages_b > 0) {
 #pragma unroll
             for (int p = 0; p < PARTS; ++p) o += red_s[p][h][r];
-            o += vm[k];
+            o = fmaf(vm[k], frac_s[h], o);          // sum_j p_j (s^_j R_V^T + v_mean): the mean carries the token mass
         }
         const size_t oi = ((size_t)b * n_q_heads + kvh * HG + h) * D + r;
         if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
@@ -790,7 +822,7 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
 
 // workspace layout
 struct WsLayout {
-    size_t qp, prefix, ml, acc, total;
+    size_t qp, prefix, qk, ml, acc, total;
 };
 WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -799,7 +831,8 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     WsLayout w;
     w.qp = 0;
     w.prefix = al(w.qp + (size_t)batch * hq * d * 4);
-    w.ml = al(w.prefix + ((size_t)batch + 1) * 4);
+    w.qk = al(w.prefix + ((size_t)batch + 1) * 4);
+    w.ml = al(w.qk + (size_t)batch * hq * 4);
     w.acc = al(w.ml + n_part * ctx->hg * 2 * 4);
     w.total = al(w.acc + n_part * ctx->hg * d * 4);
     return w;
@@ -810,18 +843,20 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                               const uint8_t* k_pages, const uint8_t* v_pages, const __nv_bfloat16* k_scales, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens,
                               int batch, float sm_scale, void* out, int out_is_fp32, void* workspace,
-                              cudaStream_t stream) {
+                              cudaStream_t stream, const float* sink_logits) {
     using C = S1<D, HG, VM>;
     const WsLayout w = ws_layout(ctx, batch);
     char* ws = (char*)workspace;
     float* qp = (float*)(ws + w.qp);
     int32_t* prefix = (int32_t*)(ws + w.prefix);
+    float* qk_off = sink_logits ? (float*)(ws + w.qk) : nullptr;
     float* part_ml = (float*)(ws + w.ml);
     float* part_acc = (float*)(ws + w.acc);
     const int hq = ctx->cfg.n_q_heads, hkv = ctx->cfg.n_kv_heads;
 
     novakv_launch_pdl(novakv_prepare_kernel<D, HG>, dim3(batch * hkv + 1), dim3(512), 0, stream, q, ly.rk_inv_t, seq_lens,
-                      batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status);
+                      batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status,
+                      ly.k_mean, qk_off);
     ctx->launches++;
 
     auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC>;
@@ -842,7 +877,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     auto merge = batch * hkv > 2 * ctx->n_sm ? novakv_decode_merge_kernel<D, HG, 2> : novakv_decode_merge_kernel<D, HG, 1>;
     novakv_launch_pdl(merge, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
                       part_ml, part_acc, prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out,
-                      out_is_fp32);
+                      out_is_fp32, sink_logits, qk_off);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
 }
@@ -854,7 +889,8 @@ size_t novakv_decode_ws_bytes(const novakv_ctx* ctx, int batch) { return ws_layo
 novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
-    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream, const __nv_bfloat16* k_scales) {
+    int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream, const __nv_bfloat16* k_scales,
+    const float* sink_logits) {
     (void)workspace_bytes;
     const int d = ctx->cfg.head_dim, hg = ctx->hg;
     if (k_scales != nullptr && ctx->value_path == 0) return NOVAKV_EUNSUPPORTED;   // scaled keys: tensor-core value side only
@@ -863,14 +899,14 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
         if (k_scales != nullptr)                                                                                 \
             return launch_decode_t<DD, HH, true, true>(ctx, ly, q, k_pages, v_pages, k_scales, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
-                                                  workspace, stream);                                            \
+                                                  workspace, stream, sink_logits);                               \
         if (ctx->value_path == 0)                                                                                \
             return launch_decode_t<DD, HH, false, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
-                                                  workspace, stream);                                            \
+                                                  workspace, stream, sink_logits);                               \
         return launch_decode_t<DD, HH, true, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table,  \
                                              max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,     \
-                                             workspace, stream);                                                 \
+                                             workspace, stream, sink_logits);                                    \
     }
     NOVAKV_DISPATCH(128, 1)
     NOVAKV_DISPATCH(128, 2)

@@ -23,6 +23,7 @@ struct novakv_layer {
     double* rk_d_mma = nullptr;   // [Hkv][d/4][d][4]: rk_d with the input dimension blocked by 4 (tensor-core fragments)
     double* rv_d_mma = nullptr;   // same for rv_d
     double* k_mean_d = nullptr;   // [Hkv][d]
+    float* k_mean = nullptr;      // [Hkv][d] (sink-logit offset q . k_mean)
     double* v_mean_d = nullptr;   // [Hkv][d]
     float* cb_k = nullptr;        // [Hkv][L][256][4]  search layout
     float* cb_v = nullptr;        // [Hkv][L][256][4]
@@ -78,7 +79,8 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
     int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream,
-    const __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */);
+    const __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */,
+    const float* sink_logits = nullptr /* learned sink: [Hq], natural-log units */);
 
 // bf16 comparator
 size_t novakv_bf16_ws_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq);

@@ -83,10 +83,14 @@ class PagedCache:
         self.ctx.novakv_encode_append(layer, k_new, v_new, tok_seq, tok_pos, self.k_pages, self.v_pages,
                                       self.page_table, self.seq_lens)
 
-    def decode(self, layer, q, out=None, sm_scale=None):
+    def decode(self, layer, q, out=None, sm_scale=None, sink_logits=None):
         if out is None:
             out = torch.empty((self.batch, self.ctx.n_q_heads, self.ctx.head_dim), dtype=torch.float32,
                               device=self.device)
+        if sink_logits is not None:
+            self.ctx.novakv_decode_attention_sink(layer, q, self.k_pages, self.v_pages, self.k_scales, sink_logits,
+                                                  self.page_table, self.seq_lens, out, self.workspace, sm_scale)
+            return out
         if self.key_scale:
             self.ctx.novakv_decode_attention_scaled(layer, q, self.k_pages, self.v_pages, self.k_scales,
                                                     self.page_table, self.seq_lens, out, self.workspace, sm_scale)

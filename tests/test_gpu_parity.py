@@ -557,3 +557,52 @@ def test_one_long_sequence_all_ctas_share_each_pair(qwen):
     assert case.ctx.novakv_last_device_status() == 0
     ref = case.oracle.decode(q[0].astype(np.float64), encs[0]["kidx"], encs[0]["vidx"])
     print(f"[one 20000-token sequence] max|delta|/||o||inf = {check_output(out[0], ref):.3e}")
+
+
+# --------------------------------------------------------------------------- learned attention-sink logit
+@pytest.mark.parametrize("name,lens", [("gptoss", [2048, 77, 0, 640]), ("qwen", [1, 64, 1000, 3001])])
+def test_sink_decode_matches_oracle(name, lens, request):
+    """Sink logits from far below to far above the token logits; key mean non-zero, so the offset
+    correction of the sink logit is exercised."""
+    case = request.getfixturevalue(name)
+    lens = np.array(lens, np.int32)
+    cache = _cache(case, lens)
+    encs = _fill_with_oracle(case, cache, lens, 900)
+    _, _, q = case.draw(901, 1, len(lens))
+    hq = case.ctx.n_q_heads
+    sink = np.linspace(-6.0, 8.0, hq).astype(np.float32)
+    assert np.abs(case.cal.k_mean).max() > 0
+    out = cache.decode(0, _dev(q, torch.bfloat16), sink_logits=_dev(sink)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    plain = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    worst = 0.0
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert not out[b].any()
+            continue
+        ref = case.oracle.decode_sink(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], sink.astype(np.float64))
+        worst = max(worst, check_output(out[b], ref))
+        if n <= 100:       # the sink is not a no-op: on a short sequence it takes a large share of the mass
+            assert np.abs(plain[b] - ref).max() > 0.05 * np.abs(ref).max()
+    print(f"[{name} {lens.tolist()}] sink: max|delta|/||o||inf = {worst:.3e}")
+
+
+def test_sink_on_scaled_key_format(qwen_scaled):
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = qwen_scaled
+    lens = np.array([700, 65], np.int32)
+    cache = PagedCache(case.ctx, lens, seed=3, key_scale=True)
+    encs = []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(950 + b, int(n), 1)
+        e = case.oracle.encode_scaled(k.astype(np.float64), v.astype(np.float64), with_gaps=False)
+        cache.store_logical(b, 0, e["kidx"], e["vidx"])
+        cache.store_scales(b, 0, e["kscale"])
+        encs.append(e)
+    _, _, q = case.draw(951, 1, 2)
+    sink = np.linspace(-3.0, 5.0, case.ctx.n_q_heads).astype(np.float32)
+    out = cache.decode(0, _dev(q, torch.bfloat16), sink_logits=_dev(sink)).cpu().numpy()
+    for b in range(2):
+        ref = case.oracle.decode_sink(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], sink.astype(np.float64),
+                                      kscale=encs[b]["kscale"])
+        check_output(out[b], ref)
