@@ -5,6 +5,8 @@
 // of the CTA's head and side stays in shared memory and every warp reads codewords as broadcasts.
 #include <math_constants.h>
 
+#include <cooperative_groups.h>
+
 #include "novakv_internal.cuh"
 
 namespace {
@@ -393,7 +395,11 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 // Everything that depends only on the calibration is staged before the grid-dependency wait, so it
 // overlaps the tail of the preceding kernel in the stream.
 // Arithmetic is identical to the tiled kernel (binary64 accumulation in index order, dist4 search).
-template <int D>
+// KSC (key format with a per-token scale): the L/4 CTAs of a (head, side) form a thread-block cluster;
+// each publishes the sums of squares of its 16 coefficients per token in its shared memory, a cluster
+// barrier makes them visible, and every CTA adds the L/4 x 4 partial sums in the same fixed order through
+// distributed shared memory, so that all of them normalise by the same rho.
+template <int D, bool KSC>
 __global__ void __launch_bounds__(128)
 novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                            const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
@@ -401,11 +407,13 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                            const double* __restrict__ rk_d, const double* __restrict__ rv_d,
                            const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
                            const float* __restrict__ cb_k, const float* __restrict__ cb_v,
-                           uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages, int n_pages,
+                           uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages,
+                           __nv_bfloat16* __restrict__ k_scales, int n_pages,
                            const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                            int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
     constexpr int L = D / NOVAKV_G;
     __shared__ __align__(16) double R_s[4][D][4];
+    __shared__ double ss_s[4][32];                  // KSC: sum of squares of a warp's 4 coefficients, per token of the pass
     __shared__ float4 cb_s[4][NOVAKV_C];
     __shared__ double mean_s[D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -485,7 +493,33 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                 acc3 = fma(xc, r23.y, acc3);
             }
         }
-        const float4 r = make_float4((float)acc0, (float)acc1, (float)acc2, (float)acc3);
+        float4 r = make_float4((float)acc0, (float)acc1, (float)acc2, (float)acc3);
+        if (KSC) {
+            namespace cg = cooperative_groups;
+            cg::cluster_group cluster = cg::this_cluster();
+            if (side == 0 && grp == 0) {
+                double ss = (double)r.x * (double)r.x;
+                ss = fma((double)r.y, (double)r.y, ss);
+                ss = fma((double)r.z, (double)r.z, ss);
+                ss = fma((double)r.w, (double)r.w, ss);
+                ss_s[warp][tok_in_pass] = ss;
+            }
+            cluster.sync();                             // every CTA of the (head, side) has published its partial sums
+            if (side == 0) {
+                double tot = 0.0;
+                for (unsigned cr = 0; cr < cluster.num_blocks(); ++cr) {
+                    const double* remote = cluster.map_shared_rank(&ss_s[0][0], cr);
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) tot += remote[w * 32 + tok_in_pass];
+                }
+                float rho = __bfloat162float(__float2bfloat16_rn((float)sqrt(tot / (double)D)));
+                if (!(rho > 0.f) || !isfinite(rho)) rho = 1.f;
+                r = make_float4(__fdiv_rn(r.x, rho), __fdiv_rn(r.y, rho), __fdiv_rn(r.z, rho), __fdiv_rn(r.w, rho));
+                if (blockIdx.x == 0 && warp == 0 && grp == 0 && page >= 0)
+                    k_scales[((size_t)page * n_kv_heads + kvh) * NOVAKV_PAGE_TOKENS + slot] = __float2bfloat16_rn(rho);
+            }
+            cluster.sync();                             // partial sums may be overwritten by the next pass / CTAs may exit
+        }
         // this lane group's range of the codebook, ascending with a strict '<' (first minimum)
         float best = dist4(r, cb_s[warp][c0]);
         int bi = c0;
@@ -547,15 +581,39 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                               int n_tokens, uint8_t* k_pages, uint8_t* v_pages, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
                               cudaStream_t stream, __nv_bfloat16* k_scales) {
-    // (the scaled key format needs all coefficients of a token in one CTA: it always takes the tiled kernel)
-    if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS && k_scales == nullptr) {
+    if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS) {
         dim3 grid(D / NOVAKV_G / 4, ctx->cfg.n_kv_heads, 2);
         novakv_prof_scope ps(ctx, 1, stream);
         int tp_log2 = 0;
         while ((1 << tp_log2) < n_tokens && tp_log2 < 5) ++tp_log2;
-        novakv_launch_pdl(novakv_encode_small_kernel<D>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos, n_tokens,
-                          tp_log2, ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, n_pages,
-                          page_table, max_pages_per_seq, n_seq, seq_lens, ctx->cfg.n_kv_heads, ctx->dev_status);
+        if (k_scales == nullptr) {
+            novakv_launch_pdl(novakv_encode_small_kernel<D, false>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos,
+                              n_tokens, tp_log2, ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages,
+                              (__nv_bfloat16*)nullptr, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
+                              ctx->cfg.n_kv_heads, ctx->dev_status);
+        } else {
+            // scaled key format: the L/4 CTAs of a (head, side) are one cluster (8 at d = 128, 4 at d = 64)
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = grid;
+            cfg.blockDim = dim3(128);
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = grid.x;
+            attr[1].val.clusterDim.y = 1;
+            attr[1].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 2;
+            const int hkv = ctx->cfg.n_kv_heads;
+            if (cudaLaunchKernelEx(&cfg, novakv_encode_small_kernel<D, true>, k_new, v_new, tok_seq, tok_pos, n_tokens, tp_log2,
+                                   (const double*)ly.rk_d, (const double*)ly.rv_d, (const double*)ly.k_mean_d,
+                                   (const double*)ly.v_mean_d, (const float*)ly.cb_k, (const float*)ly.cb_v, k_pages, v_pages,
+                                   k_scales, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens, hkv,
+                                   ctx->dev_status) != cudaSuccess)
+                return NOVAKV_ECUDA;
+        }
         ps.end();
         ctx->launches++;
         return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;

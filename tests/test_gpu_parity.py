@@ -425,14 +425,16 @@ def gptoss_scaled():
     return Case(workloads.gpt_oss_20b(batch=2, seq_len=2048, calib_tokens=4096, lloyd_iters=6), key_scale=True)
 
 
+@pytest.mark.parametrize("add", [[200, 64, 1, 130], [20, 7, 1, 3], [1, 0, 0, 0], [70, 60, 50, 40]])
 @pytest.mark.parametrize("name", ["qwen_scaled", "gptoss_scaled"])
-def test_scaled_encode_matches_oracle_indices_and_scales(name, request):
-    """Append (tiled kernel: a long run, a ragged tail, a single token) on the scaled key format:
+def test_scaled_encode_matches_oracle_indices_and_scales(name, add, request):
+    """Append on the scaled key format, through the tiled kernel (395 tokens: a long run, a ragged tail, a
+    single token) and through the clustered append kernel (31, 1 and 220 tokens: one, one and seven passes):
     indices as in the unscaled test, scales bit for bit (bfloat16)."""
     from paper_2608_04074_b200.runtime import PagedCache
     case = request.getfixturevalue(name)
     lens0 = np.array([0, 5, 63, 130], np.int32)
-    add = np.array([200, 64, 1, 130], np.int32)
+    add = np.array(add, np.int32)
     cache = PagedCache(case.ctx, lens0, capacity_tokens=lens0 + add, seed=3, key_scale=True)
     n = int(add.sum())
     k, v, _ = case.draw(210, n, 1)
@@ -453,7 +455,7 @@ def test_scaled_encode_matches_oracle_indices_and_scales(name, request):
         got_k[t], got_v[t] = kk[0], vv[0]
         got_s[t] = cache.load_scales(int(tok_seq[t]), int(tok_pos[t]), 1)[0]
     assert np.array_equal(got_s, enc["kscale"]), f"{int((got_s != enc['kscale']).sum())} scales differ"
-    assert len(np.unique(enc["kscale"])) > 8
+    assert n < 100 or len(np.unique(enc["kscale"])) > 8
     dk, nk = check_indices(got_k, enc, "k")
     dv, nv = check_indices(got_v, enc, "v")
     print(f"[{name}] scaled format: index mismatches K {dk} V {dv}; near-ties K {nk} V {nv} of {got_k.size}")
