@@ -233,7 +233,9 @@ novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, u
  *   k_new_host, v_new_host  bf16 [n_tokens][Hkv][d];  tok_seq_host, tok_pos_host int32 [n_tokens]
  *   q_host   bf16 [batch][Hq][d];  out_host  float32 [batch][Hq][d]
  *   staging  device scratch of novakv_step_staging_bytes(ctx, batch, n_tokens) bytes
- * For pinned host memory the copies are asynchronous until the final synchronise.
+ * A buffer in page-locked (pinned, device-mapped) host memory is read or written by the kernels
+ * directly across the bus; any other host buffer is staged through `staging` with a copy on `stream`.
+ * Either way the step's inputs travel host -> device and its output device -> host inside the call.
  */
 size_t novakv_step_staging_bytes(const novakv_ctx* ctx, int batch, int n_tokens);
 novakv_status novakv_step_host(novakv_ctx* ctx, int layer,

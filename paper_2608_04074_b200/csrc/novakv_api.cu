@@ -329,22 +329,52 @@ extern "C" novakv_status novakv_step_host(novakv_ctx* ctx, int layer, const void
     char* dpos = p; p += align256(tok_b);
     char* dq = p; p += align256(q_b);
     char* dout = p;
+    // Page-locked host buffers are visible to the device under unified addressing: one small kernel pulls
+    // all of the step's inputs across the bus (every byte once, coalesced) into `staging`, instead of five
+    // copy-engine operations queued one after the other; the merge kernel writes the output straight into
+    // the page-locked output buffer.  A buffer that is not page-locked (or not mapped, or not 4-byte
+    // aligned) is staged with an asynchronous copy instead.
+    auto device_view = [](const void* host_ptr) -> const void* {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return (at.type == cudaMemoryTypeHost && at.devicePointer != nullptr) ? at.devicePointer : nullptr;
+    };
+    novakv_stage_args sa;
+    sa.n = 0;
+    auto stage_in = [&](const void* host_ptr, char* dev_buf, size_t bytes) -> cudaError_t {
+        const void* view = device_view(host_ptr);
+        if (view != nullptr && ((uintptr_t)view & 3) == 0 && (bytes & 3) == 0) {
+            sa.src[sa.n] = (const uint32_t*)view;
+            sa.dst[sa.n] = (uint32_t*)dev_buf;
+            sa.words[sa.n] = (unsigned)(bytes / 4);
+            ++sa.n;
+            return cudaSuccess;
+        }
+        return cudaMemcpyAsync(dev_buf, host_ptr, bytes, cudaMemcpyHostToDevice, s);
+    };
     if (n_tokens > 0) {
-        CUDA_OK(cudaMemcpyAsync(dk, k_new_host, kv_b, cudaMemcpyHostToDevice, s));
-        CUDA_OK(cudaMemcpyAsync(dv, v_new_host, kv_b, cudaMemcpyHostToDevice, s));
-        CUDA_OK(cudaMemcpyAsync(dseq, tok_seq_host, tok_b, cudaMemcpyHostToDevice, s));
-        CUDA_OK(cudaMemcpyAsync(dpos, tok_pos_host, tok_b, cudaMemcpyHostToDevice, s));
+        CUDA_OK(stage_in(k_new_host, dk, kv_b));
+        CUDA_OK(stage_in(v_new_host, dv, kv_b));
+        CUDA_OK(stage_in(tok_seq_host, dseq, tok_b));
+        CUDA_OK(stage_in(tok_pos_host, dpos, tok_b));
     }
-    CUDA_OK(cudaMemcpyAsync(dq, q_host, q_b, cudaMemcpyHostToDevice, s));
+    CUDA_OK(stage_in(q_host, dq, q_b));
+    if (sa.n > 0) {
+        if (novakv_launch_stage(ctx, sa, s) != NOVAKV_OK) return NOVAKV_ECUDA;
+    }
+    const void *uk = dk, *uv = dv, *useq = dseq, *upos = dpos, *uq = dq;
+    void* uout = const_cast<void*>(device_view(out_host));
+    const bool out_direct = uout != nullptr;
+    if (!out_direct) uout = dout;
     if (n_tokens > 0) {
-        st = novakv_encode_append(ctx, layer, dk, dv, (const int32_t*)dseq, (const int32_t*)dpos, n_tokens,
+        st = novakv_encode_append(ctx, layer, uk, uv, (const int32_t*)useq, (const int32_t*)upos, n_tokens,
                                   k_pages, v_pages, n_pages, page_table, max_pages_per_seq, batch, seq_lens, stream);
         if (st != NOVAKV_OK) return st;
     }
-    st = novakv_decode_attention(ctx, layer, dq, k_pages, v_pages, n_pages, page_table, max_pages_per_seq,
-                                 seq_lens, batch, sm_scale, dout, 1, workspace, workspace_bytes, stream);
+    st = novakv_decode_attention(ctx, layer, uq, k_pages, v_pages, n_pages, page_table, max_pages_per_seq,
+                                 seq_lens, batch, sm_scale, uout, 1, workspace, workspace_bytes, stream);
     if (st != NOVAKV_OK) return st;
-    CUDA_OK(cudaMemcpyAsync(out_host, dout, o_b, cudaMemcpyDeviceToHost, s));
+    if (!out_direct) CUDA_OK(cudaMemcpyAsync(out_host, dout, o_b, cudaMemcpyDeviceToHost, s));
     CUDA_OK(cudaStreamSynchronize(s));
     return NOVAKV_OK;
 }

@@ -674,6 +674,29 @@ novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, cons
                                page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales);
 }
 
+// Gather of up to 5 page-locked host buffers into device staging: every 32-bit word crosses the bus
+// once, consecutive threads take consecutive words (128-byte requests per warp).
+__global__ void __launch_bounds__(256) novakv_stage_kernel(const novakv_stage_args a) {
+    const unsigned stride = gridDim.x * blockDim.x;
+#pragma unroll 1
+    for (int sgm = 0; sgm < a.n; ++sgm) {
+        const uint32_t* __restrict__ src = a.src[sgm];
+        uint32_t* __restrict__ dst = a.dst[sgm];
+        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < a.words[sgm]; i += stride) dst[i] = src[i];
+    }
+}
+
+novakv_status novakv_launch_stage(novakv_ctx* ctx, const novakv_stage_args& a, cudaStream_t stream) {
+    unsigned total = 0;
+    for (int i = 0; i < a.n; ++i) total += a.words[i];
+    if (total == 0) return NOVAKV_OK;
+    unsigned blocks = (total + 255) / 256;
+    if (blocks > (unsigned)(2 * ctx->n_sm)) blocks = 2 * ctx->n_sm;
+    novakv_stage_kernel<<<blocks, 256, 0, stream>>>(a);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
+}
+
 novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef,
     int n, uint8_t* idx_out, cudaStream_t stream) {
     if (ctx->cfg.head_dim == 128) return launch_search_t<128>(ctx, ly, which, coef, n, idx_out, stream);

@@ -82,6 +82,15 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
     const __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */,
     const float* sink_logits = nullptr /* learned sink: [Hq], natural-log units */);
 
+// gather of page-locked host buffers into device staging (one kernel for up to 5 segments of 32-bit words)
+struct novakv_stage_args {
+    const uint32_t* src[5];
+    uint32_t* dst[5];
+    unsigned words[5];
+    int n;
+};
+novakv_status novakv_launch_stage(novakv_ctx* ctx, const novakv_stage_args& a, cudaStream_t stream);
+
 // bf16 comparator
 size_t novakv_bf16_ws_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq);
 novakv_status novakv_launch_bf16_decode(novakv_ctx* ctx, const __nv_bfloat16* q,

@@ -205,7 +205,7 @@ def test_bf16_output_and_custom_scale(qwen):
 def test_step_host_equals_device_calls(qwen):
     case = qwen
     lens0 = np.array([300, 65], np.int32)
-    caches = [_cache(case, lens0, capacity=lens0 + 1, seed=9) for _ in range(2)]
+    caches = [_cache(case, lens0, capacity=lens0 + 1, seed=9) for _ in range(3)]
     for c in caches:
         _fill_with_oracle(case, c, lens0, 700)
     k1, v1, q = case.draw(701, 2, 2)
@@ -223,6 +223,16 @@ def test_step_host_equals_device_calls(qwen):
                               staging, c.workspace)
     assert torch.equal(out_h, ref)
     assert torch.equal(caches[0].k_pages, c.k_pages) and torch.equal(caches[0].v_pages, c.v_pages)
+    # pageable (not page-locked) host buffers take the staged-copy route: same result
+    c = caches[2]
+    host = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(dt) if dt else torch.from_numpy(np.ascontiguousarray(a)).clone())
+    out_p = torch.empty((2, case.ctx.n_q_heads, case.ctx.head_dim), dtype=torch.float32)
+    case.ctx.novakv_step_host(0, host(k1, torch.bfloat16), host(v1, torch.bfloat16), host(seq), host(pos),
+                              host(q, torch.bfloat16), c.k_pages, c.v_pages, c.page_table, c.seq_lens, out_p,
+                              staging, c.workspace)
+    assert torch.equal(out_p, ref)
+    assert torch.equal(caches[0].k_pages, c.k_pages) and torch.equal(caches[0].v_pages, c.v_pages)
+    assert case.ctx.novakv_last_device_status() == 0
 
 
 # --------------------------------------------------------------------------- T7: host-injected faults
