@@ -245,6 +245,28 @@ class Oracle:
                                    ctypes.c_void_p(out.ctypes.data))
         return out
 
+    def decode_banded(self, q, kidx, vidx, k_exact, v_exact, band_mask, kscale=None, sink=None,
+                      sm_scale: float | None = None):
+        """Decode step on a cache whose tokens are partly held exactly (Fig. "Cache layout at decoding
+        position t": the first n_sink and the most recent n_rec tokens stay in BF16, the tokens in between
+        are quantised).  Every position is dequantised explicitly; positions with band_mask[j] set take the
+        exact (bf16-representable) key and value instead; textbook attention follows.
+
+        kidx, vidx [S][Hkv][L] (entries at band positions are ignored), k_exact / v_exact [S][Hkv][d],
+        band_mask bool [S]."""
+        band_mask = np.asarray(band_mask, bool)
+        if kscale is None:
+            k_hat, v_hat = self.reconstruct(kidx, vidx)
+        else:
+            k_hat, v_hat = self.reconstruct_scaled(kidx, vidx, kscale)
+        k_hat[band_mask] = _f64(k_exact)[band_mask]
+        v_hat[band_mask] = _f64(v_exact)[band_mask]
+        if k_hat.shape[0] == 0:
+            return np.zeros((np.asarray(q).shape[0], self.d))
+        if sink is None:
+            return attention(q, k_hat, v_hat, sm_scale)
+        return attention_sink(q, k_hat, v_hat, sink, sm_scale)
+
 
 def attention_sink(q, k, v, sink, sm_scale: float | None = None):
     """Textbook attention with an extra value-less logit per head: q [Hq][d], k/v [S][Hkv][d], sink [Hq]."""

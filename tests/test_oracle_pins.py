@@ -538,3 +538,32 @@ def test_sink_breaks_key_offset_invariance(tiny_case):
     assert np.abs(moved - base).max() > 1e-3 * np.abs(base).max()
     fixed = o2.decode_sink(q, e["kidx"], e["vidx"], sink + (q @ shift[0]) / np.sqrt(o.d))
     np.testing.assert_allclose(fixed, base, rtol=0, atol=1e-12)
+
+
+# ---- BF16 sink-plus-recent band (Fig. "Cache layout at decoding position t") ----
+def test_banded_decode_limits_and_mixture(tiny_case):
+    o = tiny_case["oracle"]
+    k, v, q = tiny_case["k"][:200], tiny_case["v"][:200], tiny_case["q"]
+    e = o.encode(k, v, with_gaps=False)
+    hq = q.shape[0]
+    hg = hq // o.n_kv_heads
+    scale = 1.0 / np.sqrt(o.d)
+    # (a) no band: the plain quantised decode
+    none = np.zeros(200, bool)
+    np.testing.assert_allclose(o.decode_banded(q, e["kidx"], e["vidx"], k, v, none),
+                               o.decode(q, e["kidx"], e["vidx"]), rtol=0, atol=1e-13)
+    # (b) everything in the band: exact attention on the raw keys and values, the indices are irrelevant
+    full = np.ones(200, bool)
+    junk = np.zeros_like(e["kidx"])
+    exact = np.stack([np_attention(q[h], k[:, h // hg, :], v[:, h // hg, :], scale) for h in range(hq)])
+    np.testing.assert_allclose(o.decode_banded(q, junk, junk, k, v, full), exact, rtol=0, atol=1e-12)
+    # (c) sink of 64 and 100 recent tokens: an independent mixture of exact and dequantised rows
+    mask = np.zeros(200, bool); mask[:64] = True; mask[100:] = True
+    k_hat, v_hat = o.reconstruct(e["kidx"], e["vidx"])
+    km, vm = np.where(mask[:, None, None], k, k_hat), np.where(mask[:, None, None], v, v_hat)
+    ref = np.stack([np_attention(q[h], km[:, h // hg, :], vm[:, h // hg, :], scale) for h in range(hq)])
+    got = o.decode_banded(q, e["kidx"], e["vidx"], k, v, mask)
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-12)
+    # the band matters: the result moves towards the exact attention
+    plain = o.decode(q, e["kidx"], e["vidx"])
+    assert np.abs(got - exact).max() < np.abs(plain - exact).max()
