@@ -543,7 +543,8 @@ def test_sink_breaks_key_offset_invariance(tiny_case):
 # ---- BF16 sink-plus-recent band (Fig. "Cache layout at decoding position t") ----
 def test_banded_decode_limits_and_mixture(tiny_case):
     o = tiny_case["oracle"]
-    k, v, q = tiny_case["k"][:200], tiny_case["v"][:200], tiny_case["q"]
+    k, v, q = (np.asarray(tiny_case[n], np.float64) for n in ("k", "v", "q"))
+    k, v = k[:200], v[:200]
     e = o.encode(k, v, with_gaps=False)
     hq = q.shape[0]
     hg = hq // o.n_kv_heads
