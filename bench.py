@@ -461,6 +461,28 @@ def run_ours(args):
                       "device_status": ctx.novakv_last_device_status()})
         del c6, q6, o6
         torch.cuda.empty_cache()
+        # BF16 sink-plus-recent band (64 + 256 tokens in bf16, the rest in the index cache), primary key format
+        from paper_2608_04074_b200.runtime import BandedCache
+        c7 = BandedCache(ctx, b6, s6 + 64, n_sink=64, n_rec=256, block=8, seed=43, device=dev)
+        fill_cache_gpu(ctx, c7.paged, laws, wl6.seq_lens, seed=9300, share_content=True)
+        c7.total[:] = s6
+        c7.quant[:] = s6 - 64 - 256
+        c7.ring_len[:] = 256
+        c7.band_k.normal_(); c7.band_v.normal_()
+        c7._sync_meta()
+        q7 = bf16_tensor(synth.draw_q(laws, 7500, b6), dev)
+        o7 = torch.empty((b6, s.n_q_heads, s.head_dim), dtype=torch.float32, device=dev)
+        td7 = time_steps(lambda: c7.decode(0, q7, out=o7), max(5, args.steps // 2), 3, lambda: None)
+        ms7 = statistics.median(td7)
+        ab7 = ab6 - int(wl6.seq_lens.astype(np.int64).sum()) * s.n_kv_heads * 2            # no scales here
+        ab7 += b6 * s.n_kv_heads * 320 * (2 * s.head_dim * 2 - 2 * (s.head_dim // 4))          # 320 tokens in bf16 instead of indices
+        sweep.append({"workload": f"BF16 sink-plus-recent band (64 + 256 tokens exact, deferred quantisation in blocks of 8), "
+                                  f"qwen3_8b_shape B={b6} S={s6}: decode only (timing only: band content random)",
+                      "ms": round(ms7, 4), "gbps": round(ab7 / (ms7 * 1e-3) / 1e9, 1),
+                      "pct_of_8TBps": round(100 * ab7 / (ms7 * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
+                      "algorithmic_bytes": ab7, "device_status": ctx.novakv_last_device_status()})
+        del c7, q7, o7
+        torch.cuda.empty_cache()
         # GPT-OSS-20B-shaped hybrid pair: full-attention layer on the 2-bit cache + sliding-window (128) layer in bf16
         wl4 = workloads.gpt_oss_20b(batch=16, seq_len=65536)
         laws4 = wl4.laws()

@@ -201,6 +201,32 @@ novakv_status novakv_decode_attention_sink(novakv_ctx* ctx, int layer, const voi
     novakv_stream stream);
 
 /*
+ * Decode step on a cache with a BF16 sink-plus-recent band (Sec. 5 "Baselines"; App. B "Sink-plus-recent
+ * band" and its figure "Cache layout at decoding position t"): the first n_sink tokens and the most
+ * recent tokens of a sequence are held exactly in bf16 and excluded from quantisation; the tokens in
+ * between are read from the index cache.  The softmax runs over all of them: the band contributes one
+ * more partial (max, sum, sum_j p_j v_j in the original value domain) to the exact merge.
+ *   index cache  positions n_sink .. n_sink + quant_lens[b] - 1 of sequence b (page column n_sink/64
+ *                onwards of its page-table row); quant_lens device int32 [batch]; n_sink a multiple of 64
+ *   band_k, band_v  device bf16 [batch][band_cap][Hkv][d].  Of sequence b, slots 0 .. sink_cnt-1 hold
+ *                its first tokens, and slots n_sink + (ring_start + i) % (band_cap - n_sink),
+ *                i < ring_len, its most recent ones (a ring: "new tokens enter the BF16 recent band and
+ *                are quantized in blocks of eight steps" - the caller appends to the ring and, when it
+ *                has grown by eight, passes the eight oldest to novakv_encode_append[_scaled] and
+ *                advances ring_start and quant_lens)
+ *   band_meta    device int32 [batch][3] = (sink_cnt, ring_start, ring_len); values are clamped to the
+ *                buffer
+ *   k_scales, sink_logits  NULL or as in novakv_decode_attention_scaled / _sink
+ * A sequence with no token at all yields zeros.  Other arguments and errors as novakv_decode_attention.
+ */
+novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, const float* sink_logits,
+    int n_pages, const int32_t* page_table, int max_pages_per_seq, const int32_t* quant_lens,
+    const void* band_k, const void* band_v, int band_cap, int n_sink, const int32_t* band_meta,
+    int batch, float sm_scale, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
+    novakv_stream stream);
+
+/*
  * The same decode step for callers that cannot supply a workspace and cannot allocate one: an
  * engine that gave all device memory to its own pool, a plug-in inside it, a serving loop that must
  * never call cudaMalloc (the call synchronises the device).  (The paper has no counterpart; this is

@@ -22,7 +22,7 @@ EXPORTED = [
     "novakv_bf16_decode_attention", "novakv_profile_enable", "novakv_profile_read",
     "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc", "novakv_debug_set_value_path",
     "novakv_scale_page_bytes", "novakv_encode_append_scaled", "novakv_decode_attention_scaled",
-    "novakv_decode_attention_sink",
+    "novakv_decode_attention_sink", "novakv_decode_attention_banded",
 ]
 
 
@@ -78,6 +78,10 @@ def load_library(path=None):
     lib.novakv_decode_attention_sink.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                  c_int, c_void_p, c_int, c_void_p, c_int, c_float, c_void_p, c_int,
                                                  c_void_p, c_size_t, c_void_p]
+    lib.novakv_decode_attention_banded.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                                   c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_int,
+                                                   c_void_p, c_int, c_float, c_void_p, c_int, c_void_p, c_size_t,
+                                                   c_void_p]
     lib.novakv_decode_attention_noalloc.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                                     c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p]
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
@@ -214,6 +218,20 @@ class Context:
             _ptr(sink_logits), int(k_pages.shape[0]), _ptr(page_table), int(page_table.shape[1]), _ptr(seq_lens),
             batch, scale, _ptr(out), 1 if out.dtype == torch.float32 else 0, _ptr(workspace),
             int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_sink")
+
+    def novakv_decode_attention_banded(self, layer, q, k_pages, v_pages, k_scales, sink_logits, page_table,
+                                       quant_lens, band_k, band_v, n_sink, band_meta, out, workspace, sm_scale=None):
+        """Decode step on a cache with a BF16 sink-plus-recent band (band_k/band_v [batch][cap][Hkv][d])."""
+        import torch
+        batch = int(q.shape[0])
+        scale = float(self.head_dim) ** -0.5 if sm_scale is None else float(sm_scale)
+        _check(self.lib, self.lib.novakv_decode_attention_banded(
+            self.handle, layer, _ptr(q), _ptr(k_pages), _ptr(v_pages),
+            _ptr(k_scales) if k_scales is not None else None, _ptr(sink_logits) if sink_logits is not None else None,
+            int(k_pages.shape[0]), _ptr(page_table), int(page_table.shape[1]), _ptr(quant_lens), _ptr(band_k),
+            _ptr(band_v), int(band_k.shape[1]), int(n_sink), _ptr(band_meta), batch, scale, _ptr(out),
+            1 if out.dtype == torch.float32 else 0, _ptr(workspace),
+            int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_banded")
 
     def novakv_decode_attention_noalloc(self, layer, q, k_pages, v_pages, page_table, seq_lens, out, sm_scale=None):
         """Decode step whose scratch is the library's fixed device array (no workspace argument)."""

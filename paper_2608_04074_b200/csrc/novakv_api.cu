@@ -284,6 +284,35 @@ extern "C" novakv_status novakv_decode_attention_sink(novakv_ctx* ctx, int layer
                                 sink_logits);
 }
 
+extern "C" novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, const float* sink_logits, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, const int32_t* quant_lens, const void* band_k,
+    const void* band_v, int band_cap, int n_sink, const int32_t* band_meta, int batch, float sm_scale, void* out,
+    int out_is_fp32, void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!q || !k_pages || !v_pages || !page_table || !quant_lens || !band_k || !band_v || !band_meta || !out) return NOVAKV_EINVAL;
+    if (n_sink < 0 || n_sink % NOVAKV_PAGE_TOKENS != 0 || band_cap < n_sink) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= n_sink / NOVAKV_PAGE_TOKENS) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_pages & 15) || ((uintptr_t)v_pages & 15) || ((uintptr_t)k_scales & 1) || ((uintptr_t)sink_logits & 3) ||
+        ((uintptr_t)band_k & 3) || ((uintptr_t)band_v & 3)) return NOVAKV_EINVAL;
+    if (!(sm_scale == sm_scale)) return NOVAKV_EINVAL;
+    if (!workspace || workspace_bytes < novakv_decode_ws_bytes(ctx, batch) || ((uintptr_t)workspace & 255)) return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    novakv_band_args band;
+    band.k = (const __nv_bfloat16*)band_k;
+    band.v = (const __nv_bfloat16*)band_v;
+    band.cap = band_cap;
+    band.n_sink = n_sink;
+    band.meta = band_meta;
+    return novakv_launch_decode(ctx, ctx->layers[layer], (const __nv_bfloat16*)q, k_pages, v_pages, n_pages,
+                                page_table, max_pages_per_seq, quant_lens, batch, sm_scale, out, out_is_fp32,
+                                workspace, workspace_bytes, (cudaStream_t)stream, (const __nv_bfloat16*)k_scales,
+                                sink_logits, &band);
+}
+
 extern "C" novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word) {
     if (!ctx || !word) return NOVAKV_EINVAL;
     cudaStream_t s = (cudaStream_t)stream;

@@ -351,7 +351,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                             const int32_t* __restrict__ page_table, int max_pages_per_seq,
                             const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ page_prefix,
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
-                            float* __restrict__ part_acc, uint32_t* __restrict__ dev_status) {
+                            float* __restrict__ part_acc, uint32_t* __restrict__ dev_status, int pt_stride) {
+    // page_table points at the first column that is scanned; rows are pt_stride entries apart and
+    // max_pages_per_seq bounds the pages of a row that may be read from there
     using C = S1<D, HG, VM>;
     constexpr int L = C::L, GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, NGB = C::NGB, KPL = C::KPL;
     constexpr int TILE_BYTES = C::TILE_BYTES, PAGE_BYTES = 2 * TILE_BYTES;
@@ -408,7 +410,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
         // this warp's tiles of the segment: half pages hp = warp, warp + NCW, ...
         const int n_it = (2 * sg.npg > warp) ? (2 * sg.npg - warp + NCW - 1) / NCW : 0;
-        const int32_t* pt = page_table + (size_t)sg.b * max_pages_per_seq + sg.pg0;
+        const int32_t* pt = page_table + (size_t)sg.b * pt_stride + sg.pg0;
         // page ids of 32 consecutive tiles of this warp, one per lane (coalesced gather, loaded a batch ahead)
         auto load_ids = [&](int batch_i) {
             const int it = batch_i * 32 + lane;
@@ -723,9 +725,12 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
                            const float* __restrict__ rv_t, const float* __restrict__ v_mean,
                            void* __restrict__ out, int out_is_fp32,
                            const float* __restrict__ sink_logits /* [Hq] natural-log units, or null */,
-                           const float* __restrict__ qk_off /* [batch][Hq], base-2 units */) {
+                           const float* __restrict__ qk_off /* [batch][Hq], base-2 units */,
+                           const float* __restrict__ band_ml /* [batch][Hq][2] (max, sum) of the BF16 band, or null */,
+                           const float* __restrict__ band_acc /* [batch][Hq][D] sum p v of the band, original value domain */) {
     __shared__ float o_s[HG * D];
-    __shared__ float frac_s[HG];      // share of the softmax mass that sits on tokens (1 without a sink)
+    __shared__ float frac_s[HG];      // share of the softmax mass on quantised tokens (1 without sink and band)
+    __shared__ float bsc_s[HG];       // multiplier of the band accumulator (0 without a band)
     constexpr int NT = HG * D > 512 ? 512 : HG * D;
     constexpr int PARTS = NT / D, COLS = D / PARTS;
     const int pair = blockIdx.x;
@@ -748,18 +753,16 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
     const int slot0 = kvh * batch + b;                     // the scan kernel's pair index (walk order)
     for (int i = threadIdx.x; i < HG * D; i += blockDim.x) {
         const int h = i / D, c = i - h * D;
-        float val = 0.f;
+        float M = M_INIT, a = 0.f, lsum = 0.f;
         if (pages_b > 0) {
             const long u0 = (long)kvh * P + page_prefix[b], u1 = u0 + pages_b;
             // CTA of unit u: the largest c with floor(c*U/G) <= u
             const int c_first = (int)(((u0 + 1) * grid_s1 - 1) / U), c_last = (int)((u1 * grid_s1 - 1) / U);
             // CTAs in between whose own range is empty wrote nothing: skip them
-            float M = M_INIT;
             for (int cta = c_first; cta <= c_last; ++cta) {
                 if (((long)cta * U) / grid_s1 >= ((long)(cta + 1) * U) / grid_s1) continue;
                 M = fmaxf(M, part_ml[(((size_t)slot0 + cta) * HG + h) * 2]);
             }
-            float a = 0.f, lsum = 0.f;
             for (int cta = c_first; cta <= c_last; ++cta) {
                 if (((long)cta * U) / grid_s1 >= ((long)(cta + 1) * U) / grid_s1) continue;
                 const size_t pidx = (size_t)slot0 + cta;
@@ -767,22 +770,35 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
                 a = fmaf(sc, part_acc[(pidx * HG + h) * D + c], a);
                 lsum = fmaf(sc, part_ml[(pidx * HG + h) * 2 + 1], lsum);
             }
-            float frac = 1.f;
-            if (sink_logits != nullptr) {
-                // learned sink: an extra logit in the normaliser, added exactly once, after the cross-split
-                // combine; it is shifted by the per-query constant the token logits dropped (q . k_mean)
-                const int hq = kvh * HG + h;
-                const float s2 = sink_logits[hq] * 1.4426950408889634f - qk_off[(size_t)b * n_q_heads + hq];
-                const float M2 = fmaxf(M, s2);
-                const float w = ex2(M - M2);
-                const float ltok = lsum * w;
-                lsum = ltok + ex2(s2 - M2);
-                a *= w;
-                frac = ltok / lsum;
-            }
-            val = a / lsum;
-            if (c == 0) frac_s[h] = frac;
         }
+        float lq = lsum;          // mass of the quantised tokens at the running scale
+        float wb = 0.f;           // weight of the band accumulator at the running scale
+        const int hq = kvh * HG + h;
+        if (band_ml != nullptr) {
+            // BF16 sink-plus-recent band: one more partial, accumulated in the original value domain
+            const float mb = band_ml[((size_t)b * n_q_heads + hq) * 2], lb = band_ml[((size_t)b * n_q_heads + hq) * 2 + 1];
+            const float M2 = fmaxf(M, mb);
+            const float wq = ex2(M - M2);
+            wb = ex2(mb - M2);
+            a *= wq;
+            lq *= wq;
+            lsum = fmaf(lb, wb, lq);
+            M = M2;
+        }
+        if (sink_logits != nullptr) {
+            // learned sink: an extra logit in the normaliser, added exactly once, after the cross-split
+            // combine; it is shifted by the per-query constant the token logits dropped (q . k_mean)
+            const float s2 = sink_logits[hq] * 1.4426950408889634f - qk_off[(size_t)b * n_q_heads + hq];
+            const float M2 = fmaxf(M, s2);
+            const float w = ex2(M - M2);
+            a *= w;
+            lq *= w;
+            wb *= w;
+            lsum = fmaf(lsum, w, ex2(s2 - M2));
+        }
+        float val = 0.f, frac = 0.f, bsc = 0.f;
+        if (lsum > 0.f) { val = a / lsum; frac = lq / lsum; bsc = wb / lsum; }
+        if (c == 0) { frac_s[h] = frac; bsc_s[h] = bsc; }
         o_s[i] = val;
     }
     __syncthreads();
@@ -809,20 +825,128 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         if (i >= HG * D) break;
         const int h = i / D, r = i - h * D;
         float o = 0.f;
-        if (pages_b > 0) {
 #pragma unroll
-            for (int p = 0; p < PARTS; ++p) o += red_s[p][h][r];
-            o = fmaf(vm[k], frac_s[h], o);          // sum_j p_j (s^_j R_V^T + v_mean): the mean carries the token mass
-        }
+        for (int p = 0; p < PARTS; ++p) o += red_s[p][h][r];
+        o = fmaf(vm[k], frac_s[h], o);              // sum_j p_j (s^_j R_V^T + v_mean): the mean carries the quantised-token mass
         const size_t oi = ((size_t)b * n_q_heads + kvh * HG + h) * D + r;
+        if (band_acc != nullptr) o = fmaf(band_acc[oi], bsc_s[h], o);
         if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
         else reinterpret_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// BF16 sink-plus-recent band: exact attention partial over the tokens that are not quantised
+// ------------------------------------------------------------------------------------------------
+// One CTA per (sequence, KV head), 16 warps; a warp takes 4 band tokens at a time (their 8 row loads in
+// flight together), lanes hold D/32 dimensions, logits by warp reduction, online softmax per warp, then a
+// merge of the warps.  Output: (max, sum) and sum_j p_j v_j per query head, base-2 domain, unnormalised.
+// Band buffers: bf16 [batch][band_cap][Hkv][D]; of sequence b, slots 0 .. sink_cnt-1 hold the sink tokens
+// and slots n_sink + (ring_start + i) % (band_cap - n_sink), i < ring_len, the recent tokens.
+constexpr int BAND_WARPS = 16, BAND_U = 4;
+template <int D, int HG>
+__global__ void __launch_bounds__(BAND_WARPS * 32)
+novakv_band_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ band_k,
+                   const __nv_bfloat16* __restrict__ band_v, int band_cap, int n_sink,
+                   const int32_t* __restrict__ band_meta, int n_q_heads, int n_kv_heads, float scale_log2,
+                   const float* __restrict__ k_mean, float* __restrict__ band_ml, float* __restrict__ band_acc) {
+    constexpr int DPL = D / 32;
+    __shared__ float m_s[BAND_WARPS][HG], l_s[BAND_WARPS][HG];
+    __shared__ float acc_s[BAND_WARPS][HG][D];
+    novakv_grid_dependency_wait();
+    const int b = blockIdx.x / n_kv_heads, kvh = blockIdx.x - b * n_kv_heads;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ring_cap = band_cap - n_sink;
+    const int sink_cnt = min(max(band_meta[b * 3 + 0], 0), n_sink);
+    const int ring_start = max(band_meta[b * 3 + 1], 0);
+    const int ring_len = ring_cap > 0 ? min(max(band_meta[b * 3 + 2], 0), ring_cap) : 0;
+    const int n = sink_cnt + ring_len;
+    float qr[HG][DPL];
+#pragma unroll
+    for (int h = 0; h < HG; ++h)
+#pragma unroll
+        for (int i = 0; i < DPL; ++i)
+            qr[h][i] = __bfloat162float(q[((size_t)b * n_q_heads + kvh * HG + h) * D + lane * DPL + i]) * scale_log2;
+    // the quantised tokens' logits omit the constant q . k_mean * sm_scale (Lemma S1): the band's logits must
+    // sit on the same scale, so the same constant is subtracted here
+    float zoff[HG];
+#pragma unroll
+    for (int h = 0; h < HG; ++h) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) t = fmaf(qr[h][i], k_mean[(size_t)kvh * D + lane * DPL + i], t);
+        zoff[h] = warp_sum_f(t);
+    }
+    float m[HG], l[HG], acc[HG][DPL];
+#pragma unroll
+    for (int h = 0; h < HG; ++h) {
+        m[h] = M_INIT; l[h] = 0.f;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[h][i] = 0.f;
+    }
+    for (int base = warp * BAND_U; base < n; base += BAND_WARPS * BAND_U) {
+        float kf[BAND_U][DPL], vf[BAND_U][DPL];
+#pragma unroll
+        for (int u = 0; u < BAND_U; ++u) {
+            const int i = base + u;
+            const int ii = i < n ? i : base;               // a valid row; its weight is zeroed below
+            const int slot = ii < sink_cnt ? ii : n_sink + (ring_start + (ii - sink_cnt)) % ring_cap;
+            const size_t off = (((size_t)b * band_cap + slot) * n_kv_heads + kvh) * D + lane * DPL;
+#pragma unroll
+            for (int j = 0; j < DPL; j += 2) {
+                const __nv_bfloat162 k2 = *reinterpret_cast<const __nv_bfloat162*>(band_k + off + j);
+                const __nv_bfloat162 v2 = *reinterpret_cast<const __nv_bfloat162*>(band_v + off + j);
+                kf[u][j] = __bfloat162float(k2.x); kf[u][j + 1] = __bfloat162float(k2.y);
+                vf[u][j] = __bfloat162float(v2.x); vf[u][j + 1] = __bfloat162float(v2.y);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < BAND_U; ++u) {
+            const bool valid = base + u < n;
+#pragma unroll
+            for (int h = 0; h < HG; ++h) {
+                float z = 0.f;
+#pragma unroll
+                for (int i = 0; i < DPL; ++i) z = fmaf(qr[h][i], kf[u][i], z);
+                z = warp_sum_f(z) - zoff[h];
+                if (!valid) z = -CUDART_INF_F;
+                const float m_new = fmaxf(m[h], z);
+                const float alpha = ex2(m[h] - m_new), p = ex2(z - m_new);
+                l[h] = fmaf(l[h], alpha, p);
+#pragma unroll
+                for (int i = 0; i < DPL; ++i) acc[h][i] = fmaf(acc[h][i], alpha, p * vf[u][i]);
+                m[h] = m_new;
+            }
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < HG; ++h) {
+        if (lane == 0) { m_s[warp][h] = m[h]; l_s[warp][h] = l[h]; }
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc_s[warp][h][lane * DPL + i] = acc[h][i];
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < HG * D; idx += BAND_WARPS * 32) {
+        const int h = idx / D, c = idx - h * D;
+        float M = M_INIT;
+#pragma unroll
+        for (int w = 0; w < BAND_WARPS; ++w) M = fmaxf(M, m_s[w][h]);
+        float a = 0.f, L = 0.f;
+#pragma unroll
+        for (int w = 0; w < BAND_WARPS; ++w) {
+            const float sc = ex2(m_s[w][h] - M);
+            a = fmaf(sc, acc_s[w][h][c], a);
+            L = fmaf(sc, l_s[w][h], L);
+        }
+        const size_t o = (size_t)b * n_q_heads + kvh * HG + h;
+        band_acc[o * D + c] = a;
+        if (c == 0) { band_ml[o * 2] = M; band_ml[o * 2 + 1] = L; }
+    }
+}
+
 // workspace layout
 struct WsLayout {
-    size_t qp, prefix, qk, ml, acc, total;
+    size_t qp, prefix, qk, bml, bacc, ml, acc, total;
 };
 WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -832,7 +956,9 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     w.qp = 0;
     w.prefix = al(w.qp + (size_t)batch * hq * d * 4);
     w.qk = al(w.prefix + ((size_t)batch + 1) * 4);
-    w.ml = al(w.qk + (size_t)batch * hq * 4);
+    w.bml = al(w.qk + (size_t)batch * hq * 4);
+    w.bacc = al(w.bml + (size_t)batch * hq * 2 * 4);
+    w.ml = al(w.bacc + (size_t)batch * hq * d * 4);
     w.acc = al(w.ml + n_part * ctx->hg * 2 * 4);
     w.total = al(w.acc + n_part * ctx->hg * d * 4);
     return w;
@@ -843,13 +969,23 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                               const uint8_t* k_pages, const uint8_t* v_pages, const __nv_bfloat16* k_scales, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens,
                               int batch, float sm_scale, void* out, int out_is_fp32, void* workspace,
-                              cudaStream_t stream, const float* sink_logits) {
+                              cudaStream_t stream, const float* sink_logits, const novakv_band_args* band) {
     using C = S1<D, HG, VM>;
+    // with a BF16 band the index cache holds positions n_sink .. n_sink + seq_lens[b] - 1: the scan starts at
+    // page column n_sink / 64 of every row
+    const int pt_stride = max_pages_per_seq;
+    if (band != nullptr) {
+        const int shift = band->n_sink / NOVAKV_PAGE_TOKENS;
+        page_table += shift;
+        max_pages_per_seq -= shift;
+    }
     const WsLayout w = ws_layout(ctx, batch);
     char* ws = (char*)workspace;
     float* qp = (float*)(ws + w.qp);
     int32_t* prefix = (int32_t*)(ws + w.prefix);
     float* qk_off = sink_logits ? (float*)(ws + w.qk) : nullptr;
+    float* band_ml = band ? (float*)(ws + w.bml) : nullptr;
+    float* band_acc = band ? (float*)(ws + w.bacc) : nullptr;
     float* part_ml = (float*)(ws + w.ml);
     float* part_acc = (float*)(ws + w.acc);
     const int hq = ctx->cfg.n_q_heads, hkv = ctx->cfg.n_kv_heads;
@@ -870,14 +1006,20 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         novakv_prof_scope ps(ctx, 0, stream);
         novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut, ly.cb_v_mma, k_pages, v_pages,
                           k_scales, n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
-                          ctx->dev_status);
+                          ctx->dev_status, pt_stride);
         ps.end();
+        ctx->launches++;
+    }
+    if (band != nullptr) {
+        novakv_launch_pdl(novakv_band_kernel<D, HG>, dim3(batch * hkv), dim3(BAND_WARPS * 32), 0, stream, q, band->k, band->v,
+                          band->cap, band->n_sink, band->meta, hq, hkv, sm_scale * 1.4426950408889634f, ly.k_mean, band_ml,
+                          band_acc);
         ctx->launches++;
     }
     auto merge = batch * hkv > 2 * ctx->n_sm ? novakv_decode_merge_kernel<D, HG, 2> : novakv_decode_merge_kernel<D, HG, 1>;
     novakv_launch_pdl(merge, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
                       part_ml, part_acc, prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out,
-                      out_is_fp32, sink_logits, qk_off);
+                      out_is_fp32, sink_logits, qk_off, (const float*)band_ml, (const float*)band_acc);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
 }
@@ -890,7 +1032,7 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
     int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream, const __nv_bfloat16* k_scales,
-    const float* sink_logits) {
+    const float* sink_logits, const novakv_band_args* band) {
     (void)workspace_bytes;
     const int d = ctx->cfg.head_dim, hg = ctx->hg;
     if (k_scales != nullptr && ctx->value_path == 0) return NOVAKV_EUNSUPPORTED;   // scaled keys: tensor-core value side only
@@ -899,14 +1041,14 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
         if (k_scales != nullptr)                                                                                 \
             return launch_decode_t<DD, HH, true, true>(ctx, ly, q, k_pages, v_pages, k_scales, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
-                                                  workspace, stream, sink_logits);                               \
+                                                  workspace, stream, sink_logits, band);                               \
         if (ctx->value_path == 0)                                                                                \
             return launch_decode_t<DD, HH, false, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
-                                                  workspace, stream, sink_logits);                               \
+                                                  workspace, stream, sink_logits, band);                               \
         return launch_decode_t<DD, HH, true, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table,  \
                                              max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,     \
-                                             workspace, stream, sink_logits);                                    \
+                                             workspace, stream, sink_logits, band);                                    \
     }
     NOVAKV_DISPATCH(128, 1)
     NOVAKV_DISPATCH(128, 2)

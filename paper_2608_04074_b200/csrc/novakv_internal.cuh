@@ -74,13 +74,21 @@ novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int 
     int n, uint8_t* idx_out, cudaStream_t stream);
 
 // decode
+struct novakv_band_args {
+    const __nv_bfloat16* k;     // [batch][cap][Hkv][d]
+    const __nv_bfloat16* v;
+    int cap;                    // slots per sequence: n_sink sink slots + a ring of cap - n_sink
+    int n_sink;                 // multiple of 64
+    const int32_t* meta;        // device [batch][3]: sink count, ring start, ring length
+};
 size_t novakv_decode_ws_bytes(const novakv_ctx* ctx, int batch);
 novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
     int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream,
     const __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */,
-    const float* sink_logits = nullptr /* learned sink: [Hq], natural-log units */);
+    const float* sink_logits = nullptr /* learned sink: [Hq], natural-log units */,
+    const novakv_band_args* band = nullptr /* BF16 sink-plus-recent band */);
 
 // gather of page-locked host buffers into device staging (one kernel for up to 5 segments of 32-bit words)
 struct novakv_stage_args {

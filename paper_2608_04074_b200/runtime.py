@@ -100,6 +100,107 @@ class PagedCache:
         return out
 
 
+class BandedCache:
+    """Index cache plus a BF16 sink-plus-recent band: the first ``n_sink`` tokens of a sequence and its most
+    recent ``n_rec`` .. ``n_rec + block - 1`` tokens stay in bf16; whenever the recent ring has grown by
+    ``block`` tokens the ``block`` oldest are quantised into the index cache (deferred quantisation in
+    blocks of eight steps).  Only bookkeeping and tensor copies happen here; encoding and attention are
+    the library's calls."""
+
+    def __init__(self, ctx: Context, batch: int, capacity_tokens: int, n_sink: int = 64, n_rec: int = 256,
+                 block: int = 8, seed: int = 0, device="cuda:0", key_scale: bool = False):
+        assert n_sink % cache_format.PAGE_TOKENS == 0
+        self.ctx, self.batch, self.n_sink, self.n_rec, self.block = ctx, batch, n_sink, n_rec, block
+        self.device = torch.device(device)
+        self.paged = PagedCache(ctx, np.zeros(batch, np.int32), capacity_tokens=np.full(batch, capacity_tokens, np.int32),
+                                seed=seed, device=device, key_scale=key_scale)
+        self.ring_cap = n_rec + block
+        self.cap = n_sink + self.ring_cap
+        shape = (batch, self.cap, ctx.n_kv_heads, ctx.head_dim)
+        self.band_k = torch.zeros(shape, dtype=torch.bfloat16, device=self.device)
+        self.band_v = torch.zeros(shape, dtype=torch.bfloat16, device=self.device)
+        self.total = np.zeros(batch, np.int64)          # tokens of each sequence
+        self.quant = np.zeros(batch, np.int64)          # of which quantised (positions n_sink .. n_sink + quant - 1)
+        self.ring_start = np.zeros(batch, np.int64)
+        self.ring_len = np.zeros(batch, np.int64)
+        self.band_meta = torch.zeros((batch, 3), dtype=torch.int32, device=self.device)
+        self.quant_lens = torch.zeros(batch, dtype=torch.int32, device=self.device)
+
+    def _sync_meta(self):
+        meta = np.stack([np.minimum(self.total, self.n_sink), self.ring_start, self.ring_len], axis=1).astype(np.int32)
+        self.band_meta.copy_(torch.from_numpy(meta))
+        self.quant_lens.copy_(torch.from_numpy(self.quant.astype(np.int32)))
+
+    def _flush(self, layer, items):
+        """items: list of (b, n_tokens): quantise the n oldest ring tokens of sequence b."""
+        ks, vs, seqs, poss = [], [], [], []
+        for b, n in items:
+            slots = self.n_sink + (self.ring_start[b] + np.arange(n)) % self.ring_cap
+            idx = torch.from_numpy(slots).to(self.device)
+            ks.append(self.band_k[b, idx]); vs.append(self.band_v[b, idx])
+            seqs.append(np.full(n, b, np.int32))
+            poss.append((self.n_sink + self.quant[b] + np.arange(n)).astype(np.int32))
+            self.ring_start[b] = (self.ring_start[b] + n) % self.ring_cap
+            self.ring_len[b] -= n
+            self.quant[b] += n
+        if not ks:
+            return
+        self.paged.append(layer, torch.cat(ks).contiguous(), torch.cat(vs).contiguous(),
+                          torch.from_numpy(np.concatenate(seqs)).to(self.device),
+                          torch.from_numpy(np.concatenate(poss)).to(self.device))
+
+    def prefill(self, layer, b: int, k: torch.Tensor, v: torch.Tensor):
+        """Tokens 0 .. n-1 of an empty sequence b (bf16 [n][Hkv][d]): sink, quantised middle, recent ring."""
+        assert self.total[b] == 0
+        n = int(k.shape[0])
+        ns = min(n, self.n_sink)
+        self.band_k[b, :ns] = k[:ns]; self.band_v[b, :ns] = v[:ns]
+        rest = n - ns
+        nrec = min(rest, self.n_rec)
+        nq = rest - nrec
+        if nq > 0:
+            self.paged.append(layer, k[ns:ns + nq].contiguous(), v[ns:ns + nq].contiguous(),
+                              torch.full((nq,), b, dtype=torch.int32, device=self.device),
+                              torch.arange(ns, ns + nq, dtype=torch.int32, device=self.device))
+        if nrec > 0:
+            self.band_k[b, self.n_sink:self.n_sink + nrec] = k[ns + nq:]
+            self.band_v[b, self.n_sink:self.n_sink + nrec] = v[ns + nq:]
+        self.total[b], self.quant[b], self.ring_start[b], self.ring_len[b] = n, nq, 0, nrec
+        self._sync_meta()
+
+    def append_step(self, layer, k_new: torch.Tensor, v_new: torch.Tensor):
+        """One new token for every sequence (bf16 [batch][Hkv][d]); quantises blocks that leave the band."""
+        flush = []
+        for b in range(self.batch):
+            pos = self.total[b]
+            if pos < self.n_sink:
+                slot = pos
+            else:
+                slot = self.n_sink + (self.ring_start[b] + self.ring_len[b]) % self.ring_cap
+                self.ring_len[b] += 1
+            self.band_k[b, slot] = k_new[b]; self.band_v[b, slot] = v_new[b]
+            self.total[b] += 1
+            if self.ring_len[b] >= self.n_rec + self.block:
+                flush.append((b, self.block))
+        self._flush(layer, flush)
+        self._sync_meta()
+
+    def band_mask(self, b: int) -> np.ndarray:
+        """bool [total[b]]: positions held in bf16."""
+        pos = np.arange(self.total[b])
+        return (pos < self.n_sink) | (pos >= self.n_sink + self.quant[b])
+
+    def decode(self, layer, q, out=None, sm_scale=None, sink_logits=None):
+        if out is None:
+            out = torch.empty((self.batch, self.ctx.n_q_heads, self.ctx.head_dim), dtype=torch.float32,
+                              device=self.device)
+        p = self.paged
+        self.ctx.novakv_decode_attention_banded(layer, q, p.k_pages, p.v_pages, p.k_scales, sink_logits, p.page_table,
+                                                self.quant_lens, self.band_k, self.band_v, self.n_sink,
+                                                self.band_meta, out, p.workspace, sm_scale)
+        return out
+
+
 def bf16_tensor(x: np.ndarray, device="cuda:0") -> torch.Tensor:
     """float array holding bf16-representable values -> torch bf16 tensor on the device."""
     return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.bfloat16).to(device)

@@ -618,3 +618,61 @@ def test_sink_on_scaled_key_format(qwen_scaled):
         ref = case.oracle.decode_sink(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], sink.astype(np.float64),
                                       kscale=encs[b]["kscale"])
         check_output(out[b], ref)
+
+
+# --------------------------------------------------------------------------- BF16 sink-plus-recent band
+@pytest.mark.parametrize("name,n_sink,n_rec", [("qwen", 64, 256), ("gptoss", 64, 256), ("qwen", 0, 32), ("qwen", 128, 8)])
+def test_banded_decode_matches_oracle(name, n_sink, n_rec, request):
+    """Sequences shorter than the sink, inside the band, just past it and far past it; bulk prefill followed
+    by single-token steps that wrap the ring and trigger the deferred block quantisation."""
+    from paper_2608_04074_b200.runtime import BandedCache
+    case = request.getfixturevalue(name)
+    lens = np.array([700, 30, 64, 65, 330, 321, 0], np.int32)
+    steps = 21
+    cache = BandedCache(case.ctx, len(lens), int(lens.max()) + steps + 64, n_sink=n_sink, n_rec=n_rec, block=8, seed=12)
+    ks, vs = [], []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(1000 + b, int(n) + steps, 1)
+        ks.append(k); vs.append(v)
+        if n > 0:
+            cache.prefill(0, b, _dev(k[:n], torch.bfloat16), _dev(v[:n], torch.bfloat16))
+    for t in range(steps):
+        cache.append_step(0, _dev(np.stack([ks[b][lens[b] + t] for b in range(len(lens))]), torch.bfloat16),
+                          _dev(np.stack([vs[b][lens[b] + t] for b in range(len(lens))]), torch.bfloat16))
+    assert case.ctx.novakv_last_device_status() == 0
+    assert (cache.total == lens + steps).all()
+    assert (cache.ring_len >= 0).all() and (cache.ring_len < n_rec + 8).all()
+    _, _, q = case.draw(1001, 1, len(lens))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    worst, n_quant = 0.0, 0
+    for b in range(len(lens)):
+        k, v = ks[b].astype(np.float64), vs[b].astype(np.float64)
+        e = case.oracle.encode(k, v, with_gaps=False)
+        mask = cache.band_mask(b)
+        n_quant += int((~mask).sum())
+        ref = case.oracle.decode_banded(q[b].astype(np.float64), e["kidx"], e["vidx"], k, v, mask)
+        worst = max(worst, check_output(out[b], ref))
+    assert n_quant > 300          # the quantised middle is exercised
+    print(f"[{name} sink {n_sink} recent {n_rec}] banded: {n_quant} quantised positions, max|delta|/||o||inf = {worst:.3e}")
+
+
+def test_banded_with_scale_and_sink(qwen_scaled):
+    from paper_2608_04074_b200.runtime import BandedCache
+    case = qwen_scaled
+    lens = np.array([500, 100], np.int32)
+    cache = BandedCache(case.ctx, 2, 700, n_sink=64, n_rec=64, block=8, seed=13, key_scale=True)
+    ks, vs = [], []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(1100 + b, int(n), 1)
+        ks.append(k); vs.append(v)
+        cache.prefill(0, b, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16))
+    _, _, q = case.draw(1101, 1, 2)
+    sink = np.linspace(-2.0, 6.0, case.ctx.n_q_heads).astype(np.float32)
+    out = cache.decode(0, _dev(q, torch.bfloat16), sink_logits=_dev(sink)).cpu().numpy()
+    for b in range(2):
+        k, v = ks[b].astype(np.float64), vs[b].astype(np.float64)
+        e = case.oracle.encode_scaled(k, v, with_gaps=False)
+        ref = case.oracle.decode_banded(q[b].astype(np.float64), e["kidx"], e["vidx"], k, v, cache.band_mask(b),
+                                        kscale=e["kscale"], sink=sink.astype(np.float64))
+        check_output(out[b], ref)
