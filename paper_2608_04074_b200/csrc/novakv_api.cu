@@ -65,7 +65,7 @@ static void free_layer(novakv_layer& ly) {
     cudaFree(ly.rk_d); cudaFree(ly.rv_d); cudaFree(ly.k_mean_d); cudaFree(ly.v_mean_d);
     cudaFree(ly.rk_d_mma); cudaFree(ly.rv_d_mma); cudaFree(ly.k_mean);
     cudaFree(ly.cb_k); cudaFree(ly.cb_v); cudaFree(ly.rk_inv_t); cudaFree(ly.rv_t);
-    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_half); cudaFree(ly.cb_v_mma);
+    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_mma);
     ly = novakv_layer();
 }
 
@@ -96,9 +96,8 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
     const size_t n_mat = (size_t)H * d * d, n_vec = (size_t)H * d, n_cb = (size_t)H * L * C * g;
 
     // value codewords must survive the binary16 round trip exactly
-    // cbv_grp: slot = group (scratch);  cbv_half: slot = index row of the group (CUDA-core value side)
+    // cbv_grp: slot = group (scratch for the image below)
     std::vector<__half> cbv_grp((size_t)H * C * 32 * g, __float2half(0.f));
-    std::vector<__half> cbv_half((size_t)H * C * 32 * g, __float2half(0.f));
     std::vector<__half> cbv_mma((size_t)H * C * 32 * g, __float2half(0.f));
     for (int hh = 0; hh < H; ++hh)
         for (int l = 0; l < L; ++l)
@@ -108,7 +107,6 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
                     __half hx = __float2half_rn(x);
                     if (!(__half2float(hx) == x)) return NOVAKV_EUNSUPPORTED;
                     cbv_grp[(((size_t)hh * C + c) * 32 + l) * g + i] = hx;
-                    cbv_half[(((size_t)hh * C + c) * 32 + ((l & 7) * (L / 8) + (l >> 3))) * g + i] = hx;
                 }
     // tensor-core value side: slot pos = 16*rho + 4*xb + r' holds group 8*(xb mod NGB) + 4*rho + r'
     // (NGB = L/8 group blocks; for L = 16 every group appears twice).  The four lanes of an MMA quad
@@ -166,7 +164,7 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
               upload(&ly.cb_k, cbk) == cudaSuccess && upload(&ly.cb_v, cbv) == cudaSuccess &&
               upload(&ly.rk_inv_t, rkinv) == cudaSuccess && upload(&ly.rv_t, rvt) == cudaSuccess &&
               upload(&ly.v_mean, vm_f) == cudaSuccess && upload(&ly.k_mean, km_f) == cudaSuccess && upload(&ly.cb_k_lut, cbk_lut) == cudaSuccess &&
-              upload(&ly.cb_v_half, cbv_half) == cudaSuccess && upload(&ly.cb_v_mma, cbv_mma) == cudaSuccess;
+              upload(&ly.cb_v_mma, cbv_mma) == cudaSuccess;
     if (!ok) { free_layer(ly); return NOVAKV_ECUDA; }
     ly.loaded = true;
     return NOVAKV_OK;

@@ -13,20 +13,19 @@ namespace {
 
 constexpr int ENC_THREADS = 512;
 constexpr int ENC_TILE = 64;   // tokens per tile (search granularity)
-constexpr int ENC_XT = 32;     // tokens per transform pass (bounds the binary64 staging buffer)
 #ifndef NOVAKV_SMALL_APPEND_TOKENS
 #define NOVAKV_SMALL_APPEND_TOKENS 256   // batches up to this size take the per-group append kernel
 #endif
 
+// Shared-memory plan of the search-only kernel: codebook, one tile of coefficients, its indices.
 template <int D>
 struct EncSmem {
     static constexpr int L = D / NOVAKV_G;
     static constexpr int RSTRIDE = D + 4;                       // floats; keeps 128-bit row reads conflict-free
     static constexpr size_t cb_bytes = (size_t)L * NOVAKV_C * NOVAKV_G * sizeof(float);
-    static constexpr size_t xc_bytes = (size_t)ENC_XT * D * sizeof(double);
     static constexpr size_t r_bytes = (size_t)ENC_TILE * RSTRIDE * sizeof(float);
     static constexpr size_t idx_bytes = (size_t)ENC_TILE * L;
-    static constexpr size_t total = cb_bytes + xc_bytes + r_bytes + idx_bytes + 3 * ENC_TILE * sizeof(int);
+    static constexpr size_t total = cb_bytes + r_bytes + idx_bytes;
 };
 
 // Squared distance in the arithmetic the public header fixes: fma(e3,e3,fma(e2,e2,fma(e1,e1,e0*e0))).
@@ -551,8 +550,8 @@ novakv_search_kernel(const float* __restrict__ coef, int n, const float* __restr
     constexpr int RS = EncSmem<D>::RSTRIDE;
     extern __shared__ __align__(16) unsigned char smem[];
     float4* cb_s = reinterpret_cast<float4*>(smem);
-    float* r_s = reinterpret_cast<float*>(smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes);
-    uint8_t* idx_s = smem + EncSmem<D>::cb_bytes + EncSmem<D>::xc_bytes + EncSmem<D>::r_bytes;
+    float* r_s = reinterpret_cast<float*>(smem + EncSmem<D>::cb_bytes);
+    uint8_t* idx_s = smem + EncSmem<D>::cb_bytes + EncSmem<D>::r_bytes;
     const int kvh = blockIdx.y;
     const float4* cb_g = reinterpret_cast<const float4*>(cb_all + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
     fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);

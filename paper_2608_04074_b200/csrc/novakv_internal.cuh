@@ -32,7 +32,6 @@ struct novakv_layer {
     float* rv_t = nullptr;        // [Hkv][d][d]  transposed R_V: rv_t[c][r] = R_V[r][c]
     float* v_mean = nullptr;      // [Hkv][d]
     float* cb_k_lut = nullptr;    // [Hkv][plane][256][16][4]  the order the score table is built in
-    __half* cb_v_half = nullptr;  // [Hkv][256][32][4]         row of 256 bytes per code, slot = group (CUDA-core value side)
     __half* cb_v_mma = nullptr;   // [Hkv][256][32][4]         same codewords, slots permuted for the tensor-core value side
 };
 
