@@ -322,6 +322,44 @@ def test_bench_configuration_sampled():
               f"{ratio:.3e} (tensor-core value side) {ratio_cc:.3e} (CUDA-core value side)")
 
 
+def test_long_context_configuration_sampled():
+    """Qwen3-8B shape, B = 64, S = 32768 (1 GB of indices, larger than L2), the sweep configuration of
+    bench.py: one drawn sequence is encoded by the GPU and its pages are copied to distinct physical pages of
+    every other sequence (as the benchmark does); queries differ per sequence.  Outputs are checked on
+    sampled sequences against the oracle's decode of the indices the GPU stored; indices on sampled tokens."""
+    S, B = 32768, 64
+    wl = workloads.qwen3_8b(batch=B, seq_len=S, calib_tokens=4096, lloyd_iters=6)
+    case = Case(wl)
+    from paper_2608_04074_b200.runtime import PagedCache
+    cache = PagedCache(case.ctx, wl.seq_lens, seed=21)
+    cache.seq_lens.zero_()
+    k, v, _ = case.draw(1200, S, 1)
+    for t0 in range(0, S, 8192):
+        cache.append(0, _dev(k[t0:t0 + 8192], torch.bfloat16), _dev(v[t0:t0 + 8192], torch.bfloat16),
+                     _dev(np.zeros(8192, np.int32)), _dev(np.arange(t0, t0 + 8192, dtype=np.int32)))
+    src = cache.page_table[0].long()
+    for b in range(1, B):
+        dst = cache.page_table[b].long()
+        cache.k_pages[dst] = cache.k_pages[src]
+        cache.v_pages[dst] = cache.v_pages[src]
+    cache.seq_lens.copy_(torch.from_numpy(wl.seq_lens.astype(np.int32)).cuda())
+    _, _, q = case.draw(1201, 1, B)
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    gk, gv = cache.load_logical(0, 0, S)
+    pick = np.sort(synth.rng(78).choice(S, size=512, replace=False))
+    enc = case.oracle.encode(k[pick].astype(np.float64), v[pick].astype(np.float64))
+    dk, _ = check_indices(gk[pick], enc, "k")
+    dv, _ = check_indices(gv[pick], enc, "v")
+    worst = 0.0
+    for b in (0, 17, 63):
+        gkb, gvb = cache.load_logical(b, 0, S)
+        assert np.array_equal(gkb, gk) and np.array_equal(gvb, gv)
+        ref = case.oracle.decode(q[b].astype(np.float64), gk, gv)
+        worst = max(worst, check_output(out[b], ref))
+    print(f"[B=64 S=32768] sampled index mismatches K {dk} V {dv}; max|delta|/||o||inf {worst:.3e}")
+
+
 # --------------------------------------------------------------------------- uncompressed comparator
 @pytest.mark.parametrize("name,window", [("qwen", 0), ("qwen", 128), ("gptoss", 0), ("gptoss", 128)])
 def test_bf16_comparator_matches_textbook_attention(name, window, request):
