@@ -235,7 +235,7 @@ novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int layer, const v
  * every GPU that loads the library holds it until the process exits.
  *   - Arguments and results are those of novakv_decode_attention without workspace/workspace_bytes.
  *   - Returns NOVAKV_EWORKSPACE when novakv_decode_workspace_bytes(ctx, batch) exceeds
- *     NOVAKV_NOALLOC_SCRATCH_BYTES (for the Qwen3-8B shape that is a batch of about 100 sequences).
+ *     NOVAKV_NOALLOC_SCRATCH_BYTES (for the Qwen3-8B shape that is a batch of more than 78 sequences).
  *   - Calls no cudaMalloc, cudaFree or other allocating routine, and records no timing events.
  *   - All calls on a device share the array: calls that overlap on the GPU (other streams, other
  *     contexts) race; calls on one stream are ordered and safe.  Every scratch word is written
