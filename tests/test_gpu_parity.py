@@ -71,11 +71,14 @@ def test_search_from_oracle_coefficients_is_exact(name, request):
 
 
 # --------------------------------------------------------------------------- T2: transform + search + paged store
+@pytest.mark.parametrize("add", [[200, 64, 1, 130], [20, 7, 1, 3], [1, 0, 0, 0], [70, 60, 50, 40], [0, 2, 0, 0]])
 @pytest.mark.parametrize("name", ["tiny", "qwen", "gptoss"])
-def test_encode_append_matches_oracle_indices(name, request):
+def test_encode_append_matches_oracle_indices(name, add, request):
+    """395 tokens take the tiled (prefill) kernel; 31, 1, 220 and 2 tokens the per-group append kernel with
+    1, 1, 7 and 1 passes and 1, 32, 1 and 16 lane groups per token."""
     case = request.getfixturevalue(name)
     lens0 = np.array([0, 5, 63, 130], np.int32)          # existing lengths; tokens are appended after them
-    add = np.array([200, 64, 1, 130], np.int32)
+    add = np.array(add, np.int32)
     cache = _cache(case, lens0, capacity=lens0 + add)
     n = int(add.sum())
     k, v, _ = case.draw(200, n, 1)
@@ -97,6 +100,9 @@ def test_encode_append_matches_oracle_indices(name, request):
     # bytes of positions that were not appended stay untouched (zero)
     kk, _ = cache.load_logical(1, 0, 5)
     assert not kk.any()
+    if add[3] > 0:
+        kk, _ = cache.load_logical(3, 0, 130)
+        assert not kk.any()
 
 
 # --------------------------------------------------------------------------- T3/T5: decode on the oracle's indices
