@@ -429,3 +429,69 @@ void oracle_decode_sink(const oracle_tables* t, const double* q, const uint8_t* 
     free(k_hat);
     free(v_hat);
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Scalar value codec of the deployed format (Sec. 5 "Bit rate": "The V cache is INT2 with a BF16
+ * scale and offset (zero-point), giving 2.000 + 32/128 = 2.250"; App. B read path: "the INT2 code is
+ * dequantized in the ... rotation basis"), in the Corollary 1 basis R_V:
+ *     s = (v - vbar) R_V,   code_i = clamp(round((s_i - zero) / scale), 0, 3),
+ *     s^_i = zero + scale * code_i,   v^ = s^ R_V^T + vbar,
+ * one (scale, zero) pair per token and KV head.  Where floating point decides stored bits the
+ * arithmetic is the one the library boundary documents: s is the binary32-rounded coefficient
+ * vector; zero = bf16(min_i s_i); scale = bf16((max_i s_i - zero) / 3) evaluated in binary32, replaced
+ * by 1 if it is not positive and finite; code_i = clamp(rint((s_i - zero) / scale), 0, 3) with the
+ * subtraction and the division in binary32 and ties to even.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_int2_quantise(const double* coef, int d, uint8_t* codes, float* scale_out, float* zero_out)
+{
+    float mn = (float)coef[0], mx = (float)coef[0];
+    for (int i = 1; i < d; ++i) {
+        const float s = (float)coef[i];
+        if (s < mn) mn = s;
+        if (s > mx) mx = s;
+    }
+    const float zero = bf16_round(mn);
+    float scale = bf16_round((mx - zero) / 3.0f);
+    if (!(scale > 0.f) || !isfinite(scale)) scale = 1.f;
+    for (int i = 0; i < d; ++i) {
+        const float t = (float)coef[i] - zero;
+        float u = rintf(t / scale);
+        if (!(u > 0.f)) u = 0.f;
+        if (u > 3.f) u = 3.f;
+        codes[i] = (uint8_t)u;
+    }
+    *scale_out = scale;
+    *zero_out = zero;
+}
+
+/* Values of n tokens -> codes [n][Hkv][d] (one code per byte, 0..3) and meta [n][Hkv][2] = (scale, zero). */
+void oracle_encode_values_int2(const oracle_tables* t, const double* v, long n, uint8_t* codes, float* meta)
+{
+    const int d = t->head_dim, H = t->n_kv_heads;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long j = 0; j < n; ++j)
+        for (int h = 0; h < H; ++h) {
+            double* coef = (double*)malloc(sizeof(double) * d);
+            long o = j * H + h;
+            oracle_coefficients(v + o * d, t->v_mean + (long)h * d, t->rv + (long)h * d * d, d, coef);
+            oracle_int2_quantise(coef, d, codes + o * d, meta + o * 2, meta + o * 2 + 1);
+            free(coef);
+        }
+}
+
+/* codes [S][Hkv][d], meta [S][Hkv][2] -> v_hat [S][Hkv][d] */
+void oracle_reconstruct_values_int2(const oracle_tables* t, const uint8_t* codes, const float* meta, long S,
+                                    double* v_hat)
+{
+    const int d = t->head_dim, H = t->n_kv_heads;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long j = 0; j < S; ++j)
+        for (int h = 0; h < H; ++h) {
+            long o = j * H + h;
+            double* s = (double*)malloc(sizeof(double) * d);
+            for (int i = 0; i < d; ++i) s[i] = (double)meta[o * 2 + 1] + (double)meta[o * 2] * (double)codes[o * d + i];
+            rowvec_mat_t(s, t->rv + (long)h * d * d, d, v_hat + o * d);
+            for (int i = 0; i < d; ++i) v_hat[o * d + i] += t->v_mean[(long)h * d + i];
+            free(s);
+        }
+}

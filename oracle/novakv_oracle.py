@@ -228,6 +228,47 @@ class Oracle:
                               ctypes.c_void_p(out.ctypes.data))
         return out
 
+    # -- scalar INT2 value codec of the deployed format ------------------------------------
+    def encode_values_int2(self, v):
+        """v [n][Hkv][d] -> (codes uint8 [n][Hkv][d] in 0..3, meta float32 [n][Hkv][2] = (scale, zero),
+        both bfloat16 values)."""
+        v = _f64(v)
+        n = v.shape[0]
+        codes = np.empty((n, self.n_kv_heads, self.d), np.uint8)
+        meta = np.empty((n, self.n_kv_heads, 2), np.float32)
+        _load().oracle_encode_values_int2(ctypes.byref(self._t), ctypes.c_void_p(v.ctypes.data), ctypes.c_long(n),
+                                          ctypes.c_void_p(codes.ctypes.data), ctypes.c_void_p(meta.ctypes.data))
+        return codes, meta
+
+    def reconstruct_values_int2(self, codes, meta):
+        codes = _u8(codes)
+        meta = np.ascontiguousarray(meta, np.float32)
+        s = codes.shape[0]
+        v_hat = np.empty((s, self.n_kv_heads, self.d))
+        _load().oracle_reconstruct_values_int2(ctypes.byref(self._t), ctypes.c_void_p(codes.ctypes.data),
+                                               ctypes.c_void_p(meta.ctypes.data), ctypes.c_long(s),
+                                               ctypes.c_void_p(v_hat.ctypes.data))
+        return v_hat
+
+    def decode_deployed(self, q, kidx, kscale, vcodes, vmeta, k_exact=None, v_exact=None, band_mask=None,
+                        sink=None, sm_scale: float | None = None):
+        """Decode step on the deployed format: scaled vector-quantised keys, INT2 scalar values, optionally a
+        BF16 band (exact rows where band_mask is set) and a sink logit.  Explicit dequantisation, then
+        textbook attention."""
+        kidx = _u8(kidx)
+        dummy_v = np.zeros_like(kidx)
+        k_hat, _ = self.reconstruct_scaled(kidx, dummy_v, kscale)
+        v_hat = self.reconstruct_values_int2(vcodes, vmeta)
+        if band_mask is not None:
+            band_mask = np.asarray(band_mask, bool)
+            k_hat[band_mask] = _f64(k_exact)[band_mask]
+            v_hat[band_mask] = _f64(v_exact)[band_mask]
+        if k_hat.shape[0] == 0:
+            return np.zeros((np.asarray(q).shape[0], self.d))
+        if sink is None:
+            return attention(q, k_hat, v_hat, sm_scale)
+        return attention_sink(q, k_hat, v_hat, sink, sm_scale)
+
     def decode_sink(self, q, kidx, vidx, sink, kscale=None, sm_scale: float | None = None):
         """Decode step with a learned sink logit per query head (sink [Hq], natural-log units)."""
         q = _f64(q)

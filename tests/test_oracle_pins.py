@@ -568,3 +568,81 @@ def test_banded_decode_limits_and_mixture(tiny_case):
     # the band matters: the result moves towards the exact attention
     plain = o.decode(q, e["kidx"], e["vidx"])
     assert np.abs(got - exact).max() < np.abs(plain - exact).max()
+
+
+# ---- scalar INT2 value codec of the deployed format (Sec. 5 "Bit rate"; App. B read path) ----
+def test_int2_value_codec_properties(tiny_case):
+    o = tiny_case["oracle"]
+    v = np.asarray(tiny_case["v"][:64], np.float64)
+    codes, meta = o.encode_values_int2(v)
+    assert codes.max() <= 3 and set(np.unique(codes)) == {0, 1, 2, 3}
+    scale, zero = meta[..., 0].astype(np.float64), meta[..., 1].astype(np.float64)
+    np.testing.assert_array_equal(meta, _bf16_values(meta))                     # both are bfloat16 values
+    s = o.coefficients(v, "v").astype(np.float32).astype(np.float64)
+    mn, mx = s.min(axis=2), s.max(axis=2)
+    np.testing.assert_array_equal(meta[..., 1], _bf16_values(mn.astype(np.float32)))
+    # the 4 levels span the token's range: zero ~ min, zero + 3 scale ~ max (bfloat16 slack 2^-8 relative)
+    span = mx - mn
+    assert (np.abs(zero + 3 * scale - mx) <= 3 * 2.0 ** -8 * (np.abs(scale) * 3 + np.abs(zero)) + 1e-12).all()
+    # nearest level: reconstruction error at most half a step, plus the clamp slack at the two ends
+    rec = zero[..., None] + scale[..., None] * codes
+    err = np.abs(rec - s)
+    assert (err <= 0.5 * scale[..., None] * (1 + 1e-6) + 2.0 ** -7 * span[..., None]).all()
+    # explicit reconstruction = s^ R_V^T + vbar
+    v_hat = o.reconstruct_values_int2(codes, meta)
+    np.testing.assert_allclose(v_hat[:, 0, :], rec[:, 0, :] @ o.rv[0].T + o.v_mean[0], rtol=0, atol=1e-12)
+
+
+def test_int2_value_codec_exact_cases():
+    d = 64
+    eye = np.eye(d)[None]
+    cb = np.zeros((1, d // 4, 256, 4), np.float32)
+    o = O.Oracle(eye, eye, eye, np.zeros((1, d)), np.zeros((1, d)), cb, cb)
+    gen = np.random.Generator(np.random.PCG64(9))
+    want = gen.integers(0, 4, size=(16, 1, d)).astype(np.uint8)
+    want[:, 0, 0], want[:, 0, 1] = 0, 3                                      # both ends present
+    zero, scale = -1.5, 0.375                                                # bfloat16-representable
+    v = zero + scale * want.astype(np.float64)
+    codes, meta = o.encode_values_int2(v)
+    np.testing.assert_array_equal(codes, want)
+    assert (meta[..., 0] == scale).all() and (meta[..., 1] == zero).all()
+    np.testing.assert_array_equal(o.reconstruct_values_int2(codes, meta), v)   # exact round trip
+    # power-of-two scaling and a bfloat16-exact shift move (scale, zero) and keep the codes
+    codes2, meta2 = o.encode_values_int2(4.0 * v + 2.0)
+    np.testing.assert_array_equal(codes2, want)
+    assert (meta2[..., 0] == 4 * scale).all() and (meta2[..., 1] == 4 * zero + 2.0).all()
+    # a constant vector: scale falls back to 1, every code 0, reconstruction = the constant
+    c, m = o.encode_values_int2(np.full((1, 1, d), 0.25))
+    assert not c.any() and m[0, 0, 0] == 1.0 and m[0, 0, 1] == 0.25
+    # ties go to even: a coefficient exactly half way between levels 0 and 1, and between 1 and 2
+    vv = zero + scale * want[:1].astype(np.float64)
+    vv[0, 0, 2], vv[0, 0, 3] = zero + 0.5 * scale, zero + 1.5 * scale
+    ct, _ = o.encode_values_int2(vv)
+    assert ct[0, 0, 2] == 0 and ct[0, 0, 3] == 2
+
+
+def test_int2_equals_product_codebook_with_affine_map(tiny_case):
+    """Four 2-bit codes in a byte index the 256-entry product codebook {0,1,2,3}^4: the scalar codec is a
+    vector quantiser with that fixed codebook and a per-token affine map (the identity the read path uses)."""
+    o = tiny_case["oracle"]
+    v = np.asarray(tiny_case["v"][:32], np.float64)
+    codes, meta = o.encode_values_int2(v)
+    table = np.stack([(np.arange(256) >> (2 * i)) & 3 for i in range(4)], axis=1).astype(np.float64)   # [256][4]
+    packed = (codes.reshape(32, o.n_kv_heads, o.d // 4, 4).astype(np.uint32) << (2 * np.arange(4))).sum(axis=3)
+    rec_table = table[packed].reshape(32, o.n_kv_heads, o.d)
+    np.testing.assert_array_equal(rec_table, codes.astype(np.float64))
+
+
+def test_deployed_decode_is_textbook_attention(tiny_case):
+    o = tiny_case["oracle"]
+    k, v, q = (np.asarray(tiny_case[n], np.float64) for n in ("k", "v", "q"))
+    k, v = k[:120], v[:120]
+    e = o.encode_scaled(k, v, with_gaps=False)
+    codes, meta = o.encode_values_int2(v)
+    ks, _ = o.reconstruct_scaled(e["kidx"], e["vidx"], e["kscale"])
+    vh = o.reconstruct_values_int2(codes, meta)
+    hq = q.shape[0]
+    hg = hq // o.n_kv_heads
+    ref = np.stack([np_attention(q[h], ks[:, h // hg, :], vh[:, h // hg, :], 1.0 / np.sqrt(o.d)) for h in range(hq)])
+    np.testing.assert_allclose(o.decode_deployed(q, e["kidx"], e["kscale"], codes, meta), ref, rtol=0, atol=1e-12)
+    assert cache_format.bits_per_element(128, key_scale_bits=16, value_meta_bits=32)[1] == 2.25
