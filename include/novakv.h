@@ -227,6 +227,38 @@ novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int layer, const v
     novakv_stream stream);
 
 /*
+ * The paper's deployed cache format (Sec. 5 "Bit rate": keys 2.125 bits per element, "the V cache is INT2
+ * with a BF16 scale and offset (zero-point), giving 2.000 + 32/128 = 2.250"; App. B read path: "the INT2
+ * code is dequantized in the ... rotation basis"): keys as in novakv_encode_append_scaled; values scalar
+ * quantised to 2 bits in the Corollary 1 basis R_V (which stands in for the rotation the paper takes from
+ * prior work), one bf16 (scale, zero) pair per token and KV head:
+ *     s = (v - v_mean) rv                      binary32 coefficients, as in novakv_encode_append
+ *     zero  = bf16(min_i s_i)
+ *     scale = bf16((max_i s_i - zero) / 3)     in binary32; replaced by 1 if not positive and finite
+ *     code_i = clamp(rint((s_i - zero) / scale), 0, 3)      binary32 subtraction and division, ties to even
+ *     read:  s^_i = zero + scale * code_i,  o_h = (sum_j p_hj s^_j) rv^T + v_mean
+ * The byte of group l in the value pool holds code_{4l} | code_{4l+1} << 2 | code_{4l+2} << 4 |
+ * code_{4l+3} << 6, at the position the vector-quantised format gives that group's index; cb_v of the
+ * calibration is not used.
+ *   v_meta  device, bf16 [n_pages][Hkv][64][2] = (scale, zero); novakv_value_meta_page_bytes() per page
+ * novakv_decode_attention_deployed takes the arguments of novakv_decode_attention_banded plus v_meta;
+ * band_k = band_v = band_meta = NULL reads the whole sequence from the index cache (quant_lens are then
+ * the sequence lengths, n_sink and band_cap are ignored); sink_logits may be NULL.
+ */
+size_t novakv_value_meta_page_bytes(const novakv_ctx* ctx);
+novakv_status novakv_encode_append_deployed(novakv_ctx* ctx, int layer,
+    const void* k_new, const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos,
+    int n_tokens, uint8_t* k_pages, uint8_t* v_pages, void* k_scales, void* v_meta, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
+    novakv_stream stream);
+novakv_status novakv_decode_attention_deployed(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, const void* v_meta,
+    const float* sink_logits, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+    const int32_t* quant_lens, const void* band_k, const void* band_v, int band_cap, int n_sink,
+    const int32_t* band_meta, int batch, float sm_scale, void* out, int out_is_fp32, void* workspace,
+    size_t workspace_bytes, novakv_stream stream);
+
+/*
  * The same decode step for callers that cannot supply a workspace and cannot allocate one: an
  * engine that gave all device memory to its own pool, a plug-in inside it, a serving loop that must
  * never call cudaMalloc (the call synchronises the device).  (The paper has no counterpart; this is

@@ -23,6 +23,7 @@ EXPORTED = [
     "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc", "novakv_debug_set_value_path",
     "novakv_scale_page_bytes", "novakv_encode_append_scaled", "novakv_decode_attention_scaled",
     "novakv_decode_attention_sink", "novakv_decode_attention_banded",
+    "novakv_value_meta_page_bytes", "novakv_encode_append_deployed", "novakv_decode_attention_deployed",
 ]
 
 
@@ -82,6 +83,15 @@ def load_library(path=None):
                                                    c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_int,
                                                    c_void_p, c_int, c_float, c_void_p, c_int, c_void_p, c_size_t,
                                                    c_void_p]
+    lib.novakv_value_meta_page_bytes.argtypes = [c_void_p]
+    lib.novakv_value_meta_page_bytes.restype = c_size_t
+    lib.novakv_encode_append_deployed.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
+                                                  c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int,
+                                                  c_int, c_void_p, c_void_p]
+    lib.novakv_decode_attention_deployed.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                                     c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                                     c_int, c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p,
+                                                     c_size_t, c_void_p]
     lib.novakv_decode_attention_noalloc.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                                     c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p]
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
@@ -232,6 +242,32 @@ class Context:
             _ptr(band_v), int(band_k.shape[1]), int(n_sink), _ptr(band_meta), batch, scale, _ptr(out),
             1 if out.dtype == torch.float32 else 0, _ptr(workspace),
             int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_banded")
+
+    def novakv_value_meta_page_bytes(self):
+        return int(self.lib.novakv_value_meta_page_bytes(self.handle))
+
+    def novakv_encode_append_deployed(self, layer, k_new, v_new, tok_seq, tok_pos, k_pages, v_pages, k_scales, v_meta,
+                                      page_table, seq_lens):
+        n_tokens = int(k_new.shape[0]) if k_new is not None else 0
+        _check(self.lib, self.lib.novakv_encode_append_deployed(
+            self.handle, layer, _ptr(k_new), _ptr(v_new), _ptr(tok_seq), _ptr(tok_pos), n_tokens,
+            _ptr(k_pages), _ptr(v_pages), _ptr(k_scales), _ptr(v_meta), int(k_pages.shape[0]), _ptr(page_table),
+            int(page_table.shape[1]), int(page_table.shape[0]), _ptr(seq_lens), _stream()),
+            "novakv_encode_append_deployed")
+
+    def novakv_decode_attention_deployed(self, layer, q, k_pages, v_pages, k_scales, v_meta, sink_logits, page_table,
+                                         quant_lens, band_k, band_v, n_sink, band_meta, out, workspace, sm_scale=None):
+        """Decode on the deployed format; band_k = band_v = band_meta = None: no BF16 band."""
+        import torch
+        batch = int(q.shape[0])
+        scale = float(self.head_dim) ** -0.5 if sm_scale is None else float(sm_scale)
+        opt = lambda t: _ptr(t) if t is not None else None
+        _check(self.lib, self.lib.novakv_decode_attention_deployed(
+            self.handle, layer, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(k_scales), _ptr(v_meta), opt(sink_logits),
+            int(k_pages.shape[0]), _ptr(page_table), int(page_table.shape[1]), _ptr(quant_lens), opt(band_k),
+            opt(band_v), int(band_k.shape[1]) if band_k is not None else 0, int(n_sink), opt(band_meta), batch, scale,
+            _ptr(out), 1 if out.dtype == torch.float32 else 0, _ptr(workspace),
+            int(workspace.numel() * workspace.element_size()), _stream()), "novakv_decode_attention_deployed")
 
     def novakv_decode_attention_noalloc(self, layer, q, k_pages, v_pages, page_table, seq_lens, out, sm_scale=None):
         """Decode step whose scratch is the library's fixed device array (no workspace argument)."""

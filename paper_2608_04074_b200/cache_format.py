@@ -53,6 +53,12 @@ def value_offset(t, l, n_groups_: int):
     return (t >> 4) * (n_groups_ * 16) + (fr * 4 + fc) * (ngb * 4) + x * 4 + b
 
 
+def pack_int2(codes: np.ndarray) -> np.ndarray:
+    """Scalar 2-bit codes [..][d] (0..3) -> one byte per group of 4: c0 | c1 << 2 | c2 << 4 | c3 << 6 ([..][d/4])."""
+    c = np.asarray(codes, np.uint8).reshape(codes.shape[:-1] + (codes.shape[-1] // 4, 4))
+    return (c[..., 0] | (c[..., 1] << 2) | (c[..., 2] << 4) | (c[..., 3] << 6)).astype(np.uint8)
+
+
 def index_bytes_per_token_per_kv_head(head_dim: int) -> int:
     """Key plus value index bytes of one token of one KV head."""
     return 2 * n_groups(head_dim)

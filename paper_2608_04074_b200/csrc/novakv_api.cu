@@ -57,6 +57,24 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
         delete ctx;
         return NOVAKV_ECUDA;
     }
+    {
+        // product codebook of the scalar INT2 value codec: byte c decodes to (c & 3, (c >> 2) & 3, (c >> 4) & 3, c >> 6),
+        // the same for every group and head, replicated in the layout the value gather reads
+        const size_t n = (size_t)cfg->n_kv_heads * NOVAKV_C * 32 * NOVAKV_G;
+        std::vector<__half> img(n);
+        for (size_t i = 0; i < n; ++i) {
+            const int comp = (int)(i % NOVAKV_G), code = (int)((i / (32 * NOVAKV_G)) % NOVAKV_C);
+            img[i] = __float2half((float)((code >> (2 * comp)) & 3));
+        }
+        if (cudaMalloc(&ctx->int2_img, n * sizeof(__half)) != cudaSuccess ||
+            cudaMemcpy(ctx->int2_img, img.data(), n * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(ctx->dev_status);
+    cudaFree(ctx->int2_img);
+            cudaFree(ctx->int2_img);
+            delete ctx;
+            return NOVAKV_ECUDA;
+        }
+    }
     *out = ctx;
     return NOVAKV_OK;
 }
@@ -309,6 +327,60 @@ extern "C" novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int lay
                                 page_table, max_pages_per_seq, quant_lens, batch, sm_scale, out, out_is_fp32,
                                 workspace, workspace_bytes, (cudaStream_t)stream, (const __nv_bfloat16*)k_scales,
                                 sink_logits, &band);
+}
+
+extern "C" size_t novakv_value_meta_page_bytes(const novakv_ctx* ctx) {
+    return ctx ? (size_t)ctx->cfg.n_kv_heads * NOVAKV_PAGE_TOKENS * 4 : 0;
+}
+
+extern "C" novakv_status novakv_encode_append_deployed(novakv_ctx* ctx, int layer, const void* k_new,
+    const void* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens, uint8_t* k_pages,
+    uint8_t* v_pages, void* k_scales, void* v_meta, int n_pages, const int32_t* page_table, int max_pages_per_seq,
+    int n_seq, int32_t* seq_lens, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (n_tokens < 0) return NOVAKV_EINVAL;
+    if (n_tokens == 0) return NOVAKV_OK;
+    if (!k_new || !v_new || !tok_seq || !tok_pos || !k_pages || !v_pages || !k_scales || !v_meta || !page_table || !seq_lens)
+        return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0 || n_seq <= 0) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_scales & 1) || ((uintptr_t)v_meta & 3)) return NOVAKV_EINVAL;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    return novakv_launch_encode(ctx, ctx->layers[layer], (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new,
+                                tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages, page_table,
+                                max_pages_per_seq, n_seq, seq_lens, (cudaStream_t)stream, (__nv_bfloat16*)k_scales,
+                                (__nv_bfloat16*)v_meta);
+}
+
+extern "C" novakv_status novakv_decode_attention_deployed(novakv_ctx* ctx, int layer, const void* q,
+    const uint8_t* k_pages, const uint8_t* v_pages, const void* k_scales, const void* v_meta, const float* sink_logits,
+    int n_pages, const int32_t* page_table, int max_pages_per_seq, const int32_t* quant_lens, const void* band_k,
+    const void* band_v, int band_cap, int n_sink, const int32_t* band_meta, int batch, float sm_scale, void* out,
+    int out_is_fp32, void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!q || !k_pages || !v_pages || !k_scales || !v_meta || !page_table || !quant_lens || !out) return NOVAKV_EINVAL;
+    const bool banded = band_k != nullptr || band_v != nullptr || band_meta != nullptr;
+    if (banded && (!band_k || !band_v || !band_meta)) return NOVAKV_EINVAL;
+    if (banded && (n_sink < 0 || n_sink % NOVAKV_PAGE_TOKENS != 0 || band_cap < n_sink)) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= (banded ? n_sink / NOVAKV_PAGE_TOKENS : 0)) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_pages & 15) || ((uintptr_t)v_pages & 15) || ((uintptr_t)k_scales & 1) || ((uintptr_t)v_meta & 3) ||
+        ((uintptr_t)sink_logits & 3) || ((uintptr_t)band_k & 3) || ((uintptr_t)band_v & 3)) return NOVAKV_EINVAL;
+    if (!(sm_scale == sm_scale)) return NOVAKV_EINVAL;
+    if (!workspace || workspace_bytes < novakv_decode_ws_bytes(ctx, batch) || ((uintptr_t)workspace & 255)) return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    novakv_band_args band;
+    band.k = (const __nv_bfloat16*)band_k;
+    band.v = (const __nv_bfloat16*)band_v;
+    band.cap = band_cap;
+    band.n_sink = n_sink;
+    band.meta = band_meta;
+    return novakv_launch_decode(ctx, ctx->layers[layer], (const __nv_bfloat16*)q, k_pages, v_pages, n_pages,
+                                page_table, max_pages_per_seq, quant_lens, batch, sm_scale, out, out_is_fp32,
+                                workspace, workspace_bytes, (cudaStream_t)stream, (const __nv_bfloat16*)k_scales,
+                                sink_logits, banded ? &band : nullptr, (const __nv_bfloat16*)v_meta);
 }
 
 extern "C" novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, uint32_t* word) {

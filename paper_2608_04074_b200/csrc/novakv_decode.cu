@@ -63,7 +63,7 @@ struct S1 {
     // one partial per lane column (4 per warp)
     static constexpr int MERGE_SLOTS = VM ? NCW : NCW * 4;
     static constexpr int MERGE_ACC_BYTES = MERGE_SLOTS * HPAD * D * 4;
-    static_assert(MERGE_ACC_BYTES + NCW * HPAD * 8 <= LUT_BYTES, "merge buffer must fit in the table");
+    static_assert(MERGE_ACC_BYTES + NCW * HPAD * 12 <= LUT_BYTES, "merge buffer must fit in the table");
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
@@ -339,15 +339,21 @@ struct TileRegs {
     uint32_t kw[L / 4];
     uint32_t vw[2][L / 8];
     uint32_t ks;          // this lane's token: bfloat16 key scale in the high half (a binary32 bit pattern), if used
+    uint32_t vm;          // this lane's token: bfloat16 value scale (low half) and zero-point (high half), if used
 };
 
 // KSC: the key format carries a per-token bfloat16 scale (k_scales [n_pages][Hkv][64]); the logits of a
 // token are multiplied by it once, after the table lookups are summed.
-template <int D, int HG, bool VM, bool KSC>
+// VSQ: scalar INT2 values with a per-token bfloat16 scale and zero-point (v_meta [n_pages][Hkv][64][2]).
+// A byte of four 2-bit codes indexes the product codebook {0,1,2,3}^4, so the value side is the same gather
+// with that fixed table as cb_v_img; the weight of a token's codes is p * scale and the zero-points enter
+// through one extra running sum per head, sum_j p_j zero_j, added to every coefficient in the epilogue.
+template <int D, int HG, bool VM, bool KSC, bool VSQ>
 __global__ void __launch_bounds__(S1_THREADS, 1)
 novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restrict__ cb_k_lut,
                             const __half* __restrict__ cb_v_img, const uint8_t* __restrict__ k_pages,
-                            const uint8_t* __restrict__ v_pages, const __nv_bfloat16* __restrict__ k_scales, int n_pages,
+                            const uint8_t* __restrict__ v_pages, const __nv_bfloat16* __restrict__ k_scales,
+                            const __nv_bfloat16* __restrict__ v_meta, int n_pages,
                             const int32_t* __restrict__ page_table, int max_pages_per_seq,
                             const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ page_prefix,
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
@@ -370,6 +376,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
     // per-warp running state
     float m_run[HPAD], l_run[HPAD];
+    float lz_run[VSQ ? HPAD : 1];                //  VSQ: running sum_j p_j zero_j per head (this lane's tokens)
+#pragma unroll
+    for (int h = 0; h < (VSQ ? HPAD : 1); ++h) lz_run[h] = 0.f;
     float macc[HSETS][NGB][4];                   //  VM: lane (fr, fc): head 4 hs + fc, group 8 gb + fr, 4 coefficients
     uint64_t acc[VM ? 1 : NGB][VM ? 1 : HPAD][2];  // !VM: lane (fr, fc): load x (group 8((x+fc)%NGB)+fr), head, 4 coefficients
 #pragma unroll
@@ -431,6 +440,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                                                  ((size_t)page * n_kv_heads + sg.kvh) * NOVAKV_PAGE_TOKENS + half * 32 + lane);
                 t.ks = (uint32_t)raw << 16;
             }
+            if (VSQ)
+                t.vm = __ldg(reinterpret_cast<const uint32_t*>(v_meta) +
+                             ((size_t)page * n_kv_heads + sg.kvh) * NOVAKV_PAGE_TOKENS + half * 32 + lane);
             const uint8_t* kp = k_pages + off + lane * 16;
             const uint8_t* vp = v_pages + off + lane * (NGB * 4);
 #pragma unroll
@@ -518,6 +530,11 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     zf[h] = __half2float(ph[h]);
                 }
                 l_run[h] = fmaf(l_run[h], alpha[h], zf[h]);
+                if (VSQ) {
+                    const float vscale = __uint_as_float(cur.vm << 16), vzero = __uint_as_float(cur.vm & 0xffff0000u);
+                    lz_run[h] = fmaf(lz_run[h], alpha[h], lane < nvalid ? zf[h] * vzero : 0.f);
+                    ph[h] = __float2half_rn(zf[h] * vscale);      // the weight of the token's integer codes
+                }
             }
 
             if (VM) {
@@ -653,10 +670,16 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         __syncthreads();                                   // scan done everywhere: the table is dead
         float* m_acc = reinterpret_cast<float*>(smem + C::OFF_LUT);                    // [MERGE_SLOTS][HPAD][D]
         float* m_ml = reinterpret_cast<float*>(smem + C::OFF_LUT + C::MERGE_ACC_BYTES);  // [NCW][HPAD][2]
+        float* m_lz = m_ml + NCW * HPAD * 2;                                             // [NCW][HPAD]  (VSQ)
 #pragma unroll
         for (int h = 0; h < HPAD; ++h) {
             const float lsum = warp_sum(l_run[h]);
             if (lane == 0) { m_ml[(warp * HPAD + h) * 2] = m_run[h]; m_ml[(warp * HPAD + h) * 2 + 1] = lsum; }
+            if (VSQ) {
+                const float lz = warp_sum(lz_run[h]);
+                if (lane == 0) m_lz[warp * HPAD + h] = lz;
+                lz_run[h] = 0.f;
+            }
             m_run[h] = M_INIT; l_run[h] = 0.f;
         }
         if (VM) {
@@ -700,6 +723,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     float aw = 0.f;
 #pragma unroll
                     for (int s = 0; s < SPW; ++s) aw += m_acc[((size_t)(w * SPW + s) * HPAD + h) * D + c];
+                    if (VSQ) aw += m_lz[w * HPAD + h];              // zero-points: the same amount on every coefficient
                     a = fmaf(sc, aw, a);
                     lsum = fmaf(sc, m_ml[(w * HPAD + h) * 2 + 1], lsum);
                 }
@@ -964,9 +988,10 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     return w;
 }
 
-template <int D, int HG, bool VM, bool KSC>
+template <int D, int HG, bool VM, bool KSC, bool VSQ>
 novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* q,
-                              const uint8_t* k_pages, const uint8_t* v_pages, const __nv_bfloat16* k_scales, int n_pages,
+                              const uint8_t* k_pages, const uint8_t* v_pages, const __nv_bfloat16* k_scales,
+                              const __nv_bfloat16* v_meta, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, const int32_t* seq_lens,
                               int batch, float sm_scale, void* out, int out_is_fp32, void* workspace,
                               cudaStream_t stream, const float* sink_logits, const novakv_band_args* band) {
@@ -995,7 +1020,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                       ly.k_mean, qk_off);
     ctx->launches++;
 
-    auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC>;
+    auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC, VSQ>;
     static bool smem_opt_in = false;      // per template instantiation; the attribute is sticky
     if (!smem_opt_in) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
@@ -1004,8 +1029,8 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
     {
         novakv_prof_scope ps(ctx, 0, stream);
-        novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut, ly.cb_v_mma, k_pages, v_pages,
-                          k_scales, n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
+        novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut,
+                          VSQ ? (const __half*)ctx->int2_img : (const __half*)ly.cb_v_mma, k_pages, v_pages, k_scales, v_meta, n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
                           ctx->dev_status, pt_stride);
         ps.end();
         ctx->launches++;
@@ -1032,21 +1057,26 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
     const uint8_t* k_pages, const uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, const int32_t* seq_lens, int batch, float sm_scale, void* out,
     int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream, const __nv_bfloat16* k_scales,
-    const float* sink_logits, const novakv_band_args* band) {
+    const float* sink_logits, const novakv_band_args* band, const __nv_bfloat16* v_meta) {
     (void)workspace_bytes;
     const int d = ctx->cfg.head_dim, hg = ctx->hg;
     if (k_scales != nullptr && ctx->value_path == 0) return NOVAKV_EUNSUPPORTED;   // scaled keys: tensor-core value side only
+    if (v_meta != nullptr && k_scales == nullptr) return NOVAKV_EUNSUPPORTED;      // INT2 values come with scaled keys (deployed format)
 #define NOVAKV_DISPATCH(DD, HH)                                                                             \
     if (d == DD && hg == HH) {                                                                                   \
+        if (v_meta != nullptr)                                                                                   \
+            return launch_decode_t<DD, HH, true, true, true>(ctx, ly, q, k_pages, v_pages, k_scales, v_meta, n_pages, page_table, \
+                                                  max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
+                                                  workspace, stream, sink_logits, band);                         \
         if (k_scales != nullptr)                                                                                 \
-            return launch_decode_t<DD, HH, true, true>(ctx, ly, q, k_pages, v_pages, k_scales, n_pages, page_table, \
+            return launch_decode_t<DD, HH, true, true, false>(ctx, ly, q, k_pages, v_pages, k_scales, nullptr, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
                                                   workspace, stream, sink_logits, band);                               \
         if (ctx->value_path == 0)                                                                                \
-            return launch_decode_t<DD, HH, false, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table, \
+            return launch_decode_t<DD, HH, false, false, false>(ctx, ly, q, k_pages, v_pages, nullptr, nullptr, n_pages, page_table, \
                                                   max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32, \
                                                   workspace, stream, sink_logits, band);                               \
-        return launch_decode_t<DD, HH, true, false>(ctx, ly, q, k_pages, v_pages, nullptr, n_pages, page_table,  \
+        return launch_decode_t<DD, HH, true, false, false>(ctx, ly, q, k_pages, v_pages, nullptr, nullptr, n_pages, page_table,  \
                                              max_pages_per_seq, seq_lens, batch, sm_scale, out, out_is_fp32,     \
                                              workspace, stream, sink_logits, band);                                    \
     }

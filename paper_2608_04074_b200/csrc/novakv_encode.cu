@@ -174,8 +174,8 @@ struct EncPipe {
     static constexpr size_t off_idx = off_slab + 2 * slab_bytes;
     static constexpr size_t off_pos = off_idx + idx_bytes;                          // [2][2][ENC_TILE] ints
     static constexpr size_t off_mean = off_pos + 4 * ENC_TILE * sizeof(int);        // [D] doubles
-    static constexpr size_t off_rho = off_mean + D * sizeof(double);                // [2][ENC_TILE] floats (key scales)
-    static constexpr size_t total = off_rho + 2 * ENC_TILE * sizeof(float);
+    static constexpr size_t off_rho = off_mean + D * sizeof(double);                // [2][2][ENC_TILE] floats (key scale | value scale, zero)
+    static constexpr size_t total = off_rho + 4 * ENC_TILE * sizeof(float);
     static_assert(total <= 232448, "shared memory budget");
 };
 
@@ -189,7 +189,12 @@ struct EncPipe {
 // in binary64), round it to binary32 and then to bfloat16 (a scale that is not positive and finite becomes
 // 1), divide the coefficients by it in binary32 (IEEE division) and hand rho to the search warps, which
 // store it beside the indices (k_scales [n_pages][Hkv][64]).  Values are not scaled.
-template <int D, bool KSC>
+// VSQ (scalar INT2 value codec of the deployed format): after the value transform of a tile the transform
+// warps form zero = bf16(min) and scale = bf16((max - zero) / 3) per token, replace each coefficient by its
+// level clamp(rint((s - zero) / scale), 0, 3), and the other warps pack four levels per byte (the byte of a
+// group) instead of searching; (scale, zero) go to v_meta [n_pages][Hkv][64][2].
+// FMT: 0 = 2-bit keys and values (vector quantised), 1 = KSC, 2 = KSC and VSQ.
+template <int D, int FMT>
 __global__ void __launch_bounds__(ENC_THREADS, 1)
 novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                      const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
@@ -197,10 +202,11 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                      const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
                      const float* __restrict__ cb_k, const float* __restrict__ cb_v,
                      uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages,
-                     __nv_bfloat16* __restrict__ k_scales, int n_pages,
+                     __nv_bfloat16* __restrict__ k_scales, __nv_bfloat16* __restrict__ v_meta, int n_pages,
                      const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                      int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
                      uint32_t* __restrict__ dev_status) {
+    constexpr bool KSC = FMT >= 1, VSQ = FMT == 2;
     using P = EncPipe<D>;
     constexpr int L = D / NOVAKV_G, RS = P::RS, NT = ENC_HALF_THREADS;
     extern __shared__ __align__(16) unsigned char smem[];
@@ -208,7 +214,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     uint8_t* idx_s = smem + P::off_idx;
     int* pos_s = reinterpret_cast<int*>(smem + P::off_pos);                // [buf][page|slot][ENC_TILE]
     double* mean_s = reinterpret_cast<double*>(smem + P::off_mean);
-    float* rho_s = reinterpret_cast<float*>(smem + P::off_rho);            // [buf][ENC_TILE]
+    float* rho_s = reinterpret_cast<float*>(smem + P::off_rho);            // [buf][2][ENC_TILE]
 
     const int kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
@@ -217,7 +223,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
 
     // codebook of this (head, side) -> shared memory, once per CTA
-    fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);
+    if (!(VSQ && side == 1)) fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);
     for (int i = threadIdx.x; i < D; i += ENC_THREADS) mean_s[i] = mean[i];
     __syncthreads();
 
@@ -348,7 +354,27 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                 if (!(rho > 0.f) || !isfinite(rho)) rho = 1.f;
 #pragma unroll 8
                 for (int i = 0; i < D / 4; ++i) row[4 * i] = __fdiv_rn(row[4 * i], rho);
-                if (part == 0) rho_s[buf * ENC_TILE + t] = rho;
+                if (part == 0) rho_s[(buf * 2) * ENC_TILE + t] = rho;
+            }
+            if (VSQ && side == 1) {
+                nbar_sync(BAR_T, NT);
+                const int t = tid >> 2, part = tid & 3;
+                float* row = r_s + (size_t)t * RS + part;
+                float mn = row[0], mx = row[0];
+#pragma unroll 8
+                for (int i = 1; i < D / 4; ++i) { mn = fminf(mn, row[4 * i]); mx = fmaxf(mx, row[4 * i]); }
+                mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float zero = __bfloat162float(__float2bfloat16_rn(mn));
+                float scale = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(__fsub_rn(mx, zero), 3.0f)));
+                if (!(scale > 0.f) || !isfinite(scale)) scale = 1.f;
+#pragma unroll 8
+                for (int i = 0; i < D / 4; ++i) {
+                    float u = rintf(__fdiv_rn(__fsub_rn(row[4 * i], zero), scale));
+                    if (!(u > 0.f)) u = 0.f;
+                    row[4 * i] = fminf(u, 3.f);
+                }
+                if (part == 0) { rho_s[(buf * 2) * ENC_TILE + t] = scale; rho_s[(buf * 2 + 1) * ENC_TILE + t] = zero; }
             }
             __threadfence_block();
             nbar_arrive(BAR_FULL + buf, ENC_THREADS);            // hand tile i to the search warps
@@ -361,7 +387,16 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
             const int n_valid = min(ENC_TILE, n_tokens - t0);
             const float* r_s = reinterpret_cast<const float*>(smem + P::off_r + buf * P::r_bytes);
             nbar_sync(BAR_FULL + buf, ENC_THREADS);
-            search_tile<D>(r_s, cb_s, idx_s, n_valid, tid >> 5, NT / 32);
+            if (VSQ && side == 1) {
+                // four levels (0..3, held as floats) per byte: the byte of group l
+                for (int e = tid; e < ENC_TILE * L; e += NT) {
+                    const int t = e / L, l = e - t * L;
+                    const float4 c = *reinterpret_cast<const float4*>(r_s + (size_t)t * RS + l * 4);
+                    idx_s[e] = (uint8_t)((int)c.x | ((int)c.y << 2) | ((int)c.z << 4) | ((int)c.w << 6));
+                }
+            } else {
+                search_tile<D>(r_s, cb_s, idx_s, n_valid, tid >> 5, NT / 32);
+            }
             nbar_sync(BAR_S, NT);
             for (int e = tid; e < n_valid * L; e += NT) {
                 const int t = e / L, l = e - t * L;
@@ -376,7 +411,14 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                 const int page = pos_s[(buf * 2 + 0) * ENC_TILE + tid];
                 if (page >= 0)
                     k_scales[((size_t)page * n_kv_heads + kvh) * NOVAKV_PAGE_TOKENS + pos_s[(buf * 2 + 1) * ENC_TILE + tid]] =
-                        __float2bfloat16_rn(rho_s[buf * ENC_TILE + tid]);
+                        __float2bfloat16_rn(rho_s[(buf * 2) * ENC_TILE + tid]);
+            }
+            if (VSQ && side == 1 && tid < n_valid) {
+                const int page = pos_s[(buf * 2 + 0) * ENC_TILE + tid];
+                if (page >= 0)
+                    reinterpret_cast<__nv_bfloat162*>(v_meta)[((size_t)page * n_kv_heads + kvh) * NOVAKV_PAGE_TOKENS +
+                                                              pos_s[(buf * 2 + 1) * ENC_TILE + tid]] =
+                        __floats2bfloat162_rn(rho_s[(buf * 2) * ENC_TILE + tid], rho_s[(buf * 2 + 1) * ENC_TILE + tid]);
             }
             nbar_sync(BAR_S, NT);                                // idx_s and the buffer are free again
             if (i + 2 < n_local) nbar_arrive(BAR_EMPTY + buf, ENC_THREADS);
@@ -398,7 +440,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 // each publishes the sums of squares of its 16 coefficients per token in its shared memory, a cluster
 // barrier makes them visible, and every CTA adds the L/4 x 4 partial sums in the same fixed order through
 // distributed shared memory, so that all of them normalise by the same rho.
-template <int D, bool KSC>
+template <int D, int FMT>
 __global__ void __launch_bounds__(128)
 novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                            const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
@@ -407,12 +449,14 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                            const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
                            const float* __restrict__ cb_k, const float* __restrict__ cb_v,
                            uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages,
-                           __nv_bfloat16* __restrict__ k_scales, int n_pages,
+                           __nv_bfloat16* __restrict__ k_scales, __nv_bfloat16* __restrict__ v_meta, int n_pages,
                            const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                            int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
     constexpr int L = D / NOVAKV_G;
+    constexpr bool KSC = FMT >= 1, VSQ = FMT == 2;
     __shared__ __align__(16) double R_s[4][D][4];
     __shared__ double ss_s[4][32];                  // KSC: sum of squares of a warp's 4 coefficients, per token of the pass
+    __shared__ float mx_s[4][32];                   // VSQ: maximum of a warp's 4 value coefficients (the minimum rides in ss_s)
     __shared__ float4 cb_s[4][NOVAKV_C];
     __shared__ double mean_s[D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -493,6 +537,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             }
         }
         float4 r = make_float4((float)acc0, (float)acc1, (float)acc2, (float)acc3);
+        int vsq_byte = 0;
         if (KSC) {
             namespace cg = cooperative_groups;
             cg::cluster_group cluster = cg::this_cluster();
@@ -517,6 +562,36 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                 if (blockIdx.x == 0 && warp == 0 && grp == 0 && page >= 0)
                     k_scales[((size_t)page * n_kv_heads + kvh) * NOVAKV_PAGE_TOKENS + slot] = __float2bfloat16_rn(rho);
             }
+            if (VSQ && side == 1 && grp == 0) {
+                // value side: the warp's minimum and maximum travel in the same slots (as doubles)
+                ss_s[warp][tok_in_pass] = (double)fminf(fminf(r.x, r.y), fminf(r.z, r.w));
+                mx_s[warp][tok_in_pass] = fmaxf(fmaxf(r.x, r.y), fmaxf(r.z, r.w));
+            }
+            if (VSQ) cluster.sync();
+            if (VSQ && side == 1) {
+                float mn = CUDART_INF_F, mx = -CUDART_INF_F;
+                for (unsigned cr = 0; cr < cluster.num_blocks(); ++cr) {
+                    const double* rmn = cluster.map_shared_rank(&ss_s[0][0], cr);
+                    const float* rmx = cluster.map_shared_rank(&mx_s[0][0], cr);
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        mn = fminf(mn, (float)rmn[w * 32 + tok_in_pass]);
+                        mx = fmaxf(mx, rmx[w * 32 + tok_in_pass]);
+                    }
+                }
+                const float zero = __bfloat162float(__float2bfloat16_rn(mn));
+                float scale = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(__fsub_rn(mx, zero), 3.0f)));
+                if (!(scale > 0.f) || !isfinite(scale)) scale = 1.f;
+                auto level = [&](float x) {
+                    float u = rintf(__fdiv_rn(__fsub_rn(x, zero), scale));
+                    if (!(u > 0.f)) u = 0.f;
+                    return (int)fminf(u, 3.f);
+                };
+                vsq_byte = level(r.x) | (level(r.y) << 2) | (level(r.z) << 4) | (level(r.w) << 6);
+                if (blockIdx.x == 0 && warp == 0 && grp == 0 && page >= 0)
+                    reinterpret_cast<__nv_bfloat162*>(v_meta)[((size_t)page * n_kv_heads + kvh) * NOVAKV_PAGE_TOKENS + slot] =
+                        __floats2bfloat162_rn(scale, zero);
+            }
             cluster.sync();                             // partial sums may be overwritten by the next pass / CTAs may exit
         }
         // this lane group's range of the codebook, ascending with a strict '<' (first minimum)
@@ -533,6 +608,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
             if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
         }
+        if (VSQ && side == 1) bi = vsq_byte;             // scalar codec: the byte holds four levels, no search result
         if (grp == 0 && page >= 0) {
             const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
             if (side == 0) k_pages[base + novakv_k_offset<L>(slot, l)] = (uint8_t)bi;
@@ -579,16 +655,16 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                               const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos,
                               int n_tokens, uint8_t* k_pages, uint8_t* v_pages, int n_pages,
                               const int32_t* page_table, int max_pages_per_seq, int n_seq, int32_t* seq_lens,
-                              cudaStream_t stream, __nv_bfloat16* k_scales) {
+                              cudaStream_t stream, __nv_bfloat16* k_scales, __nv_bfloat16* v_meta) {
     if (n_tokens <= NOVAKV_SMALL_APPEND_TOKENS) {
         dim3 grid(D / NOVAKV_G / 4, ctx->cfg.n_kv_heads, 2);
         novakv_prof_scope ps(ctx, 1, stream);
         int tp_log2 = 0;
         while ((1 << tp_log2) < n_tokens && tp_log2 < 5) ++tp_log2;
         if (k_scales == nullptr) {
-            novakv_launch_pdl(novakv_encode_small_kernel<D, false>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos,
+            novakv_launch_pdl(novakv_encode_small_kernel<D, 0>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos,
                               n_tokens, tp_log2, ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages,
-                              (__nv_bfloat16*)nullptr, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
+                              (__nv_bfloat16*)nullptr, (__nv_bfloat16*)nullptr, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
                               ctx->cfg.n_kv_heads, ctx->dev_status);
         } else {
             // scaled key format: the L/4 CTAs of a (head, side) are one cluster (8 at d = 128, 4 at d = 64)
@@ -606,10 +682,11 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
             cfg.attrs = attr;
             cfg.numAttrs = 2;
             const int hkv = ctx->cfg.n_kv_heads;
-            if (cudaLaunchKernelEx(&cfg, novakv_encode_small_kernel<D, true>, k_new, v_new, tok_seq, tok_pos, n_tokens, tp_log2,
+            auto small = v_meta ? novakv_encode_small_kernel<D, 2> : novakv_encode_small_kernel<D, 1>;
+            if (cudaLaunchKernelEx(&cfg, small, k_new, v_new, tok_seq, tok_pos, n_tokens, tp_log2,
                                    (const double*)ly.rk_d, (const double*)ly.rv_d, (const double*)ly.k_mean_d,
                                    (const double*)ly.v_mean_d, (const float*)ly.cb_k, (const float*)ly.cb_v, k_pages, v_pages,
-                                   k_scales, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens, hkv,
+                                   k_scales, v_meta, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens, hkv,
                                    ctx->dev_status) != cudaSuccess)
                 return NOVAKV_ECUDA;
         }
@@ -617,7 +694,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         ctx->launches++;
         return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
     }
-    auto kern = k_scales ? novakv_encode_kernel<D, true> : novakv_encode_kernel<D, false>;
+    auto kern = v_meta ? novakv_encode_kernel<D, 2> : (k_scales ? novakv_encode_kernel<D, 1> : novakv_encode_kernel<D, 0>);
     const size_t smem = EncPipe<D>::total;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return NOVAKV_ECUDA;
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
@@ -639,7 +716,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     novakv_prof_scope ps(ctx, 1, stream);
     kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d_mma, ly.rv_d_mma,
                                                ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, k_scales,
-                                               n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
+                                               v_meta, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
                                                ctx->cfg.n_kv_heads, tiles_per_cta, ctx->dev_status);
     ps.end();
     ctx->launches++;
@@ -665,12 +742,14 @@ novakv_status launch_search_t(novakv_ctx* ctx, const novakv_layer& ly, int which
 novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, const __nv_bfloat16* k_new,
     const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens,
     uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
-    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream, __nv_bfloat16* k_scales) {
+    int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream, __nv_bfloat16* k_scales,
+    __nv_bfloat16* v_meta) {
+    if (v_meta != nullptr && k_scales == nullptr) return NOVAKV_EUNSUPPORTED;   // INT2 values come with scaled keys
     if (ctx->cfg.head_dim == 128)
         return launch_encode_t<128>(ctx, ly, k_new, v_new, tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages,
-                                    page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales);
+                                    page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales, v_meta);
     return launch_encode_t<64>(ctx, ly, k_new, v_new, tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages,
-                               page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales);
+                               page_table, max_pages_per_seq, n_seq, seq_lens, stream, k_scales, v_meta);
 }
 
 // Gather of up to 5 page-locked host buffers into device staging: every 32-bit word crosses the bus

@@ -44,6 +44,7 @@ struct novakv_ctx {
     int hg = 0, n_groups = 0, n_sm = 0;
     std::vector<novakv_layer> layers;
     uint32_t* dev_status = nullptr;
+    void* int2_img = nullptr;     // binary16 [Hkv][256][32][4]: the product codebook {0,1,2,3}^4 in the value-gather layout
     bool profile = false;
     std::vector<novakv_event_pair> prof[3];
     std::vector<novakv_event_pair> prof_free;
@@ -68,7 +69,8 @@ novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, cons
     const __nv_bfloat16* v_new, const int32_t* tok_seq, const int32_t* tok_pos, int n_tokens,
     uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, int n_seq, int32_t* seq_lens, cudaStream_t stream,
-    __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */);
+    __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */,
+    __nv_bfloat16* v_meta = nullptr /* INT2 value codec: (scale, zero) [n_pages][Hkv][64][2] */);
 novakv_status novakv_launch_search(novakv_ctx* ctx, const novakv_layer& ly, int which, const float* coef,
     int n, uint8_t* idx_out, cudaStream_t stream);
 
@@ -87,7 +89,8 @@ novakv_status novakv_launch_decode(novakv_ctx* ctx, const novakv_layer& ly, cons
     int out_is_fp32, void* workspace, size_t workspace_bytes, cudaStream_t stream,
     const __nv_bfloat16* k_scales = nullptr /* scaled key format: [n_pages][Hkv][64] */,
     const float* sink_logits = nullptr /* learned sink: [Hq], natural-log units */,
-    const novakv_band_args* band = nullptr /* BF16 sink-plus-recent band */);
+    const novakv_band_args* band = nullptr /* BF16 sink-plus-recent band */,
+    const __nv_bfloat16* v_meta = nullptr /* INT2 value codec: (scale, zero) [n_pages][Hkv][64][2] */);
 
 // gather of page-locked host buffers into device staging (one kernel for up to 5 segments of 32-bit words)
 struct novakv_stage_args {

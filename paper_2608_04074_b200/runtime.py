@@ -16,9 +16,11 @@ class PagedCache:
     """Key/value index pools plus page table and lengths for a batch of sequences."""
 
     def __init__(self, ctx: Context, seq_lens, capacity_tokens=None, seed: int = 0, device="cuda:0",
-                 key_scale: bool = False):
+                 key_scale: bool = False, int2_values: bool = False):
         self.ctx = ctx
-        self.key_scale = key_scale
+        self.key_scale = key_scale or int2_values
+        self.int2_values = int2_values
+        key_scale = self.key_scale
         self.device = torch.device(device)
         seq_lens = np.asarray(seq_lens, dtype=np.int32)
         cap = seq_lens if capacity_tokens is None else np.maximum(np.asarray(capacity_tokens, np.int32), seq_lens)
@@ -32,6 +34,9 @@ class PagedCache:
         # scaled key format: one bf16 scale per token and KV head, [n_pages][Hkv][64]
         self.k_scales = (torch.ones((self.n_pages, ctx.n_kv_heads, cache_format.PAGE_TOKENS), dtype=torch.bfloat16,
                                     device=self.device) if key_scale else None)
+        # deployed format: scalar INT2 values with a bf16 (scale, zero) pair per token and KV head
+        self.v_meta = (torch.zeros((self.n_pages, ctx.n_kv_heads, cache_format.PAGE_TOKENS, 2), dtype=torch.bfloat16,
+                                   device=self.device) if int2_values else None)
         # unused table entries point at page 0 so that a wrong read stays in bounds
         self.page_table = torch.from_numpy(np.where(table < 0, 0, table).astype(np.int32)).to(self.device)
         self.seq_lens = torch.from_numpy(seq_lens.copy()).to(self.device)
@@ -75,7 +80,23 @@ class PagedCache:
         return sp[self.page_table_host[seq][pos // cache_format.PAGE_TOKENS], :, pos % cache_format.PAGE_TOKENS]
 
     # ---- hot path calls
+    def load_value_meta(self, seq: int, pos0: int, n: int) -> np.ndarray:
+        """(scale, zero) [n][Hkv][2] of positions pos0.. of one sequence."""
+        mp = self.v_meta.float().cpu().numpy()
+        pos = pos0 + np.arange(n)
+        return mp[self.page_table_host[seq][pos // cache_format.PAGE_TOKENS], :, pos % cache_format.PAGE_TOKENS, :]
+
+    def store_value_meta(self, seq: int, pos0: int, meta: np.ndarray):
+        mp = self.v_meta.float().cpu().numpy()
+        pos = pos0 + np.arange(meta.shape[0])
+        mp[self.page_table_host[seq][pos // cache_format.PAGE_TOKENS], :, pos % cache_format.PAGE_TOKENS, :] = meta
+        self.v_meta.copy_(torch.from_numpy(mp).to(torch.bfloat16))
+
     def append(self, layer, k_new, v_new, tok_seq, tok_pos):
+        if self.int2_values:
+            self.ctx.novakv_encode_append_deployed(layer, k_new, v_new, tok_seq, tok_pos, self.k_pages, self.v_pages,
+                                                   self.k_scales, self.v_meta, self.page_table, self.seq_lens)
+            return
         if self.key_scale:
             self.ctx.novakv_encode_append_scaled(layer, k_new, v_new, tok_seq, tok_pos, self.k_pages, self.v_pages,
                                                  self.k_scales, self.page_table, self.seq_lens)
@@ -87,6 +108,11 @@ class PagedCache:
         if out is None:
             out = torch.empty((self.batch, self.ctx.n_q_heads, self.ctx.head_dim), dtype=torch.float32,
                               device=self.device)
+        if self.int2_values:
+            self.ctx.novakv_decode_attention_deployed(layer, q, self.k_pages, self.v_pages, self.k_scales, self.v_meta,
+                                                      sink_logits, self.page_table, self.seq_lens, None, None, 0, None,
+                                                      out, self.workspace, sm_scale)
+            return out
         if sink_logits is not None:
             self.ctx.novakv_decode_attention_sink(layer, q, self.k_pages, self.v_pages, self.k_scales, sink_logits,
                                                   self.page_table, self.seq_lens, out, self.workspace, sm_scale)
@@ -108,12 +134,12 @@ class BandedCache:
     the library's calls."""
 
     def __init__(self, ctx: Context, batch: int, capacity_tokens: int, n_sink: int = 64, n_rec: int = 256,
-                 block: int = 8, seed: int = 0, device="cuda:0", key_scale: bool = False):
+                 block: int = 8, seed: int = 0, device="cuda:0", key_scale: bool = False, int2_values: bool = False):
         assert n_sink % cache_format.PAGE_TOKENS == 0
         self.ctx, self.batch, self.n_sink, self.n_rec, self.block = ctx, batch, n_sink, n_rec, block
         self.device = torch.device(device)
         self.paged = PagedCache(ctx, np.zeros(batch, np.int32), capacity_tokens=np.full(batch, capacity_tokens, np.int32),
-                                seed=seed, device=device, key_scale=key_scale)
+                                seed=seed, device=device, key_scale=key_scale, int2_values=int2_values)
         self.ring_cap = n_rec + block
         self.cap = n_sink + self.ring_cap
         shape = (batch, self.cap, ctx.n_kv_heads, ctx.head_dim)
@@ -195,6 +221,11 @@ class BandedCache:
             out = torch.empty((self.batch, self.ctx.n_q_heads, self.ctx.head_dim), dtype=torch.float32,
                               device=self.device)
         p = self.paged
+        if p.int2_values:
+            self.ctx.novakv_decode_attention_deployed(layer, q, p.k_pages, p.v_pages, p.k_scales, p.v_meta, sink_logits,
+                                                      p.page_table, self.quant_lens, self.band_k, self.band_v,
+                                                      self.n_sink, self.band_meta, out, p.workspace, sm_scale)
+            return out
         self.ctx.novakv_decode_attention_banded(layer, q, p.k_pages, p.v_pages, p.k_scales, sink_logits, p.page_table,
                                                 self.quant_lens, self.band_k, self.band_v, self.n_sink,
                                                 self.band_meta, out, p.workspace, sm_scale)

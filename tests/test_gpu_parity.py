@@ -720,3 +720,107 @@ def test_banded_with_scale_and_sink(qwen_scaled):
         ref = case.oracle.decode_banded(q[b].astype(np.float64), e["kidx"], e["vidx"], k, v, cache.band_mask(b),
                                         kscale=e["kscale"], sink=sink.astype(np.float64))
         check_output(out[b], ref)
+
+
+# --------------------------------------------------------------------------- deployed format: scaled VQ keys + INT2 values
+@pytest.mark.parametrize("add", [[200, 64, 1, 130], [20, 7, 1, 3], [1, 0, 0, 0], [70, 60, 50, 40]])
+@pytest.mark.parametrize("name", ["qwen_scaled", "gptoss_scaled"])
+def test_deployed_encode_matches_oracle(name, add, request):
+    """Keys as in the scaled format; value bytes (four 2-bit levels each) and (scale, zero) bit for bit."""
+    from paper_2608_04074_b200 import cache_format
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = request.getfixturevalue(name)
+    lens0 = np.array([0, 5, 63, 130], np.int32)
+    add = np.array(add, np.int32)
+    cache = PagedCache(case.ctx, lens0, capacity_tokens=lens0 + add, seed=3, int2_values=True)
+    n = int(add.sum())
+    k, v, _ = case.draw(1300, n, 1)
+    v = synth.to_bf16_representable(v * (2.0 ** synth.rng(16).integers(-2, 3, size=(n, 1, 1))) + 0.25)
+    tok_seq = np.concatenate([np.full(a, b, np.int32) for b, a in enumerate(add)])
+    tok_pos = np.concatenate([lens0[b] + np.arange(a, dtype=np.int32) for b, a in enumerate(add)])
+    perm = synth.rng(17).permutation(n)
+    k, v, tok_seq, tok_pos = k[perm], v[perm], tok_seq[perm], tok_pos[perm]
+    cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(tok_seq), _dev(tok_pos))
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens0 + add)
+    enc = case.oracle.encode_scaled(k.astype(np.float64), v.astype(np.float64))
+    codes, meta = case.oracle.encode_values_int2(v.astype(np.float64))
+    want_v = cache_format.pack_int2(codes)
+    got_k = np.empty_like(enc["kidx"]); got_v = np.empty_like(want_v)
+    got_s = np.empty_like(enc["kscale"]); got_m = np.empty_like(meta)
+    for t in range(n):
+        kk, vv = cache.load_logical(int(tok_seq[t]), int(tok_pos[t]), 1)
+        got_k[t], got_v[t] = kk[0], vv[0]
+        got_s[t] = cache.load_scales(int(tok_seq[t]), int(tok_pos[t]), 1)[0]
+        got_m[t] = cache.load_value_meta(int(tok_seq[t]), int(tok_pos[t]), 1)[0]
+    assert np.array_equal(got_s, enc["kscale"])
+    assert np.array_equal(got_m, meta), f"{int((got_m != meta).sum())} value (scale, zero) entries differ"
+    assert np.array_equal(got_v, want_v), f"{int((got_v != want_v).sum())} value bytes differ of {want_v.size}"
+    check_indices(got_k, enc, "k")
+
+
+@pytest.mark.parametrize("name,lens", [("qwen_scaled", [1, 63, 64, 65, 1000, 0, 3001]), ("gptoss_scaled", [2048, 77, 640])])
+def test_deployed_decode_matches_oracle(name, lens, request):
+    from paper_2608_04074_b200 import cache_format
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = request.getfixturevalue(name)
+    lens = np.array(lens, np.int32)
+    cache = PagedCache(case.ctx, lens, seed=3, int2_values=True)
+    encs = []
+    for b, n in enumerate(lens):
+        if n == 0:
+            encs.append(None)
+            continue
+        k, v, _ = case.draw(1400 + b, int(n), 1)
+        v = synth.to_bf16_representable(v * (2.0 ** synth.rng(18 + b).integers(-2, 3, size=(int(n), 1, 1))) - 0.5)
+        e = case.oracle.encode_scaled(k.astype(np.float64), v.astype(np.float64), with_gaps=False)
+        codes, meta = case.oracle.encode_values_int2(v.astype(np.float64))
+        cache.store_logical(b, 0, e["kidx"], cache_format.pack_int2(codes))
+        cache.store_scales(b, 0, e["kscale"])
+        cache.store_value_meta(b, 0, meta)
+        encs.append((e, codes, meta))
+    _, _, q = case.draw(1401, 1, len(lens))
+    sink = np.linspace(-4.0, 4.0, case.ctx.n_q_heads).astype(np.float32)
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    out_sink = cache.decode(0, _dev(q, torch.bfloat16), sink_logits=_dev(sink)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    worst = 0.0
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert not out[b].any() and not out_sink[b].any()
+            continue
+        e, codes, meta = encs[b]
+        ref = case.oracle.decode_deployed(q[b].astype(np.float64), e["kidx"], e["kscale"], codes, meta)
+        worst = max(worst, check_output(out[b], ref))
+        ref_s = case.oracle.decode_deployed(q[b].astype(np.float64), e["kidx"], e["kscale"], codes, meta,
+                                            sink=sink.astype(np.float64))
+        worst = max(worst, check_output(out_sink[b], ref_s))
+    print(f"[{name} {lens.tolist()}] deployed format: max|delta|/||o||inf = {worst:.3e}")
+
+
+def test_deployed_banded_end_to_end(qwen_scaled):
+    """The whole deployed format: scaled keys, INT2 values, BF16 band with deferred quantisation, sink logit."""
+    from paper_2608_04074_b200.runtime import BandedCache
+    case = qwen_scaled
+    lens = np.array([600, 90, 330], np.int32)
+    steps = 17
+    cache = BandedCache(case.ctx, 3, 700, n_sink=64, n_rec=256, block=8, seed=14, int2_values=True)
+    ks, vs = [], []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(1500 + b, int(n) + steps, 1)
+        ks.append(k); vs.append(v)
+        cache.prefill(0, b, _dev(k[:n], torch.bfloat16), _dev(v[:n], torch.bfloat16))
+    for t in range(steps):
+        cache.append_step(0, _dev(np.stack([ks[b][lens[b] + t] for b in range(3)]), torch.bfloat16),
+                          _dev(np.stack([vs[b][lens[b] + t] for b in range(3)]), torch.bfloat16))
+    _, _, q = case.draw(1501, 1, 3)
+    sink = np.linspace(-1.0, 5.0, case.ctx.n_q_heads).astype(np.float32)
+    out = cache.decode(0, _dev(q, torch.bfloat16), sink_logits=_dev(sink)).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    for b in range(3):
+        k, v = ks[b].astype(np.float64), vs[b].astype(np.float64)
+        e = case.oracle.encode_scaled(k, v, with_gaps=False)
+        codes, meta = case.oracle.encode_values_int2(v)
+        ref = case.oracle.decode_deployed(q[b].astype(np.float64), e["kidx"], e["kscale"], codes, meta, k_exact=k,
+                                          v_exact=v, band_mask=cache.band_mask(b), sink=sink.astype(np.float64))
+        check_output(out[b], ref)
