@@ -1021,10 +1021,11 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     ctx->launches++;
 
     auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC, VSQ>;
-    static bool smem_opt_in = false;      // per template instantiation; the attribute is sticky
-    if (!smem_opt_in) {
+    // the opt-in is per device and per kernel instantiation: remembered in the context (one device each)
+    constexpr unsigned inst_bit = 1u << ((VM ? 1 : 0) + (KSC ? 2 : 0) + (VSQ ? 4 : 0));
+    if (!(ctx->smem_opt_in & inst_bit)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
-        smem_opt_in = true;
+        ctx->smem_opt_in |= inst_bit;
     }
     const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
     {
