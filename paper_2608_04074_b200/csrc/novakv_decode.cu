@@ -258,27 +258,20 @@ __device__ __forceinline__ uint2 ldg_stream_64(const void* p) {
     return v;
 }
 
-// Segment prologue pieces, kept out of line so that their register-hungry load batches do not
-// disturb the register allocation of the scan loop.
-// 64 KB image (value codebook of a KV head, or one plane of its key codebook) -> shared memory.
-__device__ __noinline__ void stage_image_64k(unsigned char* dst_smem, const void* __restrict__ src_g) {
-    const uint4* src = reinterpret_cast<const uint4*>(src_g);
-    uint4* dst = reinterpret_cast<uint4*>(dst_smem);
-    // all loads of a thread in flight before the first store (one L2 latency for the whole copy)
-    constexpr int NV4 = (VCB_BYTES / 16 + S1_THREADS - 1) / S1_THREADS;
-    uint4 tmp[NV4];
-#pragma unroll
-    for (int k = 0; k < NV4; ++k) {
-        const int i = threadIdx.x + k * S1_THREADS;
-        if (i < VCB_BYTES / 16) tmp[k] = src[i];
-    }
-#pragma unroll
-    for (int k = 0; k < NV4; ++k) {
-        const int i = threadIdx.x + k * S1_THREADS;
-        if (i < VCB_BYTES / 16) dst[i] = tmp[k];
-    }
+// 64 KB image (the value codebook of a KV head) -> shared memory, without registers: asynchronous 16-byte
+// copies that land while the caller does other work (segment lookup, page ids, table build);
+// async_copies_wait() before the barrier that publishes the image.
+__device__ __forceinline__ void stage_image_64k_async(unsigned char* dst_smem, const void* __restrict__ src_g) {
+    const uint32_t dst = smem_u32(dst_smem);
+    const char* src = reinterpret_cast<const char*>(src_g);
+    for (int i = threadIdx.x; i < VCB_BYTES / 16; i += S1_THREADS)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * 16), "l"(src + (size_t)i * 16) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
 }
+__device__ __forceinline__ void async_copies_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
+// The table build is kept out of line so that its register-hungry load batch does not disturb the
+// register allocation of the scan loop.
 // LUT[hs][plane][code][e] = <q'_h segment of group l(e, plane), key codeword> for 4 heads per entry.
 template <int D, int HG, bool VM>
 __device__ __noinline__ void build_score_table(unsigned char* smem,
@@ -365,6 +358,11 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     constexpr int TILE_BYTES = C::TILE_BYTES, PAGE_BYTES = 2 * TILE_BYTES;
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_found[4];
+    // With the KV-head-major walk the first KV head of CTA c is floor(c * Hkv / G) whatever the lengths are:
+    // its (constant) value codebook starts flowing into shared memory before the grid-dependency wait and
+    // lands behind the segment lookup and the first table build.
+    int vcb_head = (int)(((long)blockIdx.x * n_kv_heads) / gridDim.x);   // KV head whose value codebook is resident
+    stage_image_64k_async(smem + C::OFF_VCB, cb_v_img + (size_t)vcb_head * (VCB_BYTES / 2));
     novakv_grid_dependency_wait();
     const uint32_t s_base = smem_u32(smem);
     const uint32_t s_lut = s_base + C::OFF_LUT, s_vcb = s_base + C::OFF_VCB, s_p = s_base + C::OFF_P;
@@ -372,7 +370,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long U = (long)page_prefix[batch] * n_kv_heads;
     const long u_begin = ((long)blockIdx.x * U) / gridDim.x, u_end = ((long)(blockIdx.x + 1) * U) / gridDim.x;
-    if (u_begin >= u_end) return;
+    if (u_begin >= u_end) { async_copies_wait(); return; }
 
     // per-warp running state
     float m_run[HPAD], l_run[HPAD];
@@ -405,7 +403,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     for (int x = 0; x < NGB; ++x) pos8[x] = (16 * (fr >> 2) + 4 * ((x + fc) & 3) + (fr & 3)) * 8;
     const uint32_t s_pw = s_p + warp * C::P_WARP_BYTES;
 
-    int vcb_head = -1;       // KV head whose value codebook is resident
     long u = u_begin;
     while (u < u_end) {
         const Segment sg = locate(page_prefix, seq_lens, batch, max_pages_per_seq, u, u_end, s_found);
@@ -413,7 +410,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
         // ---- segment prologue -----------------------------------------------------------------
         if (vcb_head != sg.kvh) {
-            stage_image_64k(smem + C::OFF_VCB, cb_v_img + (size_t)sg.kvh * (VCB_BYTES / 2));
+            stage_image_64k_async(smem + C::OFF_VCB, cb_v_img + (size_t)sg.kvh * (VCB_BYTES / 2));
             vcb_head = sg.kvh;
         }
 
@@ -468,6 +465,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         if (n_it > 0) load_tile(0, nxt);
         build_score_table<D, HG, VM>(smem, cb_k_lut + (size_t)sg.kvh * C::PLANES * (LUT_PLANE_BYTES / 4),
                                      qp + ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D);
+        async_copies_wait();
         __syncthreads();     // table and value codebook complete
 
         // ---- scan: 32-token tiles, loads of the next tile in flight while this one is consumed ------
@@ -741,7 +739,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 // ------------------------------------------------------------------------------------------------
 // MINB = resident blocks per SM the register budget allows for: 1 keeps the prefetched constants in
 // registers (lowest latency, small batches), 2 trades a few spills for occupancy (many pairs).
-template <int D, int HG, int MINB>
+// EXT = the call carries a learned sink logit and/or a BF16 band partial; without it that code is compiled out.
+template <int D, int HG, int MINB, bool EXT>
 __global__ void __launch_bounds__(HG * D > 512 ? 512 : HG * D, MINB)
 novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __restrict__ part_acc,
                            const int32_t* __restrict__ page_prefix, const int32_t* __restrict__ seq_lens,
@@ -798,7 +797,7 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         float lq = lsum;          // mass of the quantised tokens at the running scale
         float wb = 0.f;           // weight of the band accumulator at the running scale
         const int hq = kvh * HG + h;
-        if (band_ml != nullptr) {
+        if (EXT && band_ml != nullptr) {
             // BF16 sink-plus-recent band: one more partial, accumulated in the original value domain
             const float mb = band_ml[((size_t)b * n_q_heads + hq) * 2], lb = band_ml[((size_t)b * n_q_heads + hq) * 2 + 1];
             const float M2 = fmaxf(M, mb);
@@ -809,7 +808,7 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
             lsum = fmaf(lb, wb, lq);
             M = M2;
         }
-        if (sink_logits != nullptr) {
+        if (EXT && sink_logits != nullptr) {
             // learned sink: an extra logit in the normaliser, added exactly once, after the cross-split
             // combine; it is shifted by the per-query constant the token logits dropped (q . k_mean)
             const float s2 = sink_logits[hq] * 1.4426950408889634f - qk_off[(size_t)b * n_q_heads + hq];
@@ -821,8 +820,11 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
             lsum = fmaf(lsum, w, ex2(s2 - M2));
         }
         float val = 0.f, frac = 0.f, bsc = 0.f;
-        if (lsum > 0.f) { val = a / lsum; frac = lq / lsum; bsc = wb / lsum; }
-        if (c == 0) { frac_s[h] = frac; bsc_s[h] = bsc; }
+        if (lsum > 0.f) {
+            val = a / lsum;
+            if (EXT) { frac = lq / lsum; bsc = wb / lsum; }
+        }
+        if (EXT && c == 0) { frac_s[h] = frac; bsc_s[h] = bsc; }
         o_s[i] = val;
     }
     __syncthreads();
@@ -851,9 +853,11 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         float o = 0.f;
 #pragma unroll
         for (int p = 0; p < PARTS; ++p) o += red_s[p][h][r];
-        o = fmaf(vm[k], frac_s[h], o);              // sum_j p_j (s^_j R_V^T + v_mean): the mean carries the quantised-token mass
+        // sum_j p_j (s^_j R_V^T + v_mean): the mean carries the quantised-token mass (all of it without sink and band)
+        if (EXT) o = fmaf(vm[k], frac_s[h], o);
+        else if (pages_b > 0) o += vm[k];
         const size_t oi = ((size_t)b * n_q_heads + kvh * HG + h) * D + r;
-        if (band_acc != nullptr) o = fmaf(band_acc[oi], bsc_s[h], o);
+        if (EXT && band_acc != nullptr) o = fmaf(band_acc[oi], bsc_s[h], o);
         if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
         else reinterpret_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
     }
@@ -1042,7 +1046,10 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                           band_acc);
         ctx->launches++;
     }
-    auto merge = batch * hkv > 2 * ctx->n_sm ? novakv_decode_merge_kernel<D, HG, 2> : novakv_decode_merge_kernel<D, HG, 1>;
+    const bool ext = sink_logits != nullptr || band != nullptr;
+    auto merge = batch * hkv > 2 * ctx->n_sm
+                     ? (ext ? novakv_decode_merge_kernel<D, HG, 2, true> : novakv_decode_merge_kernel<D, HG, 2, false>)
+                     : (ext ? novakv_decode_merge_kernel<D, HG, 1, true> : novakv_decode_merge_kernel<D, HG, 1, false>);
     novakv_launch_pdl(merge, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
                       part_ml, part_acc, prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out,
                       out_is_fp32, sink_logits, qk_off, (const float*)band_ml, (const float*)band_acc);
