@@ -117,7 +117,9 @@ size_t novakv_decode_workspace_bytes(const novakv_ctx* ctx, int batch);
 
 /*
  * Write path (Algorithm 1 line 7; Sec. 4 "Complexity"): for each new token t and KV head,
- *     r = (k_t - k_mean) rk,   s = (v_t - v_mean) rv          accumulated in binary64,
+ *     r = (k_t - k_mean) rk,   s = (v_t - v_mean) rv          exact products accumulated in binary64
+ * (in index order for append-sized batches, in blocks of four input dimensions on the fp64 tensor path
+ * for larger ones: the two differ by less than an ulp of binary64 before the rounding that follows),
  * each coefficient rounded once to binary32, then for every group l the index of the nearest
  * codeword (exact Euclidean search, App. B "Calibration").  The squared distance is evaluated
  * in binary32 as fma(e3,e3, fma(e2,e2, fma(e1,e1, e0*e0))), e_i = coef_i - codeword_i, visiting
