@@ -70,6 +70,16 @@ def bits_per_element(head_dim: int, key_scale_bits: int = 0, value_meta_bits: in
     return (8 * l + key_scale_bits) / head_dim, (8 * l + value_meta_bits) / head_dim
 
 
+def deployed_bits_per_element(context_tokens: int, head_dim: int = 128, n_sink: int = 64, n_rec: int = 256) -> float:
+    """Average cache rate of the deployed format over keys and values at a given context length
+    (Sec. 5 "Bit rate"): scaled 2-bit keys and INT2 values with their per-token metadata, and the
+    n_sink + n_rec band tokens at 16 bits per element."""
+    kb, vb = bits_per_element(head_dim, key_scale_bits=16, value_meta_bits=32)
+    quant = 0.5 * (kb + vb)
+    band = min(context_tokens, n_sink + n_rec)
+    return quant + band * (16.0 - quant) / context_tokens
+
+
 def table_scalars(head_dim: int, with_value_codebooks: bool = False) -> int:
     """Scalars stored once per (layer, KV head): 3 d^2 + d + L * 256 * g (+ value codebooks)."""
     l = n_groups(head_dim)

@@ -485,6 +485,13 @@ def test_scaled_key_rate_matches_paper_arithmetic():
     assert kb == gold["bpe_keys_deployed"] and vb == gold["bpe_values_deployed"]
     assert (kb + vb) / 2 == gold["bpe_mean_deployed"]
     assert cache_format.bits_per_element(128, key_scale_bits=16)[0] - cache_format.bits_per_element(128)[0] == 16 / 128
+    # the band's share at 128K context and the total, to the digits the paper prints
+    total = cache_format.deployed_bits_per_element(128 * 1024)
+    assert round(total - gold["bpe_mean_deployed"], 3) == gold["bpe_band_extra_128k"]
+    assert round(total, 2) == gold["bpe_total_deployed_128k"]
+    # the band's share vanishes as the context grows and is everything for a context inside the band
+    assert cache_format.deployed_bits_per_element(320) == 16.0
+    assert cache_format.deployed_bits_per_element(10 ** 9) - gold["bpe_mean_deployed"] < 1e-5
 
 
 # ---- learned attention sink (App. "Attention sinks in the quantized serving path") ----
