@@ -824,3 +824,21 @@ def test_deployed_banded_end_to_end(qwen_scaled):
         ref = case.oracle.decode_deployed(q[b].astype(np.float64), e["kidx"], e["kscale"], codes, meta, k_exact=k,
                                           v_exact=v, band_mask=cache.band_mask(b), sink=sink.astype(np.float64))
         check_output(out[b], ref)
+
+
+# --------------------------------------------------------------------------- extreme softmax temperatures
+@pytest.mark.parametrize("factor", [16.0, 1e-3])
+def test_near_one_hot_and_near_uniform_attention(qwen, factor):
+    """Logits scaled by 16 (attention close to one-hot: the running maximum changes abruptly and most
+    weights underflow) and by 1e-3 (close to uniform: the output is the mean of the values)."""
+    case = qwen
+    lens = np.array([1500, 129], np.int32)
+    cache = _cache(case, lens, seed=15)
+    encs = _fill_with_oracle(case, cache, lens, 1600)
+    _, _, q = case.draw(1601, 1, 2)
+    scale = factor / np.sqrt(case.ctx.head_dim)
+    out = cache.decode(0, _dev(q, torch.bfloat16), sm_scale=scale).cpu().numpy()
+    assert case.ctx.novakv_last_device_status() == 0
+    for b in range(2):
+        ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], sm_scale=scale)
+        check_output(out[b], ref)
