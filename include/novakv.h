@@ -352,6 +352,15 @@ novakv_status novakv_debug_set_scan_ctas(novakv_ctx* ctx, int n_ctas);
  */
 novakv_status novakv_debug_set_value_path(novakv_ctx* ctx, int path);
 
+/*
+ * Work split of the index scan.  The scan kernel walks all (sequence, KV head) pairs page by page and
+ * cuts the walk into one contiguous piece per CTA.  Each pair a CTA touches costs it a fixed set-up (the
+ * per-query score table), so the cut is even not in pages but in pages + `pages` per pair touched: a CTA
+ * that has to set up several pairs gets fewer pages.  `pages` = 0 gives the even split in pages; the
+ * default is 24.  Results do not depend on it beyond binary32 rounding (it only moves split points).
+ */
+novakv_status novakv_debug_set_segment_weight(novakv_ctx* ctx, int pages);
+
 /* Kernels this library launched since the context was created (all kinds). */
 long novakv_launch_count(const novakv_ctx* ctx);
 

@@ -564,6 +564,12 @@ extern "C" novakv_status novakv_debug_set_scan_ctas(novakv_ctx* ctx, int n_ctas)
     return NOVAKV_OK;
 }
 
+extern "C" novakv_status novakv_debug_set_segment_weight(novakv_ctx* ctx, int pages) {
+    if (!ctx || pages < 0 || pages > 4096) return NOVAKV_EINVAL;
+    ctx->seg_weight = pages;
+    return NOVAKV_OK;
+}
+
 extern "C" novakv_status novakv_debug_set_value_path(novakv_ctx* ctx, int path) {
     if (!ctx || (path != 0 && path != 1)) return NOVAKV_EINVAL;
     ctx->value_path = path;

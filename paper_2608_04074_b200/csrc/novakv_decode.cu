@@ -88,7 +88,8 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                       const int32_t* __restrict__ seq_lens, int batch, int n_q_heads, int n_kv_heads,
                       int max_pages_per_seq, float scale_log2, float* __restrict__ qp,
                       int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status,
-                      const float* __restrict__ k_mean /* [Hkv][D] */, float* __restrict__ qk_off /* [batch][Hq] or null */) {
+                      const float* __restrict__ k_mean /* [Hkv][D] */, float* __restrict__ qk_off /* [batch][Hq] or null */,
+                      int32_t* __restrict__ cost_prefix /* [batch + 1] */, int seg_weight) {
     const int blk = blockIdx.x;
     constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
@@ -103,9 +104,12 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
     }
     novakv_grid_dependency_wait();
     if (blk == batch * n_kv_heads) {
-        // exclusive prefix over sequences of their page counts; small, done by one warp
+        // exclusive prefix over sequences of their page counts; small, done by one warp.  Beside it the same
+        // prefix in "cost" units, in which every non-empty sequence weighs seg_weight pages more: the scan
+        // kernel splits the walk evenly in cost, so that a CTA that has to set up several (sequence, KV head)
+        // segments gets fewer pages.
         if (threadIdx.x < 32) {
-            int carry = 0;
+            int carry = 0, carry_ne = 0;
             for (int b0 = 0; b0 < batch; b0 += 32) {
                 const int b = b0 + threadIdx.x;
                 int v = 0;
@@ -115,16 +119,22 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                     if (raw != len) atomicOr(dev_status, NOVAKV_DEV_BAD_LENGTH);
                     v = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
                 }
-                int incl = v;
+                const int ne = v > 0 ? 1 : 0;
+                int incl = v, incl_ne = ne;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const int t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if ((int)threadIdx.x >= o) incl += t;
+                    const int tn = __shfl_up_sync(0xffffffffu, incl_ne, o);
+                    if ((int)threadIdx.x >= o) { incl += t; incl_ne += tn; }
                 }
-                if (b < batch) page_prefix[b] = carry + incl - v;
+                if (b < batch) {
+                    page_prefix[b] = carry + incl - v;
+                    cost_prefix[b] = carry + incl - v + seg_weight * (carry_ne + incl_ne - ne);
+                }
                 carry += __shfl_sync(0xffffffffu, incl, 31);
+                carry_ne += __shfl_sync(0xffffffffu, incl_ne, 31);
             }
-            if (threadIdx.x == 0) page_prefix[batch] = carry;
+            if (threadIdx.x == 0) { page_prefix[batch] = carry; cost_prefix[batch] = carry + seg_weight * carry_ne; }
         }
         return;
     }
@@ -350,7 +360,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                             const int32_t* __restrict__ page_table, int max_pages_per_seq,
                             const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ page_prefix,
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
-                            float* __restrict__ part_acc, uint32_t* __restrict__ dev_status, int pt_stride) {
+                            float* __restrict__ part_acc, uint32_t* __restrict__ dev_status, int pt_stride,
+                            const int32_t* __restrict__ cost_prefix, int seg_weight, long* __restrict__ cta_range) {
     // page_table points at the first column that is scanned; rows are pt_stride entries apart and
     // max_pages_per_seq bounds the pages of a row that may be read from there
     using C = S1<D, HG, VM>;
@@ -368,8 +379,38 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     const uint32_t s_lut = s_base + C::OFF_LUT, s_vcb = s_base + C::OFF_VCB, s_p = s_base + C::OFF_P;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long U = (long)page_prefix[batch] * n_kv_heads;
-    const long u_begin = ((long)blockIdx.x * U) / gridDim.x, u_end = ((long)(blockIdx.x + 1) * U) / gridDim.x;
+    // This CTA's range of the walk [u_begin, u_end).  The walk is cut evenly in cost units, cost = pages +
+    // seg_weight per (sequence, KV head) pair: cost point t lies in the pair whose cost interval contains it
+    // and maps to unit  start + clamp(t - cost_start - seg_weight, 0, pages)  (the first seg_weight cost units
+    // of a pair stand for setting up its score table).  seg_weight = 0 is the even split in pages.
+    long u_begin, u_end;
+    {
+        const long P = page_prefix[batch], U = P * n_kv_heads;
+        if (seg_weight == 0) {
+            u_begin = ((long)blockIdx.x * U) / gridDim.x;
+            u_end = ((long)(blockIdx.x + 1) * U) / gridDim.x;
+        } else {
+            const long cper = cost_prefix[batch], T = cper * n_kv_heads;
+            const long t0 = ((long)blockIdx.x * T) / gridDim.x, t1 = ((long)(blockIdx.x + 1) * T) / gridDim.x;
+            __shared__ long s_bnd[2];
+            if (threadIdx.x < 2) s_bnd[threadIdx.x] = U;              // a cost point at the very end
+            __syncthreads();
+            if (cper > 0) {
+                const long kv0 = t0 / cper, kv1 = t1 / cper;
+                const long rem0 = t0 - kv0 * cper, rem1 = t1 - kv1 * cper;
+                for (int t = threadIdx.x; t < batch; t += S1_THREADS) {
+                    const long lo = cost_prefix[t], hi = cost_prefix[t + 1];
+                    const long p0 = page_prefix[t], pg = page_prefix[t + 1] - p0;
+                    if (t0 < T && lo <= rem0 && rem0 < hi) s_bnd[0] = kv0 * P + p0 + min(max(rem0 - lo - seg_weight, 0l), pg);
+                    if (t1 < T && lo <= rem1 && rem1 < hi) s_bnd[1] = kv1 * P + p0 + min(max(rem1 - lo - seg_weight, 0l), pg);
+                }
+            }
+            __syncthreads();
+            u_begin = s_bnd[0];
+            u_end = s_bnd[1];
+        }
+        if (threadIdx.x == 0) { cta_range[blockIdx.x * 2] = u_begin; cta_range[blockIdx.x * 2 + 1] = u_end; }
+    }
     if (u_begin >= u_end) { async_copies_wait(); return; }
 
     // per-warp running state
@@ -750,7 +791,8 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
                            const float* __restrict__ sink_logits /* [Hq] natural-log units, or null */,
                            const float* __restrict__ qk_off /* [batch][Hq], base-2 units */,
                            const float* __restrict__ band_ml /* [batch][Hq][2] (max, sum) of the BF16 band, or null */,
-                           const float* __restrict__ band_acc /* [batch][Hq][D] sum p v of the band, original value domain */) {
+                           const float* __restrict__ band_acc /* [batch][Hq][D] sum p v of the band, original value domain */,
+                           const int32_t* __restrict__ cost_prefix, int seg_weight, const long* __restrict__ cta_range) {
     __shared__ float o_s[HG * D];
     __shared__ float frac_s[HG];      // share of the softmax mass on quantised tokens (1 without sink and band)
     __shared__ float bsc_s[HG];       // multiplier of the band accumulator (0 without a band)
@@ -772,22 +814,28 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
     novakv_grid_dependency_wait();
     const int len = clamp_len(seq_lens[b], max_pages_per_seq);
     const int pages_b = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
-    const long P = page_prefix[batch], U = P * n_kv_heads;
+    const long P = page_prefix[batch];
     const int slot0 = kvh * batch + b;                     // the scan kernel's pair index (walk order)
     for (int i = threadIdx.x; i < HG * D; i += blockDim.x) {
         const int h = i / D, c = i - h * D;
         float M = M_INIT, a = 0.f, lsum = 0.f;
         if (pages_b > 0) {
             const long u0 = (long)kvh * P + page_prefix[b], u1 = u0 + pages_b;
-            // CTA of unit u: the largest c with floor(c*U/G) <= u
-            const int c_first = (int)(((u0 + 1) * grid_s1 - 1) / U), c_last = (int)((u1 * grid_s1 - 1) / U);
-            // CTAs in between whose own range is empty wrote nothing: skip them
+            // CTAs that may hold a piece of this pair: those whose cost range meets the pair's (the largest c
+            // with floor(c*T/G) <= x for its first and last cost unit), widened by one on each side; the
+            // ranges the scan CTAs recorded decide
+            const long T = (long)cost_prefix[batch] * n_kv_heads;
+            const long x0 = (long)kvh * cost_prefix[batch] + cost_prefix[b] + seg_weight, x1 = x0 + pages_b - 1;
+            const int c_first = max((int)(((x0 + 1) * grid_s1 - 1) / T) - 1, 0);
+            const int c_last = min((int)(((x1 + 1) * grid_s1 - 1) / T) + 1, grid_s1 - 1);
             for (int cta = c_first; cta <= c_last; ++cta) {
-                if (((long)cta * U) / grid_s1 >= ((long)(cta + 1) * U) / grid_s1) continue;
+                const long r0 = cta_range[cta * 2], r1 = cta_range[cta * 2 + 1];
+                if (r0 >= r1 || r1 <= u0 || r0 >= u1) continue;
                 M = fmaxf(M, part_ml[(((size_t)slot0 + cta) * HG + h) * 2]);
             }
             for (int cta = c_first; cta <= c_last; ++cta) {
-                if (((long)cta * U) / grid_s1 >= ((long)(cta + 1) * U) / grid_s1) continue;
+                const long r0 = cta_range[cta * 2], r1 = cta_range[cta * 2 + 1];
+                if (r0 >= r1 || r1 <= u0 || r0 >= u1) continue;
                 const size_t pidx = (size_t)slot0 + cta;
                 const float sc = ex2(part_ml[(pidx * HG + h) * 2] - M);
                 a = fmaf(sc, part_acc[(pidx * HG + h) * D + c], a);
@@ -974,7 +1022,7 @@ novakv_band_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 
 // workspace layout
 struct WsLayout {
-    size_t qp, prefix, qk, bml, bacc, ml, acc, total;
+    size_t qp, prefix, cost, range, qk, bml, bacc, ml, acc, total;
 };
 WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -983,7 +1031,9 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     WsLayout w;
     w.qp = 0;
     w.prefix = al(w.qp + (size_t)batch * hq * d * 4);
-    w.qk = al(w.prefix + ((size_t)batch + 1) * 4);
+    w.cost = al(w.prefix + ((size_t)batch + 1) * 4);
+    w.range = al(w.cost + ((size_t)batch + 1) * 4);
+    w.qk = al(w.range + (size_t)ctx->n_sm * 2 * sizeof(long));
     w.bml = al(w.qk + (size_t)batch * hq * 4);
     w.bacc = al(w.bml + (size_t)batch * hq * 2 * 4);
     w.ml = al(w.bacc + (size_t)batch * hq * d * 4);
@@ -1012,6 +1062,8 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     char* ws = (char*)workspace;
     float* qp = (float*)(ws + w.qp);
     int32_t* prefix = (int32_t*)(ws + w.prefix);
+    int32_t* cost_prefix = (int32_t*)(ws + w.cost);
+    long* cta_range = (long*)(ws + w.range);
     float* qk_off = sink_logits ? (float*)(ws + w.qk) : nullptr;
     float* band_ml = band ? (float*)(ws + w.bml) : nullptr;
     float* band_acc = band ? (float*)(ws + w.bacc) : nullptr;
@@ -1021,7 +1073,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
 
     novakv_launch_pdl(novakv_prepare_kernel<D, HG>, dim3(batch * hkv + 1), dim3(512), 0, stream, q, ly.rk_inv_t, seq_lens,
                       batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status,
-                      ly.k_mean, qk_off);
+                      ly.k_mean, qk_off, cost_prefix, ctx->seg_weight);
     ctx->launches++;
 
     auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC, VSQ>;
@@ -1036,7 +1088,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         novakv_prof_scope ps(ctx, 0, stream);
         novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut,
                           VSQ ? (const __half*)ctx->int2_img : (const __half*)ly.cb_v_mma, k_pages, v_pages, k_scales, v_meta, n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
-                          ctx->dev_status, pt_stride);
+                          ctx->dev_status, pt_stride, (const int32_t*)cost_prefix, ctx->seg_weight, cta_range);
         ps.end();
         ctx->launches++;
     }
@@ -1052,7 +1104,8 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                      : (ext ? novakv_decode_merge_kernel<D, HG, 1, true> : novakv_decode_merge_kernel<D, HG, 1, false>);
     novakv_launch_pdl(merge, dim3(batch * hkv), dim3(HG * D > 512 ? 512 : HG * D), 0, stream,
                       part_ml, part_acc, prefix, seq_lens, batch, hq, hkv, max_pages_per_seq, grid, ly.rv_t, ly.v_mean, out,
-                      out_is_fp32, sink_logits, qk_off, (const float*)band_ml, (const float*)band_acc);
+                      out_is_fp32, sink_logits, qk_off, (const float*)band_ml, (const float*)band_acc,
+                      (const int32_t*)cost_prefix, ctx->seg_weight, (const long*)cta_range);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
 }

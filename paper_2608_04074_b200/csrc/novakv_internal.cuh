@@ -51,6 +51,7 @@ struct novakv_ctx {
     long launches = 0;
     int scan_ctas = 0;            // 0 = one per SM
     int value_path = 1;           // 1 = tensor cores, 0 = CUDA cores
+    int seg_weight = 24;          // pages one (sequence, KV head) segment weighs extra in the scan kernel's work split
     unsigned smem_opt_in = 0;     // scan-kernel instantiations whose shared-memory opt-in was set on this device
 };
 

@@ -842,3 +842,32 @@ def test_near_one_hot_and_near_uniform_attention(qwen, factor):
     for b in range(2):
         ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"], sm_scale=scale)
         check_output(out[b], ref)
+
+
+# --------------------------------------------------------------------------- work split of the scan
+@pytest.mark.parametrize("weight", [0, 1, 24, 200, 4096])
+def test_segment_weight_moves_split_points_only(qwen, weight):
+    """The cost-weighted split (0 = even in pages; large values push whole pairs to single CTAs) must give
+    the same attention output: ragged lengths, empty sequences, pairs much shorter than the weight."""
+    case = qwen
+    lens = np.array([3001, 0, 64, 1, 777, 130, 0, 2000, 65], np.int32)
+    cache = _cache(case, lens, seed=16)
+    encs = _fill_with_oracle(case, cache, lens, 1700)
+    _, _, q = case.draw(1701, 1, len(lens))
+    case.ctx.novakv_debug_set_segment_weight(weight)
+    try:
+        outs = []
+        for ctas in (0, 5):
+            case.ctx.novakv_debug_set_scan_ctas(ctas)
+            outs.append(cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy())
+        assert case.ctx.novakv_last_device_status() == 0
+    finally:
+        case.ctx.novakv_debug_set_segment_weight(24)
+        case.ctx.novakv_debug_set_scan_ctas(0)
+    for b, n in enumerate(lens):
+        for out in outs:
+            if n == 0:
+                assert not out[b].any()
+                continue
+            ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
+            check_output(out[b], ref)
