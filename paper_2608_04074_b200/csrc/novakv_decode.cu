@@ -52,7 +52,7 @@ struct S1 {
     static constexpr int LUT_BYTES = HSETS * PLANES * LUT_PLANE_BYTES;
     // per-warp staging of the softmax weights of one 32-token tile
     //   VM: fp16 [HPAD][4 k-slot pairs][8 tokens]        otherwise: fp32 [32 tokens][HPAD]
-    static constexpr int P_WARP_BYTES = VM ? HPAD * 64 : 32 * HPAD * 4;
+    static constexpr int P_WARP_BYTES = VM ? HPAD * 128 : 32 * HPAD * 4;   // VM: two fp16 arrays (weights, and their residuals for the INT2 value codec)
     static constexpr int P_BYTES = NCW * P_WARP_BYTES;
     static constexpr int OFF_LUT = 0;
     static constexpr int OFF_VCB = OFF_LUT + LUT_BYTES;
@@ -553,6 +553,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             bool rescale = false;
             float alpha[HPAD];
             __half ph[HPAD];
+            __half pl[VSQ ? HPAD : 1];
 #pragma unroll
             for (int h = 0; h < HPAD; ++h) {
                 if (lane >= nvalid) zf[h] = -CUDART_INF_F;
@@ -572,7 +573,11 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 if (VSQ) {
                     const float vscale = __uint_as_float(cur.vm << 16), vzero = __uint_as_float(cur.vm & 0xffff0000u);
                     lz_run[h] = fmaf(lz_run[h], alpha[h], lane < nvalid ? zf[h] * vzero : 0.f);
-                    ph[h] = __float2half_rn(zf[h] * vscale);      // the weight of the token's integer codes
+                    // the weight of the token's integer codes, p * scale, as a binary16 pair (value + residual):
+                    // a single binary16 rounding here would not cancel against the normaliser as it does for p
+                    const float wv = zf[h] * vscale;
+                    ph[h] = __float2half_rn(wv);
+                    pl[h] = __float2half_rn(wv - __half2float(ph[h]));
                 }
             }
 
@@ -602,12 +607,22 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 #pragma unroll
                     for (int h = 0; h < HPAD; ++h)
                         asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + h * 64), "h"(__half_as_ushort(ph[h])) : "memory");
+                    if (VSQ) {
+#pragma unroll
+                        for (int h = 0; h < HPAD; ++h)
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + (HPAD + h) * 64), "h"(__half_as_ushort(pl[VSQ ? h : 0])) : "memory");
+                    }
                 }
                 __syncwarp();
                 // B-fragment sources: 8 weights of head (4 hs + fr/2) for the tokens with (token & 3) == fc
                 uint4 pw[HSETS];
 #pragma unroll
                 for (int hs = 0; hs < HSETS; ++hs) pw[hs] = lds_u128(s_pw + (hs * 4 + (fr >> 1)) * 64 + fc * 16);
+                uint4 pwl[VSQ ? HSETS : 1];
+                if (VSQ) {
+#pragma unroll
+                    for (int hs = 0; hs < HSETS; ++hs) pwl[hs] = lds_u128(s_pw + (HPAD + hs * 4 + (fr >> 1)) * 64 + fc * 16);
+                }
 #pragma unroll
                 for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
@@ -657,6 +672,17 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                                     "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                                     : "+f"(macc[hs][gb][0]), "+f"(macc[hs][gb][1]), "+f"(macc[hs][gb][2]), "+f"(macc[hs][gb][3])
                                     : "r"(Y[gb][0][0]), "r"(Y[gb][0][1]), "r"(Y[gb][1][0]), "r"(Y[gb][1][1]), "r"(b0), "r"(b1));
+                            }
+                            if (VSQ) {
+                                const uint32_t wl = t == 0 ? pwl[VSQ ? hs : 0].x : (t == 1 ? pwl[VSQ ? hs : 0].y : (t == 2 ? pwl[VSQ ? hs : 0].z : pwl[VSQ ? hs : 0].w));
+                                const uint32_t c0 = __byte_perm(wl, 0u, sel_b0), c1 = __byte_perm(wl, 0u, sel_b1);
+#pragma unroll
+                                for (int gb = 0; gb < NGB; ++gb) {
+                                    asm volatile(
+                                        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                        : "+f"(macc[hs][gb][0]), "+f"(macc[hs][gb][1]), "+f"(macc[hs][gb][2]), "+f"(macc[hs][gb][3])
+                                        : "r"(Y[gb][0][0]), "r"(Y[gb][0][1]), "r"(Y[gb][1][0]), "r"(Y[gb][1][1]), "r"(c0), "r"(c1));
+                                }
                             }
                         }
                     }
