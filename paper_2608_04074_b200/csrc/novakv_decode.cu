@@ -52,7 +52,7 @@ struct S1 {
     static constexpr int LUT_BYTES = HSETS * PLANES * LUT_PLANE_BYTES;
     // per-warp staging of the softmax weights of one 32-token tile
     //   VM: fp16 [HPAD][4 k-slot pairs][8 tokens]        otherwise: fp32 [32 tokens][HPAD]
-    static constexpr int P_WARP_BYTES = VM ? HPAD * 128 : 32 * HPAD * 4;   // VM: two fp16 arrays (weights, and their residuals for the INT2 value codec)
+    static constexpr int P_WARP_BYTES = VM ? HPAD * 64 : 32 * HPAD * 4;
     static constexpr int P_BYTES = NCW * P_WARP_BYTES;
     static constexpr int OFF_LUT = 0;
     static constexpr int OFF_VCB = OFF_LUT + LUT_BYTES;
@@ -553,7 +553,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             bool rescale = false;
             float alpha[HPAD];
             __half ph[HPAD];
-            __half pl[VSQ ? HPAD : 1];
 #pragma unroll
             for (int h = 0; h < HPAD; ++h) {
                 if (lane >= nvalid) zf[h] = -CUDART_INF_F;
@@ -569,16 +568,17 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     ph[h] = __float2half_rn(zf[h]);
                     zf[h] = __half2float(ph[h]);
                 }
-                l_run[h] = fmaf(l_run[h], alpha[h], zf[h]);
                 if (VSQ) {
+                    // INT2 values: the tensor-core product needs the weight of the token's integer codes,
+                    // w = p * scale, in binary16.  As for p above, the rounding must not separate numerator and
+                    // normaliser: the weight that counts is p' = fp16(p * scale) / scale, used for the
+                    // normaliser and for the zero-point sum as well (an exact softmax of perturbed logits).
                     const float vscale = __uint_as_float(cur.vm << 16), vzero = __uint_as_float(cur.vm & 0xffff0000u);
-                    lz_run[h] = fmaf(lz_run[h], alpha[h], lane < nvalid ? zf[h] * vzero : 0.f);
-                    // the weight of the token's integer codes, p * scale, as a binary16 pair (value + residual):
-                    // a single binary16 rounding here would not cancel against the normaliser as it does for p
-                    const float wv = zf[h] * vscale;
-                    ph[h] = __float2half_rn(wv);
-                    pl[h] = __float2half_rn(wv - __half2float(ph[h]));
+                    ph[h] = __float2half_rn(zf[h] * vscale);
+                    zf[h] = lane < nvalid ? __fdividef(__half2float(ph[h]), vscale) : 0.f;   // (slots beyond the length hold no metadata)
+                    lz_run[h] = fmaf(lz_run[h], alpha[h], zf[h] * vzero);
                 }
+                l_run[h] = fmaf(l_run[h], alpha[h], zf[h]);
             }
 
             if (VM) {
@@ -607,22 +607,12 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 #pragma unroll
                     for (int h = 0; h < HPAD; ++h)
                         asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + h * 64), "h"(__half_as_ushort(ph[h])) : "memory");
-                    if (VSQ) {
-#pragma unroll
-                        for (int h = 0; h < HPAD; ++h)
-                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + (HPAD + h) * 64), "h"(__half_as_ushort(pl[VSQ ? h : 0])) : "memory");
-                    }
                 }
                 __syncwarp();
                 // B-fragment sources: 8 weights of head (4 hs + fr/2) for the tokens with (token & 3) == fc
                 uint4 pw[HSETS];
 #pragma unroll
                 for (int hs = 0; hs < HSETS; ++hs) pw[hs] = lds_u128(s_pw + (hs * 4 + (fr >> 1)) * 64 + fc * 16);
-                uint4 pwl[VSQ ? HSETS : 1];
-                if (VSQ) {
-#pragma unroll
-                    for (int hs = 0; hs < HSETS; ++hs) pwl[hs] = lds_u128(s_pw + (HPAD + hs * 4 + (fr >> 1)) * 64 + fc * 16);
-                }
 #pragma unroll
                 for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
@@ -672,17 +662,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                                     "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                                     : "+f"(macc[hs][gb][0]), "+f"(macc[hs][gb][1]), "+f"(macc[hs][gb][2]), "+f"(macc[hs][gb][3])
                                     : "r"(Y[gb][0][0]), "r"(Y[gb][0][1]), "r"(Y[gb][1][0]), "r"(Y[gb][1][1]), "r"(b0), "r"(b1));
-                            }
-                            if (VSQ) {
-                                const uint32_t wl = t == 0 ? pwl[VSQ ? hs : 0].x : (t == 1 ? pwl[VSQ ? hs : 0].y : (t == 2 ? pwl[VSQ ? hs : 0].z : pwl[VSQ ? hs : 0].w));
-                                const uint32_t c0 = __byte_perm(wl, 0u, sel_b0), c1 = __byte_perm(wl, 0u, sel_b1);
-#pragma unroll
-                                for (int gb = 0; gb < NGB; ++gb) {
-                                    asm volatile(
-                                        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                        : "+f"(macc[hs][gb][0]), "+f"(macc[hs][gb][1]), "+f"(macc[hs][gb][2]), "+f"(macc[hs][gb][3])
-                                        : "r"(Y[gb][0][0]), "r"(Y[gb][0][1]), "r"(Y[gb][1][0]), "r"(Y[gb][1][1]), "r"(c0), "r"(c1));
-                                }
                             }
                         }
                     }
