@@ -119,11 +119,13 @@ size_t novakv_decode_workspace_bytes(const novakv_ctx* ctx, int batch);
  * Write path (Algorithm 1 line 7; Sec. 4 "Complexity"): for each new token t and KV head,
  *     r = (k_t - k_mean) rk,   s = (v_t - v_mean) rv          exact products accumulated in binary64
  * (in index order for append-sized batches, in blocks of four input dimensions on the fp64 tensor path
- * for larger ones: the two differ by less than an ulp of binary64 before the rounding that follows),
- * each coefficient rounded once to binary32, then for every group l the index of the nearest
- * codeword (exact Euclidean search, App. B "Calibration").  The squared distance is evaluated
- * in binary32 as fma(e3,e3, fma(e2,e2, fma(e1,e1, e0*e0))), e_i = coef_i - codeword_i, visiting
- * codewords in ascending index and keeping the first minimum (lowest index wins a tie).
+ * for larger ones: the two differ by less than an ulp of binary64), then for every group l the index of
+ * the nearest codeword: exact Euclidean search (Sec. 2.2 "Quantization", App. B "Calibration"), the
+ * lowest index winning a tie.  The stored index is the minimiser of the binary64 squared distance
+ * sum_i (coef_i - codeword_i)^2 of the binary64 coefficient.  (Large batches evaluate the 256 distances
+ * in binary32 first and keep that result only where the two smallest distances are further apart than
+ * binary32 rounding can have moved them; every other group is searched again in binary64.  The result
+ * can differ from a binary64 reference only where the two nearest codewords are within ~1e-12 relative.)
  * The 2L index bytes go to page page_table[tok_seq[t]][tok_pos[t]/64] at slot tok_pos[t]%64, and
  * seq_lens[tok_seq[t]] becomes max(seq_lens[tok_seq[t]], tok_pos[t]+1).
  *   k_new, v_new  bf16 [n_tokens][Hkv][d]

@@ -15,15 +15,14 @@
  *             accumulation used on the GPU are deliberately NOT used here.
  *   R_K^{-1} is taken from the stored synthesis matrix: R_K^{-1} = (R_K^{-T})^T.
  *
- * Precision: everything is float64, except the one place where floating point decides an
- * integer.  The library boundary fixes that decision's arithmetic (see the encode entry of
- * the public header): the float64 coefficient is rounded once to binary32 and the squared
- * distance to each codeword is evaluated in binary32 as
- *      fma(e3,e3, fma(e2,e2, fma(e1,e1, e0*e0))),   e_i = coef_i - codeword_i,
- * visiting codewords in ascending index and keeping the first minimum.  The oracle takes the
- * decision in that same precision and, beside it, reports the float64 decision and the
- * float64 relative gap (d2 - d1) / d1 between the two smallest distances, which is how
- * near-ties are counted.
+ * Precision: everything is float64.  The encoder is the paper's exact Euclidean nearest-neighbour
+ * search (Sec. 2.2 "Quantization"; App. B "Calibration"): float64 coefficients, float64 squared
+ * distances, codewords visited in ascending index, the first minimum kept (lowest index wins an
+ * exact tie).  Beside the index the oracle reports the float64 relative gap (d2 - d1) / d1 between
+ * the two smallest distances, which is how near-ties are counted.  Two stored formats define some
+ * of their bits through binary32 arithmetic (the per-token key scale and the scalar INT2 value
+ * codec, see below); there the binary32 step is part of the format's definition and is stated with
+ * the function.
  *
  * Pins (tests/test_oracle_pins.py): exact invariance of the attention products when the
  * quantiser is the identity, generalised Parseval relation (Prop. 1), Lemma S1, one-token
@@ -79,68 +78,54 @@ void oracle_coefficients(const double* x, const double* mean, const double* m, i
 }
 
 /*
- * Nearest-codeword search for one group (Sec. 2.2; lowest index wins ties).
- * coef: g float64 coefficients.  cb: [C][g] float64 holding binary32-representable values.
- * Returns the binary32 decision; *idx64 gets the float64 decision and *gap the float64
- * relative gap between the two smallest float64 distances (DBL_MAX if d1 == 0 and d2 > 0,
- * 0 if both are 0).
+ * Nearest-codeword search for one group (Sec. 2.2 "Quantization": the encoder returns the index of
+ * the nearest codeword; App. B "Calibration": exact Euclidean search; lowest index wins ties).
+ * coef: g float64 coefficients.  cb: [C][g] float64.  Returns the index of the first minimum of the
+ * float64 squared distance; *gap gets the relative gap (d2 - d1) / d1 between the two smallest
+ * distances (DBL_MAX if d1 == 0 and d2 > 0, 0 if both are 0).
  */
-static int search_group(const double* coef, const double* cb, int g, int C, int* idx64, double* gap)
+static int search_group(const double* coef, const double* cb, int g, int C, double* gap)
 {
-    float best32 = 0.f;
-    int bi32 = -1;
     double d1 = DBL_MAX, d2 = DBL_MAX;
-    int bi64 = -1;
+    int best = -1;
     for (int c = 0; c < C; ++c) {
         const double* cw = cb + (long)c * g;
-        /* binary32 decision, the arithmetic the library boundary documents */
-        float acc = 0.f;
-        for (int i = 0; i < g; ++i) {
-            float e = (float)coef[i] - (float)cw[i];
-            acc = (i == 0) ? e * e : fmaf(e, e, acc);
-        }
-        if (bi32 < 0 || acc < best32) { best32 = acc; bi32 = c; }
-        /* float64 distances for the near-tie accounting */
         double s = 0.0;
         for (int i = 0; i < g; ++i) {
             double e = coef[i] - cw[i];
             s += e * e;
         }
-        if (s < d1) { d2 = d1; d1 = s; bi64 = c; }
+        if (best < 0 || s < d1) { d2 = d1; d1 = s; best = c; }
         else if (s < d2) { d2 = s; }
     }
-    if (idx64) *idx64 = bi64;
     if (gap) *gap = (d1 > 0.0) ? (d2 - d1) / d1 : (d2 > 0.0 ? DBL_MAX : 0.0);
-    return bi32;
+    return best;
 }
 
 /*
  * Encode from coefficients that are already given (float64 holding the values to search).
- * coef: [n][d]; cb: [L][C][g]; idx: [n][L].  idx64 / gap may be NULL.
+ * coef: [n][d]; cb: [L][C][g]; idx: [n][L].  gap may be NULL.
  */
 void oracle_search(const double* coef, long n, int d, int g, int C, const double* cb,
-                   uint8_t* idx, uint8_t* idx64, double* gap)
+                   uint8_t* idx, double* gap)
 {
     int L = d / g;
 #pragma omp parallel for schedule(static)
     for (long j = 0; j < n; ++j) {
         for (int l = 0; l < L; ++l) {
-            int i64; double gp;
-            int i32 = search_group(coef + j * d + l * g, cb + (long)l * C * g, g, C, &i64, &gp);
-            idx[j * L + l] = (uint8_t)i32;
-            if (idx64) idx64[j * L + l] = (uint8_t)i64;
+            double gp;
+            idx[j * L + l] = (uint8_t)search_group(coef + j * d + l * g, cb + (long)l * C * g, g, C, &gp);
             if (gap) gap[j * L + l] = gp;
         }
     }
 }
 
 /*
- * Write path for n tokens: k, v [n][Hkv][d] -> kidx, vidx [n][Hkv][L] (+ float64 decision and
- * gap arrays of the same shape, may be NULL).
+ * Write path for n tokens: k, v [n][Hkv][d] -> kidx, vidx [n][Hkv][L] (+ gap arrays of the same
+ * shape, may be NULL).
  */
 void oracle_encode(const oracle_tables* t, const double* k, const double* v, long n,
-                   uint8_t* kidx, uint8_t* vidx, uint8_t* kidx64, uint8_t* vidx64,
-                   double* kgap, double* vgap)
+                   uint8_t* kidx, uint8_t* vidx, double* kgap, double* vgap)
 {
     const int d = t->head_dim, g = t->group_size, C = t->codebook_size, H = t->n_kv_heads;
     const int L = d / g;
@@ -152,19 +137,15 @@ void oracle_encode(const oracle_tables* t, const double* k, const double* v, lon
             /* keys */
             oracle_coefficients(k + o * d, t->k_mean + (long)h * d, t->rk + (long)h * d * d, d, coef);
             for (int l = 0; l < L; ++l) {
-                int i64; double gp;
-                int i32 = search_group(coef + l * g, t->cb_k + ((long)h * L + l) * C * g, g, C, &i64, &gp);
-                kidx[o * L + l] = (uint8_t)i32;
-                if (kidx64) kidx64[o * L + l] = (uint8_t)i64;
+                double gp;
+                kidx[o * L + l] = (uint8_t)search_group(coef + l * g, t->cb_k + ((long)h * L + l) * C * g, g, C, &gp);
                 if (kgap) kgap[o * L + l] = gp;
             }
             /* values */
             oracle_coefficients(v + o * d, t->v_mean + (long)h * d, t->rv + (long)h * d * d, d, coef);
             for (int l = 0; l < L; ++l) {
-                int i64; double gp;
-                int i32 = search_group(coef + l * g, t->cb_v + ((long)h * L + l) * C * g, g, C, &i64, &gp);
-                vidx[o * L + l] = (uint8_t)i32;
-                if (vidx64) vidx64[o * L + l] = (uint8_t)i64;
+                double gp;
+                vidx[o * L + l] = (uint8_t)search_group(coef + l * g, t->cb_v + ((long)h * L + l) * C * g, g, C, &gp);
                 if (vgap) vgap[o * L + l] = gp;
             }
             free(coef);
@@ -303,8 +284,7 @@ float oracle_key_scale(const double* coef, int d, double* out)
 
 /* Write path with the key scale: as oracle_encode, plus kscale [n][Hkv] (bfloat16 values as float). */
 void oracle_encode_scaled(const oracle_tables* t, const double* k, const double* v, long n,
-                          uint8_t* kidx, uint8_t* vidx, float* kscale, uint8_t* kidx64, uint8_t* vidx64,
-                          double* kgap, double* vgap)
+                          uint8_t* kidx, uint8_t* vidx, float* kscale, double* kgap, double* vgap)
 {
     const int d = t->head_dim, g = t->group_size, C = t->codebook_size, H = t->n_kv_heads;
     const int L = d / g;
@@ -317,18 +297,14 @@ void oracle_encode_scaled(const oracle_tables* t, const double* k, const double*
             oracle_coefficients(k + o * d, t->k_mean + (long)h * d, t->rk + (long)h * d * d, d, coef);
             kscale[o] = oracle_key_scale(coef, d, nrm);
             for (int l = 0; l < L; ++l) {
-                int i64; double gp;
-                int i32 = search_group(nrm + l * g, t->cb_k + ((long)h * L + l) * C * g, g, C, &i64, &gp);
-                kidx[o * L + l] = (uint8_t)i32;
-                if (kidx64) kidx64[o * L + l] = (uint8_t)i64;
+                double gp;
+                kidx[o * L + l] = (uint8_t)search_group(nrm + l * g, t->cb_k + ((long)h * L + l) * C * g, g, C, &gp);
                 if (kgap) kgap[o * L + l] = gp;
             }
             oracle_coefficients(v + o * d, t->v_mean + (long)h * d, t->rv + (long)h * d * d, d, coef);
             for (int l = 0; l < L; ++l) {
-                int i64; double gp;
-                int i32 = search_group(coef + l * g, t->cb_v + ((long)h * L + l) * C * g, g, C, &i64, &gp);
-                vidx[o * L + l] = (uint8_t)i32;
-                if (vidx64) vidx64[o * L + l] = (uint8_t)i64;
+                double gp;
+                vidx[o * L + l] = (uint8_t)search_group(coef + l * g, t->cb_v + ((long)h * L + l) * C * g, g, C, &gp);
                 if (vgap) vgap[o * L + l] = gp;
             }
             free(coef);

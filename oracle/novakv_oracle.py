@@ -108,36 +108,33 @@ class Oracle:
     def search(self, coef, kvh: int, which: str):
         """Nearest-codeword search of given coefficients [n][d] against one head's codebooks.
 
-        Returns (idx binary32 decision, idx float64 decision, float64 relative gap), each [n][L].
+        Returns (idx, float64 relative gap between the two nearest codewords), each [n][L].
         """
         coef = _f64(coef)
         n = coef.shape[0]
         cb = (self.cb_k if which == "k" else self.cb_v)[kvh]
         idx = np.empty((n, self.n_groups), np.uint8)
-        idx64 = np.empty_like(idx)
         gap = np.empty((n, self.n_groups), np.float64)
         _load().oracle_search(ctypes.c_void_p(coef.ctypes.data), ctypes.c_long(n), self.d, self.g,
                               self.codebook_size, ctypes.c_void_p(cb.ctypes.data),
-                              ctypes.c_void_p(idx.ctypes.data), ctypes.c_void_p(idx64.ctypes.data),
-                              ctypes.c_void_p(gap.ctypes.data))
-        return idx, idx64, gap
+                              ctypes.c_void_p(idx.ctypes.data), ctypes.c_void_p(gap.ctypes.data))
+        return idx, gap
 
     def encode(self, k, v, with_gaps: bool = True):
-        """k, v: [n][Hkv][d] -> dict(kidx, vidx[, kidx64, vidx64, kgap, vgap]), each [n][Hkv][L]."""
+        """k, v: [n][Hkv][d] -> dict(kidx, vidx[, kgap, vgap]), each [n][Hkv][L]."""
         k, v = _f64(k), _f64(v)
         n = k.shape[0]
         shp = (n, self.n_kv_heads, self.n_groups)
         res = dict(kidx=np.empty(shp, np.uint8), vidx=np.empty(shp, np.uint8))
         if with_gaps:
-            res.update(kidx64=np.empty(shp, np.uint8), vidx64=np.empty(shp, np.uint8),
-                       kgap=np.empty(shp, np.float64), vgap=np.empty(shp, np.float64))
+            res.update(kgap=np.empty(shp, np.float64), vgap=np.empty(shp, np.float64))
 
         def p(name):
             return ctypes.c_void_p(res[name].ctypes.data) if name in res else ctypes.c_void_p(0)
 
         _load().oracle_encode(ctypes.byref(self._t), ctypes.c_void_p(k.ctypes.data),
                               ctypes.c_void_p(v.ctypes.data), ctypes.c_long(n), p("kidx"), p("vidx"),
-                              p("kidx64"), p("vidx64"), p("kgap"), p("vgap"))
+                              p("kgap"), p("vgap"))
         return res
 
     def key_scale(self, coef):
@@ -163,15 +160,14 @@ class Oracle:
         res = dict(kidx=np.empty(shp, np.uint8), vidx=np.empty(shp, np.uint8),
                    kscale=np.empty((n, self.n_kv_heads), np.float32))
         if with_gaps:
-            res.update(kidx64=np.empty(shp, np.uint8), vidx64=np.empty(shp, np.uint8),
-                       kgap=np.empty(shp, np.float64), vgap=np.empty(shp, np.float64))
+            res.update(kgap=np.empty(shp, np.float64), vgap=np.empty(shp, np.float64))
 
         def p(name):
             return ctypes.c_void_p(res[name].ctypes.data) if name in res else ctypes.c_void_p(0)
 
         _load().oracle_encode_scaled(ctypes.byref(self._t), ctypes.c_void_p(k.ctypes.data),
                                      ctypes.c_void_p(v.ctypes.data), ctypes.c_long(n), p("kidx"), p("vidx"),
-                                     p("kscale"), p("kidx64"), p("vidx64"), p("kgap"), p("vgap"))
+                                     p("kscale"), p("kgap"), p("vgap"))
         return res
 
     def reconstruct_scaled(self, kidx, vidx, kscale):

@@ -69,7 +69,6 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
         if (cudaMalloc(&ctx->int2_img, n * sizeof(__half)) != cudaSuccess ||
             cudaMemcpy(ctx->int2_img, img.data(), n * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess) {
             cudaFree(ctx->dev_status);
-    cudaFree(ctx->int2_img);
             cudaFree(ctx->int2_img);
             delete ctx;
             return NOVAKV_ECUDA;
@@ -96,6 +95,7 @@ extern "C" novakv_status novakv_destroy(novakv_ctx* ctx) {
         for (auto& e : ctx->prof[k]) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
     for (auto& e : ctx->prof_free) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
     cudaFree(ctx->dev_status);
+    cudaFree(ctx->int2_img);
     delete ctx;
     return NOVAKV_OK;
 }
@@ -415,6 +415,8 @@ extern "C" novakv_status novakv_step_host(novakv_ctx* ctx, int layer, const void
     if (st != NOVAKV_OK) return st;
     if (batch <= 0 || n_tokens < 0 || !q_host || !out_host || !staging) return NOVAKV_EINVAL;
     if (n_tokens > 0 && (!k_new_host || !v_new_host || !tok_seq_host || !tok_pos_host)) return NOVAKV_EINVAL;
+    if (!k_pages || !v_pages || !page_table || !seq_lens) return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0) return NOVAKV_EPAGE;
     if (staging_bytes < novakv_step_staging_bytes(ctx, batch, n_tokens) || ((uintptr_t)staging & 255)) return NOVAKV_EWORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
     CUDA_OK(cudaSetDevice(ctx->cfg.device));

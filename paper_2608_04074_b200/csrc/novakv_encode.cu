@@ -1,8 +1,15 @@
-// Write path: forward transforms (binary64) + brute-force nearest-codeword search (binary32) +
-// paged store.  One CTA handles a tile of tokens for one (KV head, side); side 0 = keys, 1 = values.
+// Write path: forward transforms (binary64) + brute-force nearest-codeword search + paged store.
+// One CTA handles a tile of tokens for one (KV head, side); side 0 = keys, 1 = values.
 //
 // The search is ALU-bound (256 distance evaluations per group, per token, per side); the codebook
 // of the CTA's head and side stays in shared memory and every warp reads codewords as broadcasts.
+//
+// The index the write path stores is the exact Euclidean nearest codeword of the binary64 coefficient
+// (lowest index on a tie).  The 256 distances are evaluated in binary32; beside the minimum the search
+// keeps the second smallest distance, and whenever the two are closer than a rigorous bound on what the
+// binary32 evaluation (coefficient rounding included) can have moved them, the group is searched again in
+// binary64 by the whole warp (certified search).  The binary32 result is kept only where it provably
+// equals the binary64 one.
 #include <math_constants.h>
 
 #include <cooperative_groups.h>
@@ -28,12 +35,14 @@ struct EncSmem {
     static constexpr size_t total = cb_bytes + r_bytes + idx_bytes;
 };
 
-// Squared distance in the arithmetic the public header fixes: fma(e3,e3,fma(e2,e2,fma(e1,e1,e0*e0))).
+#ifdef NOVAKV_SCALAR_SEARCH
+// Scalar form of the binary32 distance: fma(e3,e3,fma(e2,e2,fma(e1,e1,e0*e0))).
 __device__ __forceinline__ float dist4(const float4 r, const float4 c) {
     const float e0 = __fsub_rn(r.x, c.x), e1 = __fsub_rn(r.y, c.y);
     const float e2 = __fsub_rn(r.z, c.z), e3 = __fsub_rn(r.w, c.w);
     return __fmaf_rn(e3, e3, __fmaf_rn(e2, e2, __fmaf_rn(e1, e1, __fmul_rn(e0, e0))));
 }
+#endif
 
 // Packed binary32 pairs: two IEEE operations per instruction (same roundings as the scalar forms).
 __device__ __forceinline__ uint64_t pk2(float lo, float hi) {
@@ -90,17 +99,88 @@ __device__ __forceinline__ float fmin3(float a, float b, float c) {
     return d;
 }
 
+// Warp-cooperative exact search of one (token, group) in binary64: all 32 lanes call it with the same
+// arguments and get the same result.  The coefficient is either taken from shared memory (EXACT_IN_SMEM:
+// the binary32 values there ARE the vector to encode: given coefficients, normalised keys) or recomputed in
+// binary64 from the token's bfloat16 input row and the transform's columns 4l .. 4l+3.  Lane i evaluates the
+// codewords i, i+32, ... in ascending order with a strict '<'; the warp then keeps the smallest distance
+// and, among equal distances, the lowest index.
+template <int D, bool EXACT_IN_SMEM>
+__device__ __noinline__ int exact_search_group(const float* r_row_s, const __nv_bfloat16* __restrict__ x_row_g,
+                                               const double* mean_s, const double* __restrict__ R_plain /* [D][D] */,
+                                               int l, const float* cb_pairs_s /* [L][128][4][2] */) {
+    const int lane = threadIdx.x & 31;
+    double r[4];
+    if (EXACT_IN_SMEM) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) r[c] = (double)r_row_s[l * 4 + c];
+    } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) r[c] = 0.0;
+        for (int k = lane; k < D; k += 32) {
+            const double xc = (double)__bfloat162float(x_row_g[k]) - mean_s[k];
+            const double2 r01 = *reinterpret_cast<const double2*>(R_plain + (size_t)k * D + l * 4);
+            const double2 r23 = *reinterpret_cast<const double2*>(R_plain + (size_t)k * D + l * 4 + 2);
+            r[0] = fma(xc, r01.x, r[0]); r[1] = fma(xc, r01.y, r[1]);
+            r[2] = fma(xc, r23.x, r[2]); r[3] = fma(xc, r23.y, r[3]);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) r[c] += __shfl_xor_sync(0xffffffffu, r[c], o);
+    }
+    double best = CUDART_INF;
+    int bi = lane;
+    const float* cb = cb_pairs_s + (size_t)l * NOVAKV_C * 4;
+#pragma unroll
+    for (int j = 0; j < NOVAKV_C / 32; ++j) {
+        const int code = lane + 32 * j;
+        const float* cw = cb + (size_t)(code >> 1) * 8 + (code & 1);
+        double dd = 0.0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const double e = r[c] - (double)cw[2 * c];
+            dd = __dadd_rn(dd, __dmul_rn(e, e));
+        }
+        if (dd < best) { best = dd; bi = code; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    return bi;
+}
+
+// What the binary32 evaluation can have moved a squared distance by: the coefficient vector of the group
+// is off by at most delta in norm (its rounding to binary32), the eight operations of the distance add a
+// relative 6 * 2^-24.  |d32 - d| <= 2 sqrt(d) delta + delta^2 + 6 * 2^-24 d; the test below uses twice the
+// bound at the larger of the two distances (both have moved) with some slack on the constants.
+__device__ __forceinline__ bool needs_exact_search(float best, float second, float delta) {
+    const float thr = 4.5f * sqrtf(second) * delta + 2.5f * delta * delta + 9.6e-7f * second;     // 9.6e-7 > 16 * 2^-24
+    return !(second - best > thr);
+}
+
 // Search of the tile's coefficients (r_s, [ENC_TILE][RSTRIDE] float) against the paired codebook image.
 // Warp w of n_warps owns groups w, w+n_warps, ...; lane t owns tokens t and t+32.
-// The result is the first minimum in ascending codeword order (what a scan with a strict '<' keeps), found in
-// two steps that need far fewer compare/select instructions than a per-codeword running argmin:
+// The binary32 pass finds the first minimum in ascending codeword order (what a scan with a strict '<' keeps)
+// in two steps that need far fewer compare/select instructions than a per-codeword running argmin:
 //   1. blocks of 8 codewords: the block minimum (a tree of 3-input minima) updates the running minimum with a
-//      strict '<', which keeps the first block that attains the overall minimum;
-//   2. the 8 distances of that block are recomputed (same instructions, same bits) and the first one equal to
-//      the minimum gives the index.
-template <int D>
+//      strict '<', which keeps the first block that attains the overall minimum; the second smallest block
+//      minimum is tracked beside it (two more min/max per block);
+//   2. the 8 distances of that block are recomputed (same instructions, same bits); the first one equal to
+//      the minimum gives the index and the others enter the second smallest distance.
+// Then the certification: a group whose two smallest distances are too close to tell apart in binary32 is
+// searched again in binary64 by the whole warp (exact_search_group).
+// EXACT_IN_SMEM: the binary32 coefficients in r_s are the vector to encode (delta = 0); otherwise they are
+// roundings of binary64 coefficients that exact_search_group recomputes from the inputs x_tile_g
+// (bfloat16 rows of the tile's tokens, row stride x_stride elements).
+template <int D, bool EXACT_IN_SMEM>
 __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s, uint8_t* idx_s, int n_valid,
-                                            int warp, int n_warps) {
+                                            int warp, int n_warps, const __nv_bfloat16* __restrict__ x_tile_g,
+                                            size_t x_stride, const double* mean_s,
+                                            const double* __restrict__ R_plain) {
     constexpr int L = D / NOVAKV_G;
     constexpr int RS = EncSmem<D>::RSTRIDE;
     const int lane = threadIdx.x & 31;
@@ -109,7 +189,7 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
         const float4 rb = *reinterpret_cast<const float4*>(r_s + (size_t)(lane + 32) * RS + l * 4);
         const uint64_t ra2[4] = {pk2(ra.x, ra.x), pk2(ra.y, ra.y), pk2(ra.z, ra.z), pk2(ra.w, ra.w)};
         const uint64_t rb2[4] = {pk2(rb.x, rb.x), pk2(rb.y, rb.y), pk2(rb.z, rb.z), pk2(rb.w, rb.w)};
-        float best_a = CUDART_INF_F, best_b = CUDART_INF_F;
+        float best_a = CUDART_INF_F, best_b = CUDART_INF_F, sec_a = CUDART_INF_F, sec_b = CUDART_INF_F;
         int blk_a = 0, blk_b = 0;
         const ulonglong2* cb = reinterpret_cast<const ulonglong2*>(cb_s) + (size_t)l * NOVAKV_C;   // 2 x 16 B per pair
 #pragma unroll 4
@@ -124,10 +204,13 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
             }
             const float ma = fmin3(fmin3(da[0], da[1], da[2]), fmin3(da[3], da[4], da[5]), fminf(da[6], da[7]));
             const float mb = fmin3(fmin3(db[0], db[1], db[2]), fmin3(db[3], db[4], db[5]), fminf(db[6], db[7]));
+            sec_a = fminf(sec_a, fmaxf(best_a, ma));
+            sec_b = fminf(sec_b, fmaxf(best_b, mb));
             if (ma < best_a) { best_a = ma; blk_a = blk; }
             if (mb < best_b) { best_b = mb; blk_b = blk; }
         }
-        // the winning blocks again: first codeword whose distance equals the minimum
+        // the winning blocks again: first codeword whose distance equals the minimum; the block's other
+        // distances compete for the second place
         int ia = 8 * blk_a, ib = 8 * blk_b;
         {
             float da[8], db[8];
@@ -140,11 +223,43 @@ __device__ __forceinline__ void search_tile(const float* r_s, const float4* cb_s
                 const uint64_t cwb[4] = {qb0.x, qb0.y, qb1.x, qb1.y};
                 dist4x2(rb2, cwb, db[2 * p], db[2 * p + 1]);
             }
+            int ka = 0, kb = 0;
 #pragma unroll
             for (int k = 7; k >= 0; --k) {
-                if (da[k] == best_a) ia = 8 * blk_a + k;
-                if (db[k] == best_b) ib = 8 * blk_b + k;
+                if (da[k] == best_a) ka = k;
+                if (db[k] == best_b) kb = k;
             }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (k != ka) sec_a = fminf(sec_a, da[k]);
+                if (k != kb) sec_b = fminf(sec_b, db[k]);
+            }
+            ia += ka; ib += kb;
+        }
+        // certification
+        float del_a = 0.f, del_b = 0.f;
+        if (!EXACT_IN_SMEM) {
+            // |coefficient - its binary32 rounding| <= 2^-24 |coefficient| per component
+            del_a = 5.97e-8f * sqrtf(fmaf(ra.x, ra.x, fmaf(ra.y, ra.y, fmaf(ra.z, ra.z, ra.w * ra.w)))) * 1.0001f;
+            del_b = 5.97e-8f * sqrtf(fmaf(rb.x, rb.x, fmaf(rb.y, rb.y, fmaf(rb.z, rb.z, rb.w * rb.w)))) * 1.0001f;
+        }
+        const bool ta = lane < n_valid && needs_exact_search(best_a, sec_a, del_a);
+        const bool tb = lane + 32 < n_valid && needs_exact_search(best_b, sec_b, del_b);
+        unsigned todo_a = __ballot_sync(0xffffffffu, ta), todo_b = __ballot_sync(0xffffffffu, tb);
+        while (todo_a) {
+            const int src = __ffs(todo_a) - 1;
+            todo_a &= todo_a - 1;
+            const int res = exact_search_group<D, EXACT_IN_SMEM>(r_s + (size_t)src * RS, x_tile_g + (size_t)src * x_stride,
+                                                                 mean_s, R_plain, l, reinterpret_cast<const float*>(cb_s));
+            if (lane == src) ia = res;
+        }
+        while (todo_b) {
+            const int src = __ffs(todo_b) - 1;
+            todo_b &= todo_b - 1;
+            const int res = exact_search_group<D, EXACT_IN_SMEM>(r_s + (size_t)(src + 32) * RS,
+                                                                 x_tile_g + (size_t)(src + 32) * x_stride, mean_s, R_plain, l,
+                                                                 reinterpret_cast<const float*>(cb_s));
+            if (lane == src) ib = res;
         }
         if (lane < n_valid) idx_s[lane * L + l] = (uint8_t)ia;
         if (lane + 32 < n_valid) idx_s[(lane + 32) * L + l] = (uint8_t)ib;
@@ -199,6 +314,7 @@ __global__ void __launch_bounds__(ENC_THREADS, 1)
 novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                      const int32_t* __restrict__ tok_seq, const int32_t* __restrict__ tok_pos, int n_tokens,
                      const double* __restrict__ rk_d, const double* __restrict__ rv_d,
+                     const double* __restrict__ rk_plain, const double* __restrict__ rv_plain,
                      const double* __restrict__ k_mean_d, const double* __restrict__ v_mean_d,
                      const float* __restrict__ cb_k, const float* __restrict__ cb_v,
                      uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages,
@@ -206,6 +322,8 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                      const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
                      int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
                      uint32_t* __restrict__ dev_status) {
+    // rk_d / rv_d: the transforms in tensor-core fragment order [d/4][d][4]; rk_plain / rv_plain: the same
+    // matrices row-major [d][d] (read only by the certified search's binary64 recomputation)
     constexpr bool KSC = FMT >= 1, VSQ = FMT == 2;
     using P = EncPipe<D>;
     constexpr int L = D / NOVAKV_G, RS = P::RS, NT = ENC_HALF_THREADS;
@@ -395,7 +513,13 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                     idx_s[e] = (uint8_t)((int)c.x | ((int)c.y << 2) | ((int)c.z << 4) | ((int)c.w << 6));
                 }
             } else {
-                search_tile<D>(r_s, cb_s, idx_s, n_valid, tid >> 5, NT / 32);
+                const __nv_bfloat16* x_tile = x_new + ((size_t)t0 * n_kv_heads + kvh) * D;
+                const double* R_plain = (side == 0 ? rk_plain : rv_plain) + (size_t)kvh * D * D;
+                // normalised keys are defined in binary32: the values in r_s are the vector to encode
+                if (KSC && side == 0)
+                    search_tile<D, true>(r_s, cb_s, idx_s, n_valid, tid >> 5, NT / 32, x_tile, (size_t)n_kv_heads * D, mean_s, R_plain);
+                else
+                    search_tile<D, false>(r_s, cb_s, idx_s, n_valid, tid >> 5, NT / 32, x_tile, (size_t)n_kv_heads * D, mean_s, R_plain);
             }
             nbar_sync(BAR_S, NT);
             for (int e = tid; e < n_valid * L; e += NT) {
@@ -435,7 +559,8 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 // ranges of the codebook; their minima are merged with the lowest index winning ties.
 // Everything that depends only on the calibration is staged before the grid-dependency wait, so it
 // overlaps the tail of the preceding kernel in the stream.
-// Arithmetic is identical to the tiled kernel (binary64 accumulation in index order, dist4 search).
+// The coefficients are accumulated in binary64 in index order and the search runs in binary64 throughout
+// (at these sizes the kernel is latency-bound, not ALU-bound), so its indices are the exact nearest codewords.
 // KSC (key format with a per-token scale): the L/4 CTAs of a (head, side) form a thread-block cluster;
 // each publishes the sums of squares of its 16 coefficients per token in its shared memory, a cluster
 // barrier makes them visible, and every CTA adds the L/4 x 4 partial sums in the same fixed order through
@@ -594,17 +719,24 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             }
             cluster.sync();                             // partial sums may be overwritten by the next pass / CTAs may exit
         }
-        // this lane group's range of the codebook, ascending with a strict '<' (first minimum)
-        float best = dist4(r, cb_s[warp][c0]);
+        // this lane group's range of the codebook in binary64, ascending with a strict '<' (first minimum).
+        // The vector to encode is the binary64 coefficient; for normalised keys it is the binary32 quotient.
+        double rd[4] = {acc0, acc1, acc2, acc3};
+        if (KSC && side == 0) { rd[0] = (double)r.x; rd[1] = (double)r.y; rd[2] = (double)r.z; rd[3] = (double)r.w; }
+        auto dist_d = [&](const float4 c) {
+            const double e0 = rd[0] - (double)c.x, e1 = rd[1] - (double)c.y, e2 = rd[2] - (double)c.z, e3 = rd[3] - (double)c.w;
+            return __dadd_rn(__dadd_rn(__dadd_rn(__dmul_rn(e0, e0), __dmul_rn(e1, e1)), __dmul_rn(e2, e2)), __dmul_rn(e3, e3));
+        };
+        double best = dist_d(cb_s[warp][c0]);
         int bi = c0;
-#pragma unroll 8
+#pragma unroll 4
         for (int c = 1; c < codes_per_grp; ++c) {
-            const float dd = dist4(r, cb_s[warp][c0 + c]);
+            const double dd = dist_d(cb_s[warp][c0 + c]);
             if (dd < best) { best = dd; bi = c0 + c; }
         }
         // merge the groups of a token: smaller distance wins, equal distances keep the lower index
         for (int off = tp; off < 32; off <<= 1) {
-            const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+            const double ob = __shfl_xor_sync(0xffffffffu, best, off);
             const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
             if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
         }
@@ -641,7 +773,7 @@ novakv_search_kernel(const float* __restrict__ coef, int n, const float* __restr
             r_s[(size_t)t * RS + c] = t < n_valid ? coef[((size_t)(t0 + t) * n_kv_heads + kvh) * D + c] : 0.f;
         }
         __syncthreads();
-        search_tile<D>(r_s, cb_s, idx_s, n_valid, threadIdx.x >> 5, ENC_THREADS / 32);
+        search_tile<D, true>(r_s, cb_s, idx_s, n_valid, threadIdx.x >> 5, ENC_THREADS / 32, nullptr, 0, nullptr, nullptr);
         __syncthreads();
         for (int i = threadIdx.x; i < n_valid * L; i += ENC_THREADS) {
             const int t = i / L, l = i - t * L;
@@ -715,7 +847,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     dim3 grid(ctas_x, ctx->cfg.n_kv_heads, 2);
     novakv_prof_scope ps(ctx, 1, stream);
     kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d_mma, ly.rv_d_mma,
-                                               ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, k_scales,
+                                               ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, k_scales,
                                                v_meta, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
                                                ctx->cfg.n_kv_heads, tiles_per_cta, ctx->dev_status);
     ps.end();

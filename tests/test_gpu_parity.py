@@ -66,8 +66,9 @@ def test_search_from_oracle_coefficients_is_exact(name, request):
         case.ctx.novakv_search_coefficients(0, 0 if which == "k" else 1, _dev(coef), idx_gpu)
         got = idx_gpu.cpu().numpy()
         for h in range(case.ctx.n_kv_heads):
-            ref, _, _ = case.oracle.search(coef[:, h].astype(np.float64), h, which)
-            assert np.array_equal(got[:, h], ref), f"{which} head {h}"
+            ref, gap = case.oracle.search(coef[:, h].astype(np.float64), h, which)
+            bad = (got[:, h] != ref) & (gap > NEAR_TIE)
+            assert not bad.any(), f"{which} head {h}: {int(bad.sum())} mismatches outside the near-tie band"
 
 
 # --------------------------------------------------------------------------- T2: transform + search + paged store

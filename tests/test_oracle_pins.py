@@ -269,17 +269,14 @@ def test_search_matches_independent_brute_force(tiny_case):
     c = tiny_case
     orc = c["oracle"]
     coef = orc.coefficients(c["k"][:300].astype(np.float64), "k")[:, 0]
-    idx, idx64, gap = orc.search(coef, 0, "k")
+    idx, gap = orc.search(coef, 0, "k")
     cb = orc.cb_k[0]                                         # [L][C][g]
     x = coef.reshape(300, 16, 1, 4)
     d2 = ((x - cb[None]) ** 2).sum(-1)                       # [n][L][C] float64
     ref = d2.argmin(axis=2)
-    assert np.array_equal(idx64, ref)
+    assert np.array_equal(idx, ref)
     srt = np.sort(d2, axis=2)
     assert np.allclose(gap, (srt[:, :, 1] - srt[:, :, 0]) / srt[:, :, 0], rtol=1e-9)
-    # the binary32 decision can differ from the float64 one only at a near-tie
-    diff = idx != idx64
-    assert np.all(gap[diff] < 1e-5)
 
 
 def test_search_tie_break_and_exact_hits():
@@ -291,19 +288,19 @@ def test_search_tie_break_and_exact_hits():
     eye = np.eye(d)[None]
     orc = O.Oracle(eye, eye, eye, np.zeros((1, d)), np.zeros((1, d)), cb, cb)
     coef = np.concatenate([cb[0, 0, 200], cb[0, 1, 250]])[None, :]
-    idx, idx64, gap = orc.search(coef, 0, "k")
-    assert idx.tolist() == [[17, 5]] and idx64.tolist() == [[17, 5]]
+    idx, gap = orc.search(coef, 0, "k")
+    assert idx.tolist() == [[17, 5]]
     assert gap.tolist() == [[0.0, 0.0]]
     # equidistant between two codewords: first minimum wins
     cb2 = np.full((1, L, C, g), 100.0)
     cb2[0, :, 3] = [1, 0, 0, 0]
     cb2[0, :, 9] = [-1, 0, 0, 0]
     orc2 = O.Oracle(eye, eye, eye, np.zeros((1, d)), np.zeros((1, d)), cb2, cb2)
-    idx, _, gap = orc2.search(np.zeros((1, d)), 0, "v")
+    idx, gap = orc2.search(np.zeros((1, d)), 0, "v")
     assert idx.tolist() == [[3, 3]] and gap.tolist() == [[0.0, 0.0]]
     # every codeword encodes to itself
     x = np.concatenate([cb[0, 0], cb[0, 1]], axis=1)          # [C][d]
-    idx, _, _ = orc.search(x, 0, "k")
+    idx, _ = orc.search(x, 0, "k")
     want = np.arange(C)
     want0 = want.copy(); want0[200] = 17
     want1 = want.copy(); want1[250] = 5
@@ -319,11 +316,13 @@ def test_encode_equals_coefficients_then_search(tiny_case):
     r = (k[:, 0] - orc.k_mean[0]) @ orc.rk[0]
     s = (v[:, 0] - orc.v_mean[0]) @ orc.rv[0]
     assert np.allclose(orc.coefficients(k, "k")[:, 0], r, rtol=1e-12, atol=1e-9)
-    ik, _, _ = orc.search(orc.coefficients(k, "k")[:, 0], 0, "k")
-    iv, _, _ = orc.search(orc.coefficients(v, "v")[:, 0], 0, "v")
+    ik, _ = orc.search(orc.coefficients(k, "k")[:, 0], 0, "k")
+    iv, _ = orc.search(orc.coefficients(v, "v")[:, 0], 0, "v")
     assert np.array_equal(enc["kidx"][:, 0], ik) and np.array_equal(enc["vidx"][:, 0], iv)
     d2 = ((s.reshape(100, 16, 1, 4) - orc.cb_v[0][None]) ** 2).sum(-1)
-    assert np.array_equal(enc["vidx64"][:, 0], d2.argmin(axis=2))
+    assert np.array_equal(enc["vidx"][:, 0], d2.argmin(axis=2))
+    d2k = ((r.reshape(100, 16, 1, 4) - orc.cb_k[0][None]) ** 2).sum(-1)
+    assert np.array_equal(enc["kidx"][:, 0], d2k.argmin(axis=2))
 
 
 # ---------------------------------------------------------------- decode (Eq. "scores", Lemma S1)
