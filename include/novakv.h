@@ -11,9 +11,9 @@
  * per-token metadata.  Pages hold 64 tokens.  Two caller-owned device pools of equal geometry,
  * uint8 [n_pages][Hkv][64*L] each: one contiguous chunk of 64*L bytes per (page, KV head) for keys
  * and one for values.  Inside a chunk (t = token slot in the page, l = group):
- *     keys    [tile = t/32][plane][t%32][16 bytes]: a token's L bytes are 8 "slots" of L/8 consecutive
- *             groups, stored rotated: position j holds slot (j + t%8 + (t/8)%4) % 8; plane = byte / 16.
- *     values  [block = t/16][fr = l%8][fc = t%4][x][b = (t%16)/4],  x = (l/8 - fc) mod (L/8).
+ *     keys    [tile = t/32][plane][t%32][16 bytes]: byte j of a token's L bytes holds the code of group
+ *             j ^ (t % 8) for j < 16 and of group j ^ (t % 16) for j >= 16; plane = j / 16.
+ *     values  [block = t/16][fr = l%8][fc = t%4][gb = l/8][b = (t%16)/4].
  * Both orders make every lane of a decode warp load exactly the bytes it consumes with coalesced
  * 128-bit loads, and keep its shared-memory table gathers free of bank conflicts.
  * page_table[seq][i] (int32, row length max_pages_per_seq) names the page of tokens 64i..64i+63.
@@ -53,7 +53,7 @@ typedef enum {
     NOVAKV_EPAGE = 4,         /* page-table geometry inconsistent */
     NOVAKV_EWORKSPACE = 5,    /* workspace NULL or too small */
     NOVAKV_ECUDA = 6,         /* a CUDA runtime call failed */
-    NOVAKV_EUNSUPPORTED = 7   /* value codebook not binary16-representable, etc. */
+    NOVAKV_EUNSUPPORTED = 7   /* value codebook off its 8-bit grid, etc. */
 } novakv_status;
 
 /* Bits of the device status word. */
@@ -61,6 +61,7 @@ typedef enum {
 #define NOVAKV_DEV_BAD_LENGTH    2u   /* a sequence length exceeded 64 * max_pages_per_seq */
 #define NOVAKV_DEV_WAIT_TIMEOUT  4u   /* reserved: no kernel of this build waits on another thread or copy */
 #define NOVAKV_DEV_BAD_TOKEN     8u   /* an appended token named a sequence slot or position out of range */
+#define NOVAKV_DEV_SMEM_LAYOUT  16u   /* the scan kernel could not place its tables in shared memory (no output was produced) */
 
 typedef struct {
     int n_layers;
@@ -85,7 +86,9 @@ typedef struct {
  *   k_mean    [Hkv][d]      may be NULL (= 0)
  *   v_mean    [Hkv][d]      may be NULL (= 0)
  *   cb_k      [Hkv][L][256][4]
- *   cb_v      [Hkv][L][256][4]   every entry must be exactly representable in IEEE binary16
+ *   cb_v      [Hkv][L][256][4]   every coordinate (head, l, component) on its own 8-bit grid:
+ *                                lo + u (hi - lo) / 255, u = 0..255, lo / hi = its smallest / largest value
+ *                                over the 256 codewords, evaluated in binary64, rounded once to binary32
  */
 typedef struct {
     const float* rk;
@@ -104,8 +107,8 @@ const char* novakv_status_string(novakv_status s);
 /*
  * Algorithm 1 lines 1-6 produce these tables offline; this call copies them to the device
  * (synchronous; the caller keeps its memory).  Returns NOVAKV_EUNSUPPORTED if cb_v holds a value
- * that binary16 cannot represent exactly (the decode kernel keeps value codewords in binary16;
- * snap them offline, as the paper does for its codebooks, so that encoder and decoder agree).
+ * off its 8-bit grid (the decode kernel keeps a value codeword as four grid indices; snap the
+ * codebooks offline, as the paper does for its own, so that encoder, decoder and any reference agree).
  */
 novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, const novakv_calibration* host);
 

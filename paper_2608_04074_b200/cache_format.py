@@ -9,12 +9,11 @@ in the key pool and one in the value pool (``uint8 [n_pages][Hkv][64*L]`` each).
 the bytes are ordered so that each lane of a decode warp loads, with one or two coalesced 128-bit
 loads, exactly the bytes it consumes:
 
-* keys:   ``[tile = t // 32][plane][t % 32][16 bytes]``.  A token's L bytes are split into 8
-  "slots" of L/8 consecutive groups; they are stored rotated, position j holding slot
-  ``(j + t % 8 + (t // 8) % 4) % 8`` (the lanes of a quarter warp then read 8 different banks of
-  the score table at every step); plane = byte position // 16.
-* values: ``[block = t // 16][fr = l % 8][fc = t % 4][x][b = (t % 16) // 4]`` with
-  ``x = (l // 8 - fc) mod (L // 8)``: the 16 (or 8) bytes of MMA lane (fr, fc) are contiguous.
+* keys:   ``[tile = t // 32][plane][t % 32][16 bytes]``.  Byte j of a token's L bytes holds the code
+  of group ``j ^ (t % 8)`` for j < 16 and of group ``j ^ (t % 16)`` for j >= 16 (neighbouring lanes
+  then read different columns of the score table at every step); plane = j // 16.
+* values: ``[block = t // 16][fr = l % 8][fc = t % 4][gb = l // 8][b = (t % 16) // 4]``: the 16 (or
+  8) bytes of MMA lane (fr, fc) are contiguous.
 
 (t = token slot in the page, l = group.)
 
@@ -37,11 +36,9 @@ def n_groups(head_dim: int) -> int:
 
 def key_offset(t, l, n_groups_: int):
     """Byte offset of (token slot t, group l) inside a key chunk (numpy arrays broadcast)."""
-    gps, kpl = n_groups_ // 8, n_groups_ // 16
-    sigma, m = l // gps, l % gps
-    rot = ((t & 7) + ((t >> 3) & 3)) & 7
-    bytepos = ((sigma - rot) & 7) * gps + m
-    return (((t >> 5) * kpl + (bytepos >> 4)) * 32 + (t & 31)) * 16 + (bytepos & 15)
+    kpl = n_groups_ // 16
+    j = l ^ (t & np.where(np.asarray(l) < 16, 7, 15))
+    return (((t >> 5) * kpl + (j >> 4)) * 32 + (t & 31)) * 16 + (j & 15)
 
 
 def value_offset(t, l, n_groups_: int):
@@ -49,8 +46,7 @@ def value_offset(t, l, n_groups_: int):
     ngb = n_groups_ // 8
     tb = t & 15
     fc, b, fr = tb & 3, tb >> 2, l & 7
-    x = ((l >> 3) - fc) & (ngb - 1)
-    return (t >> 4) * (n_groups_ * 16) + (fr * 4 + fc) * (ngb * 4) + x * 4 + b
+    return (t >> 4) * (n_groups_ * 16) + (fr * 4 + fc) * (ngb * 4) + (l >> 3) * 4 + b
 
 
 def pack_int2(codes: np.ndarray) -> np.ndarray:

@@ -21,9 +21,9 @@ transform coefficients on the calibration values; eigenvector signs are fixed so
 entry of largest magnitude is positive; k-means is seeded with distinct training vectors and
 runs a fixed number of iterations; the per-token scale of Algorithm 3 is off (it is outside
 Theorem 2's model and would break the exact 2 bits/element).
-Value codebooks are finally snapped to IEEE binary16-representable numbers (the paper snaps
-its codebooks to a narrower format offline as well); the encoder and the decoder therefore
-see the same centroids.
+Value codebooks are finally snapped to an 8-bit grid per (KV head, group, coordinate) (the paper
+snaps its codebooks to an 8-bit format offline as well): encoder, decoder and oracle therefore see
+the same centroids, and the decode kernel can keep a value codeword in four bytes.
 """
 from __future__ import annotations
 
@@ -131,6 +131,23 @@ def equalizing_order(variances: np.ndarray, n_groups: int) -> np.ndarray:
     return order
 
 
+def snap_to_u8_grid(cb: np.ndarray) -> np.ndarray:
+    """Round every codebook coordinate to its own 8-bit grid and return float32 values.
+
+    cb: [..][C][g].  Coordinate i of a codebook takes the values lo_i + u (hi_i - lo_i) / 255, u = 0 .. 255,
+    where lo_i / hi_i are the smallest / largest float32 value of that coordinate over the C codewords; the
+    grid is evaluated in float64 and rounded once to float32 (``novakv_load_calibration`` re-derives the
+    grid from the snapped values with the same arithmetic and refuses anything else).
+    """
+    cb32 = np.asarray(cb, dtype=np.float32)
+    lo = cb32.min(axis=-2, keepdims=True).astype(np.float64)
+    hi = cb32.max(axis=-2, keepdims=True).astype(np.float64)
+    step = (hi - lo) / 255.0
+    step = np.where(step > 0, step, 1.0)
+    u = np.clip(np.rint((cb32.astype(np.float64) - lo) / step), 0, 255)
+    return (lo + step * u).astype(np.float32)
+
+
 def _lloyd_c(x_groups: np.ndarray, init: np.ndarray, iters: int):
     lib = ctypes.CDLL(str(_build.build_calib_host()))
     fn = lib.novakv_calib_lloyd
@@ -170,7 +187,7 @@ def train_codebooks(coef: np.ndarray, n_groups: int, codebook_size: int, iters: 
 def calibrate(q_cal: np.ndarray, k_cal: np.ndarray, v_cal: np.ndarray, *, n_kv_heads: int,
               group_size: int = 4, codebook_size: int = 256, lloyd_iters: int = 25,
               seed: int = 0, n_q_for_values: int | None = None,
-              snap_value_codebook_fp16: bool = True, key_scale: bool = False) -> Calibration:
+              snap_value_codebook: bool = True, key_scale: bool = False) -> Calibration:
     """Run the whole offline calibration for one layer.
 
     q_cal: [N][Hq][d], k_cal / v_cal: [M][Hkv][d] (float64).
@@ -218,9 +235,14 @@ def calibrate(q_cal: np.ndarray, k_cal: np.ndarray, v_cal: np.ndarray, *, n_kv_h
         info["value_coef_var"].append(var_v[order_v])
         info["key_distortion"].append(dist_k); info["value_distortion"].append(dist_v)
     f32 = {name: np.ascontiguousarray(np.stack(vals), dtype=np.float32) for name, vals in out.items()}
-    if snap_value_codebook_fp16:
-        f32["cb_v"] = f32["cb_v"].astype(np.float16).astype(np.float32)
+    if snap_value_codebook:
+        unsnapped = f32["cb_v"]
+        f32["cb_v"] = snap_to_u8_grid(unsnapped)
+        info["value_snap_rms"] = np.sqrt(((f32["cb_v"].astype(np.float64) - unsnapped) ** 2).mean(axis=(1, 2, 3)))
+        info["value_codeword_rms"] = np.sqrt((unsnapped.astype(np.float64) ** 2).mean(axis=(1, 2, 3)))
+    extra = {k_: info.pop(k_) for k_ in ("value_snap_rms", "value_codeword_rms") if k_ in info}
     info = {k_: np.stack(v_) for k_, v_ in info.items()}
+    info.update(extra)
     info["lloyd_iters"] = lloyd_iters
     info["seed"] = seed
     return Calibration(head_dim=d, group_size=group_size, codebook_size=codebook_size, info=info,

@@ -1,4 +1,5 @@
 // Host side of the C ABI: context, calibration upload, argument validation, dispatch.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -58,16 +59,17 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
         return NOVAKV_ECUDA;
     }
     {
-        // product codebook of the scalar INT2 value codec: byte c decodes to (c & 3, (c >> 2) & 3, (c >> 4) & 3, c >> 6),
-        // the same for every group and head, replicated in the layout the value gather reads
-        const size_t n = (size_t)cfg->n_kv_heads * NOVAKV_C * 32 * NOVAKV_G;
-        std::vector<__half> img(n);
+        // product codebook of the scalar INT2 value codec: byte c decodes to the levels (c & 3, (c >> 2) & 3,
+        // (c >> 4) & 3, c >> 6), the same for every group and head, in the layout the value gather reads
+        // (uint8 [256 codes][32 slots][4])
+        const size_t n = (size_t)NOVAKV_C * 32 * NOVAKV_G;
+        std::vector<uint8_t> img(n);
         for (size_t i = 0; i < n; ++i) {
-            const int comp = (int)(i % NOVAKV_G), code = (int)((i / (32 * NOVAKV_G)) % NOVAKV_C);
-            img[i] = __float2half((float)((code >> (2 * comp)) & 3));
+            const int comp = (int)(i % NOVAKV_G), code = (int)(i / (32 * NOVAKV_G));
+            img[i] = (uint8_t)((code >> (2 * comp)) & 3);
         }
-        if (cudaMalloc(&ctx->int2_img, n * sizeof(__half)) != cudaSuccess ||
-            cudaMemcpy(ctx->int2_img, img.data(), n * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess) {
+        if (cudaMalloc(&ctx->int2_img, n) != cudaSuccess ||
+            cudaMemcpy(ctx->int2_img, img.data(), n, cudaMemcpyHostToDevice) != cudaSuccess) {
             cudaFree(ctx->dev_status);
             cudaFree(ctx->int2_img);
             delete ctx;
@@ -82,7 +84,8 @@ static void free_layer(novakv_layer& ly) {
     cudaFree(ly.rk_d); cudaFree(ly.rv_d); cudaFree(ly.k_mean_d); cudaFree(ly.v_mean_d);
     cudaFree(ly.rk_d_mma); cudaFree(ly.rv_d_mma); cudaFree(ly.k_mean);
     cudaFree(ly.cb_k); cudaFree(ly.cb_v); cudaFree(ly.rk_inv_t); cudaFree(ly.rv_t);
-    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_mma);
+    cudaFree(ly.v_mean); cudaFree(ly.cb_k_lut); cudaFree(ly.cb_v_u8); cudaFree(ly.v_scale); cudaFree(ly.v_off);
+    cudaFree(ly.k_mean_eff); cudaFree(ly.k_center);
     ly = novakv_layer();
 }
 
@@ -113,29 +116,35 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
     const int H = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim, L = ctx->n_groups, C = NOVAKV_C, g = NOVAKV_G;
     const size_t n_mat = (size_t)H * d * d, n_vec = (size_t)H * d, n_cb = (size_t)H * L * C * g;
 
-    // value codewords must survive the binary16 round trip exactly
-    // cbv_grp: slot = group (scratch for the image below)
-    std::vector<__half> cbv_grp((size_t)H * C * 32 * g, __float2half(0.f));
-    std::vector<__half> cbv_mma((size_t)H * C * 32 * g, __float2half(0.f));
+    // Value codewords: every coordinate (KV head, group l, component i) must lie on its own 8-bit grid
+    // lo + u (hi - lo) / 255, u = 0 .. 255, with lo / hi the smallest / largest value that coordinate takes over
+    // the 256 codewords (the calibrator snaps them after Lloyd, as the paper snaps its codebooks to a narrow
+    // format offline).  The kernel keeps the indices u (4 bytes per codeword) and applies step and offset once
+    // per output coefficient.  The grid is evaluated in binary64 and rounded to binary32 exactly as below.
+    std::vector<uint8_t> cbv_u8((size_t)H * C * 32 * g, 0);
+    std::vector<float> v_scale((size_t)H * d, 1.f), v_off((size_t)H * d, 0.f);
     for (int hh = 0; hh < H; ++hh)
         for (int l = 0; l < L; ++l)
-            for (int c = 0; c < C; ++c)
-                for (int i = 0; i < g; ++i) {
-                    float x = h->cb_v[(((size_t)hh * L + l) * C + c) * g + i];
-                    __half hx = __float2half_rn(x);
-                    if (!(__half2float(hx) == x)) return NOVAKV_EUNSUPPORTED;
-                    cbv_grp[(((size_t)hh * C + c) * 32 + l) * g + i] = hx;
+            for (int i = 0; i < g; ++i) {
+                float lo = h->cb_v[(((size_t)hh * L + l) * C) * g + i], hi = lo;
+                for (int c = 1; c < C; ++c) {
+                    const float x = h->cb_v[(((size_t)hh * L + l) * C + c) * g + i];
+                    if (!(x == x)) return NOVAKV_EUNSUPPORTED;
+                    lo = x < lo ? x : lo;
+                    hi = x > hi ? x : hi;
                 }
-    // tensor-core value side: slot pos = 16*rho + 4*xb + r' holds group 8*(xb mod NGB) + 4*rho + r'
-    // (NGB = L/8 group blocks; for L = 16 every group appears twice).  The four lanes of an MMA quad
-    // then read four different 8-byte bank pairs whatever codes their tokens carry.
-    for (int hh = 0; hh < H; ++hh)
-        for (int c = 0; c < C; ++c)
-            for (int pos = 0; pos < 32; ++pos) {
-                const int rho = pos >> 4, xb = (pos >> 2) & 3, rp = pos & 3;
-                const int l = 8 * (xb % (L / 8)) + 4 * rho + rp;
-                for (int i = 0; i < g; ++i)
-                    cbv_mma[(((size_t)hh * C + c) * 32 + pos) * g + i] = cbv_grp[(((size_t)hh * C + c) * 32 + l) * g + i];
+                double step = ((double)hi - (double)lo) / 255.0;
+                if (!(step > 0.0) || !(step < 1e300)) step = 1.0;
+                for (int c = 0; c < C; ++c) {
+                    const float x = h->cb_v[(((size_t)hh * L + l) * C + c) * g + i];
+                    double u = nearbyint(((double)x - (double)lo) / step);
+                    if (u < 0.0) u = 0.0;
+                    if (u > 255.0) u = 255.0;
+                    if ((float)((double)lo + step * u) != x) return NOVAKV_EUNSUPPORTED;
+                    cbv_u8[(((size_t)hh * C + c) * 32 + l) * g + i] = (uint8_t)u;
+                }
+                v_scale[(size_t)hh * d + l * g + i] = (float)step;
+                v_off[(size_t)hh * d + l * g + i] = (float)((double)lo + 128.0 * step);
             }
 
     std::vector<double> rk_d(n_mat), rv_d(n_mat), km_d(n_vec, 0.0), vm_d(n_vec, 0.0);
@@ -153,20 +162,32 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
     if (h->k_mean) for (size_t i = 0; i < n_vec; ++i) { km_d[i] = (double)h->k_mean[i]; km_f[i] = h->k_mean[i]; }
     if (h->v_mean) for (size_t i = 0; i < n_vec; ++i) { vm_d[i] = (double)h->v_mean[i]; vm_f[i] = h->v_mean[i]; }
 
-    // key codebook in score-table order: [Hkv][plane][code][e = (m%2)*8 + sigma][4],
-    // group l = sigma*GPS + plane*2 + (m%2), GPS = L/8 groups per slot.
-    const int GPS = L / 8, planes = GPS / 2;
-    std::vector<float> cbk_lut((size_t)H * planes * C * 16 * g);
+    // Key codebook in score-table order [Hkv][code][l][4], centred: every (group, component) has the midrange of
+    // its 256 codeword values subtracted, which shrinks the table entries (they are kept in binary16).  The
+    // softmax does not see the shift: it moves all logits of a query by the same <q', centre>.
+    std::vector<float> cbk_lut((size_t)H * C * L * g), kcen((size_t)H * d, 0.f), km_eff(n_vec, 0.f);
     for (int hh = 0; hh < H; ++hh)
-        for (int pl = 0; pl < planes; ++pl)
-            for (int c = 0; c < C; ++c)
-                for (int e = 0; e < 16; ++e) {
-                    int sigma = e & 7, mpar = e >> 3;
-                    int l = sigma * GPS + pl * 2 + mpar;
-                    for (int i = 0; i < g; ++i)
-                        cbk_lut[((((size_t)hh * planes + pl) * C + c) * 16 + e) * g + i] =
-                            h->cb_k[(((size_t)hh * L + l) * C + c) * g + i];
+        for (int l = 0; l < L; ++l)
+            for (int i = 0; i < g; ++i) {
+                float lo = h->cb_k[(((size_t)hh * L + l) * C) * g + i], hi = lo;
+                for (int c = 1; c < C; ++c) {
+                    const float x = h->cb_k[(((size_t)hh * L + l) * C + c) * g + i];
+                    lo = x < lo ? x : lo;
+                    hi = x > hi ? x : hi;
                 }
+                const float cen = (float)(0.5 * ((double)lo + (double)hi));
+                kcen[(size_t)hh * d + l * g + i] = cen;
+                for (int c = 0; c < C; ++c)
+                    cbk_lut[(((size_t)hh * C + c) * L + l) * g + i] =
+                        (float)((double)h->cb_k[(((size_t)hh * L + l) * C + c) * g + i] - (double)cen);
+            }
+    // what the centred table drops from a logit, <q rk_inv_t, centre> = q . (rk_inv_t centre^T), joins q . k_mean
+    for (int hh = 0; hh < H; ++hh)
+        for (int r = 0; r < d; ++r) {
+            double acc = km_d[(size_t)hh * d + r];
+            for (int c = 0; c < d; ++c) acc += (double)h->rk_inv_t[((size_t)hh * d + r) * d + c] * (double)kcen[(size_t)hh * d + c];
+            km_eff[(size_t)hh * d + r] = (float)acc;
+        }
 
     CUDA_OK(cudaSetDevice(ctx->cfg.device));
     novakv_layer& ly = ctx->layers[layer];
@@ -182,7 +203,9 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
               upload(&ly.cb_k, cbk) == cudaSuccess && upload(&ly.cb_v, cbv) == cudaSuccess &&
               upload(&ly.rk_inv_t, rkinv) == cudaSuccess && upload(&ly.rv_t, rvt) == cudaSuccess &&
               upload(&ly.v_mean, vm_f) == cudaSuccess && upload(&ly.k_mean, km_f) == cudaSuccess && upload(&ly.cb_k_lut, cbk_lut) == cudaSuccess &&
-              upload(&ly.cb_v_mma, cbv_mma) == cudaSuccess;
+              upload(&ly.cb_v_u8, cbv_u8) == cudaSuccess && upload(&ly.v_scale, v_scale) == cudaSuccess &&
+              upload(&ly.v_off, v_off) == cudaSuccess && upload(&ly.k_mean_eff, km_eff) == cudaSuccess &&
+              upload(&ly.k_center, kcen) == cudaSuccess;
     if (!ok) { free_layer(ly); return NOVAKV_ECUDA; }
     ly.loaded = true;
     return NOVAKV_OK;

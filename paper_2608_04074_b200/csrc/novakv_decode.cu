@@ -5,22 +5,33 @@
 //   stage 1  : persistent scan kernel, one CTA per SM.  Each CTA takes a contiguous range of the
 //              global page sequence, so that consecutive pages mostly belong to the same
 //              (sequence, KV head) and reuse its score table.  Per (sequence, KV head) segment:
-//                - score table LUT[h][l][c] = <q'_h[4l..4l+3], cb_k[l][c]> in shared memory (fp32),
+//                - score table LUT[code][l][h] = <q'_h[4l..4l+3], cb_k[l][code] - centre_l> in shared memory,
+//                  all heads of the KV head side by side in one entry.  The first K32 groups, which carry
+//                  the high-variance coordinates and hence the large entries, are kept in binary32; the
+//                  others (head dimension 128 only) in binary16,
 //                - every warp streams its own 32-token tiles with coalesced 128-bit loads straight into
 //                  registers, the next tile's loads in flight while the current tile is consumed (the
 //                  cache layout is such that each lane's bytes are exactly the ones it consumes),
-//                - key side: lane <-> token, 32 table lookups summed in registers (no cross-lane
-//                  reduction), online softmax per 32-token tile,
+//                - key side: lane <-> token, L table lookups summed in registers (no cross-lane
+//                  reduction): binary32 adds for the binary32 entries, short binary16 chains, each
+//                  flushed into the binary32 sum, for the others,
+//                - online softmax per 32-token tile with a lazily updated running maximum,
 //                - value side: sum_j p_j * value-codeword_j in the value-transform domain, a dense
-//                  [heads x tokens] x [tokens x d] contraction, run on tensor cores (mma.sync, fp16
-//                  operands, fp32 accumulators) or, as the selectable alternative, on CUDA cores in fp32,
+//                  [heads x tokens] x [tokens x d] contraction, run on tensor cores (mma.sync, binary16
+//                  operands, binary32 accumulators) or, as the selectable alternative, on CUDA cores in
+//                  binary32; value codewords are 8-bit grid indices (4 bytes per codeword) that expand to
+//                  binary16 with one byte permutation per pair,
 //                - the warps' partial (m, l, acc) are merged and written once per segment.
 //   merge    : exact log-sum-exp merge of the partials of every (sequence, KV head), then the inverse
 //              value transform o = o' rv^T + v_mean, once per head.
 //
-// Shared-memory gathers are laid out so that they never bank-conflict: on the key side the 8 lanes of a
-// quarter warp always address 8 different 16-byte bank groups of the table ("slots"); on the value
-// side the 16 lanes of a half warp address 16 different 8-byte slots of a codebook row.
+// Shared-memory gathers are laid out against bank conflicts: byte j of a token's key bytes holds group
+// j ^ (token % 8) (j ^ (token % 16) for j >= 16), so that at every step the lanes of a quarter warp read 8
+// different 16-byte columns of a binary32 table row and the lanes of a half warp 16 different 8-byte
+// columns of a binary16 row (8 for steps 8..15: a two-way conflict on those 8 of 32 steps); on the value
+// side the 32 lanes of a warp read 32 different 4-byte slots, because the lane columns fc = 0,1 and fc = 2,3
+// use two copies of the value codebook whose slots are rotated by 16, and odd columns take the group
+// blocks in swapped order.
 // The kernel contains no spin wait.
 #include <math_constants.h>
 
@@ -29,12 +40,21 @@
 namespace {
 
 #ifndef NOVAKV_NCW
-#define NOVAKV_NCW 12
+#define NOVAKV_NCW 16
+#endif
+#ifndef NOVAKV_CHAIN
+#define NOVAKV_CHAIN 4        // table lookups summed in binary16 before a flush into the binary32 logit
+#endif
+#ifndef NOVAKV_WINDOW
+#define NOVAKV_WINDOW 8       // tiles whose tensor-core sums are accumulated before the offset of the 8-bit grid is removed
 #endif
 constexpr int NCW = NOVAKV_NCW;               // warps of the scan kernel
 constexpr int S1_THREADS = NCW * 32;
-constexpr int LUT_PLANE_BYTES = 256 * 256;    // 256 codes x 16 entries x 16 bytes
-constexpr int VCB_BYTES = 256 * 256;          // 256 codes x 32 slots x 4 halves
+constexpr int T16_BYTES = 65536;              // binary16 table: 256 codes x 256-byte rows
+constexpr int T16_ROW = 256;
+constexpr int VCB_COPY_BYTES = 32768;         // 256 codes x 32 slots x 4 bytes
+constexpr int VCB_ROW = 128;
+constexpr int S1_SMEM_BYTES = 229376;         // dynamic shared memory requested (224 KB; the CTA also has a few static words)
 constexpr float M_INIT = -1.0e30f;
 
 // VM selects the value side: true = tensor cores (mma.sync m16n8k16, fp16 weights and codewords,
@@ -42,29 +62,38 @@ constexpr float M_INIT = -1.0e30f;
 template <int D, int HG, bool VM>
 struct S1 {
     static constexpr int L = D / NOVAKV_G;
-    static constexpr int GPS = L / 8;                         // groups per slot: 4 (d=128) or 2 (d=64)
-    static constexpr int PLANES = GPS / 2;                    // 64 KB planes of the score table per head set
     static constexpr int NGB = L / 8;                         // group blocks of 8 groups (value side)
     static constexpr int KPL = L / 16;                        // 16-byte planes of a key tile: 2 or 1
-    static constexpr int HSETS = HG <= 4 ? 1 : 2;             // table entries are 4 heads wide
+    static constexpr int HSETS = HG <= 4 ? 1 : 2;             // sets of 4 heads
     static constexpr int HPAD = HSETS * 4;
+    // Score table.  Groups 0 .. K32-1 (the equal-volume dealing puts the coordinates of largest variance there)
+    // have binary32 entries, 16 bytes per head set: T32[hs][code][K32][4 heads].  The other groups have
+    // binary16 entries, 8 bytes: T16[code][32 columns][4 heads], rows of 256 bytes (only for d = 128, where
+    // Hq/Hkv <= 4).  For d = 64 every group is binary32.
+    static constexpr int K32 = D == 128 ? 8 : L;
+    static constexpr bool HAS16 = K32 < L;
+    static_assert(!HAS16 || HSETS == 1, "binary16 entries hold one head set");
+    static constexpr int ROW32 = K32 * 16;
+    static constexpr int PLANE32 = 256 * ROW32;
+    static constexpr int T32_BYTES = HSETS * PLANE32;
     static constexpr int TILE_BYTES = 32 * L;                 // index bytes of a 32-token tile, K or V
-    static constexpr int LUT_BYTES = HSETS * PLANES * LUT_PLANE_BYTES;
     // per-warp staging of the softmax weights of one 32-token tile
     //   VM: fp16 [HPAD][4 k-slot pairs][8 tokens]        otherwise: fp32 [32 tokens][HPAD]
     static constexpr int P_WARP_BYTES = VM ? HPAD * 64 : 32 * HPAD * 4;
     static constexpr int P_BYTES = NCW * P_WARP_BYTES;
-    static constexpr int OFF_LUT = 0;
-    static constexpr int OFF_VCB = OFF_LUT + LUT_BYTES;
-    static constexpr int OFF_P = OFF_VCB + VCB_BYTES;
-    static constexpr int OFF_BAR = OFF_P + P_BYTES;
-    static constexpr int SMEM = OFF_BAR + 64;
-    // merge buffer (aliases the table once a segment's scan is done); the CUDA-core value side keeps
-    // one partial per lane column (4 per warp)
-    static constexpr int MERGE_SLOTS = VM ? NCW : NCW * 4;
-    static constexpr int MERGE_ACC_BYTES = MERGE_SLOTS * HPAD * D * 4;
-    static_assert(MERGE_ACC_BYTES + NCW * HPAD * 12 <= LUT_BYTES, "merge buffer must fit in the table");
-    static_assert(SMEM <= 232448, "shared memory budget");
+    // Shared-memory map.  Below the binary16 table: T32, the weight staging, q' of the pair.  The binary16 table
+    // sits at the first 64 KB boundary of the shared address window that leaves that much room (a row then
+    // starts at an address whose low 16 bits are code * 256, so that one byte permutation builds a gather
+    // address); without a binary16 table nothing needs aligning.  The two copies of the value codebook follow.
+    static constexpr int OFFB_T32 = 0;
+    static constexpr int OFFB_P = OFFB_T32 + T32_BYTES;
+    static constexpr int OFFB_Q = OFFB_P + P_BYTES;                     // fp32 [HPAD][D]
+    static constexpr int BELOW_BYTES = OFFB_Q + HPAD * D * 4;
+    // merge buffer (aliases the larger table once a segment's scan is done)
+    static constexpr int MERGE_ACC_BYTES = NCW * HPAD * D * 4;
+    static_assert(MERGE_ACC_BYTES + NCW * HPAD * 16 <= (HAS16 ? T16_BYTES : T32_BYTES), "merge buffer must fit in a table");
+    static_assert(BELOW_BYTES + (HAS16 ? T16_BYTES : 0) + 2 * VCB_COPY_BYTES <= S1_SMEM_BYTES, "shared memory budget (before alignment)");
+    static_assert(S1_THREADS % L == 0, "table build mapping");
 };
 
 __device__ __forceinline__ float warp_sum_f(float v) {
@@ -89,7 +118,8 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                       int max_pages_per_seq, float scale_log2, float* __restrict__ qp,
                       int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status,
                       const float* __restrict__ k_mean /* [Hkv][D] */, float* __restrict__ qk_off /* [batch][Hq] or null */,
-                      int32_t* __restrict__ cost_prefix /* [batch + 1] */, int seg_weight) {
+                      int32_t* __restrict__ cost_prefix /* [batch + 1] */, int seg_weight,
+                      const float* __restrict__ k_center /* [Hkv][D], transform domain */, float* __restrict__ qc /* [batch][Hq] or null */) {
     const int blk = blockIdx.x;
     constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
@@ -158,10 +188,12 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         float v = 0.f;
 #pragma unroll
         for (int p = 0; p < PARTS; ++p) v += red_s[p][h][cc];
-        qp[((size_t)b * n_q_heads + kvh * HG + h) * D + cc] = v * scale_log2;
+        v *= scale_log2;
+        qp[((size_t)b * n_q_heads + kvh * HG + h) * D + cc] = v;
+        if (qc != nullptr) red_s[0][h][cc] = v * k_center[(size_t)kvh * D + cc];       // (each thread rewrites only what it read)
     }
     // the constant the read path drops from every logit of a query, q . k_mean * sm_scale (base-2 units):
-    // only a learned sink logit needs it (it must be shifted by the same amount)
+    // only a learned sink logit and the BF16 band need it (they must be shifted by the same amount)
     if (qk_off != nullptr && (threadIdx.x >> 5) < HG) {
         const int h = threadIdx.x >> 5, lane = threadIdx.x & 31;
         float acc = 0.f;
@@ -169,22 +201,36 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         acc = warp_sum_f(acc);
         if (lane == 0) qk_off[(size_t)b * n_q_heads + kvh * HG + h] = acc * scale_log2;
     }
+    // scaled key format: the table is built from centred codewords, and the centre's share <q', centre> of
+    // every logit is added back before the per-token scale multiplies it
+    if (qc != nullptr) {
+        __syncthreads();
+        if ((threadIdx.x >> 5) < HG) {
+            const int h = threadIdx.x >> 5, lane = threadIdx.x & 31;
+            float acc = 0.f;
+            for (int i = lane; i < D; i += 32) acc += red_s[0][h][i];
+            acc = warp_sum_f(acc);
+            if (lane == 0) qc[(size_t)b * n_q_heads + kvh * HG + h] = acc;
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
 // stage 1 helpers
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void lds_2x64(uint32_t addr, uint64_t& a, uint64_t& b) {
-    asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr));
+__device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ uint4 lds_u128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
@@ -205,6 +251,22 @@ __device__ __forceinline__ void ffma2(uint64_t& d, uint64_t a, uint64_t b) {
 __device__ __forceinline__ void fmul2(uint64_t& d, uint64_t a) {
     asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(d) : "l"(a));
 }
+// packed binary16 pairs
+__device__ __forceinline__ uint32_t hadd2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("add.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// lo += low half of h, hi += high half of h (binary16 widened exactly, binary32 addition)
+__device__ __forceinline__ void flush_h2(uint32_t h, float& lo, float& hi) {
+    asm("{\n\t.reg .b16 l, u;\n\tmov.b32 {l, u}, %2;\n\tadd.rn.f32.f16 %0, l, %0;\n\tadd.rn.f32.f16 %1, u, %1;\n\t}"
+        : "+f"(lo), "+f"(hi) : "r"(h));
+}
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -221,6 +283,11 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 struct Segment {
@@ -268,75 +335,83 @@ __device__ __forceinline__ uint2 ldg_stream_64(const void* p) {
     return v;
 }
 
-// 64 KB image (the value codebook of a KV head) -> shared memory, without registers: asynchronous 16-byte
+// Value codebook of a KV head (32 KB image, uint8 [256 codes][32 slots][4], slot = group) -> two copies in
+// shared memory, copy c holding group g in slot (g + 16 c) % 32, without registers: asynchronous 16-byte
 // copies that land while the caller does other work (segment lookup, page ids, table build);
-// async_copies_wait() before the barrier that publishes the image.
-__device__ __forceinline__ void stage_image_64k_async(unsigned char* dst_smem, const void* __restrict__ src_g) {
-    const uint32_t dst = smem_u32(dst_smem);
-    const char* src = reinterpret_cast<const char*>(src_g);
-    for (int i = threadIdx.x; i < VCB_BYTES / 16; i += S1_THREADS)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * 16), "l"(src + (size_t)i * 16) : "memory");
+// async_copies_wait() before the barrier that publishes the copies.  A 16-byte chunk holds 4 slots, so the
+// rotation by 16 slots moves whole chunks.  INTERLEAVED: the two copies share 256-byte rows
+// [code][copy][32 slots] (a row then starts at code * 256 of a 64 KB block); otherwise copy 1 follows copy 0.
+template <bool INTERLEAVED>
+__device__ __forceinline__ void stage_value_codebook_async(unsigned char* vcb, const uint8_t* __restrict__ src_g) {
+    const uint32_t d0 = smem_u32(vcb);
+    for (int i = threadIdx.x; i < VCB_COPY_BYTES / 16; i += S1_THREADS) {
+        const int row = i >> 3, ch = i & 7;
+        const uint8_t* src = src_g + (size_t)i * 16;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            const uint32_t dst = d0 + (INTERLEAVED ? row * (2 * VCB_ROW) + c * VCB_ROW : c * VCB_COPY_BYTES + row * VCB_ROW) +
+                                 ((ch + 4 * c) & 7) * 16;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+        }
+    }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 __device__ __forceinline__ void async_copies_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-// The table build is kept out of line so that its register-hungry load batch does not disturb the
-// register allocation of the scan loop.
-// LUT[hs][plane][code][e] = <q'_h segment of group l(e, plane), key codeword> for 4 heads per entry.
+// The table build is kept out of line so that its load batches do not disturb the register allocation of
+// the scan loop.  Entry (code, l, h) = <q'_h segment of group l, centred key codeword (l, code)>, heads beyond
+// HG zero: binary32 in T32 for l < K32, binary16 in T16 otherwise.
 template <int D, int HG, bool VM>
-__device__ __noinline__ void build_score_table(unsigned char* smem,
-                                               const float* __restrict__ cb_k_planes /* key codewords of the KV head, table order */,
-                                               const float* __restrict__ q_pair /* q' of the pair's heads, [HG][D] */) {
+__device__ __noinline__ void build_score_table(unsigned char* t32, unsigned char* t16,
+                                               const float* __restrict__ cb_k_lut /* [256][L][4] of the KV head */,
+                                               const float* q_s /* shared: q' of the pair, [HPAD][D] */) {
     using C = S1<D, HG, VM>;
-    constexpr int GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, PLANES = C::PLANES;
-    constexpr int CPI = NCW * 2;                                   // codes per iteration (16 entries each)
-    constexpr int NIT = (256 + CPI - 1) / CPI;
-    const int e = threadIdx.x & 15, code0 = threadIdx.x >> 4;
-    const int sigma = e & 7, mpar = e >> 3;
-    const float4* cbk = reinterpret_cast<const float4*>(cb_k_planes);
-    // every load of the thread (query segments and codewords of all planes) is issued before the first
-    // use: one memory latency for the whole table
-    float4 qseg[PLANES][HPAD];                    // heads beyond HG are zero
-    float4 cwv[PLANES][NIT];
+    constexpr int L = C::L, HPAD = C::HPAD, HSETS = C::HSETS, K32 = C::K32;
+    constexpr int CSTEP = S1_THREADS / L;                       // codes per pass of the CTA
+    constexpr int NIT = (256 + CSTEP - 1) / CSTEP;
+    constexpr int BATCH = 8;                                    // loads in flight per thread
+    const int g = threadIdx.x % L, code0 = threadIdx.x / L;
+    float4 qs[HPAD];
 #pragma unroll
-    for (int pl = 0; pl < PLANES; ++pl) {
-        const int l = sigma * GPS + pl * 2 + mpar;
+    for (int h = 0; h < HPAD; ++h) qs[h] = *reinterpret_cast<const float4*>(q_s + h * D + g * 4);
+    const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut);
+#pragma unroll 1
+    for (int it0 = 0; it0 < NIT; it0 += BATCH) {
+        float4 cw[BATCH];
 #pragma unroll
-        for (int h = 0; h < HPAD; ++h)
-            qseg[pl][h] = h < HG ? *reinterpret_cast<const float4*>(q_pair + h * D + l * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int code = code0 + it * CPI;
-            if (code < 256) cwv[pl][it] = cbk[((size_t)pl * 256 + code) * 16 + e];
+        for (int u = 0; u < BATCH; ++u) {
+            const int code = code0 + (it0 + u) * CSTEP;
+            if (it0 + u < NIT && code < 256) cw[u] = cbk[(size_t)code * L + g];
         }
-    }
 #pragma unroll
-    for (int pl = 0; pl < PLANES; ++pl)
+        for (int u = 0; u < BATCH; ++u) {
+            const int code = code0 + (it0 + u) * CSTEP;
+            if (it0 + u < NIT && code < 256) {
+                float o[HPAD];
 #pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int code = code0 + it * CPI;
-            if (code < 256) {
-                const float4 cw = cwv[pl][it];
+                for (int h = 0; h < HPAD; ++h)
+                    o[h] = fmaf(qs[h].w, cw[u].w, fmaf(qs[h].z, cw[u].z, fmaf(qs[h].y, cw[u].y, qs[h].x * cw[u].x)));
+                if (g < K32) {
 #pragma unroll
-                for (int hs = 0; hs < HSETS; ++hs) {
-                    const float4* q = &qseg[pl][hs * 4];
-                    float4 o;
-                    o.x = fmaf(q[0].w, cw.w, fmaf(q[0].z, cw.z, fmaf(q[0].y, cw.y, q[0].x * cw.x)));
-                    o.y = fmaf(q[1].w, cw.w, fmaf(q[1].z, cw.z, fmaf(q[1].y, cw.y, q[1].x * cw.x)));
-                    o.z = fmaf(q[2].w, cw.w, fmaf(q[2].z, cw.z, fmaf(q[2].y, cw.y, q[2].x * cw.x)));
-                    o.w = fmaf(q[3].w, cw.w, fmaf(q[3].z, cw.z, fmaf(q[3].y, cw.y, q[3].x * cw.x)));
-                    *reinterpret_cast<float4*>(smem + C::OFF_LUT + (hs * PLANES + pl) * LUT_PLANE_BYTES + code * 256 + e * 16) = o;
+                    for (int hs = 0; hs < HSETS; ++hs)
+                        *reinterpret_cast<float4*>(t32 + hs * C::PLANE32 + code * C::ROW32 + g * 16) =
+                            make_float4(o[hs * 4], o[hs * 4 + 1], o[hs * 4 + 2], o[hs * 4 + 3]);
+                } else if (C::HAS16) {
+                    // (a table entry beyond the binary16 range would be a logit share of 2^16 bits; clamped, never inf)
+                    *reinterpret_cast<uint2*>(t16 + code * T16_ROW + g * 8) =
+                        make_uint2(pack_h2(fminf(fmaxf(o[0], -60000.f), 60000.f), fminf(fmaxf(o[1], -60000.f), 60000.f)),
+                                   pack_h2(fminf(fmaxf(o[2], -60000.f), 60000.f), fminf(fmaxf(o[3], -60000.f), 60000.f)));
                 }
             }
         }
+    }
 }
 
 // Index bytes of one 32-token tile as one lane holds them.
-//   kw: this lane's token (lane = token within the tile), L bytes in rotated slot order: position j
-//       holds slot (j + lane%8 + lane/8) % 8, so that step j of every lane reads a different slot.
+//   kw: this lane's token (lane = token within the tile), L bytes: byte j holds the code of group
+//       j ^ (lane % 8) for j < 16 and j ^ (lane % 16) for j >= 16.
 //   vw: per 16-token block, the codes of this lane's MMA coordinates (fr = lane/4, fc = lane%4):
-//       word x holds, for the four tokens 8ts + 4u + fc (byte 2ts+u), the code of group
-//       8*((x + fc) % NGB) + fr.
+//       word gb holds, for the four tokens 4u + fc of the block (byte u), the code of group 8 gb + fr.
 template <int L>
 struct TileRegs {
     uint32_t kw[L / 4];
@@ -346,37 +421,70 @@ struct TileRegs {
 };
 
 // KSC: the key format carries a per-token bfloat16 scale (k_scales [n_pages][Hkv][64]); the logits of a
-// token are multiplied by it once, after the table lookups are summed.
+// token are multiplied by it once, after the table lookups are summed (and the centre's share added back).
 // VSQ: scalar INT2 values with a per-token bfloat16 scale and zero-point (v_meta [n_pages][Hkv][64][2]).
 // A byte of four 2-bit codes indexes the product codebook {0,1,2,3}^4, so the value side is the same gather
-// with that fixed table as cb_v_img; the weight of a token's codes is p * scale and the zero-points enter
-// through one extra running sum per head, sum_j p_j zero_j, added to every coefficient in the epilogue.
+// with that fixed table as the value-codebook image; the weight of a token's codes is p * scale and the
+// zero-points enter through one extra running sum per head, sum_j p_j zero_j, added to every coefficient
+// in the epilogue.
+//
+// Numerics of the tensor-core value side.  A softmax weight enters the product as the binary16 number
+// w = fp16(2^15 p) (p <= 1 relative to the running maximum, so w <= 2^15; weights down to 2^-39 stay
+// non-zero), and the same rounded w is what the normaliser sums: the result is an exact softmax of slightly
+// perturbed logits.  A value codeword is four 8-bit grid indices u; the byte permutation that widens them
+// yields the binary16 numbers 1024 + u, so an accumulator gains sum_j w_j (1024 + u_j).  Every NOVAKV_WINDOW
+// tiles, and before any rescaling, that offset is removed with the weight sum of the same tokens, which the
+// tensor core accumulates beside the products (an all-ones operand): acc -= 1152 sum_j w_j leaves
+// sum_j w_j (u_j - 128), so that the long-running sums stay centred and small.
 template <int D, int HG, bool VM, bool KSC, bool VSQ>
 __global__ void __launch_bounds__(S1_THREADS, 1)
 novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restrict__ cb_k_lut,
-                            const __half* __restrict__ cb_v_img, const uint8_t* __restrict__ k_pages,
+                            const uint8_t* __restrict__ cb_v_img, const float* __restrict__ v_scale,
+                            const float* __restrict__ v_off, const uint8_t* __restrict__ k_pages,
                             const uint8_t* __restrict__ v_pages, const __nv_bfloat16* __restrict__ k_scales,
                             const __nv_bfloat16* __restrict__ v_meta, int n_pages,
                             const int32_t* __restrict__ page_table, int max_pages_per_seq,
                             const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ page_prefix,
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
                             float* __restrict__ part_acc, uint32_t* __restrict__ dev_status, int pt_stride,
-                            const int32_t* __restrict__ cost_prefix, int seg_weight, long* __restrict__ cta_range) {
+                            const int32_t* __restrict__ cost_prefix, int seg_weight, long* __restrict__ cta_range,
+                            const float* __restrict__ qc, int vcb_per_head) {
     // page_table points at the first column that is scanned; rows are pt_stride entries apart and
     // max_pages_per_seq bounds the pages of a row that may be read from there
     using C = S1<D, HG, VM>;
-    constexpr int L = C::L, GPS = C::GPS, HPAD = C::HPAD, HSETS = C::HSETS, NGB = C::NGB, KPL = C::KPL;
+    constexpr int L = C::L, HPAD = C::HPAD, HSETS = C::HSETS, NGB = C::NGB, KPL = C::KPL, K32 = C::K32;
+    constexpr bool HAS16 = C::HAS16;
     constexpr int TILE_BYTES = C::TILE_BYTES, PAGE_BYTES = 2 * TILE_BYTES;
+    constexpr float SH = VM ? 15.f : 0.f;                     // weights are scaled by 2^SH before the binary16 rounding
+    constexpr float CEN = VSQ ? 1024.f : 1152.f;              // what one unit of weight adds to a tensor-core sum beyond u - centre
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_found[4];
+    __shared__ long s_bnd[2];
+    // ---- shared-memory map (see S1)
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t t16_abs = HAS16 ? ((s_base + C::BELOW_BYTES + 65535u) & ~65535u) : s_base + C::BELOW_BYTES;
+    const uint32_t pad = t16_abs - s_base;
+    if (pad + (HAS16 ? T16_BYTES : 0) + 2 * VCB_COPY_BYTES > (uint32_t)S1_SMEM_BYTES || (s_base & 255u) != 0u) {
+        // cannot happen with the shared address window of this architecture; reported, never trapped
+        if (threadIdx.x == 0) {
+            atomicOr(dev_status, NOVAKV_DEV_SMEM_LAYOUT);
+            cta_range[blockIdx.x * 2] = 0; cta_range[blockIdx.x * 2 + 1] = 0;
+        }
+        return;
+    }
+    unsigned char* const t32_p = smem + C::OFFB_T32;
+    unsigned char* const t16_p = smem + pad;
+    unsigned char* const vcb_p = t16_p + (HAS16 ? T16_BYTES : 0);
+    const uint32_t vcb_abs = t16_abs + (HAS16 ? T16_BYTES : 0);
+    float* const q_s = reinterpret_cast<float*>(smem + C::OFFB_Q);
+    const uint32_t s_p = s_base + C::OFFB_P;
+
     // With the KV-head-major walk the first KV head of CTA c is floor(c * Hkv / G) whatever the lengths are:
     // its (constant) value codebook starts flowing into shared memory before the grid-dependency wait and
     // lands behind the segment lookup and the first table build.
     int vcb_head = (int)(((long)blockIdx.x * n_kv_heads) / gridDim.x);   // KV head whose value codebook is resident
-    stage_image_64k_async(smem + C::OFF_VCB, cb_v_img + (size_t)vcb_head * (VCB_BYTES / 2));
+    stage_value_codebook_async<HAS16>(vcb_p, cb_v_img + (size_t)vcb_head * vcb_per_head);
     novakv_grid_dependency_wait();
-    const uint32_t s_base = smem_u32(smem);
-    const uint32_t s_lut = s_base + C::OFF_LUT, s_vcb = s_base + C::OFF_VCB, s_p = s_base + C::OFF_P;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // This CTA's range of the walk [u_begin, u_end).  The walk is cut evenly in cost units, cost = pages +
@@ -392,7 +500,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         } else {
             const long cper = cost_prefix[batch], T = cper * n_kv_heads;
             const long t0 = ((long)blockIdx.x * T) / gridDim.x, t1 = ((long)(blockIdx.x + 1) * T) / gridDim.x;
-            __shared__ long s_bnd[2];
             if (threadIdx.x < 2) s_bnd[threadIdx.x] = U;              // a cost point at the very end
             __syncthreads();
             if (cper > 0) {
@@ -413,36 +520,76 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     }
     if (u_begin >= u_end) { async_copies_wait(); return; }
 
-    // per-warp running state
-    float m_run[HPAD], l_run[HPAD];
-    float lz_run[VSQ ? HPAD : 1];                //  VSQ: running sum_j p_j zero_j per head (this lane's tokens)
+    // ---- lane roles and constants
+    const int fr = lane >> 2, fc = lane & 3;          // value side: MMA fragment coordinates
+    // key side: token = lane; its byte j holds group j ^ (lane & 7) (j < 16) or j ^ (lane & 15) (j >= 16).
+    //   binary32 entries (steps j < K32): address = T32 + code * ROW32 + ((j ^ lane%8) * 16): the column part is
+    //     one xor with a constant away from a per-lane word, the row part one multiply-add;
+    //   binary16 entries: address = T16 + code * 256 + ((j ^ mask) * 8) = a byte permutation of (index word,
+    //     column word): the column word holds the column bytes of an even / odd step in bytes 0 / 1 and the
+    //     table's upper address half in bytes 2, 3; stepping to another pair of j is one xor with a constant.
+    const uint32_t col32 = s_base + C::OFFB_T32 + (lane & 7) * 16;
+    const uint32_t colword7 = t16_abs | (uint32_t)((lane & 7) * 8) * 0x0101u;
+    const uint32_t colword15 = t16_abs | (uint32_t)((lane & 15) * 8) * 0x0101u;
+    // value side: lane column fc reads copy fc / 2 of the value codebook; odd columns take the group blocks in
+    // swapped order (x ^ 1), so that the 32 lanes of a gather hit 32 different slots.  With the binary16 table
+    // (d = 128) the codebook block is 64 KB aligned too and its two copies share 256-byte rows, so that a gather
+    // address is one byte permutation of (code word, pos); otherwise address = pos + code * 128.
+    uint32_t pos[NGB];
 #pragma unroll
-    for (int h = 0; h < (VSQ ? HPAD : 1); ++h) lz_run[h] = 0.f;
+    for (int x = 0; x < NGB; ++x) {
+        const uint32_t slot4 = ((8 * (x ^ (fc & 1)) + fr + 16 * (fc >> 1)) & 31) * 4;
+        pos[x] = HAS16 ? (vcb_abs | ((fc >> 1) * VCB_ROW + slot4)) : vcb_abs + (fc >> 1) * VCB_COPY_BYTES + slot4;
+    }
+    // address of the codeword whose code is byte b of word w, for load x
+    auto vaddr = [&](uint32_t w, int b, int x) -> uint32_t {
+        return HAS16 ? __byte_perm(w, pos[x], 0x7604u | (b << 4)) : pos[x] + __byte_perm(w, 0u, 0x4440u | b) * VCB_ROW;
+    };
+    const bool odd_col = fc & 1;
+    // B fragments carry a weight in the low or high half depending on the column parity (fr & 1)
+    const uint32_t sel_b0 = (fr & 1) ? 0x1044u : 0x4410u, sel_b1 = (fr & 1) ? 0x3244u : 0x4432u;
+    const uint32_t s_pw = s_p + warp * C::P_WARP_BYTES;
+
+    // ---- per-warp running state
+    float m_run[HPAD];                           // running maximum of the logits (base 2), the same in every lane
     float macc[HSETS][NGB][4];                   //  VM: lane (fr, fc): head 4 hs + fc, group 8 gb + fr, 4 coefficients
-    uint64_t acc[VM ? 1 : NGB][VM ? 1 : HPAD][2];  // !VM: lane (fr, fc): load x (group 8((x+fc)%NGB)+fr), head, 4 coefficients
+    float eacc[HSETS][4];                        //  VM: weight sums of head 4 hs + fc since the last offset removal (four equal numbers)
+    float l_run[HPAD];                           //  VM: [hs] weight sum of head 4 hs + fc (every lane); else this lane's tokens, per head
+    float lz_run[VSQ ? HPAD : 1];                //  VSQ: running sum_j p_j zero_j per head (this lane's tokens)
+    uint64_t acc[VM ? 1 : NGB][VM ? 1 : HPAD][2];  // !VM: lane (fr, fc): group 8 gb + fr, head, 4 coefficients, its own tokens
+    float esh_pow = 0.f;                         //  VSQ: 2^E with E >= log2 of every value scale seen so far (weights carry 2^-E)
 #pragma unroll
     for (int h = 0; h < HPAD; ++h) { m_run[h] = M_INIT; l_run[h] = 0.f; }
 #pragma unroll
-    for (int hs = 0; hs < HSETS; ++hs)
+    for (int h = 0; h < (VSQ ? HPAD : 1); ++h) lz_run[h] = 0.f;
+#pragma unroll
+    for (int hs = 0; hs < HSETS; ++hs) {
 #pragma unroll
         for (int gb = 0; gb < NGB; ++gb)
 #pragma unroll
             for (int i = 0; i < 4; ++i) macc[hs][gb][i] = 0.f;
 #pragma unroll
+        for (int i = 0; i < 4; ++i) eacc[hs][i] = 0.f;
+    }
+#pragma unroll
     for (int x = 0; x < (VM ? 1 : NGB); ++x)
 #pragma unroll
         for (int h = 0; h < (VM ? 1 : HPAD); ++h) { acc[x][h][0] = 0ull; acc[x][h][1] = 0ull; }
 
-    // lane roles
-    const int q4 = lane >> 3, i8 = lane & 7;          // key side: token = lane, slot rotation i8 + q4
-    const int fr = lane >> 2, fc = lane & 3;          // value side: MMA fragment coordinates
-    // B fragments carry a weight in the low or high half depending on the column parity (fr & 1)
-    const uint32_t sel_b0 = (fr & 1) ? 0x1044u : 0x4410u, sel_b1 = (fr & 1) ? 0x3244u : 0x4432u;
-    // byte offset of this lane's codeword slot in a value-codebook row, per load x
-    uint32_t pos8[NGB];
+    // remove the offset of the 8-bit grid from the sums of the tiles since the last call (tensor-core value side)
+    auto flush_window = [&]() {
 #pragma unroll
-    for (int x = 0; x < NGB; ++x) pos8[x] = (16 * (fr >> 2) + 4 * ((x + fc) & 3) + (fr & 3)) * 8;
-    const uint32_t s_pw = s_p + warp * C::P_WARP_BYTES;
+        for (int hs = 0; hs < HSETS; ++hs) {
+            const float w = eacc[hs][0];
+#pragma unroll
+            for (int gb = 0; gb < NGB; ++gb)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) macc[hs][gb][i] = fmaf(-CEN, w, macc[hs][gb][i]);
+            if (!VSQ) l_run[hs] += w;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) eacc[hs][i] = 0.f;
+        }
+    };
 
     long u = u_begin;
     while (u < u_end) {
@@ -451,8 +598,20 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
         // ---- segment prologue -----------------------------------------------------------------
         if (vcb_head != sg.kvh) {
-            stage_image_64k_async(smem + C::OFF_VCB, cb_v_img + (size_t)sg.kvh * (VCB_BYTES / 2));
+            stage_value_codebook_async<HAS16>(vcb_p, cb_v_img + (size_t)sg.kvh * vcb_per_head);
             vcb_head = sg.kvh;
+        }
+        // q' of the pair's heads -> shared memory (rows beyond HG are zero)
+        for (int i = threadIdx.x; i < HPAD * D / 4; i += S1_THREADS) {
+            const int h = i / (D / 4);
+            const float4 v = h < HG ? reinterpret_cast<const float4*>(qp + ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D)[i]
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+            reinterpret_cast<float4*>(q_s)[i] = v;
+        }
+        float qcen[KSC ? HPAD : 1];
+        if (KSC) {
+#pragma unroll
+            for (int h = 0; h < HPAD; ++h) qcen[h] = h < HG ? qc[(size_t)sg.b * n_q_heads + sg.kvh * HG + h] : 0.f;
         }
 
         // this warp's tiles of the segment: half pages hp = warp, warp + NCW, ...
@@ -469,7 +628,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             return page;
         };
         int ids_cur = load_ids(0), ids_next = load_ids(1);
+        // tiles are loaded in ascending order, one ahead of the tile being consumed
         auto load_tile = [&](int it, TileRegs<L>& t) {
+            if ((it & 31) == 0 && it > 0) { ids_cur = ids_next; ids_next = load_ids((it >> 5) + 1); }
             const int page = __shfl_sync(0xffffffffu, ids_cur, it & 31);
             const int half = (warp + NCW * it) & 1;
             const size_t off = ((size_t)page * n_kv_heads + sg.kvh) * PAGE_BYTES + half * TILE_BYTES;
@@ -500,113 +661,154 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             }
         };
 
-        // ---- score table: LUT[hs][plane][code][e] (4 heads per entry) ----------------------------
-        // (the first tile's loads are issued before, so that they fly during the table build)
-        TileRegs<L> nxt;
-        if (n_it > 0) load_tile(0, nxt);
-        build_score_table<D, HG, VM>(smem, cb_k_lut + (size_t)sg.kvh * C::PLANES * (LUT_PLANE_BYTES / 4),
-                                     qp + ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D);
-        async_copies_wait();
-        __syncthreads();     // table and value codebook complete
-
-        // ---- scan: 32-token tiles, loads of the next tile in flight while this one is consumed ------
-        for (int it = 0; it < n_it; ++it) {
-            const TileRegs<L> cur = nxt;
-            if (((it + 1) & 31) == 0) { ids_cur = ids_next; ids_next = load_ids(((it + 1) >> 5) + 1); }
-            if (it + 1 < n_it) load_tile(it + 1, nxt);
+        // ---- one 32-token tile -------------------------------------------------------------------
+        auto process = [&](const TileRegs<L>& cur, int it) {
             const int hp = warp + NCW * it;
             const int tok0 = (sg.pg0 + (hp >> 1)) * NOVAKV_PAGE_TOKENS + (hp & 1) * 32;
             const int nvalid = min(32, sg.len - tok0);
-            if (nvalid <= 0) continue;
+            if (nvalid <= 0) return;
 
-            // ---- key side: lane <-> token; step j reads slot (i8 + q4 + j) % 8 of the table ---------
-            uint64_t z[HPAD / 2];
+            // ---- key side: lane <-> token; step j gathers the entry of (code_j, group j ^ lane bits) ------
+            float zf[HPAD];
+            {
+                uint64_t z2[HPAD / 2];
 #pragma unroll
-            for (int h = 0; h < HPAD / 2; ++h) z[h] = 0ull;
+                for (int k = 0; k < HPAD / 2; ++k) z2[k] = 0ull;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t sg16 = ((i8 + q4 + j) & 7) * 16;
-                const uint32_t w = GPS == 4 ? cur.kw[j] : cur.kw[j >> 1];
-#pragma unroll
-                for (int mm = 0; mm < GPS; ++mm) {
-                    const int byte = GPS == 4 ? mm : mm + 2 * (j & 1);
-                    // index byte -> bits 8..15, slot offset -> bits 0..7
-                    const uint32_t a = __byte_perm(w, sg16, 0x5504 | (byte << 4)) + s_lut + (mm >> 1) * LUT_PLANE_BYTES + (mm & 1) * 128;
+                for (int j = 0; j < K32; ++j) {
+                    const uint32_t code = __byte_perm(cur.kw[j >> 2], 0u, 0x4440u | (j & 3));
+                    const uint32_t a = (col32 ^ (uint32_t)(j * 16)) + code * C::ROW32;
 #pragma unroll
                     for (int hs = 0; hs < HSETS; ++hs) {
-                        uint64_t e01, e23;
-                        lds_2x64(a + hs * C::PLANES * LUT_PLANE_BYTES, e01, e23);
-                        fadd2(z[hs * 2 + 0], e01);
-                        fadd2(z[hs * 2 + 1], e23);
+                        const uint4 v = lds_u128(a + hs * C::PLANE32);
+                        fadd2(z2[2 * hs], (uint64_t)v.x | ((uint64_t)v.y << 32));
+                        fadd2(z2[2 * hs + 1], (uint64_t)v.z | ((uint64_t)v.w << 32));
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < HPAD / 2; ++k) unpack2(z2[k], zf[2 * k], zf[2 * k + 1]);
+            }
+            if (HAS16) {
+                uint32_t ch[2];
+#pragma unroll
+                for (int j = K32; j < L; ++j) {
+                    const uint32_t cw2 = (j < 16 ? colword7 : colword15) ^ (uint32_t)(((j & ~1) * 8) | (((j | 1) * 8) << 8));
+                    const uint2 v = lds_u64(__byte_perm(cur.kw[j >> 2], cw2, 0x7600u | ((j & 3) << 4) | (4 + (j & 1))));
+                    if ((j - K32) % NOVAKV_CHAIN == 0) { ch[0] = v.x; ch[1] = v.y; }
+                    else { ch[0] = hadd2(ch[0], v.x); ch[1] = hadd2(ch[1], v.y); }
+                    if ((j - K32) % NOVAKV_CHAIN == NOVAKV_CHAIN - 1 || j == L - 1) {
+                        flush_h2(ch[0], zf[0], zf[1]);
+                        flush_h2(ch[1], zf[2], zf[3]);
                     }
                 }
             }
-            // ---- online softmax over the tile (base-2 domain) -----------------------------------------
-            float zf[HPAD];
-#pragma unroll
-            for (int h = 0; h < HPAD / 2; ++h) unpack2(z[h], zf[2 * h], zf[2 * h + 1]);
+            float vscale = 1.f, vzero = 0.f, vsmax = 0.f;     // vsmax: this lane's scale as it enters the running bound (0 beyond the length)
             if (KSC) {
                 const float rho = __uint_as_float(cur.ks);
 #pragma unroll
-                for (int h = 0; h < HPAD; ++h) zf[h] *= rho;
+                for (int h = 0; h < HPAD; ++h) zf[h] = (zf[h] + qcen[h]) * rho;
             }
-            bool rescale = false;
-            float alpha[HPAD];
-            __half ph[HPAD];
+            if (VSQ && lane < nvalid) {
+                // (slots beyond the length hold no metadata; a scale that is not positive and finite counts as 1)
+                vscale = __uint_as_float(cur.vm << 16);
+                vzero = __uint_as_float(cur.vm & 0xffff0000u);
+                if (!(vscale > 0.f && vscale < CUDART_INF_F)) vscale = 1.f;
+                vsmax = vscale;
+            }
+            if (nvalid < 32 && lane >= nvalid) {
 #pragma unroll
-            for (int h = 0; h < HPAD; ++h) {
-                if (lane >= nvalid) zf[h] = -CUDART_INF_F;
-                const float mx = warp_max(zf[h]);
-                const float m_new = fmaxf(m_run[h], mx);
-                alpha[h] = ex2(m_run[h] - m_new);
-                rescale |= (m_new != m_run[h]);
-                m_run[h] = m_new;
-                zf[h] = ex2(zf[h] - m_new);                 // p
-                if (VM) {
-                    // the weight that multiplies the value and the one summed into the normaliser are the
-                    // same fp16-rounded number, so the result is an exact softmax of perturbed logits
-                    ph[h] = __float2half_rn(zf[h]);
-                    zf[h] = __half2float(ph[h]);
+                for (int h = 0; h < HPAD; ++h) zf[h] = -CUDART_INF_F;
+            }
+            // ---- online softmax (base 2): the running maximum moves only when a logit exceeds it ---------
+            {
+                bool up = false;
+#pragma unroll
+                for (int h = 0; h < HPAD; ++h) up |= zf[h] > m_run[h];
+                if (VSQ) up |= vsmax >= esh_pow;
+                if (__any_sync(0xffffffffu, up)) {
+                    if (VM) flush_window();
+                    float alpha[HPAD];
+#pragma unroll
+                    for (int h = 0; h < HPAD; ++h) {
+                        const float m_new = fmaxf(m_run[h], warp_max(zf[h]));
+                        alpha[h] = ex2(m_run[h] - m_new);
+                        m_run[h] = m_new;
+                    }
+                    float vsc = 1.f;                     // VSQ: 2^(E_old - E_new)
+                    if (VSQ) {
+                        // E = exponent of the largest scale so far + 1 (scale < 2^E), an exact power of two
+                        const float smax = warp_max(vsmax);
+                        const float e_new = __uint_as_float((__float_as_uint(smax) & 0x7f800000u) + 0x00800000u);
+                        if (e_new > esh_pow) { vsc = esh_pow / e_new; esh_pow = e_new; }
+                    }
+                    if (VM) {
+#pragma unroll
+                        for (int hs = 0; hs < HSETS; ++hs) {
+                            const float a01 = fc & 1 ? alpha[hs * 4 + 1] : alpha[hs * 4 + 0];
+                            const float a23 = fc & 1 ? alpha[hs * 4 + 3] : alpha[hs * 4 + 2];
+                            const float al = fc & 2 ? a23 : a01;
+#pragma unroll
+                            for (int gb = 0; gb < NGB; ++gb)
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) macc[hs][gb][i] *= al * vsc;
+                            if (!VSQ) l_run[hs] *= al;
+                        }
+                        if (VSQ) {
+#pragma unroll
+                            for (int h = 0; h < HPAD; ++h) { l_run[h] *= alpha[h]; lz_run[h] *= alpha[h]; }
+                        }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < HPAD; ++h) {
+                            const uint64_t a2 = pack2(alpha[h], alpha[h]);
+#pragma unroll
+                            for (int x = 0; x < NGB; ++x) { fmul2(acc[VM ? 0 : x][VM ? 0 : h][0], a2); fmul2(acc[VM ? 0 : x][VM ? 0 : h][1], a2); }
+                            l_run[h] *= alpha[h];
+                        }
+                    }
                 }
-                if (VSQ) {
-                    // INT2 values: the tensor-core product needs the weight of the token's integer codes,
-                    // w = p * scale, in binary16.  As for p above, the rounding must not separate numerator and
-                    // normaliser: the weight that counts is p' = fp16(p * scale) / scale, used for the
-                    // normaliser and for the zero-point sum as well (an exact softmax of perturbed logits).
-                    const float vscale = __uint_as_float(cur.vm << 16), vzero = __uint_as_float(cur.vm & 0xffff0000u);
-                    ph[h] = __float2half_rn(zf[h] * vscale);
-                    zf[h] = lane < nvalid ? __fdividef(__half2float(ph[h]), vscale) : 0.f;   // (slots beyond the length hold no metadata)
-                    lz_run[h] = fmaf(lz_run[h], alpha[h], zf[h] * vzero);
+            }
+            // weights
+            uint32_t ph[HPAD / 2];
+            if (VSQ) {
+                // INT2 values: the tensor-core product needs the weight of the token's integer codes,
+                // w = p * scale (times 2^15 / 2^E), in binary16.  The rounding must not separate numerator and
+                // normaliser: the weight that counts is p' = fp16(w) / (scale 2^-E), used for the normaliser and
+                // for the zero-point sum as well (an exact softmax of perturbed logits).
+                const float wmul = __fdividef(vscale, esh_pow), winv = __fdividef(esh_pow, vscale);
+#pragma unroll
+                for (int h = 0; h < HPAD; h += 2) {
+                    const float w0 = ex2(zf[h] - m_run[h] + SH) * wmul, w1 = ex2(zf[h + 1] - m_run[h + 1] + SH) * wmul;
+                    ph[h / 2] = pack_h2(w0, w1);
+                    const float2 wf = __half22float2(*reinterpret_cast<const __half2*>(&ph[h / 2]));
+                    const float p0 = wf.x * winv, p1 = wf.y * winv;
+                    l_run[h] += p0; l_run[h + 1] += p1;
+                    lz_run[h] = fmaf(p0, vzero, lz_run[h]); lz_run[h + 1] = fmaf(p1, vzero, lz_run[h + 1]);
                 }
-                l_run[h] = fmaf(l_run[h], alpha[h], zf[h]);
+            } else if (VM) {
+#pragma unroll
+                for (int h = 0; h < HPAD; h += 2)
+                    ph[h / 2] = pack_h2(ex2(zf[h] - m_run[h] + SH), ex2(zf[h + 1] - m_run[h + 1] + SH));
+            } else {
+#pragma unroll
+                for (int h = 0; h < HPAD; ++h) { zf[h] = ex2(zf[h] - m_run[h]); l_run[h] += zf[h]; }
             }
 
             if (VM) {
                 // ---- value side on tensor cores ---------------------------------------------------------
                 // D[m][n] += sum_k A[m][k] B[k][n], m16 n8 k16, per 8-token sub-tile and group block gb:
                 //   k = (token j of the sub-tile, sub-coefficient i in {0,1}),
-                //   A[m][(j,i)] = codeword(token j, group 8gb + (m & 7))[2 (m >> 3) + i]      fp16
-                //   B[(j,i)][(h,i')] = p_h(token j) * [i == i']                                fp16
+                //   A[m][(j,i)] = 1024 + grid index of codeword(token j, group 8gb + (m & 7))[2 (m >> 3) + i]     fp16
+                //   B[(j,i)][(h,i')] = w_h(token j) * [i == i']                                                fp16
                 //   D[m][(h,i')] = partial of head h, group 8gb + (m & 7), coefficient 2 (m >> 3) + i'
-                if (rescale) {
-#pragma unroll
-                    for (int hs = 0; hs < HSETS; ++hs) {
-                        const float a01 = fc & 1 ? alpha[hs * 4 + 1] : alpha[hs * 4 + 0];
-                        const float a23 = fc & 1 ? alpha[hs * 4 + 3] : alpha[hs * 4 + 2];
-                        const float al = fc & 2 ? a23 : a01;
-#pragma unroll
-                        for (int gb = 0; gb < NGB; ++gb)
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) macc[hs][gb][i] *= al;
-                    }
-                }
                 // weights -> shared memory as fp16, [head][k-slot pair = token & 3][token >> 3, (token >> 2) & 1]
                 __syncwarp();      // previous tile's readers of the P area are done
                 {
                     const uint32_t wa = s_pw + (lane & 3) * 16 + ((lane >> 3) * 2 + ((lane >> 2) & 1)) * 2;
 #pragma unroll
                     for (int h = 0; h < HPAD; ++h)
-                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + h * 64), "h"(__half_as_ushort(ph[h])) : "memory");
+                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(wa + h * 64),
+                                     "h"((unsigned short)((h & 1) ? (ph[h / 2] >> 16) : (ph[h / 2] & 0xffffu))) : "memory");
                 }
                 __syncwarp();
                 // B-fragment sources: 8 weights of head (4 hs + fr/2) for the tokens with (token & 3) == fc
@@ -617,65 +819,36 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
                     for (int ts = 0; ts < 2; ++ts) {                       // 8-token sub-tiles of the block
-                        // gather: X[x][u] = codeword (token 8ts + 4u + fc, group of load x), 2 registers each
-                        uint32_t X[NGB][2][2];
-#pragma unroll
-                        for (int x = 0; x < NGB; ++x)
-#pragma unroll
-                            for (int uu = 0; uu < 2; ++uu) {
-                                const uint32_t a = __byte_perm(cur.vw[blk][x], pos8[x], 0x5504 | ((2 * ts + uu) << 4)) + s_vcb;
-                                const uint2 cw = lds_u64(a);
-                                X[x][uu][0] = cw.x; X[x][uu][1] = cw.y;
-                            }
-                        // un-rotate: Y[gb] = X[(gb - fc) mod NGB]
-                        uint32_t Y[NGB][2][2];
-                        if (NGB == 4) {
-                            uint32_t T[4][2][2];
-#pragma unroll
-                            for (int gb = 0; gb < 4; ++gb)
-#pragma unroll
-                                for (int uu = 0; uu < 2; ++uu)
-#pragma unroll
-                                    for (int i = 0; i < 2; ++i) T[gb][uu][i] = (fc & 1) ? X[(gb + 3) & 3][uu][i] : X[gb][uu][i];
-#pragma unroll
-                            for (int gb = 0; gb < 4; ++gb)
-#pragma unroll
-                                for (int uu = 0; uu < 2; ++uu)
-#pragma unroll
-                                    for (int i = 0; i < 2; ++i) Y[gb][uu][i] = (fc & 2) ? T[(gb + 2) & 3][uu][i] : T[gb][uu][i];
-                        } else {
-#pragma unroll
-                            for (int gb = 0; gb < NGB; ++gb)
-#pragma unroll
-                                for (int uu = 0; uu < 2; ++uu)
-#pragma unroll
-                                    for (int i = 0; i < 2; ++i) Y[gb][uu][i] = (fc & 1) ? X[(gb + 1) & 1][uu][i] : X[gb][uu][i];
-                        }
                         const int t = blk * 2 + ts;                         // sub-tile index within the 32-token tile
+                        uint32_t b0[HSETS], b1[HSETS];
 #pragma unroll
                         for (int hs = 0; hs < HSETS; ++hs) {
                             const uint32_t w = t == 0 ? pw[hs].x : (t == 1 ? pw[hs].y : (t == 2 ? pw[hs].z : pw[hs].w));
-                            const uint32_t b0 = __byte_perm(w, 0u, sel_b0), b1 = __byte_perm(w, 0u, sel_b1);
+                            b0[hs] = __byte_perm(w, 0u, sel_b0);
+                            b1[hs] = __byte_perm(w, 0u, sel_b1);
+                            mma_f16(eacc[hs], 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b0[hs], b1[hs]);
+                        }
+                        // gather: X[x][u] = codeword of token 8ts + 4u + fc of the block, group block x ^ (fc & 1), row fr
+                        uint32_t X[NGB][2];
 #pragma unroll
-                            for (int gb = 0; gb < NGB; ++gb) {
-                                asm volatile(
-                                    "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                    : "+f"(macc[hs][gb][0]), "+f"(macc[hs][gb][1]), "+f"(macc[hs][gb][2]), "+f"(macc[hs][gb][3])
-                                    : "r"(Y[gb][0][0]), "r"(Y[gb][0][1]), "r"(Y[gb][1][0]), "r"(Y[gb][1][1]), "r"(b0), "r"(b1));
-                            }
+                        for (int x = 0; x < NGB; ++x) {
+                            const uint32_t vwd = odd_col ? cur.vw[blk][x ^ 1] : cur.vw[blk][x];      // codes of the group block this load fetches
+                            X[x][0] = lds_u32(vaddr(vwd, 2 * ts, x));
+                            X[x][1] = lds_u32(vaddr(vwd, 2 * ts + 1, x));
+                        }
+#pragma unroll
+                        for (int gb = 0; gb < NGB; ++gb) {
+                            const uint32_t x0 = odd_col ? X[gb ^ 1][0] : X[gb][0], x1 = odd_col ? X[gb ^ 1][1] : X[gb][1];
+                            const uint32_t a0 = __byte_perm(x0, 0x64646464u, 0x4140u), a1 = __byte_perm(x0, 0x64646464u, 0x4342u);
+                            const uint32_t a2 = __byte_perm(x1, 0x64646464u, 0x4140u), a3 = __byte_perm(x1, 0x64646464u, 0x4342u);
+#pragma unroll
+                            for (int hs = 0; hs < HSETS; ++hs) mma_f16(macc[hs][gb], a0, a1, a2, a3, b0[hs], b1[hs]);
                         }
                     }
                 }
+                if ((it & (NOVAKV_WINDOW - 1)) == NOVAKV_WINDOW - 1) flush_window();
             } else {
                 // ---- value side on CUDA cores (fp32): same lane coordinates and gathers, FMA instead of MMA ----
-                if (rescale) {
-#pragma unroll
-                    for (int h = 0; h < HPAD; ++h) {
-                        const uint64_t a2 = pack2(alpha[h], alpha[h]);
-#pragma unroll
-                        for (int x = 0; x < NGB; ++x) { fmul2(acc[VM ? 0 : x][VM ? 0 : h][0], a2); fmul2(acc[VM ? 0 : x][VM ? 0 : h][1], a2); }
-                    }
-                }
                 __syncwarp();      // previous tile's readers of the P area are done
 #pragma unroll
                 for (int h = 0; h < HPAD; h += 4)
@@ -694,10 +867,14 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                                          : "r"(s_pw + tok * (HPAD * 4) + h * 4));
 #pragma unroll
                         for (int x = 0; x < NGB; ++x) {
-                            const uint32_t a = __byte_perm(cur.vw[blk][x], pos8[x], 0x5504 | (tq << 4)) + s_vcb;
-                            const uint2 cw = lds_u64(a);
-                            const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&cw.x));
-                            const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&cw.y));
+                            // (odd lane columns fetch group block x ^ 1 with load x; their accumulator x holds that block)
+                            const uint32_t vwd = odd_col ? cur.vw[blk][x ^ 1] : cur.vw[blk][x];
+                            const uint32_t cwd = lds_u32(vaddr(vwd, tq, x));
+                            // grid indices -> binary32, centred: (1024 + u) - 1152 is exact in binary16
+                            const __half2 c1152 = __float2half2_rn(1152.f);
+                            const uint32_t h01 = __byte_perm(cwd, 0x64646464u, 0x4140u), h23 = __byte_perm(cwd, 0x64646464u, 0x4342u);
+                            const float2 f01 = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&h01), c1152));
+                            const float2 f23 = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&h23), c1152));
                             const uint64_t v01 = pack2(f01.x, f01.y), v23 = pack2(f23.x, f23.y);
 #pragma unroll
                             for (int h = 0; h < HPAD; ++h) {
@@ -708,71 +885,121 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                         }
                     }
             }
+        };
+
+        // ---- score table (the first tile's loads are issued before, so that they fly during the build)
+        TileRegs<L> ta, tb;
+        if (n_it > 0) load_tile(0, ta);
+        __syncthreads();     // q' of the pair is in shared memory
+        build_score_table<D, HG, VM>(t32_p, t16_p, cb_k_lut + (size_t)sg.kvh * 256 * L * 4, q_s);
+        async_copies_wait();
+        __syncthreads();     // table and value codebook complete
+
+        // ---- scan: 32-token tiles, two register buffers, the next tile's loads in flight while one is consumed
+        for (int it = 0; it < n_it; it += 2) {
+            if (it + 1 < n_it) load_tile(it + 1, tb);
+            process(ta, it);
+            if (it + 1 < n_it) {
+                if (it + 2 < n_it) load_tile(it + 2, ta);
+                process(tb, it + 1);
+            }
         }
 
         // ---- segment epilogue: merge the warps' partials, write one partial ---------------------
-        __syncthreads();                                   // scan done everywhere: the table is dead
-        float* m_acc = reinterpret_cast<float*>(smem + C::OFF_LUT);                    // [MERGE_SLOTS][HPAD][D]
-        float* m_ml = reinterpret_cast<float*>(smem + C::OFF_LUT + C::MERGE_ACC_BYTES);  // [NCW][HPAD][2]
-        float* m_lz = m_ml + NCW * HPAD * 2;                                             // [NCW][HPAD]  (VSQ)
+        if (VM) flush_window();
+        __syncthreads();                                   // scan done everywhere: the tables are dead
+        unsigned char* const merge_p = HAS16 ? t16_p : t32_p;
+        float* m_acc = reinterpret_cast<float*>(merge_p);                              // [NCW][HPAD][D]
+        float* m_ml = reinterpret_cast<float*>(merge_p + C::MERGE_ACC_BYTES);          // [NCW][HPAD][2]
+        float* m_lz = m_ml + NCW * HPAD * 2;                                           // [NCW][HPAD]  (VSQ)
+        if (VM && !VSQ) {
+            // lane (fr = 0, fc) holds the weight sum of heads 4 hs + fc
+            if (fr == 0) {
 #pragma unroll
-        for (int h = 0; h < HPAD; ++h) {
-            const float lsum = warp_sum(l_run[h]);
-            if (lane == 0) { m_ml[(warp * HPAD + h) * 2] = m_run[h]; m_ml[(warp * HPAD + h) * 2 + 1] = lsum; }
-            if (VSQ) {
-                const float lz = warp_sum(lz_run[h]);
-                if (lane == 0) m_lz[warp * HPAD + h] = lz;
-                lz_run[h] = 0.f;
+                for (int hs = 0; hs < HSETS; ++hs) {
+                    const float ma01 = fc & 1 ? m_run[hs * 4 + 1] : m_run[hs * 4 + 0];
+                    const float ma23 = fc & 1 ? m_run[hs * 4 + 3] : m_run[hs * 4 + 2];
+                    m_ml[(warp * HPAD + hs * 4 + fc) * 2] = fc & 2 ? ma23 : ma01;
+                    m_ml[(warp * HPAD + hs * 4 + fc) * 2 + 1] = l_run[hs];
+                }
             }
-            m_run[h] = M_INIT; l_run[h] = 0.f;
+        } else {
+#pragma unroll
+            for (int h = 0; h < HPAD; ++h) {
+                const float lsum = warp_sum(l_run[h]);
+                if (lane == 0) { m_ml[(warp * HPAD + h) * 2] = m_run[h]; m_ml[(warp * HPAD + h) * 2 + 1] = lsum; }
+                if (VSQ) {
+                    const float lz = warp_sum(lz_run[h]);
+                    if (lane == 0) m_lz[warp * HPAD + h] = lz;
+                    lz_run[h] = 0.f;
+                }
+            }
         }
+#pragma unroll
+        for (int h = 0; h < HPAD; ++h) { m_run[h] = M_INIT; l_run[h] = 0.f; }
         if (VM) {
+            // VSQ: the sums carry 2^-E of the scales; E is per warp, so it is folded back here
+            const float unsh = VSQ ? esh_pow : 1.f;
 #pragma unroll
             for (int hs = 0; hs < HSETS; ++hs)
 #pragma unroll
                 for (int gb = 0; gb < NGB; ++gb) {
                     *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + hs * 4 + fc) * D + (8 * gb + fr) * 4) =
-                        make_float4(macc[hs][gb][0], macc[hs][gb][1], macc[hs][gb][2], macc[hs][gb][3]);
+                        make_float4(macc[hs][gb][0] * unsh, macc[hs][gb][1] * unsh, macc[hs][gb][2] * unsh, macc[hs][gb][3] * unsh);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) macc[hs][gb][i] = 0.f;
                 }
+            esh_pow = 0.f;
         } else {
-            // slot (warp, fc): each lane column holds a partial over its own tokens for every group
+            // every lane column holds a partial over its own tokens (accumulator x of an odd column belongs to group
+            // block x ^ 1): add the four columns, column fc writes head 4 k + fc
 #pragma unroll
             for (int x = 0; x < NGB; ++x) {
-                const int g = 8 * ((x + fc) % NGB) + fr;
 #pragma unroll
                 for (int h = 0; h < HPAD; ++h) {
-                    float a0, a1, a2, a3;
+                    float a0, a1, a2, a3, b0, b1, b2, b3;
                     unpack2(acc[VM ? 0 : x][VM ? 0 : h][0], a0, a1);
                     unpack2(acc[VM ? 0 : x][VM ? 0 : h][1], a2, a3);
-                    *reinterpret_cast<float4*>(m_acc + ((size_t)(warp * 4 + fc) * HPAD + h) * D + g * 4) = make_float4(a0, a1, a2, a3);
-                    acc[VM ? 0 : x][VM ? 0 : h][0] = 0ull; acc[VM ? 0 : x][VM ? 0 : h][1] = 0ull;
+                    unpack2(acc[VM ? 0 : (x ^ 1)][VM ? 0 : h][0], b0, b1);
+                    unpack2(acc[VM ? 0 : (x ^ 1)][VM ? 0 : h][1], b2, b3);
+                    if (odd_col) { a0 = b0; a1 = b1; a2 = b2; a3 = b3; }           // now: this lane's partial of group block x
+#pragma unroll
+                    for (int o = 1; o <= 2; o <<= 1) {
+                        a0 += __shfl_xor_sync(0xffffffffu, a0, o); a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+                        a2 += __shfl_xor_sync(0xffffffffu, a2, o); a3 += __shfl_xor_sync(0xffffffffu, a3, o);
+                    }
+                    if ((h & 3) == fc)
+                        *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + h) * D + (8 * x + fr) * 4) = make_float4(a0, a1, a2, a3);
                 }
             }
+#pragma unroll
+            for (int x = 0; x < NGB; ++x)
+#pragma unroll
+                for (int h = 0; h < HPAD; ++h) { acc[VM ? 0 : x][VM ? 0 : h][0] = 0ull; acc[VM ? 0 : x][VM ? 0 : h][1] = 0ull; }
         }
         __syncthreads();
         {
-            constexpr int SPW = VM ? 1 : 4;                     // merge slots per warp
             const size_t pidx = (size_t)pair + blockIdx.x;      // unique: pair and CTA index both grow along the walk
+            const float unscale = VM ? 3.0517578125e-05f : 1.f;  // 2^-15: the weights carried 2^15
             for (int i = threadIdx.x; i < HG * D; i += S1_THREADS) {
                 const int h = i / D, c = i - h * D;
                 float M = M_INIT;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) M = fmaxf(M, m_ml[(w * HPAD + h) * 2]);
-                float a = 0.f, lsum = 0.f;
+                float a = 0.f, lsum = 0.f, zsum = 0.f;
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
                     const float sc = ex2(m_ml[(w * HPAD + h) * 2] - M);
-                    float aw = 0.f;
-#pragma unroll
-                    for (int s = 0; s < SPW; ++s) aw += m_acc[((size_t)(w * SPW + s) * HPAD + h) * D + c];
-                    if (VSQ) aw += m_lz[w * HPAD + h];              // zero-points: the same amount on every coefficient
-                    a = fmaf(sc, aw, a);
+                    a = fmaf(sc, m_acc[((size_t)w * HPAD + h) * D + c], a);
+                    if (VSQ) zsum = fmaf(sc, m_lz[w * HPAD + h], zsum);              // zero-points: the same amount on every coefficient
                     lsum = fmaf(sc, m_ml[(w * HPAD + h) * 2 + 1], lsum);
                 }
-                part_acc[(pidx * HG + h) * D + c] = a;
-                if (c == 0) { part_ml[(pidx * HG + h) * 2] = M; part_ml[(pidx * HG + h) * 2 + 1] = lsum; }
+                // grid index sums -> value-transform coefficients: s (u - 128) + (lo + 128 s) per unit of weight
+                float val;
+                if (VSQ) val = (a + zsum) * unscale;       // levels are the codes themselves (s = 1, no offset)
+                else val = (v_scale[(size_t)sg.kvh * D + c] * a + v_off[(size_t)sg.kvh * D + c] * lsum) * unscale;
+                part_acc[(pidx * HG + h) * D + c] = val;
+                if (c == 0) { part_ml[(pidx * HG + h) * 2] = M; part_ml[(pidx * HG + h) * 2 + 1] = lsum * unscale; }
             }
         }
         __syncthreads();                                   // merge buffer free before the next table build
@@ -1027,7 +1254,7 @@ novakv_band_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 
 // workspace layout
 struct WsLayout {
-    size_t qp, prefix, cost, range, qk, bml, bacc, ml, acc, total;
+    size_t qp, prefix, cost, range, qk, qc, bml, bacc, ml, acc, total;
 };
 WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -1039,7 +1266,8 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     w.cost = al(w.prefix + ((size_t)batch + 1) * 4);
     w.range = al(w.cost + ((size_t)batch + 1) * 4);
     w.qk = al(w.range + (size_t)ctx->n_sm * 2 * sizeof(long));
-    w.bml = al(w.qk + (size_t)batch * hq * 4);
+    w.qc = al(w.qk + (size_t)batch * hq * 4);
+    w.bml = al(w.qc + (size_t)batch * hq * 4);
     w.bacc = al(w.bml + (size_t)batch * hq * 2 * 4);
     w.ml = al(w.bacc + (size_t)batch * hq * d * 4);
     w.acc = al(w.ml + n_part * ctx->hg * 2 * 4);
@@ -1070,6 +1298,10 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     int32_t* cost_prefix = (int32_t*)(ws + w.cost);
     long* cta_range = (long*)(ws + w.range);
     float* qk_off = sink_logits ? (float*)(ws + w.qk) : nullptr;
+    float* qc = KSC ? (float*)(ws + w.qc) : nullptr;
+    // what the token logits drop: q . k_mean, and for the unscaled key format also the share of the codebook
+    // centres (k_mean_eff = k_mean + centre R_K^{-1}); with a per-token scale the centres are added back instead
+    const float* k_off_vec = KSC ? ly.k_mean : ly.k_mean_eff;
     float* band_ml = band ? (float*)(ws + w.bml) : nullptr;
     float* band_acc = band ? (float*)(ws + w.bacc) : nullptr;
     float* part_ml = (float*)(ws + w.ml);
@@ -1078,28 +1310,31 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
 
     novakv_launch_pdl(novakv_prepare_kernel<D, HG>, dim3(batch * hkv + 1), dim3(512), 0, stream, q, ly.rk_inv_t, seq_lens,
                       batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status,
-                      ly.k_mean, qk_off, cost_prefix, ctx->seg_weight);
+                      k_off_vec, qk_off, cost_prefix, ctx->seg_weight, (const float*)ly.k_center, qc);
     ctx->launches++;
 
     auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC, VSQ>;
     // the opt-in is per device and per kernel instantiation: remembered in the context (one device each)
     constexpr unsigned inst_bit = 1u << ((VM ? 1 : 0) + (KSC ? 2 : 0) + (VSQ ? 4 : 0));
     if (!(ctx->smem_opt_in & inst_bit)) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) return NOVAKV_ECUDA;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S1_SMEM_BYTES) != cudaSuccess) return NOVAKV_ECUDA;
         ctx->smem_opt_in |= inst_bit;
     }
     const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
     {
         novakv_prof_scope ps(ctx, 0, stream);
-        novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), C::SMEM, stream, qp, ly.cb_k_lut,
-                          VSQ ? (const __half*)ctx->int2_img : (const __half*)ly.cb_v_mma, k_pages, v_pages, k_scales, v_meta, n_pages, page_table, max_pages_per_seq, seq_lens, prefix, batch, hq, hkv, part_ml, part_acc,
-                          ctx->dev_status, pt_stride, (const int32_t*)cost_prefix, ctx->seg_weight, cta_range);
+        novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), S1_SMEM_BYTES, stream, qp, ly.cb_k_lut,
+                          VSQ ? (const uint8_t*)ctx->int2_img : (const uint8_t*)ly.cb_v_u8, (const float*)ly.v_scale,
+                          (const float*)ly.v_off, k_pages, v_pages, k_scales, v_meta, n_pages, page_table, max_pages_per_seq,
+                          seq_lens, prefix, batch, hq, hkv, part_ml, part_acc, ctx->dev_status, pt_stride,
+                          (const int32_t*)cost_prefix, ctx->seg_weight, cta_range, (const float*)qc,
+                          VSQ ? 0 : VCB_COPY_BYTES);
         ps.end();
         ctx->launches++;
     }
     if (band != nullptr) {
         novakv_launch_pdl(novakv_band_kernel<D, HG>, dim3(batch * hkv), dim3(BAND_WARPS * 32), 0, stream, q, band->k, band->v,
-                          band->cap, band->n_sink, band->meta, hq, hkv, sm_scale * 1.4426950408889634f, ly.k_mean, band_ml,
+                          band->cap, band->n_sink, band->meta, hq, hkv, sm_scale * 1.4426950408889634f, k_off_vec, band_ml,
                           band_acc);
         ctx->launches++;
     }

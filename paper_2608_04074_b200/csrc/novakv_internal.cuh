@@ -23,7 +23,9 @@ struct novakv_layer {
     double* rk_d_mma = nullptr;   // [Hkv][d/4][d][4]: rk_d with the input dimension blocked by 4 (tensor-core fragments)
     double* rv_d_mma = nullptr;   // same for rv_d
     double* k_mean_d = nullptr;   // [Hkv][d]
-    float* k_mean = nullptr;      // [Hkv][d] (sink-logit offset q . k_mean)
+    float* k_mean = nullptr;      // [Hkv][d] (offset q . k_mean of a sink logit / the BF16 band, scaled key format)
+    float* k_mean_eff = nullptr;  // [Hkv][d] k_mean + centre R_K^{-1}: the same offset when the table is built from centred codewords
+    float* k_center = nullptr;    // [Hkv][d] per (group, coordinate) midrange of the key codewords (transform domain)
     double* v_mean_d = nullptr;   // [Hkv][d]
     float* cb_k = nullptr;        // [Hkv][L][256][4]  search layout
     float* cb_v = nullptr;        // [Hkv][L][256][4]
@@ -31,8 +33,10 @@ struct novakv_layer {
     float* rk_inv_t = nullptr;    // [Hkv][d][d]
     float* rv_t = nullptr;        // [Hkv][d][d]  transposed R_V: rv_t[c][r] = R_V[r][c]
     float* v_mean = nullptr;      // [Hkv][d]
-    float* cb_k_lut = nullptr;    // [Hkv][plane][256][16][4]  the order the score table is built in
-    __half* cb_v_mma = nullptr;   // [Hkv][256][32][4]         same codewords, slots permuted for the tensor-core value side
+    float* cb_k_lut = nullptr;    // [Hkv][256][L][4]   key codewords minus k_center, the order the score table is built in
+    uint8_t* cb_v_u8 = nullptr;   // [Hkv][256][32][4]  value codewords as indices of their 8-bit grid, slot = group
+    float* v_scale = nullptr;     // [Hkv][d]  grid step s of each value coefficient: codeword = lo + s u
+    float* v_off = nullptr;       // [Hkv][d]  lo + 128 s
 };
 
 struct novakv_event_pair {
@@ -44,7 +48,7 @@ struct novakv_ctx {
     int hg = 0, n_groups = 0, n_sm = 0;
     std::vector<novakv_layer> layers;
     uint32_t* dev_status = nullptr;
-    void* int2_img = nullptr;     // binary16 [Hkv][256][32][4]: the product codebook {0,1,2,3}^4 in the value-gather layout
+    void* int2_img = nullptr;     // uint8 [256][32][4]: the product codebook {0,1,2,3}^4 in the value-gather layout
     bool profile = false;
     std::vector<novakv_event_pair> prof[3];
     std::vector<novakv_event_pair> prof_free;
@@ -144,23 +148,20 @@ cudaError_t novakv_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 
 // Byte offsets inside the 64*L-byte chunk of one (page, KV head); t = token slot in the page
 // (0..63), l = group.  These define the cache format (see the public header).
-//   keys:   [tile = t/32][plane][token t%32][16 bytes]; a token's L bytes are its 8 "slots" of L/8
-//           groups each, stored rotated: position j holds slot (j + t%8 + (t/8)%4) % 8.
-//   values: [block = t/16][fr = l%8][fc = t%4][x][b = (t%16)/4], x = (l/8 - fc) mod (L/8).
+//   keys:   [tile = t/32][plane][token t%32][16 bytes]; byte j of a token's L bytes (plane j/16) holds
+//           the code of group j ^ (t % 8) for j < 16 and of group j ^ (t % 16) for j >= 16.
+//   values: [block = t/16][fr = l%8][fc = t%4][gb = l/8][b = (t%16)/4].
 template <int L>
 __host__ __device__ __forceinline__ int novakv_k_offset(int t, int l) {
-    constexpr int GPS = L / 8, KPL = L / 16;
-    const int sigma = l / GPS, m = l % GPS;
-    const int rot = ((t & 7) + ((t >> 3) & 3)) & 7;
-    const int bytepos = ((sigma - rot) & 7) * GPS + m;
-    return (((t >> 5) * KPL + (bytepos >> 4)) * 32 + (t & 31)) * 16 + (bytepos & 15);
+    constexpr int KPL = L / 16;
+    const int j = l ^ (t & (l < 16 ? 7 : 15));
+    return (((t >> 5) * KPL + (j >> 4)) * 32 + (t & 31)) * 16 + (j & 15);
 }
 template <int L>
 __host__ __device__ __forceinline__ int novakv_v_offset(int t, int l) {
     constexpr int NGB = L / 8;
     const int tb = t & 15, fc = tb & 3, b = tb >> 2, fr = l & 7;
-    const int x = ((l >> 3) - fc) & (NGB - 1);
-    return (t >> 4) * (L * 16) + (fr * 4 + fc) * (NGB * 4) + x * 4 + b;
+    return (t >> 4) * (L * 16) + (fr * 4 + fc) * (NGB * 4) + (l >> 3) * 4 + b;
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

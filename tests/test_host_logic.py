@@ -59,17 +59,15 @@ def test_cache_layout_round_trip_and_positions():
     for b, n in enumerate(lens):
         k, v = cache_format.read_tokens(kp, vp, table[b], hkv, d, 0, int(n))
         assert np.array_equal(k, ref[b][0]) and np.array_equal(v, ref[b][1])
-    # documented byte positions of the chunk layouts (d = 64: L = 16, 2 groups per slot, 2 group blocks)
+    # documented byte positions of the chunk layouts (d = 64: L = 16, one 16-byte plane, 2 group blocks)
     b, pos, h, l = 0, 77, 1, 9
     page = table[b][pos // 64]
     t = pos % 64                                       # 13
-    rot = (t % 8 + (t // 8) % 4) % 8                   # slot rotation of this token
-    bytepos = ((l // 2 - rot) % 8) * 2 + l % 2
-    k_off = (((t // 32) * 1 + bytepos // 16) * 32 + t % 32) * 16 + bytepos % 16
+    j = l ^ (t % 8)                                    # byte of the token's key bytes that holds group l (l < 16)
+    k_off = (((t // 32) * 1 + j // 16) * 32 + t % 32) * 16 + j % 16
     assert kp[page, h, k_off] == ref[b][0][pos, h, l]
     fc, bb, fr = (t % 16) % 4, (t % 16) // 4, l % 8
-    x = (l // 8 - fc) % 2
-    v_off = (t // 16) * (L * 16) + (fr * 4 + fc) * 8 + x * 4 + bb
+    v_off = (t // 16) * (L * 16) + (fr * 4 + fc) * 8 + (l // 8) * 4 + bb
     assert vp[page, h, v_off] == ref[b][1][pos, h, l]
     # every byte of a chunk is hit exactly once
     tt, ll = np.meshgrid(np.arange(64), np.arange(L), indexing="ij")
