@@ -888,21 +888,18 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         };
 
         // ---- score table (the first tile's loads are issued before, so that they fly during the build)
-        TileRegs<L> ta, tb;
+        TileRegs<L> ta;
         if (n_it > 0) load_tile(0, ta);
         __syncthreads();     // q' of the pair is in shared memory
         build_score_table<D, HG, VM>(t32_p, t16_p, cb_k_lut + (size_t)sg.kvh * 256 * L * 4, q_s);
         async_copies_wait();
         __syncthreads();     // table and value codebook complete
 
-        // ---- scan: 32-token tiles, two register buffers, the next tile's loads in flight while one is consumed
-        for (int it = 0; it < n_it; it += 2) {
-            if (it + 1 < n_it) load_tile(it + 1, tb);
-            process(ta, it);
-            if (it + 1 < n_it) {
-                if (it + 2 < n_it) load_tile(it + 2, ta);
-                process(tb, it + 1);
-            }
+        // ---- scan: 32-token tiles, the next tile's loads in flight while one is consumed
+        for (int it = 0; it < n_it; ++it) {
+            const TileRegs<L> cur = ta;
+            if (it + 1 < n_it) load_tile(it + 1, ta);
+            process(cur, it);
         }
 
         // ---- segment epilogue: merge the warps' partials, write one partial ---------------------
