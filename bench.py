@@ -8,9 +8,10 @@ decode step must read (packed indices + codebooks + transforms + q/out) / time o
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-sweep]
 
-N > 1 is launched under torchrun, one rank per GPU; every rank runs its own batch (weak scaling,
-no collective on the data path), time is the max over ranks.  `--impl reference` times the CPU
-oracle on the host cores on a bounded sample of the same workload.
+N > 1: one rank per GPU under torch.distributed.run (started by this script itself when it is not
+already running under a launcher); every rank runs its own batch (weak scaling, no collective on the
+data path), time is the max over ranks.  `--impl reference` times the CPU oracle on the host cores on
+a bounded sample of the same workload.
 Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
@@ -211,6 +212,10 @@ def time_steps(fn, steps, warmup, flush, after_warmup=None):
     return [a.elapsed_time(b) for a, b in evs]
 
 
+def med_min(times):
+    return round(statistics.median(times), 5), round(min(times), 5)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -224,7 +229,7 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
 
-    wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len)
+    wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len, calib_tokens=args.calib_tokens, lloyd_iters=args.lloyd_iters)
     laws = wl.laws()
     cal = wl.calibration(laws)
     s = wl.shape
@@ -233,6 +238,24 @@ def run_ours(args):
     B, S = wl.batch, args.seq_len
     cache = PagedCache(ctx, wl.seq_lens, capacity_tokens=wl.seq_lens + 64, seed=17 + rank, device=dev)
     fill_cache_gpu(ctx, cache, laws, wl.seq_lens, seed=5000 + 100000 * rank)
+
+    # a sample of what the GPU encoder stored (the CPU-baseline leg compares it with the oracle's indices)
+    parity = None
+    if rank == 0:
+        from paper_2608_04074_b200 import cache_format
+        kp = cache.k_pages.cpu().numpy().reshape(cache.n_pages, s.n_kv_heads, -1)
+        vp = cache.v_pages.cpu().numpy().reshape(cache.n_pages, s.n_kv_heads, -1)
+        parity = {"samples": []}
+        gen = synth.rng(4711)
+        for b, chunk in ((0, 1 if S > 8192 else 0), (B - 1, 0)):
+            m = min(8192, S - chunk * 8192)
+            pick = np.sort(gen.choice(m, size=min(512, m), replace=False))
+            kk, vv = synth.draw_kv(laws, 5000 + 100000 * rank + 131 * b + chunk, m)        # what fill_cache_gpu drew
+            gk, gv = cache_format.read_tokens(kp, vp, cache.page_table_host[b], s.n_kv_heads, s.head_dim, 0, S)
+            parity["samples"].append(dict(k=synth.to_bf16_representable(kk[pick]), v=synth.to_bf16_representable(vv[pick]),
+                                          gk=gk[chunk * 8192 + pick], gv=gv[chunk * 8192 + pick]))
+        parity["seq0_idx"] = cache_format.read_tokens(kp, vp, cache.page_table_host[0], s.n_kv_heads, s.head_dim, 0, S)
+        del kp, vp
 
     # step inputs: one new token per sequence at position S, one query per sequence
     k1, v1 = synth.draw_kv(laws, 7001 + rank, B)
@@ -255,6 +278,10 @@ def run_ours(args):
 
     # ---- device-resident timing -------------------------------------------------------------
     ctx.novakv_profile_enable(False)
+    if parity is not None:
+        cache.decode(0, qd, out=out)          # before any append: attends over the S tokens sampled above
+        parity["seq0_out"] = out[0].cpu().numpy()
+        parity["seq0_q"] = synth.to_bf16_representable(q[0])
     for _ in range(2):
         step()
     torch.cuda.synchronize()
@@ -288,7 +315,7 @@ def run_ours(args):
 
     # ---- decode only / encode only (explanatory numbers) ------------------------------------
     dec_times = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, flush)
-    dec_ms = statistics.median(dec_times)
+    dec_ms, dec_min = med_min(dec_times)
     nowarm = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, lambda: None)
     dec_ms_warm_l2 = statistics.median(nowarm)
 
@@ -296,7 +323,7 @@ def run_ours(args):
     ctx.novakv_debug_set_value_path(0)
     cc_times = time_steps(lambda: cache.decode(0, qd, out=out), args.steps, 3, flush)
     ctx.novakv_debug_set_value_path(1)
-    cc_ms = statistics.median(cc_times)
+    cc_ms, cc_min = med_min(cc_times)
     bf16 = time_bf16_comparator(ctx, wl_after, dev, max(5, args.steps // 2), flush)
 
     # ---- end to end from pinned host buffers through the C ABI --------------------------------
@@ -334,7 +361,9 @@ def run_ours(args):
         result = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None,
+            "dtype": "f32 accumulation; f32/f16 score-table entries; f16 MMA operands on the value side (u8 grid codewords)",
+            "data": "synthetic", "ms_per_step_min": round(min(times), 5),
             "config": {"workload": f"qwen3_8b_shape decode step: Hq=32 Hkv=8 d=128 B={B} S={S}+1 per GPU, "
                                    "2-bit VQ K and V (g=4, 256-entry codebooks), bf16 q, 64-token pages; "
                                    "step = encode_append of B tokens + decode_attention",
@@ -353,17 +382,21 @@ def run_ours(args):
                          "avg_launch_ms": round(s1_avg_ms, 5), "launches_timed": s1_n,
                          "timing": "CUDA events around the kernel, second pass of the same K steps",
                          "traffic": ncu_traffic_per_launch("decode_stage1_qwen3_8b_B8_S16384.md")},
-            "decode_only": {"ms": round(dec_ms, 5), "gbps": round(alg_bytes / (dec_ms * 1e-3) / 1e9, 1),
+            "decode_only": {"ms": round(dec_ms, 5), "ms_min": dec_min, "gbps": round(alg_bytes / (dec_ms * 1e-3) / 1e9, 1),
                             "pct_of_8TBps": round(100 * alg_bytes / (dec_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
                             "ms_l2_not_flushed": round(dec_ms_warm_l2, 5)},
-            "decode_only_cuda_core_value_side": {"ms": round(cc_ms, 5),
-                                                 "gbps": round(alg_bytes / (cc_ms * 1e-3) / 1e9, 1)},
+            "decode_only_cuda_core_value_side": {"ms": round(cc_ms, 5), "ms_min": cc_min,
+                                                 "gbps": round(alg_bytes / (cc_ms * 1e-3) / 1e9, 1),
+                                                 "note": "the variant that keeps tensor cores out of the decode path altogether "
+                                                         "(north_star's literal reading); the headline runs the value-side "
+                                                         "contraction on tensor cores"},
             "bf16_comparator": dict(bf16, speedup_of_2bit_decode=round(bf16["ms"] / dec_ms, 2)),
             "encode_append": {"tokens": B, "avg_kernel_ms": round(enc_ms / max(enc_n, 1), 5)},
             "device_status": status,
         }
 
     # ---- sweep: long-context bandwidth configs and prefill encode (rank 0 of a 1-GPU run only) ----
+    oracle_jobs = []
     if rank == 0 and world == 1 and not args.no_sweep:
         sweep = []
         del cache
@@ -379,17 +412,21 @@ def run_ours(args):
             k_ms, k_n = ctx.novakv_profile_read(0)
             ctx.novakv_profile_enable(False)
             ab, ib = algorithmic_decode_bytes(wl2)
-            ms = statistics.median(tt)
+            ms, ms_min = med_min(tt)
+            oracle_jobs.append((f"qwen3_8b_shape B={b2} S={s2}", wl2, laws, cal))
             del c2
             torch.cuda.empty_cache()
             bf = time_bf16_comparator(ctx, wl2, dev, 5, lambda: None)
             sweep.append({"workload": f"qwen3_8b_shape B={b2} S={s2} decode only, inputs larger than L2",
-                          "ms": round(ms, 4), "gbps": round(ab / (ms * 1e-3) / 1e9, 1),
+                          "ms": round(ms, 4), "ms_min": round(ms_min, 4), "gbps": round(ab / (ms * 1e-3) / 1e9, 1),
                           "pct_of_8TBps": round(100 * ab / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBPS, 2),
                           "scan_kernel_ms": round(k_ms / max(k_n, 1), 4),
                           "scan_kernel_frac_of_measured_peak": round(ab / (k_ms / max(k_n, 1) * 1e-3) / 1e9 / measured_peak()[0], 4),
                           "algorithmic_bytes": ab,
                           "bf16_comparator": dict(bf, speedup_of_2bit_decode=round(bf["ms"] / ms, 2))})
+            result["roofline"].setdefault("long_context", []).append(
+                {"workload": f"B={b2} S={s2}", "achieved": round(ab / (k_ms / max(k_n, 1) * 1e-3) / 1e9, 1),
+                 "frac": sweep[-1]["scan_kernel_frac_of_measured_peak"], "avg_launch_ms": sweep[-1]["scan_kernel_ms"]})
             del q2, o2
             torch.cuda.empty_cache()
         # paged serving mix: 128 ragged sequences, append 128 tokens then decode (Qwen3-8B KV shape)
@@ -414,6 +451,7 @@ def run_ours(args):
         wl5b.seq_lens = wl5.seq_lens + 1
         ab5, _ = algorithmic_decode_bytes(wl5b)
         ms5, msd5 = statistics.median(tt), statistics.median(td)
+        oracle_jobs.append((f"paged mix, {n5} sequences", wl5b, laws, cal))
         sweep.append({"workload": f"paged mix: {n5} sequences, lognormal lengths {int(wl5.seq_lens.min())}..{int(wl5.seq_lens.max())} "
                                   f"(sum {int(wl5.seq_lens.sum())}), 64-token pages shuffled; step = append {n5} tokens + decode",
                       "ms": round(ms5, 4), "decode_only_ms": round(msd5, 4),
@@ -531,6 +569,7 @@ def run_ours(args):
         tt = time_steps(lambda: c4.decode(0, q4, out=o4), max(5, args.steps // 2), 3, lambda: None)
         ab4, _ = algorithmic_decode_bytes(wl4)
         ms4 = statistics.median(tt)
+        oracle_jobs.append(("gpt_oss_20b_shape B=16 S=65536", wl4, laws4, cal4))
         del c4
         torch.cuda.empty_cache()
         bf4 = time_bf16_comparator(ctx4, wl4, dev, 5, lambda: None)
@@ -553,7 +592,7 @@ def run_ours(args):
         result["sweep"] = sweep
 
     if rank == 0:
-        result["cpu_baseline"] = cpu_baseline_sample(wl, laws, cal, args)
+        result["cpu_baseline"] = cpu_baseline_sample(wl, laws, cal, args, parity, oracle_jobs)
         print(json.dumps(result))
     if world > 1:
         dist.barrier()
@@ -586,7 +625,47 @@ def oracle_step(orc, kidx, vidx, q, k1, v1):
         orc.decode(q[b].astype(np.float64), kidx, vidx)
 
 
-def cpu_baseline_sample(wl, laws, cal, args):
+def _omp_set_threads(n):
+    """Thread count of the oracle's OpenMP loops (libgomp runtime call); returns True if it could be set."""
+    import ctypes
+    try:
+        ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+        return True
+    except OSError:
+        return False
+
+
+def oracle_subset(label, wl, laws, cal):
+    """Oracle decode time on a stated subset of a sweep workload (first, last and two seeded random sequences,
+    all heads), extrapolated linearly in tokens to the whole workload."""
+    from oracle import novakv_oracle as O
+    from paper_2608_04074_b200 import synth
+    orc = O.Oracle.from_calibration(cal)
+    n = wl.batch
+    pick = sorted(set([0, n - 1] + [int(x) for x in synth.rng(99).choice(n, size=min(2, n), replace=False)]))
+    k, v = synth.draw_kv(laws, 8201, 2048)
+    enc = orc.encode(synth.to_bf16_representable(k).astype(np.float64), synth.to_bf16_representable(v).astype(np.float64),
+                     with_gaps=False)
+    q = synth.to_bf16_representable(synth.draw_q(laws, 8202, len(pick)))
+    t0 = time.perf_counter()
+    for i, b in enumerate(pick):
+        S = int(wl.seq_lens[b])
+        reps = (S + 2047) // 2048
+        orc.decode(q[i].astype(np.float64), np.tile(enc["kidx"], (reps, 1, 1))[:S], np.tile(enc["vidx"], (reps, 1, 1))[:S])
+    dt = time.perf_counter() - t0
+    sub_tokens = int(sum(int(wl.seq_lens[b]) for b in pick))
+    all_tokens = int(wl.seq_lens.astype(np.int64).sum())
+    per_tok_bytes = wl.shape.n_kv_heads * 2 * (wl.shape.head_dim // 4)
+    return {"workload": label, "sequences": pick, "tokens": sub_tokens, "seconds": round(dt, 3),
+            "gbps": round(sub_tokens * per_tok_bytes / dt / 1e9, 6),
+            "extrapolated_seconds_whole_workload": round(dt * all_tokens / max(sub_tokens, 1), 2),
+            "note": "decode only; time extrapolated linearly in tokens (labelled, not measured)"}
+
+
+def cpu_baseline_sample(wl, laws, cal, args, parity=None, jobs=()):
+    """The CPU-baseline leg: times the oracle on a bounded sample of the benchmark workload (all host cores and one
+    thread), on stated subsets of the sweep workloads, and compares what the GPU stored / produced on a sample of
+    the benchmark cache with the oracle (index mismatches against the float64 nearest codeword, near-ties)."""
     from oracle import novakv_oracle as O
     n_seq = min(wl.batch, 8)          # about 20 core-seconds of oracle work on the benchmark shape
     orc, kidx, vidx, q, k1, v1 = oracle_sample_inputs(wl, laws, cal, n_seq)
@@ -594,20 +673,70 @@ def cpu_baseline_sample(wl, laws, cal, args):
     oracle_step(orc, kidx, vidx, q, k1, v1)
     dt = time.perf_counter() - t0
     s = wl.shape
-    sample_bytes = n_seq * int(wl.seq_lens[0]) * s.n_kv_heads * 2 * (s.head_dim // 4)
-    return {"value": round(sample_bytes / dt / 1e9, 6), "unit": UNIT, "cores": O.cpu_threads(), "kind": "oracle",
-            "seconds": round(dt, 3),
-            "sample": f"{n_seq} of {wl.batch} sequences (S={int(wl.seq_lens[0])}, all heads): oracle encode of "
-                      f"{n_seq} new tokens + explicit-dequantise decode; index bytes of the sample / wall time"}
+    per_seq_bytes = int(wl.seq_lens[0]) * s.n_kv_heads * 2 * (s.head_dim // 4)
+    res = {"value": round(n_seq * per_seq_bytes / dt / 1e9, 6), "unit": UNIT, "cores": O.cpu_threads(), "kind": "oracle",
+           "seconds": round(dt, 3),
+           "sample": f"{n_seq} of {wl.batch} sequences (S={int(wl.seq_lens[0])}, all heads): oracle encode of "
+                     f"{n_seq} new tokens + explicit-dequantise decode; index bytes of the sample / wall time"}
+    if _omp_set_threads(1):
+        t0 = time.perf_counter()
+        oracle_step(orc, kidx, vidx, q[:1], k1[:1], v1[:1])
+        dt1 = time.perf_counter() - t0
+        _omp_set_threads(O.cpu_threads())
+        res["single_thread"] = {"value": round(per_seq_bytes / dt1 / 1e9, 6), "unit": UNIT, "seconds": round(dt1, 3),
+                                "sample": "1 sequence of the same workload, one thread"}
+    if jobs:
+        res["sweep_subsets"] = [oracle_subset(*j) for j in jobs]
+    if parity is not None:
+        n_groups = mism = near = bad = 0
+        max_gap = 0.0
+        for smp in parity["samples"]:
+            enc = orc.encode(smp["k"].astype(np.float64), smp["v"].astype(np.float64))
+            for side, got in (("k", smp["gk"]), ("v", smp["gv"])):
+                diff = got != enc[side + "idx"]
+                gap = enc[side + "gap"]
+                n_groups += int(diff.size)
+                mism += int(diff.sum())
+                near += int((gap <= 1e-6).sum())
+                bad += int((diff & (gap > 1e-6)).sum())
+                if diff.any():
+                    max_gap = max(max_gap, float(gap[diff].max()))
+        gk, gv = parity["seq0_idx"]
+        ref = orc.decode(parity["seq0_q"].astype(np.float64), gk, gv)
+        err = float(np.abs(parity["seq0_out"] - ref).max() / np.abs(ref).max())
+        res["parity_on_benchmark_cache"] = {
+            "groups_compared": n_groups, "index_mismatch_vs_f64": mism, "near_ties_le_1e-6": near,
+            "index_mismatch_outside_near_ties": bad, "max_gap_among_mismatches": max_gap,
+            "decode_max_abs_err_over_out_inf_norm_seq0": round(err, 7), "decode_tolerance": 2e-3,
+            "sample": "2 x 512 tokens of the GPU-encoded benchmark cache (all heads, K and V) against the oracle's float64 "
+                      "nearest codeword; GPU output of sequence 0 against the oracle's decode of the stored indices"}
+    return res
 
 
 def run_reference(args):
     rank, _, world = env_rank()
-    if rank != 0:
-        return
+    if world > 1:
+        # rank 0 alone runs and prints; the others only join the rendezvous (CPU: gloo) and leave
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        if rank != 0:
+            dist.barrier()
+            dist.destroy_process_group()
+            return
+    _run_reference_rank0(args, world)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def _run_reference_rank0(args, world):
+    if world > 1:
+        # a launcher pins every rank to one OpenMP thread; this rank is the only one that works
+        os.environ["OMP_NUM_THREADS"] = str(len(os.sched_getaffinity(0)))
     from oracle import novakv_oracle as O
     from paper_2608_04074_b200 import workloads
-    wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len)
+    wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len, calib_tokens=args.calib_tokens, lloyd_iters=args.lloyd_iters)
     laws = wl.laws()
     cal = wl.calibration(laws)
     n_seq = 1
@@ -635,6 +764,22 @@ def run_reference(args):
     }))
 
 
+def launch_ranks(n):
+    """`--gpus N` outside a launcher: re-run this script as N ranks of one node under torch.distributed.run
+    (one rank per GPU, rendezvous on 127.0.0.1) and return its exit code.  NCCL's communicator log is kept
+    (in a file per rank, so that standard output stays the one JSON line)."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_FILE", os.path.join(os.environ.get("TMPDIR", "/tmp"), "novakv_bench_nccl.%h.%p.log"))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd, env=env).returncode
+
+
 def main():
     sys.setswitchinterval(1e-4)          # let the clock-sampling thread run between short GPU calls
     ap = argparse.ArgumentParser()
@@ -645,8 +790,12 @@ def main():
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--seq-len", type=int, default=16384)
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--calib-tokens", type=int, default=8192, help="calibration tokens per KV head (set-up cost only)")
+    ap.add_argument("--lloyd-iters", type=int, default=12, help="Lloyd iterations of the calibration (set-up cost only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args.gpus))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -274,13 +274,16 @@ novakv_status novakv_decode_attention_deployed(novakv_ctx* ctx, int layer, const
  * every GPU that loads the library holds it until the process exits.
  *   - Arguments and results are those of novakv_decode_attention without workspace/workspace_bytes.
  *   - Returns NOVAKV_EWORKSPACE when novakv_decode_workspace_bytes(ctx, batch) exceeds
- *     NOVAKV_NOALLOC_SCRATCH_BYTES (for the Qwen3-8B shape that is a batch of more than 78 sequences).
+ *     NOVAKV_NOALLOC_SCRATCH_BYTES; the workspace grows with the batch and with the number of SMs of the
+ *     device (for the Qwen3-8B shape on a 148-SM device the largest batch that fits is 77 sequences).
  *   - Calls no cudaMalloc, cudaFree or other allocating routine, and records no timing events.
  *   - All calls on a device share the array: calls that overlap on the GPU (other streams, other
  *     contexts) race; calls on one stream are ordered and safe.  Every scratch word is written
  *     before it is read within a call, so nothing needs clearing between calls.
  *   - The first call on each device queries the array's device address (a synchronous runtime
- *     call); issue that first call before any stream capture begins.
+ *     call); issue that first call before any stream capture begins.  The address is cached per device
+ *     in a process-wide table that is written without a lock: the look-up gives the same value every
+ *     time, so concurrent first calls are harmless, but a context is still used from one thread at a time.
  */
 #define NOVAKV_NOALLOC_SCRATCH_BYTES (4u << 20)
 novakv_status novakv_decode_attention_noalloc(novakv_ctx* ctx, int layer, const void* q,

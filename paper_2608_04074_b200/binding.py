@@ -44,6 +44,9 @@ class CalibrationPtrs(ctypes.Structure):
 _lib = None
 
 
+NOALLOC_SCRATCH_BYTES = 4 << 20      # NOVAKV_NOALLOC_SCRATCH_BYTES of the public header
+
+
 def load_library(path=None):
     """Load libnovakv.so (built in-tree by ``build.build_cuda``); raises if it is absent."""
     global _lib

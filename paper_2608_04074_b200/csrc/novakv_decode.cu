@@ -124,16 +124,19 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
     constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
     const int c = threadIdx.x % D, part = threadIdx.x / D;
-    // this thread's slice of the (constant) transform is fetched before the grid-dependency wait, so the
-    // loads overlap the tail of the preceding kernel in the stream
+    // The query transform depends on nothing the preceding kernel of the stream (normally the append of this
+    // step's tokens) writes: queries are produced before that kernel started, the transform is a constant.  So
+    // the blocks that transform queries never wait on the grid dependency: they run beside the preceding
+    // kernel.  Only the block that forms the page prefix (it reads seq_lens, which an append updates) waits;
+    // since a grid completes only when all its blocks have, the scan kernel's own wait still covers both.
     float rv[ROWS];
     if (blk < batch * n_kv_heads) {
         const float* R = rk_inv_t + (size_t)kvh * D * D + (size_t)part * ROWS * D + c;
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) rv[r] = R[(size_t)r * D];
     }
-    novakv_grid_dependency_wait();
     if (blk == batch * n_kv_heads) {
+        novakv_grid_dependency_wait();
         // exclusive prefix over sequences of their page counts; small, done by one warp.  Beside it the same
         // prefix in "cost" units, in which every non-empty sequence weighs seg_weight pages more: the scan
         // kernel splits the walk evenly in cost, so that a CTA that has to set up several (sequence, KV head)
@@ -168,6 +171,7 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         }
         return;
     }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ float q_s[HG][D];
     __shared__ float red_s[PARTS][HG][D];
     for (int i = threadIdx.x; i < HG * D; i += 512)
@@ -199,6 +203,8 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         float acc = 0.f;
         for (int i = lane; i < D; i += 32) acc = fmaf(q_s[h][i], k_mean[(size_t)kvh * D + i], acc);
         acc = warp_sum_f(acc);
+        // (the merge kernel of a preceding decode call on this workspace reads qk_off: its grid must have completed)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (lane == 0) qk_off[(size_t)b * n_q_heads + kvh * HG + h] = acc * scale_log2;
     }
     // scaled key format: the table is built from centred codewords, and the centre's share <q', centre> of

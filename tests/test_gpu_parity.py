@@ -135,7 +135,11 @@ def test_decode_matches_oracle(name, lens, request):
 
 
 # --------------------------------------------------------------------------- T4: split invariance, determinism
-def test_split_count_invariance_and_determinism(qwen):
+@pytest.mark.parametrize("path", [1, 0])
+def test_split_count_invariance_and_determinism(qwen, path):
+    """path 1: tensor-core value side (binary16 weights: different splits see different running maxima and
+    round the weights differently, 2^-12 relative per weight, so invariance holds to ~2e-4 of the output
+    scale); path 0: CUDA-core value side, binary32 weights, invariant within binary32 rounding."""
     case = qwen
     lens = np.array([4096, 900, 2500], np.int32)
     cache = _cache(case, lens)
@@ -143,21 +147,24 @@ def test_split_count_invariance_and_determinism(qwen):
     _, _, q = case.draw(401, 1, len(lens))
     qd = _dev(q, torch.bfloat16)
     outs = {}
-    for n_ctas in (1, 2, 7, 0):
-        case.ctx.novakv_debug_set_scan_ctas(n_ctas)
-        outs[n_ctas] = cache.decode(0, qd).cpu().numpy()
-        again = cache.decode(0, qd).cpu().numpy()
-        assert np.array_equal(outs[n_ctas], again), "same launch configuration must be bitwise reproducible"
-    case.ctx.novakv_debug_set_scan_ctas(0)
+    case.ctx.novakv_debug_set_value_path(path)
+    try:
+        for n_ctas in (1, 2, 7, 0):
+            case.ctx.novakv_debug_set_scan_ctas(n_ctas)
+            outs[n_ctas] = cache.decode(0, qd).cpu().numpy()
+            again = cache.decode(0, qd).cpu().numpy()
+            assert np.array_equal(outs[n_ctas], again), "same launch configuration must be bitwise reproducible"
+    finally:
+        case.ctx.novakv_debug_set_scan_ctas(0)
+        case.ctx.novakv_debug_set_value_path(1)
+    bound = 2e-4 if path == 1 else 2e-5
     for b in range(len(lens)):
         ref = case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"])
         for n_ctas, o in outs.items():
             check_output(o[b], ref)
         scale = np.abs(ref).max()
-        # different splits see different running maxima, hence round the fp16 softmax weights of the
-        # tensor-core value side differently (2^-12 relative per weight): invariance holds to ~1e-4
         for n_ctas in (1, 2, 7):
-            assert np.abs(outs[n_ctas][b] - outs[0][b]).max() <= 2e-4 * scale
+            assert np.abs(outs[n_ctas][b] - outs[0][b]).max() <= bound * scale
 
 
 # --------------------------------------------------------------------------- T6: append then decode, end to end
@@ -283,7 +290,8 @@ def test_faults_are_reported_not_trapped(qwen):
     bad = type("C", (), {})()
     for n in ("rk", "rk_inv_t", "rv", "k_mean", "v_mean", "cb_k", "cb_v"):
         setattr(bad, n, getattr(case.cal, n))
-    bad.cb_v = case.cal.cb_v + np.float32(1e-4)             # no longer binary16-representable
+    bad.cb_v = case.cal.cb_v.copy()
+    bad.cb_v[0, 3, 100, 2] += np.float32(1e-4) * max(1.0, abs(float(bad.cb_v[0, 3, 100, 2])))   # off its 8-bit grid
     with pytest.raises(NovaKVError, match="unsupported calibration"):
         fresh.novakv_load_calibration(1, bad)
     with pytest.raises(NovaKVError, match="unsupported shape"):
@@ -767,13 +775,18 @@ def test_deployed_decode_matches_oracle(name, lens, request):
     case = request.getfixturevalue(name)
     lens = np.array(lens, np.int32)
     cache = PagedCache(case.ctx, lens, seed=3, int2_values=True)
+    # slots that hold no token (the tail of a partly filled last page) carry whatever the caller's allocator
+    # left there: NaN and infinity patterns must not reach the result
+    cache.v_meta.view(torch.int16).fill_(0x7FC0)
+    cache.k_scales.view(torch.int16).fill_(0x7F80)
     encs = []
     for b, n in enumerate(lens):
         if n == 0:
             encs.append(None)
             continue
         k, v, _ = case.draw(1400 + b, int(n), 1)
-        v = synth.to_bf16_representable(v * (2.0 ** synth.rng(18 + b).integers(-2, 3, size=(int(n), 1, 1))) - 0.5)
+        # value scales spread over 2^-9 .. 2^2 (small scales exercise the weight range of the INT2 path)
+        v = synth.to_bf16_representable(v * (2.0 ** synth.rng(18 + b).integers(-9, 3, size=(int(n), 1, 1))) - 0.5)
         e = case.oracle.encode_scaled(k.astype(np.float64), v.astype(np.float64), with_gaps=False)
         codes, meta = case.oracle.encode_values_int2(v.astype(np.float64))
         cache.store_logical(b, 0, e["kidx"], cache_format.pack_int2(codes))

@@ -149,3 +149,19 @@ def test_bench_reference_arm_prints_one_json_line():
     r = json.loads(lines[0])
     assert r["impl"] == "reference" and r["value"] > 0 and r["cpu_baseline"]["kind"] == "oracle"
     assert r["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_bench_gpus_flag_launches_ranks():
+    """`bench.py --gpus 2` outside a launcher starts two ranks itself (here the CPU reference arm, gloo
+    rendezvous on 127.0.0.1) and rank 0 prints one JSON line that says so."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                          "--warmup", "0", "--batch", "2", "--seq-len", "512", "--calib-tokens", "1024", "--lloyd-iters", "2"],
+                         capture_output=True, text=True, timeout=600, env=env)
+    assert res.returncode == 0, res.stdout + res.stderr
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    out = json.loads(lines[0])
+    assert out["impl"] == "reference" and out["n_gpus"] == 2
+    assert out["cpu_baseline"]["cores"] == len(os.sched_getaffinity(0))
