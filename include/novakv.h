@@ -369,6 +369,17 @@ novakv_status novakv_debug_set_value_path(novakv_ctx* ctx, int path);
  */
 novakv_status novakv_debug_set_segment_weight(novakv_ctx* ctx, int pages);
 
+/*
+ * Cross-split merge (App. B "Decoding kernel and read path": stage 2 combines the per-split partials).
+ * on = 0 (default): a separate merge kernel follows the scan.  on = 1: without a sink logit and without a
+ * BF16 band the scan kernel performs the merge itself - the CTA that writes the last partial of a
+ * (sequence, KV head) pair combines the pair's partials and applies the inverse value transform; an arrival
+ * counter per pair decides, nothing waits.  Results agree within binary32 rounding.  (Measured on B200 the
+ * fused form saves a launch but puts the merge on the critical path of the last CTA of every pair; it is not
+ * faster at any benchmark shape, hence not the default.)
+ */
+novakv_status novakv_debug_set_fused_merge(novakv_ctx* ctx, int on);
+
 /* Kernels this library launched since the context was created (all kinds). */
 long novakv_launch_count(const novakv_ctx* ctx);
 

@@ -24,7 +24,7 @@ EXPORTED = [
     "novakv_scale_page_bytes", "novakv_encode_append_scaled", "novakv_decode_attention_scaled",
     "novakv_decode_attention_sink", "novakv_decode_attention_banded",
     "novakv_value_meta_page_bytes", "novakv_encode_append_deployed", "novakv_decode_attention_deployed",
-    "novakv_debug_set_segment_weight",
+    "novakv_debug_set_segment_weight", "novakv_debug_set_fused_merge",
 ]
 
 
@@ -116,6 +116,7 @@ def load_library(path=None):
     lib.novakv_debug_set_scan_ctas.argtypes = [c_void_p, c_int]
     lib.novakv_debug_set_value_path.argtypes = [c_void_p, c_int]
     lib.novakv_debug_set_segment_weight.argtypes = [c_void_p, c_int]
+    lib.novakv_debug_set_fused_merge.argtypes = [c_void_p, c_int]
     lib.novakv_launch_count.restype = c_long
     if path is None:
         _lib = lib
@@ -342,6 +343,9 @@ class Context:
     def novakv_debug_set_segment_weight(self, pages):
         _check(self.lib, self.lib.novakv_debug_set_segment_weight(self.handle, int(pages)),
                "novakv_debug_set_segment_weight")
+
+    def novakv_debug_set_fused_merge(self, on):
+        _check(self.lib, self.lib.novakv_debug_set_fused_merge(self.handle, int(bool(on))), "novakv_debug_set_fused_merge")
 
     def novakv_launch_count(self):
         return int(self.lib.novakv_launch_count(self.handle))

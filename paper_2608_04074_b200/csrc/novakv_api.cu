@@ -595,6 +595,12 @@ extern "C" novakv_status novakv_debug_set_segment_weight(novakv_ctx* ctx, int pa
     return NOVAKV_OK;
 }
 
+extern "C" novakv_status novakv_debug_set_fused_merge(novakv_ctx* ctx, int on) {
+    if (!ctx || (on != 0 && on != 1)) return NOVAKV_EINVAL;
+    ctx->fused_merge = on != 0;
+    return NOVAKV_OK;
+}
+
 extern "C" novakv_status novakv_debug_set_value_path(novakv_ctx* ctx, int path) {
     if (!ctx || (path != 0 && path != 1)) return NOVAKV_EINVAL;
     ctx->value_path = path;

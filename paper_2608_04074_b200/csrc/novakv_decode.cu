@@ -34,6 +34,9 @@
 // blocks in swapped order.
 // The kernel contains no spin wait.
 #include <math_constants.h>
+#ifdef NOVAKV_TIMING
+#include <cstdio>
+#endif
 
 #include "novakv_internal.cuh"
 
@@ -56,6 +59,7 @@ constexpr int VCB_COPY_BYTES = 32768;         // 256 codes x 32 slots x 4 bytes
 constexpr int VCB_ROW = 128;
 constexpr int S1_SMEM_BYTES = 229376;         // dynamic shared memory requested (224 KB; the CTA also has a few static words)
 constexpr float M_INIT = -1.0e30f;
+constexpr int MAX_SCAN_CTAS = 255;            // scan CTAs (one per SM) the boundary table has room for
 
 // VM selects the value side: true = tensor cores (mma.sync m16n8k16, fp16 weights and codewords,
 // fp32 accumulators), false = CUDA cores (fp32 FMA).
@@ -88,7 +92,8 @@ struct S1 {
     static constexpr int OFFB_T32 = 0;
     static constexpr int OFFB_P = OFFB_T32 + T32_BYTES;
     static constexpr int OFFB_Q = OFFB_P + P_BYTES;                     // fp32 [HPAD][D]
-    static constexpr int BELOW_BYTES = OFFB_Q + HPAD * D * 4;
+    static constexpr int OFFB_BND = OFFB_Q + HPAD * D * 4;              // long [MAX_SCAN_CTAS + 1]: first unit of every CTA
+    static constexpr int BELOW_BYTES = OFFB_BND + (MAX_SCAN_CTAS + 1) * 8;
     // merge buffer (aliases the larger table once a segment's scan is done)
     static constexpr int MERGE_ACC_BYTES = NCW * HPAD * D * 4;
     static_assert(MERGE_ACC_BYTES + NCW * HPAD * 16 <= (HAS16 ? T16_BYTES : T32_BYTES), "merge buffer must fit in a table");
@@ -119,7 +124,9 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                       int32_t* __restrict__ page_prefix, uint32_t* __restrict__ dev_status,
                       const float* __restrict__ k_mean /* [Hkv][D] */, float* __restrict__ qk_off /* [batch][Hq] or null */,
                       int32_t* __restrict__ cost_prefix /* [batch + 1] */, int seg_weight,
-                      const float* __restrict__ k_center /* [Hkv][D], transform domain */, float* __restrict__ qc /* [batch][Hq] or null */) {
+                      const float* __restrict__ k_center /* [Hkv][D], transform domain */, float* __restrict__ qc /* [batch][Hq] or null */,
+                      int32_t* __restrict__ pair_count /* [Hkv * batch] arrival counters of the fused merge, or null */,
+                      void* __restrict__ out_fused /* outputs, when the scan kernel itself merges */, int out_is_fp32) {
     const int blk = blockIdx.x;
     constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
@@ -164,6 +171,17 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                     page_prefix[b] = carry + incl - v;
                     cost_prefix[b] = carry + incl - v + seg_weight * (carry_ne + incl_ne - ne);
                 }
+                // no scan CTA ever visits an empty sequence: with the merge fused into the scan its zeros are written here
+                if (out_fused != nullptr) {
+                    const unsigned empties = __ballot_sync(0xffffffffu, b < batch && v == 0);
+                    for (unsigned m = empties; m; m &= m - 1) {
+                        const size_t row = (size_t)(b0 + __ffs(m) - 1) * n_q_heads * D;
+                        for (int i = threadIdx.x; i < n_q_heads * D; i += 32) {
+                            if (out_is_fp32) reinterpret_cast<float*>(out_fused)[row + i] = 0.f;
+                            else reinterpret_cast<__nv_bfloat16*>(out_fused)[row + i] = __float2bfloat16_rn(0.f);
+                        }
+                    }
+                }
                 carry += __shfl_sync(0xffffffffu, incl, 31);
                 carry_ne += __shfl_sync(0xffffffffu, incl_ne, 31);
             }
@@ -172,6 +190,7 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
         return;
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (pair_count != nullptr && threadIdx.x == 0) pair_count[kvh * batch + b] = 0;
     __shared__ float q_s[HG][D];
     __shared__ float red_s[PARTS][HG][D];
     for (int i = threadIdx.x; i < HG * D; i += 512)
@@ -426,6 +445,82 @@ struct TileRegs {
     uint32_t vm;          // this lane's token: bfloat16 value scale (low half) and zero-point (high half), if used
 };
 
+// First unit of scan CTA c of G (c = G gives the end of the walk).  The walk is cut evenly in cost units,
+// cost = pages + seg_weight per (sequence, KV head) pair: cost point t lies in the pair whose cost interval
+// contains it and maps to unit  start + clamp(t - cost_start - seg_weight, 0, pages)  (the first seg_weight cost
+// units of a pair stand for setting up its score table).  seg_weight = 0 is the even split in pages.
+__device__ __forceinline__ long scan_boundary(int c, int G, const int32_t* __restrict__ page_prefix,
+                                              const int32_t* __restrict__ cost_prefix, int batch, int n_kv_heads, int seg_weight) {
+    const long P = page_prefix[batch], U = P * n_kv_heads;
+    if (seg_weight == 0) return ((long)c * U) / G;
+    const long cper = cost_prefix[batch], T = cper * n_kv_heads;
+    const long t = ((long)c * T) / G;
+    if (cper <= 0 || t >= T) return U;
+    const long kv = t / cper, rem = t - kv * cper;
+    int lo = 0, hi = batch - 1;                   // the last sequence whose cost interval starts at or before rem
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if ((long)cost_prefix[mid] <= rem) lo = mid; else hi = mid - 1;
+    }
+    const long p0 = page_prefix[lo], pg = page_prefix[lo + 1] - p0;
+    return kv * P + p0 + min(max(rem - cost_prefix[lo] - seg_weight, 0l), pg);
+}
+
+// Merge of one (sequence, KV head) pair inside the scan kernel, run by the CTA that wrote the pair's last
+// partial: exact log-sum-exp combination of the partials of the CTAs first .. last (those with an empty
+// range skipped), normalisation, inverse value transform o = o' rv^T + v_mean.  scratch: shared memory,
+// (1 + S1_THREADS / D) * HG * D floats.  Partials of other CTAs are read past the L1 (they were written by
+// other SMs; the arrival counter orders the accesses).
+template <int D, int HG>
+__device__ __noinline__ void fused_merge(float* scratch, const float* part_ml, const float* part_acc, int pair, int first,
+                                         int last, const long* s_bnd, const float* __restrict__ rv_t,
+                                         const float* __restrict__ v_mean, int kvh, void* __restrict__ out, int out_is_fp32,
+                                         size_t out_row /* (b * Hq + kvh * HG) * D */) {
+    constexpr int PARTS = S1_THREADS / D, COLS = D / PARTS;
+    float* o_s = scratch;                         // [HG][D]
+    float* red_s = scratch + HG * D;              // [PARTS][HG][D]
+    for (int i = threadIdx.x; i < HG * D; i += S1_THREADS) {
+        const int h = i / D, c = i - h * D;
+        float M = M_INIT;
+        for (int cta = first; cta <= last; ++cta)
+            if (s_bnd[cta] < s_bnd[cta + 1]) M = fmaxf(M, __ldcg(part_ml + (((size_t)pair + cta) * HG + h) * 2));
+        float a = 0.f, lsum = 0.f;
+        for (int cta = first; cta <= last; ++cta) {
+            if (s_bnd[cta] >= s_bnd[cta + 1]) continue;
+            const size_t pidx = (size_t)pair + cta;
+            const float sc = ex2(__ldcg(part_ml + (pidx * HG + h) * 2) - M);
+            a = fmaf(sc, __ldcg(part_acc + (pidx * HG + h) * D + c), a);
+            lsum = fmaf(sc, __ldcg(part_ml + (pidx * HG + h) * 2 + 1), lsum);
+        }
+        o_s[i] = lsum > 0.f ? a / lsum : 0.f;
+    }
+    __syncthreads();
+    {
+        const int r = threadIdx.x % D, part = threadIdx.x / D;
+        const float* R = rv_t + (size_t)kvh * D * D + (size_t)part * COLS * D + r;      // rv_t[c][r] = R_V[r][c]
+        float acc[HG];
+#pragma unroll
+        for (int h = 0; h < HG; ++h) acc[h] = 0.f;
+#pragma unroll 8
+        for (int c = 0; c < COLS; ++c) {
+            const float rv = R[(size_t)c * D];
+#pragma unroll
+            for (int h = 0; h < HG; ++h) acc[h] = fmaf(o_s[h * D + part * COLS + c], rv, acc[h]);
+        }
+#pragma unroll
+        for (int h = 0; h < HG; ++h) red_s[(part * HG + h) * D + r] = acc[h];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < HG * D; i += S1_THREADS) {
+        const int h = i / D, r = i - h * D;
+        float o = v_mean[(size_t)kvh * D + r];
+#pragma unroll
+        for (int p = 0; p < PARTS; ++p) o += red_s[(p * HG + h) * D + r];
+        if (out_is_fp32) reinterpret_cast<float*>(out)[out_row + i] = o;
+        else reinterpret_cast<__nv_bfloat16*>(out)[out_row + i] = __float2bfloat16_rn(o);
+    }
+}
+
 // KSC: the key format carries a per-token bfloat16 scale (k_scales [n_pages][Hkv][64]); the logits of a
 // token are multiplied by it once, after the table lookups are summed (and the centre's share added back).
 // VSQ: scalar INT2 values with a per-token bfloat16 scale and zero-point (v_meta [n_pages][Hkv][64][2]).
@@ -454,7 +549,12 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                             int batch, int n_q_heads, int n_kv_heads, float* __restrict__ part_ml,
                             float* __restrict__ part_acc, uint32_t* __restrict__ dev_status, int pt_stride,
                             const int32_t* __restrict__ cost_prefix, int seg_weight, long* __restrict__ cta_range,
-                            const float* __restrict__ qc, int vcb_per_head) {
+                            const float* __restrict__ qc, int vcb_per_head,
+                            int32_t* __restrict__ pair_count, const float* __restrict__ rv_t,
+                            const float* __restrict__ v_mean, void* __restrict__ out_fused, int out_is_fp32) {
+    // out_fused != null: the CTA that writes the last partial of a (sequence, KV head) pair also merges the pair's
+    // partials and applies the inverse value transform (no merge kernel follows); pair_count holds one arrival
+    // counter per pair, zero on entry and reset to zero by the merging CTA.  Nothing waits on another CTA.
     // page_table points at the first column that is scanned; rows are pt_stride entries apart and
     // max_pages_per_seq bounds the pages of a row that may be read from there
     using C = S1<D, HG, VM>;
@@ -465,7 +565,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     constexpr float CEN = VSQ ? 1024.f : 1152.f;              // what one unit of weight adds to a tensor-core sum beyond u - centre
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_found[4];
-    __shared__ long s_bnd[2];
+    __shared__ int s_arrived, s_first, s_last;
     // ---- shared-memory map (see S1)
     const uint32_t s_base = smem_u32(smem);
     const uint32_t t16_abs = HAS16 ? ((s_base + C::BELOW_BYTES + 65535u) & ~65535u) : s_base + C::BELOW_BYTES;
@@ -490,40 +590,19 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     // lands behind the segment lookup and the first table build.
     int vcb_head = (int)(((long)blockIdx.x * n_kv_heads) / gridDim.x);   // KV head whose value codebook is resident
     stage_value_codebook_async<HAS16>(vcb_p, cb_v_img + (size_t)vcb_head * vcb_per_head);
-    novakv_grid_dependency_wait();
+    // With the merge fused in, the kernels that follow (the query transform of the next call writes the same
+    // workspace) must not start before this grid is done: no early release of the dependents.
+    if (out_fused != nullptr) asm volatile("griddepcontrol.wait;" ::: "memory");
+    else novakv_grid_dependency_wait();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // This CTA's range of the walk [u_begin, u_end).  The walk is cut evenly in cost units, cost = pages +
-    // seg_weight per (sequence, KV head) pair: cost point t lies in the pair whose cost interval contains it
-    // and maps to unit  start + clamp(t - cost_start - seg_weight, 0, pages)  (the first seg_weight cost units
-    // of a pair stand for setting up its score table).  seg_weight = 0 is the even split in pages.
-    long u_begin, u_end;
-    {
-        const long P = page_prefix[batch], U = P * n_kv_heads;
-        if (seg_weight == 0) {
-            u_begin = ((long)blockIdx.x * U) / gridDim.x;
-            u_end = ((long)(blockIdx.x + 1) * U) / gridDim.x;
-        } else {
-            const long cper = cost_prefix[batch], T = cper * n_kv_heads;
-            const long t0 = ((long)blockIdx.x * T) / gridDim.x, t1 = ((long)(blockIdx.x + 1) * T) / gridDim.x;
-            if (threadIdx.x < 2) s_bnd[threadIdx.x] = U;              // a cost point at the very end
-            __syncthreads();
-            if (cper > 0) {
-                const long kv0 = t0 / cper, kv1 = t1 / cper;
-                const long rem0 = t0 - kv0 * cper, rem1 = t1 - kv1 * cper;
-                for (int t = threadIdx.x; t < batch; t += S1_THREADS) {
-                    const long lo = cost_prefix[t], hi = cost_prefix[t + 1];
-                    const long p0 = page_prefix[t], pg = page_prefix[t + 1] - p0;
-                    if (t0 < T && lo <= rem0 && rem0 < hi) s_bnd[0] = kv0 * P + p0 + min(max(rem0 - lo - seg_weight, 0l), pg);
-                    if (t1 < T && lo <= rem1 && rem1 < hi) s_bnd[1] = kv1 * P + p0 + min(max(rem1 - lo - seg_weight, 0l), pg);
-                }
-            }
-            __syncthreads();
-            u_begin = s_bnd[0];
-            u_end = s_bnd[1];
-        }
-        if (threadIdx.x == 0) { cta_range[blockIdx.x * 2] = u_begin; cta_range[blockIdx.x * 2 + 1] = u_end; }
-    }
+    // First unit of every CTA (see scan_boundary): one thread per boundary.  This CTA owns [s_bnd[c], s_bnd[c + 1]).
+    long* const s_bnd = reinterpret_cast<long*>(smem + C::OFFB_BND);
+    for (int c = threadIdx.x; c <= (int)gridDim.x; c += S1_THREADS)
+        s_bnd[c] = scan_boundary(c, gridDim.x, page_prefix, cost_prefix, batch, n_kv_heads, seg_weight);
+    __syncthreads();
+    const long u_begin = s_bnd[blockIdx.x], u_end = s_bnd[blockIdx.x + 1];
+    if (threadIdx.x == 0) { cta_range[blockIdx.x * 2] = u_begin; cta_range[blockIdx.x * 2 + 1] = u_end; }
     if (u_begin >= u_end) { async_copies_wait(); return; }
 
     // ---- lane roles and constants
@@ -597,8 +676,18 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         }
     };
 
+#ifdef NOVAKV_TIMING
+    long long tm[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long t_prev = clock64();
+    const long long t_start = t_prev;
+    int n_seg = 0;
+#define NOVAKV_TICK(i) { const long long t_now = clock64(); tm[i] += t_now - t_prev; t_prev = t_now; }
+#else
+#define NOVAKV_TICK(i)
+#endif
     long u = u_begin;
     while (u < u_end) {
+        NOVAKV_TICK(0)
         const Segment sg = locate(page_prefix, seq_lens, batch, max_pages_per_seq, u, u_end, s_found);
         const int pair = sg.kvh * batch + sg.b;            // grows along the walk
 
@@ -897,9 +986,12 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         TileRegs<L> ta;
         if (n_it > 0) load_tile(0, ta);
         __syncthreads();     // q' of the pair is in shared memory
+        NOVAKV_TICK(1)
         build_score_table<D, HG, VM>(t32_p, t16_p, cb_k_lut + (size_t)sg.kvh * 256 * L * 4, q_s);
+        NOVAKV_TICK(2)
         async_copies_wait();
         __syncthreads();     // table and value codebook complete
+        NOVAKV_TICK(3)
 
         // ---- scan: 32-token tiles, the next tile's loads in flight while one is consumed
         for (int it = 0; it < n_it; ++it) {
@@ -909,8 +1001,10 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         }
 
         // ---- segment epilogue: merge the warps' partials, write one partial ---------------------
+        NOVAKV_TICK(4)
         if (VM) flush_window();
         __syncthreads();                                   // scan done everywhere: the tables are dead
+        NOVAKV_TICK(5)
         unsigned char* const merge_p = HAS16 ? t16_p : t32_p;
         float* m_acc = reinterpret_cast<float*>(merge_p);                              // [NCW][HPAD][D]
         float* m_ml = reinterpret_cast<float*>(merge_p + C::MERGE_ACC_BYTES);          // [NCW][HPAD][2]
@@ -1005,9 +1099,44 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 if (c == 0) { part_ml[(pidx * HG + h) * 2] = M; part_ml[(pidx * HG + h) * 2 + 1] = lsum * unscale; }
             }
         }
+        if (out_fused != nullptr) {
+            // arrival: this CTA's partial is visible before its count is; the CTA that completes the count merges
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                s_arrived = atomicAdd(&pair_count[pair], 1) + 1;
+                s_first = gridDim.x;
+                s_last = -1;
+            }
+            __syncthreads();
+            const long P = page_prefix[batch];
+            const long pu0 = (long)sg.kvh * P + page_prefix[sg.b], pu1 = pu0 + (sg.len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
+            bool touches = false;                           // CTA threadIdx.x has a non-empty share of this pair
+            if (threadIdx.x < gridDim.x) {
+                const int c = threadIdx.x;
+                touches = s_bnd[c] < s_bnd[c + 1] && s_bnd[c] < pu1 && s_bnd[c + 1] > pu0;
+                if (touches) { atomicMin(&s_first, c); atomicMax(&s_last, c); }
+            }
+            const int expected = __syncthreads_count(touches);
+            if (s_arrived == expected) {
+                __threadfence();
+                fused_merge<D, HG>(reinterpret_cast<float*>(t32_p), part_ml, part_acc, pair, s_first, s_last, s_bnd, rv_t, v_mean,
+                                   sg.kvh, out_fused, out_is_fp32, ((size_t)sg.b * n_q_heads + sg.kvh * HG) * D);
+                if (threadIdx.x == 0) pair_count[pair] = 0;
+            }
+        }
         __syncthreads();                                   // merge buffer free before the next table build
+        NOVAKV_TICK(6)
+#ifdef NOVAKV_TIMING
+        ++n_seg;
+#endif
         u += sg.npg;
     }
+#ifdef NOVAKV_TIMING
+    if (threadIdx.x == 0 && (blockIdx.x % 21 == 0 || blockIdx.x == gridDim.x - 1))
+        printf("cta %3d segs %d pages %ld | clocks: pre-loop %lld locate+q %lld build %lld vcbwait %lld scan(w0) %lld barrier %lld epilogue %lld total %lld\n",
+               blockIdx.x, n_seg, (long)(u_end - u_begin), tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], clock64() - t_start);
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1257,7 +1386,7 @@ novakv_band_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 
 // workspace layout
 struct WsLayout {
-    size_t qp, prefix, cost, range, qk, qc, bml, bacc, ml, acc, total;
+    size_t qp, prefix, cost, range, qk, qc, cnt, bml, bacc, ml, acc, total;
 };
 WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     auto al = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -1270,7 +1399,8 @@ WsLayout ws_layout(const novakv_ctx* ctx, int batch) {
     w.range = al(w.cost + ((size_t)batch + 1) * 4);
     w.qk = al(w.range + (size_t)ctx->n_sm * 2 * sizeof(long));
     w.qc = al(w.qk + (size_t)batch * hq * 4);
-    w.bml = al(w.qc + (size_t)batch * hq * 4);
+    w.cnt = al(w.qc + (size_t)batch * hq * 4);
+    w.bml = al(w.cnt + (size_t)batch * ctx->cfg.n_kv_heads * 4);
     w.bacc = al(w.bml + (size_t)batch * hq * 2 * 4);
     w.ml = al(w.bacc + (size_t)batch * hq * d * 4);
     w.acc = al(w.ml + n_part * ctx->hg * 2 * 4);
@@ -1309,11 +1439,19 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
     float* band_acc = band ? (float*)(ws + w.bacc) : nullptr;
     float* part_ml = (float*)(ws + w.ml);
     float* part_acc = (float*)(ws + w.acc);
+    int32_t* pair_count = (int32_t*)(ws + w.cnt);
     const int hq = ctx->cfg.n_q_heads, hkv = ctx->cfg.n_kv_heads;
+    const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
+    if (grid > MAX_SCAN_CTAS) return NOVAKV_EUNSUPPORTED;
+    // Optionally (novakv_debug_set_fused_merge), without a sink logit or a BF16 band, the scan kernel merges each
+    // (sequence, KV head) pair itself (the CTA that writes the pair's last partial does it); otherwise the merge
+    // kernel follows.
+    const bool fuse = sink_logits == nullptr && band == nullptr && ctx->fused_merge;
 
     novakv_launch_pdl(novakv_prepare_kernel<D, HG>, dim3(batch * hkv + 1), dim3(512), 0, stream, q, ly.rk_inv_t, seq_lens,
                       batch, hq, hkv, max_pages_per_seq, sm_scale * 1.4426950408889634f, qp, prefix, ctx->dev_status,
-                      k_off_vec, qk_off, cost_prefix, ctx->seg_weight, (const float*)ly.k_center, qc);
+                      k_off_vec, qk_off, cost_prefix, ctx->seg_weight, (const float*)ly.k_center, qc,
+                      fuse ? pair_count : (int32_t*)nullptr, fuse ? out : (void*)nullptr, out_is_fp32);
     ctx->launches++;
 
     auto kern = novakv_decode_stage1_kernel<D, HG, VM, KSC, VSQ>;
@@ -1323,7 +1461,6 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S1_SMEM_BYTES) != cudaSuccess) return NOVAKV_ECUDA;
         ctx->smem_opt_in |= inst_bit;
     }
-    const int grid = ctx->scan_ctas > 0 ? (ctx->scan_ctas < ctx->n_sm ? ctx->scan_ctas : ctx->n_sm) : ctx->n_sm;
     {
         novakv_prof_scope ps(ctx, 0, stream);
         novakv_launch_pdl(kern, dim3(grid), dim3(S1_THREADS), S1_SMEM_BYTES, stream, qp, ly.cb_k_lut,
@@ -1331,7 +1468,8 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                           (const float*)ly.v_off, k_pages, v_pages, k_scales, v_meta, n_pages, page_table, max_pages_per_seq,
                           seq_lens, prefix, batch, hq, hkv, part_ml, part_acc, ctx->dev_status, pt_stride,
                           (const int32_t*)cost_prefix, ctx->seg_weight, cta_range, (const float*)qc,
-                          VSQ ? 0 : VCB_COPY_BYTES);
+                          VSQ ? 0 : VCB_COPY_BYTES, pair_count, (const float*)ly.rv_t, (const float*)ly.v_mean,
+                          fuse ? out : (void*)nullptr, out_is_fp32);
         ps.end();
         ctx->launches++;
     }
@@ -1341,6 +1479,7 @@ novakv_status launch_decode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
                           band_acc);
         ctx->launches++;
     }
+    if (fuse) return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
     const bool ext = sink_logits != nullptr || band != nullptr;
     auto merge = batch * hkv > 2 * ctx->n_sm
                      ? (ext ? novakv_decode_merge_kernel<D, HG, 2, true> : novakv_decode_merge_kernel<D, HG, 2, false>)

@@ -56,6 +56,7 @@ struct novakv_ctx {
     int scan_ctas = 0;            // 0 = one per SM
     int value_path = 1;           // 1 = tensor cores, 0 = CUDA cores
     int seg_weight = 24;          // pages one (sequence, KV head) segment weighs extra in the scan kernel's work split
+    bool fused_merge = false;     // true: the scan kernel merges the partials itself where it can (no sink, no band)
     unsigned smem_opt_in = 0;     // scan-kernel instantiations whose shared-memory opt-in was set on this device
 };
 

@@ -120,9 +120,13 @@ def test_decode_matches_oracle(name, lens, request):
     encs = _fill_with_oracle(case, cache, lens, 300)
     _, _, q = case.draw(301, 1, len(lens))
     refs = [case.oracle.decode(q[b].astype(np.float64), encs[b]["kidx"], encs[b]["vidx"]) for b in range(len(lens))]
-    for path, label in ((1, "tensor-core value side"), (0, "CUDA-core value side")):
+    for path, fused, label in ((1, 1, "tensor-core value side"), (0, 1, "CUDA-core value side"),
+                               (1, 0, "tensor-core value side, separate merge kernel")):
         case.ctx.novakv_debug_set_value_path(path)
-        out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+        case.ctx.novakv_debug_set_fused_merge(fused)
+        out = torch.full((len(lens), case.ctx.n_q_heads, case.ctx.head_dim), float("nan"), device="cuda")
+        cache.decode(0, _dev(q, torch.bfloat16), out=out)
+        out = out.cpu().numpy()
         assert case.ctx.novakv_last_device_status() == 0
         worst = 0.0
         for b, n in enumerate(lens):
@@ -132,6 +136,7 @@ def test_decode_matches_oracle(name, lens, request):
             worst = max(worst, check_output(out[b], refs[b]))
         print(f"[{name} {lens.tolist()} {label}] max|delta|/||o||inf = {worst:.3e}")
     case.ctx.novakv_debug_set_value_path(1)
+    case.ctx.novakv_debug_set_fused_merge(1)
 
 
 # --------------------------------------------------------------------------- T4: split invariance, determinism
