@@ -764,6 +764,50 @@ def _run_reference_rank0(args, world):
     }))
 
 
+def run_profile_case(args):
+    """`--profile-case NAME`: a short decode-only (or encode-only) loop of one workload shape, for profiler captures
+    of the kernels the sweep times (the captures summarised under profiles/ were taken with these commands).
+    Index bytes are random (timing and counters do not depend on them); prints a small JSON line, not the
+    benchmark contract."""
+    import torch
+    from paper_2608_04074_b200 import synth, workloads
+    from paper_2608_04074_b200.binding import Context
+    from paper_2608_04074_b200.runtime import PagedCache, bf16_tensor
+    name = args.profile_case
+    if name == "gptoss":
+        wl = workloads.gpt_oss_20b(batch=args.batch, seq_len=args.seq_len, calib_tokens=2048, lloyd_iters=2)
+    elif name == "mix":
+        wl = workloads.paged_mix(calib_tokens=2048, lloyd_iters=2)
+    elif name in ("qwen", "encode"):
+        wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len, calib_tokens=2048, lloyd_iters=2)
+    else:
+        raise SystemExit(f"unknown profile case {name}")
+    laws = wl.laws()
+    cal = wl.calibration(laws)
+    s = wl.shape
+    ctx = Context(s.n_q_heads, s.n_kv_heads, s.head_dim)
+    ctx.novakv_load_calibration(0, cal)
+    cache = PagedCache(ctx, wl.seq_lens, seed=3)
+    times = []
+    if name == "encode":
+        T = int(wl.seq_lens.sum())
+        k, v = synth.draw_kv(laws, 7200, T)
+        kd, vd = bf16_tensor(k), bf16_tensor(v)
+        ts = torch.repeat_interleave(torch.arange(wl.batch, dtype=torch.int32, device="cuda"),
+                                     torch.from_numpy(wl.seq_lens.astype(np.int64)).cuda())
+        tp = torch.cat([torch.arange(int(n), dtype=torch.int32, device="cuda") for n in wl.seq_lens])
+        fn = lambda: cache.append(0, kd, vd, ts, tp)
+    else:
+        cache.k_pages.random_(0, 256)
+        cache.v_pages.random_(0, 256)
+        q = bf16_tensor(synth.draw_q(laws, 5, wl.batch))
+        out = torch.empty((wl.batch, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda")
+        fn = lambda: cache.decode(0, q, out=out)
+    times = time_steps(fn, args.steps, args.warmup, lambda: None)
+    print(json.dumps({"profile_case": name, "batch": wl.batch, "tokens": int(wl.seq_lens.astype(np.int64).sum()),
+                      "ms_median": round(statistics.median(times), 5), "device_status": ctx.novakv_last_device_status()}))
+
+
 def launch_ranks(n):
     """`--gpus N` outside a launcher: re-run this script as N ranks of one node under torch.distributed.run
     (one rank per GPU, rendezvous on 127.0.0.1) and return its exit code.  NCCL's communicator log is kept
@@ -790,10 +834,15 @@ def main():
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--seq-len", type=int, default=16384)
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--profile-case", default=None, choices=["qwen", "gptoss", "mix", "encode"],
+                    help="profiling helper: short decode-only (encode-only) loop of one workload shape")
     ap.add_argument("--calib-tokens", type=int, default=8192, help="calibration tokens per KV head (set-up cost only)")
     ap.add_argument("--lloyd-iters", type=int, default=12, help="Lloyd iterations of the calibration (set-up cost only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.profile_case:
+        run_profile_case(args)
+        return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(launch_ranks(args.gpus))
     if args.impl == "reference":

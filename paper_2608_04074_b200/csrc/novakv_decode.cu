@@ -60,6 +60,7 @@ constexpr int VCB_ROW = 128;
 constexpr int S1_SMEM_BYTES = 229376;         // dynamic shared memory requested (224 KB; the CTA also has a few static words)
 constexpr float M_INIT = -1.0e30f;
 constexpr int MAX_SCAN_CTAS = 255;            // scan CTAs (one per SM) the boundary table has room for
+constexpr int PFX_CAP = 511;                  // batches up to this size keep their page / cost prefixes in shared memory
 
 // VM selects the value side: true = tensor cores (mma.sync m16n8k16, fp16 weights and codewords,
 // fp32 accumulators), false = CUDA cores (fp32 FMA).
@@ -93,7 +94,8 @@ struct S1 {
     static constexpr int OFFB_P = OFFB_T32 + T32_BYTES;
     static constexpr int OFFB_Q = OFFB_P + P_BYTES;                     // fp32 [HPAD][D]
     static constexpr int OFFB_BND = OFFB_Q + HPAD * D * 4;              // long [MAX_SCAN_CTAS + 1]: first unit of every CTA
-    static constexpr int BELOW_BYTES = OFFB_BND + (MAX_SCAN_CTAS + 1) * 8;
+    static constexpr int OFFB_PFX = OFFB_BND + (MAX_SCAN_CTAS + 1) * 8; // int [2][PFX_CAP + 1]: page and cost prefix of small batches
+    static constexpr int BELOW_BYTES = OFFB_PFX + 2 * (PFX_CAP + 1) * 4;
     // merge buffer (aliases the larger table once a segment's scan is done)
     static constexpr int MERGE_ACC_BYTES = NCW * HPAD * D * 4;
     static_assert(MERGE_ACC_BYTES + NCW * HPAD * 16 <= (HAS16 ? T16_BYTES : T32_BYTES), "merge buffer must fit in a table");
@@ -596,6 +598,14 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     else novakv_grid_dependency_wait();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // The two prefixes are read many times (boundaries, segment look-ups): small batches keep them in shared memory.
+    if (batch <= PFX_CAP) {
+        int32_t* pfx = reinterpret_cast<int32_t*>(smem + C::OFFB_PFX);
+        for (int i = threadIdx.x; i <= batch; i += S1_THREADS) { pfx[i] = page_prefix[i]; pfx[PFX_CAP + 1 + i] = cost_prefix[i]; }
+        __syncthreads();
+        page_prefix = pfx;
+        cost_prefix = pfx + PFX_CAP + 1;
+    }
     // First unit of every CTA (see scan_boundary): one thread per boundary.  This CTA owns [s_bnd[c], s_bnd[c + 1]).
     long* const s_bnd = reinterpret_cast<long*>(smem + C::OFFB_BND);
     for (int c = threadIdx.x; c <= (int)gridDim.x; c += S1_THREADS)
@@ -1180,31 +1190,42 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
     const int pages_b = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
     const long P = page_prefix[batch];
     const int slot0 = kvh * batch + b;                     // the scan kernel's pair index (walk order)
+    // CTAs that may hold a piece of this pair: those whose cost range meets the pair's (the largest c with
+    // floor(c*T/G) <= x for its first and last cost unit), widened by one on each side; the ranges the scan
+    // CTAs recorded decide.  Their ranges, then their (max, sum) pairs, are fetched into shared memory by
+    // parallel threads (two memory latencies, whatever the number of pieces), so that the loop below only issues
+    // independent loads of the accumulators.
+    __shared__ int cand_s[MAX_SCAN_CTAS + 1];              // 1 = this CTA holds a piece of the pair
+    __shared__ float2 ml_s[MAX_SCAN_CTAS + 1][HG];
+    int c_first = 0, n_cand = 0;
+    if (pages_b > 0) {
+        const long u0 = (long)kvh * P + page_prefix[b], u1 = u0 + pages_b;
+        const long T = (long)cost_prefix[batch] * n_kv_heads;
+        const long x0 = (long)kvh * cost_prefix[batch] + cost_prefix[b] + seg_weight, x1 = x0 + pages_b - 1;
+        c_first = max((int)(((x0 + 1) * grid_s1 - 1) / T) - 1, 0);
+        const int c_last = min((int)(((x1 + 1) * grid_s1 - 1) / T) + 1, grid_s1 - 1);
+        n_cand = min(c_last - c_first + 1, MAX_SCAN_CTAS + 1);
+        for (int t = threadIdx.x; t < n_cand; t += blockDim.x) {
+            const long r0 = cta_range[(c_first + t) * 2], r1 = cta_range[(c_first + t) * 2 + 1];
+            cand_s[t] = (r0 < r1 && r1 > u0 && r0 < u1) ? 1 : 0;
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < n_cand * HG; t += blockDim.x) {
+            const int ci = t / HG, h = t - ci * HG;
+            if (cand_s[ci]) ml_s[ci][h] = *reinterpret_cast<const float2*>(part_ml + (((size_t)slot0 + c_first + ci) * HG + h) * 2);
+        }
+        __syncthreads();
+    }
     for (int i = threadIdx.x; i < HG * D; i += blockDim.x) {
         const int h = i / D, c = i - h * D;
         float M = M_INIT, a = 0.f, lsum = 0.f;
-        if (pages_b > 0) {
-            const long u0 = (long)kvh * P + page_prefix[b], u1 = u0 + pages_b;
-            // CTAs that may hold a piece of this pair: those whose cost range meets the pair's (the largest c
-            // with floor(c*T/G) <= x for its first and last cost unit), widened by one on each side; the
-            // ranges the scan CTAs recorded decide
-            const long T = (long)cost_prefix[batch] * n_kv_heads;
-            const long x0 = (long)kvh * cost_prefix[batch] + cost_prefix[b] + seg_weight, x1 = x0 + pages_b - 1;
-            const int c_first = max((int)(((x0 + 1) * grid_s1 - 1) / T) - 1, 0);
-            const int c_last = min((int)(((x1 + 1) * grid_s1 - 1) / T) + 1, grid_s1 - 1);
-            for (int cta = c_first; cta <= c_last; ++cta) {
-                const long r0 = cta_range[cta * 2], r1 = cta_range[cta * 2 + 1];
-                if (r0 >= r1 || r1 <= u0 || r0 >= u1) continue;
-                M = fmaxf(M, part_ml[(((size_t)slot0 + cta) * HG + h) * 2]);
-            }
-            for (int cta = c_first; cta <= c_last; ++cta) {
-                const long r0 = cta_range[cta * 2], r1 = cta_range[cta * 2 + 1];
-                if (r0 >= r1 || r1 <= u0 || r0 >= u1) continue;
-                const size_t pidx = (size_t)slot0 + cta;
-                const float sc = ex2(part_ml[(pidx * HG + h) * 2] - M);
-                a = fmaf(sc, part_acc[(pidx * HG + h) * D + c], a);
-                lsum = fmaf(sc, part_ml[(pidx * HG + h) * 2 + 1], lsum);
-            }
+        for (int ci = 0; ci < n_cand; ++ci)
+            if (cand_s[ci]) M = fmaxf(M, ml_s[ci][h].x);
+        for (int ci = 0; ci < n_cand; ++ci) {
+            if (!cand_s[ci]) continue;
+            const float sc = ex2(ml_s[ci][h].x - M);
+            a = fmaf(sc, part_acc[(((size_t)slot0 + c_first + ci) * HG + h) * D + c], a);
+            lsum = fmaf(sc, ml_s[ci][h].y, lsum);
         }
         float lq = lsum;          // mass of the quantised tokens at the running scale
         float wb = 0.f;           // weight of the band accumulator at the running scale
