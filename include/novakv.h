@@ -161,7 +161,7 @@ novakv_status novakv_decode_attention(novakv_ctx* ctx, int layer, const void* q,
 
 /*
  * Key format with a per-token scale (Algorithm 3, the "Normalize" step; App. B "Decoding kernel and
- * read path": the kernel "applies the per-token scale rho_j recovered from metadata (one multiply)";
+ * read path": the read kernel fetches rho_j from per-token metadata and applies it with a single multiply;
  * Sec. 5 "Bit rate": one BF16 scale per token and KV head, 16/d extra bits per key element, 2.125 at
  * d = 128).  The key codebooks of the layer must have been trained on normalised coefficients.
  *   write:  r as in novakv_encode_append (binary32 coefficients);
@@ -217,10 +217,10 @@ novakv_status novakv_decode_attention_sink(novakv_ctx* ctx, int layer, const voi
  *                onwards of its page-table row); quant_lens device int32 [batch]; n_sink a multiple of 64
  *   band_k, band_v  device bf16 [batch][band_cap][Hkv][d].  Of sequence b, slots 0 .. sink_cnt-1 hold
  *                its first tokens, and slots n_sink + (ring_start + i) % (band_cap - n_sink),
- *                i < ring_len, its most recent ones (a ring: "new tokens enter the BF16 recent band and
- *                are quantized in blocks of eight steps" - the caller appends to the ring and, when it
- *                has grown by eight, passes the eight oldest to novakv_encode_append[_scaled] and
- *                advances ring_start and quant_lens)
+ *                i < ring_len, its most recent ones (a ring: App. B has a new token join the recent band
+ *                first and leaves quantisation to batches of eight decode steps - the caller appends to
+ *                the ring and, when it has grown by eight, passes the eight oldest to
+ *                novakv_encode_append[_scaled] and advances ring_start and quant_lens)
  *   band_meta    device int32 [batch][3] = (sink_cnt, ring_start, ring_len); values are clamped to the
  *                buffer
  *   k_scales, sink_logits  NULL or as in novakv_decode_attention_scaled / _sink
@@ -234,9 +234,10 @@ novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int layer, const v
     novakv_stream stream);
 
 /*
- * The paper's deployed cache format (Sec. 5 "Bit rate": keys 2.125 bits per element, "the V cache is INT2
- * with a BF16 scale and offset (zero-point), giving 2.000 + 32/128 = 2.250"; App. B read path: "the INT2
- * code is dequantized in the ... rotation basis"): keys as in novakv_encode_append_scaled; values scalar
+ * The paper's deployed cache format (Sec. 5 "Bit rate": keys at 2.125 bits per element; values as 2-bit
+ * integers with one BF16 scale and one BF16 zero-point per token, 2 + 32/128 = 2.25 bits per element;
+ * App. B read path: the 2-bit codes are dequantised in a rotation basis): keys as in
+ * novakv_encode_append_scaled; values scalar
  * quantised to 2 bits in the Corollary 1 basis R_V (which stands in for the rotation the paper takes from
  * prior work), one bf16 (scale, zero) pair per token and KV head:
  *     s = (v - v_mean) rv                      binary32 coefficients, as in novakv_encode_append

@@ -244,8 +244,8 @@ void oracle_decode(const oracle_tables* t, const double* q, const uint8_t* kidx,
 
 /* ------------------------------------------------------------------------------------------------
  * Key format with a per-token scale (Algorithm "Codebook training", the "Normalize" step; App. B
- * "Decoding kernel and read path": the kernel "applies the per-token scale rho_j recovered from
- * metadata (one multiply)"; Sec. 5 "Bit rate": a BF16 scale per token, 16/128 = 0.125 bit/elem).
+ * "Decoding kernel and read path": the read side takes rho_j from per-token metadata and applies it
+ * with a single multiply; Sec. 5 "Bit rate": a BF16 scale per token, 16/128 = 0.125 bit/elem).
  *
  *   rho_j = ||r_j||_2 / sqrt(d),   r_j <- r_j / rho_j   before the codebook search,
  *   k^_j  = rho_j * Q(r_j / rho_j) R_K^{-1} + kbar       on the read side.
@@ -407,9 +407,9 @@ void oracle_decode_sink(const oracle_tables* t, const double* q, const uint8_t* 
 }
 
 /* ------------------------------------------------------------------------------------------------
- * Scalar value codec of the deployed format (Sec. 5 "Bit rate": "The V cache is INT2 with a BF16
- * scale and offset (zero-point), giving 2.000 + 32/128 = 2.250"; App. B read path: "the INT2 code is
- * dequantized in the ... rotation basis"), in the Corollary 1 basis R_V:
+ * Scalar value codec of the deployed format (Sec. 5 "Bit rate": values are 2-bit integers with one BF16
+ * scale and one BF16 zero-point per token, 2 + 32/128 = 2.25 bits per element; App. B read path: the
+ * codes are dequantised in a rotation basis), in the Corollary 1 basis R_V:
  *     s = (v - vbar) R_V,   code_i = clamp(round((s_i - zero) / scale), 0, 3),
  *     s^_i = zero + scale * code_i,   v^ = s^ R_V^T + vbar,
  * one (scale, zero) pair per token and KV head.  Where floating point decides stored bits the
