@@ -362,7 +362,7 @@ def run_ours(args):
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None,
-            "dtype": "f32 accumulation; f32/f16 score-table entries; f16 MMA operands on the value side (u8 grid codewords)",
+            "dtype": "f32 accumulation; f32/f16 score-table entries; f16 MMA operands on the value side (7-bit grid codewords)",
             "data": "synthetic", "ms_per_step_min": round(min(times), 5),
             "config": {"workload": f"qwen3_8b_shape decode step: Hq=32 Hkv=8 d=128 B={B} S={S}+1 per GPU, "
                                    "2-bit VQ K and V (g=4, 256-entry codebooks), bf16 q, 64-token pages; "

@@ -13,7 +13,7 @@
  * and one for values.  Inside a chunk (t = token slot in the page, l = group):
  *     keys    [tile = t/32][plane][t%32][16 bytes]: byte j of a token's L bytes holds the code of group
  *             j ^ (t % 8) for j < 16 and of group j ^ (t % 16) for j >= 16; plane = j / 16.
- *     values  [block = t/16][fr = l%8][fc = t%4][gb = l/8][b = (t%16)/4].
+ *     values  [block = t/16][fr = l%8][fc = t%4][gb = (l/8) ^ (t%2)][b = (t%16)/4].
  * Both orders make every lane of a decode warp load exactly the bytes it consumes with coalesced
  * 128-bit loads, and keep its shared-memory table gathers free of bank conflicts.
  * page_table[seq][i] (int32, row length max_pages_per_seq) names the page of tokens 64i..64i+63.
@@ -53,7 +53,7 @@ typedef enum {
     NOVAKV_EPAGE = 4,         /* page-table geometry inconsistent */
     NOVAKV_EWORKSPACE = 5,    /* workspace NULL or too small */
     NOVAKV_ECUDA = 6,         /* a CUDA runtime call failed */
-    NOVAKV_EUNSUPPORTED = 7   /* value codebook off its 8-bit grid, etc. */
+    NOVAKV_EUNSUPPORTED = 7   /* value codebook off its 7-bit grid, etc. */
 } novakv_status;
 
 /* Bits of the device status word. */
@@ -86,8 +86,8 @@ typedef struct {
  *   k_mean    [Hkv][d]      may be NULL (= 0)
  *   v_mean    [Hkv][d]      may be NULL (= 0)
  *   cb_k      [Hkv][L][256][4]
- *   cb_v      [Hkv][L][256][4]   every coordinate (head, l, component) on its own 8-bit grid:
- *                                lo + u (hi - lo) / 255, u = 0..255, lo / hi = its smallest / largest value
+ *   cb_v      [Hkv][L][256][4]   every coordinate (head, l, component) on its own 7-bit grid:
+ *                                lo + u (hi - lo) / 127, u = 0..127, lo / hi = its smallest / largest value
  *                                over the 256 codewords, evaluated in binary64, rounded once to binary32
  */
 typedef struct {
@@ -107,7 +107,7 @@ const char* novakv_status_string(novakv_status s);
 /*
  * Algorithm 1 lines 1-6 produce these tables offline; this call copies them to the device
  * (synchronous; the caller keeps its memory).  Returns NOVAKV_EUNSUPPORTED if cb_v holds a value
- * off its 8-bit grid (the decode kernel keeps a value codeword as four grid indices; snap the
+ * off its 7-bit grid (the decode kernel keeps a value codeword as four grid indices; snap the
  * codebooks offline, as the paper does for its own, so that encoder, decoder and any reference agree).
  */
 novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, const novakv_calibration* host);

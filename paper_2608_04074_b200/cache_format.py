@@ -46,7 +46,7 @@ def value_offset(t, l, n_groups_: int):
     ngb = n_groups_ // 8
     tb = t & 15
     fc, b, fr = tb & 3, tb >> 2, l & 7
-    return (t >> 4) * (n_groups_ * 16) + (fr * 4 + fc) * (ngb * 4) + (l >> 3) * 4 + b
+    return (t >> 4) * (n_groups_ * 16) + (fr * 4 + fc) * (ngb * 4) + ((l >> 3) ^ (fc & 1)) * 4 + b
 
 
 def pack_int2(codes: np.ndarray) -> np.ndarray:

@@ -21,8 +21,8 @@ transform coefficients on the calibration values; eigenvector signs are fixed so
 entry of largest magnitude is positive; k-means is seeded with distinct training vectors and
 runs a fixed number of iterations; the per-token scale of Algorithm 3 is off (it is outside
 Theorem 2's model and would break the exact 2 bits/element).
-Value codebooks are finally snapped to an 8-bit grid per (KV head, group, coordinate) (the paper
-snaps its codebooks to an 8-bit format offline as well): encoder, decoder and oracle therefore see
+Value codebooks are finally snapped to a 7-bit grid per (KV head, group, coordinate) (the paper
+stores its codebooks in a narrow format offline as well): encoder, decoder and oracle therefore see
 the same centroids, and the decode kernel can keep a value codeword in four bytes.
 """
 from __future__ import annotations
@@ -131,10 +131,13 @@ def equalizing_order(variances: np.ndarray, n_groups: int) -> np.ndarray:
     return order
 
 
-def snap_to_u8_grid(cb: np.ndarray) -> np.ndarray:
-    """Round every codebook coordinate to its own 8-bit grid and return float32 values.
+GRID_LEVELS = 127          # a value-codebook coordinate takes the values lo + u (hi - lo) / 127, u = 0 .. 127
 
-    cb: [..][C][g].  Coordinate i of a codebook takes the values lo_i + u (hi_i - lo_i) / 255, u = 0 .. 255,
+
+def snap_to_byte_grid(cb: np.ndarray) -> np.ndarray:
+    """Round every codebook coordinate to its own 7-bit grid and return float32 values.
+
+    cb: [..][C][g].  Coordinate i of a codebook takes the values lo_i + u (hi_i - lo_i) / 127, u = 0 .. 127,
     where lo_i / hi_i are the smallest / largest float32 value of that coordinate over the C codewords; the
     grid is evaluated in float64 and rounded once to float32 (``novakv_load_calibration`` re-derives the
     grid from the snapped values with the same arithmetic and refuses anything else).
@@ -142,9 +145,9 @@ def snap_to_u8_grid(cb: np.ndarray) -> np.ndarray:
     cb32 = np.asarray(cb, dtype=np.float32)
     lo = cb32.min(axis=-2, keepdims=True).astype(np.float64)
     hi = cb32.max(axis=-2, keepdims=True).astype(np.float64)
-    step = (hi - lo) / 255.0
+    step = (hi - lo) / float(GRID_LEVELS)
     step = np.where(step > 0, step, 1.0)
-    u = np.clip(np.rint((cb32.astype(np.float64) - lo) / step), 0, 255)
+    u = np.clip(np.rint((cb32.astype(np.float64) - lo) / step), 0, GRID_LEVELS)
     return (lo + step * u).astype(np.float32)
 
 
@@ -237,7 +240,7 @@ def calibrate(q_cal: np.ndarray, k_cal: np.ndarray, v_cal: np.ndarray, *, n_kv_h
     f32 = {name: np.ascontiguousarray(np.stack(vals), dtype=np.float32) for name, vals in out.items()}
     if snap_value_codebook:
         unsnapped = f32["cb_v"]
-        f32["cb_v"] = snap_to_u8_grid(unsnapped)
+        f32["cb_v"] = snap_to_byte_grid(unsnapped)
         info["value_snap_rms"] = np.sqrt(((f32["cb_v"].astype(np.float64) - unsnapped) ** 2).mean(axis=(1, 2, 3)))
         info["value_codeword_rms"] = np.sqrt((unsnapped.astype(np.float64) ** 2).mean(axis=(1, 2, 3)))
     extra = {k_: info.pop(k_) for k_ in ("value_snap_rms", "value_codeword_rms") if k_ in info}

@@ -116,11 +116,12 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
     const int H = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim, L = ctx->n_groups, C = NOVAKV_C, g = NOVAKV_G;
     const size_t n_mat = (size_t)H * d * d, n_vec = (size_t)H * d, n_cb = (size_t)H * L * C * g;
 
-    // Value codewords: every coordinate (KV head, group l, component i) must lie on its own 8-bit grid
-    // lo + u (hi - lo) / 255, u = 0 .. 255, with lo / hi the smallest / largest value that coordinate takes over
+    // Value codewords: every coordinate (KV head, group l, component i) must lie on its own 7-bit grid
+    // lo + u (hi - lo) / 127, u = 0 .. 127, with lo / hi the smallest / largest value that coordinate takes over
     // the 256 codewords (the calibrator snaps them after Lloyd, as the paper snaps its codebooks to a narrow
-    // format offline).  The kernel keeps the indices u (4 bytes per codeword) and applies step and offset once
-    // per output coefficient.  The grid is evaluated in binary64 and rounded to binary32 exactly as below.
+    // format offline).  The kernel keeps the indices u (4 bytes per codeword, top bit clear: a byte and its
+    // replicated top bit form the binary16 number u 2^-24) and applies step and offset once per output
+    // coefficient.  The grid is evaluated in binary64 and rounded to binary32 exactly as below.
     std::vector<uint8_t> cbv_u8((size_t)H * C * 32 * g, 0);
     std::vector<float> v_scale((size_t)H * d, 1.f), v_off((size_t)H * d, 0.f);
     for (int hh = 0; hh < H; ++hh)
@@ -133,18 +134,18 @@ extern "C" novakv_status novakv_load_calibration(novakv_ctx* ctx, int layer, con
                     lo = x < lo ? x : lo;
                     hi = x > hi ? x : hi;
                 }
-                double step = ((double)hi - (double)lo) / 255.0;
+                double step = ((double)hi - (double)lo) / 127.0;
                 if (!(step > 0.0) || !(step < 1e300)) step = 1.0;
                 for (int c = 0; c < C; ++c) {
                     const float x = h->cb_v[(((size_t)hh * L + l) * C + c) * g + i];
                     double u = nearbyint(((double)x - (double)lo) / step);
                     if (u < 0.0) u = 0.0;
-                    if (u > 255.0) u = 255.0;
+                    if (u > 127.0) u = 127.0;
                     if ((float)((double)lo + step * u) != x) return NOVAKV_EUNSUPPORTED;
                     cbv_u8[(((size_t)hh * C + c) * 32 + l) * g + i] = (uint8_t)u;
                 }
                 v_scale[(size_t)hh * d + l * g + i] = (float)step;
-                v_off[(size_t)hh * d + l * g + i] = (float)((double)lo + 128.0 * step);
+                v_off[(size_t)hh * d + l * g + i] = (float)((double)lo + 64.0 * step);
             }
 
     std::vector<double> rk_d(n_mat), rv_d(n_mat), km_d(n_vec, 0.0), vm_d(n_vec, 0.0);

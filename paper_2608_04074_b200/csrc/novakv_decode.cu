@@ -255,6 +255,13 @@ __device__ __forceinline__ uint4 lds_u128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
+// Byte permutation with the full selector of the instruction: bit 3 of a selector nibble replaces the chosen
+// byte by eight copies of its top bit (the intrinsic __byte_perm documents only the low three bits).
+__device__ __forceinline__ uint32_t prmt_rep(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -425,9 +432,11 @@ __device__ __noinline__ void build_score_table(unsigned char* t32, unsigned char
                             make_float4(o[hs * 4], o[hs * 4 + 1], o[hs * 4 + 2], o[hs * 4 + 3]);
                 } else if (C::HAS16) {
                     // (a table entry beyond the binary16 range would be a logit share of 2^16 bits; clamped, never inf)
-                    *reinterpret_cast<uint2*>(t16 + code * T16_ROW + g * 8) =
-                        make_uint2(pack_h2(fminf(fmaxf(o[0], -60000.f), 60000.f), fminf(fmaxf(o[1], -60000.f), 60000.f)),
-                                   pack_h2(fminf(fmaxf(o[2], -60000.f), 60000.f), fminf(fmaxf(o[3], -60000.f), 60000.f)));
+                    const uint2 e = make_uint2(pack_h2(fminf(fmaxf(o[0], -60000.f), 60000.f), fminf(fmaxf(o[1], -60000.f), 60000.f)),
+                                               pack_h2(fminf(fmaxf(o[2], -60000.f), 60000.f), fminf(fmaxf(o[3], -60000.f), 60000.f)));
+                    *reinterpret_cast<uint2*>(t16 + code * T16_ROW + g * 8) = e;
+                    // groups 8..15 a second time in columns 0..7: the 16 lanes of a half warp then read 16 different columns
+                    if (K32 == 8 && g < 16) *reinterpret_cast<uint2*>(t16 + code * T16_ROW + (g - 8) * 8) = e;
                 }
             }
         }
@@ -534,11 +543,13 @@ __device__ __noinline__ void fused_merge(float* scratch, const float* part_ml, c
 // Numerics of the tensor-core value side.  A softmax weight enters the product as the binary16 number
 // w = fp16(2^15 p) (p <= 1 relative to the running maximum, so w <= 2^15; weights down to 2^-39 stay
 // non-zero), and the same rounded w is what the normaliser sums: the result is an exact softmax of slightly
-// perturbed logits.  A value codeword is four 8-bit grid indices u; the byte permutation that widens them
-// yields the binary16 numbers 1024 + u, so an accumulator gains sum_j w_j (1024 + u_j).  Every NOVAKV_WINDOW
-// tiles, and before any rescaling, that offset is removed with the weight sum of the same tokens, which the
-// tensor core accumulates beside the products (an all-ones operand): acc -= 1152 sum_j w_j leaves
-// sum_j w_j (u_j - 128), so that the long-running sums stay centred and small.
+// perturbed logits.  A value codeword is four 7-bit grid indices u (bytes with the top bit clear); the byte
+// permutation that widens them pairs every byte with its replicated top bit, i.e. with a zero byte: the
+// binary16 numbers u 2^-24 (subnormal, exact; the tensor core multiplies them exactly).  The same permutation
+// picks the bytes from one of two registers by lane, which undoes the block swap of the odd lane columns.
+// Every NOVAKV_WINDOW tiles, and before any rescaling, the grid centre is removed with the weight sum of
+// the same tokens, which the tensor core accumulates beside the products (an all-ones operand):
+// acc -= 64 2^-24 sum_j w_j leaves 2^-24 sum_j w_j (u_j - 64), so that the long-running sums stay centred.
 template <int D, int HG, bool VM, bool KSC, bool VSQ>
 __global__ void __launch_bounds__(S1_THREADS, 1)
 novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restrict__ cb_k_lut,
@@ -564,7 +575,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     constexpr bool HAS16 = C::HAS16;
     constexpr int TILE_BYTES = C::TILE_BYTES, PAGE_BYTES = 2 * TILE_BYTES;
     constexpr float SH = VM ? 15.f : 0.f;                     // weights are scaled by 2^SH before the binary16 rounding
-    constexpr float CEN = VSQ ? 1024.f : 1152.f;              // what one unit of weight adds to a tensor-core sum beyond u - centre
+    constexpr float U_UNIT = 5.9604644775390625e-08f;         // 2^-24: a grid index u enters a product as the binary16 subnormal u 2^-24
+    constexpr float CEN = VSQ ? 0.f : 64.f * U_UNIT;          // what one unit of weight adds to a tensor-core sum beyond u - centre
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ int s_found[4];
     __shared__ int s_arrived, s_first, s_last;
@@ -624,7 +636,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     //     column word): the column word holds the column bytes of an even / odd step in bytes 0 / 1 and the
     //     table's upper address half in bytes 2, 3; stepping to another pair of j is one xor with a constant.
     const uint32_t col32 = s_base + C::OFFB_T32 + (lane & 7) * 16;
-    const uint32_t colword7 = t16_abs | (uint32_t)((lane & 7) * 8) * 0x0101u;
     const uint32_t colword15 = t16_abs | (uint32_t)((lane & 15) * 8) * 0x0101u;
     // value side: lane column fc reads copy fc / 2 of the value codebook; odd columns take the group blocks in
     // swapped order (x ^ 1), so that the 32 lanes of a gather hit 32 different slots.  With the binary16 table
@@ -641,6 +652,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         return HAS16 ? __byte_perm(w, pos[x], 0x7604u | (b << 4)) : pos[x] + __byte_perm(w, 0u, 0x4440u | b) * VCB_ROW;
     };
     const bool odd_col = fc & 1;
+    // widening selectors: byte pairs (u, replicated top bit of u = 0) of the low / high half of a codeword, taken
+    // from the first operand in even columns and from the second in odd columns
+    const uint32_t sel_lo = odd_col ? 0xD5C4u : 0x9180u, sel_hi = odd_col ? 0xF7E6u : 0xB3A2u;
     // B fragments carry a weight in the low or high half depending on the column parity (fr & 1)
     const uint32_t sel_b0 = (fr & 1) ? 0x1044u : 0x4410u, sel_b1 = (fr & 1) ? 0x3244u : 0x4432u;
     const uint32_t s_pw = s_p + warp * C::P_WARP_BYTES;
@@ -688,6 +702,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
 #ifdef NOVAKV_TIMING
     long long tm[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    unsigned long long g_start;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_start));
     long long t_prev = clock64();
     const long long t_start = t_prev;
     int n_seg = 0;
@@ -797,7 +813,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 uint32_t ch[2];
 #pragma unroll
                 for (int j = K32; j < L; ++j) {
-                    const uint32_t cw2 = (j < 16 ? colword7 : colword15) ^ (uint32_t)(((j & ~1) * 8) | (((j | 1) * 8) << 8));
+                    const uint32_t cw2 = colword15 ^ (uint32_t)(((j & ~1) * 8) | (((j | 1) * 8) << 8));
                     const uint2 v = lds_u64(__byte_perm(cur.kw[j >> 2], cw2, 0x7600u | ((j & 3) << 4) | (4 + (j & 1))));
                     if ((j - K32) % NOVAKV_CHAIN == 0) { ch[0] = v.x; ch[1] = v.y; }
                     else { ch[0] = hadd2(ch[0], v.x); ch[1] = hadd2(ch[1], v.y); }
@@ -937,15 +953,15 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                         uint32_t X[NGB][2];
 #pragma unroll
                         for (int x = 0; x < NGB; ++x) {
-                            const uint32_t vwd = odd_col ? cur.vw[blk][x ^ 1] : cur.vw[blk][x];      // codes of the group block this load fetches
+                            const uint32_t vwd = cur.vw[blk][x];      // codes of the group block this load fetches (x ^ 1 in odd columns)
                             X[x][0] = lds_u32(vaddr(vwd, 2 * ts, x));
                             X[x][1] = lds_u32(vaddr(vwd, 2 * ts + 1, x));
                         }
 #pragma unroll
                         for (int gb = 0; gb < NGB; ++gb) {
-                            const uint32_t x0 = odd_col ? X[gb ^ 1][0] : X[gb][0], x1 = odd_col ? X[gb ^ 1][1] : X[gb][1];
-                            const uint32_t a0 = __byte_perm(x0, 0x64646464u, 0x4140u), a1 = __byte_perm(x0, 0x64646464u, 0x4342u);
-                            const uint32_t a2 = __byte_perm(x1, 0x64646464u, 0x4140u), a3 = __byte_perm(x1, 0x64646464u, 0x4342u);
+                            // bytes (u, 0) pairs from X[gb] (even columns) or X[gb ^ 1] (odd columns)
+                            const uint32_t a0 = prmt_rep(X[gb][0], X[gb ^ 1][0], sel_lo), a1 = prmt_rep(X[gb][0], X[gb ^ 1][0], sel_hi);
+                            const uint32_t a2 = prmt_rep(X[gb][1], X[gb ^ 1][1], sel_lo), a3 = prmt_rep(X[gb][1], X[gb ^ 1][1], sel_hi);
 #pragma unroll
                             for (int hs = 0; hs < HSETS; ++hs) mma_f16(macc[hs][gb], a0, a1, a2, a3, b0[hs], b1[hs]);
                         }
@@ -973,13 +989,12 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 #pragma unroll
                         for (int x = 0; x < NGB; ++x) {
                             // (odd lane columns fetch group block x ^ 1 with load x; their accumulator x holds that block)
-                            const uint32_t vwd = odd_col ? cur.vw[blk][x ^ 1] : cur.vw[blk][x];
-                            const uint32_t cwd = lds_u32(vaddr(vwd, tq, x));
-                            // grid indices -> binary32, centred: (1024 + u) - 1152 is exact in binary16
-                            const __half2 c1152 = __float2half2_rn(1152.f);
-                            const uint32_t h01 = __byte_perm(cwd, 0x64646464u, 0x4140u), h23 = __byte_perm(cwd, 0x64646464u, 0x4342u);
-                            const float2 f01 = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&h01), c1152));
-                            const float2 f23 = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&h23), c1152));
+                            const uint32_t cwd = lds_u32(vaddr(cur.vw[blk][x], tq, x));
+                            // grid indices -> binary32, centred: bytes (u, 0) are the binary16 subnormals u 2^-24
+                            const __half2 c64 = __halves2half2(__ushort_as_half((unsigned short)64), __ushort_as_half((unsigned short)64));
+                            const uint32_t h01 = __byte_perm(cwd, 0u, 0x4140u), h23 = __byte_perm(cwd, 0u, 0x4342u);
+                            const float2 f01 = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&h01), c64));
+                            const float2 f23 = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&h23), c64));
                             const uint64_t v01 = pack2(f01.x, f01.y), v23 = pack2(f23.x, f23.y);
 #pragma unroll
                             for (int h = 0; h < HPAD; ++h) {
@@ -1101,7 +1116,8 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                     if (VSQ) zsum = fmaf(sc, m_lz[w * HPAD + h], zsum);              // zero-points: the same amount on every coefficient
                     lsum = fmaf(sc, m_ml[(w * HPAD + h) * 2 + 1], lsum);
                 }
-                // grid index sums -> value-transform coefficients: s (u - 128) + (lo + 128 s) per unit of weight
+                // grid index sums -> value-transform coefficients: s (u - 64) + (lo + 64 s) per unit of weight
+                a *= 16777216.f;                           // indices entered the sums as u 2^-24
                 float val;
                 if (VSQ) val = (a + zsum) * unscale;       // levels are the codes themselves (s = 1, no offset)
                 else val = (v_scale[(size_t)sg.kvh * D + c] * a + v_off[(size_t)sg.kvh * D + c] * lsum) * unscale;
@@ -1143,9 +1159,11 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         u += sg.npg;
     }
 #ifdef NOVAKV_TIMING
-    if (threadIdx.x == 0 && (blockIdx.x % 21 == 0 || blockIdx.x == gridDim.x - 1))
-        printf("cta %3d segs %d pages %ld | clocks: pre-loop %lld locate+q %lld build %lld vcbwait %lld scan(w0) %lld barrier %lld epilogue %lld total %lld\n",
-               blockIdx.x, n_seg, (long)(u_end - u_begin), tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], clock64() - t_start);
+    unsigned long long g_end;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_end));
+    if (threadIdx.x == 0)
+        printf("cta %3d segs %d pages %ld | clocks: pre-loop %lld locate+q %lld build %lld vcbwait %lld scan(w0) %lld barrier %lld epilogue %lld total %lld | ns start %llu end %llu\n",
+               blockIdx.x, n_seg, (long)(u_end - u_begin), tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], clock64() - t_start, g_start, g_end);
 #endif
 }
 

@@ -162,7 +162,7 @@ template <int L>
 __host__ __device__ __forceinline__ int novakv_v_offset(int t, int l) {
     constexpr int NGB = L / 8;
     const int tb = t & 15, fc = tb & 3, b = tb >> 2, fr = l & 7;
-    return (t >> 4) * (L * 16) + (fr * 4 + fc) * (NGB * 4) + (l >> 3) * 4 + b;
+    return (t >> 4) * (L * 16) + (fr * 4 + fc) * (NGB * 4) + ((l >> 3) ^ (fc & 1)) * 4 + b;
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -296,7 +296,7 @@ def test_faults_are_reported_not_trapped(qwen):
     for n in ("rk", "rk_inv_t", "rv", "k_mean", "v_mean", "cb_k", "cb_v"):
         setattr(bad, n, getattr(case.cal, n))
     bad.cb_v = case.cal.cb_v.copy()
-    bad.cb_v[0, 3, 100, 2] += np.float32(1e-4) * max(1.0, abs(float(bad.cb_v[0, 3, 100, 2])))   # off its 8-bit grid
+    bad.cb_v[0, 3, 100, 2] += np.float32(1e-4) * max(1.0, abs(float(bad.cb_v[0, 3, 100, 2])))   # off its 7-bit grid
     with pytest.raises(NovaKVError, match="unsupported calibration"):
         fresh.novakv_load_calibration(1, bad)
     with pytest.raises(NovaKVError, match="unsupported shape"):

@@ -67,7 +67,7 @@ def test_cache_layout_round_trip_and_positions():
     k_off = (((t // 32) * 1 + j // 16) * 32 + t % 32) * 16 + j % 16
     assert kp[page, h, k_off] == ref[b][0][pos, h, l]
     fc, bb, fr = (t % 16) % 4, (t % 16) // 4, l % 8
-    v_off = (t // 16) * (L * 16) + (fr * 4 + fc) * 8 + (l // 8) * 4 + bb
+    v_off = (t // 16) * (L * 16) + (fr * 4 + fc) * 8 + ((l // 8) ^ (t % 2)) * 4 + bb   # odd tokens: group blocks swapped
     assert vp[page, h, v_off] == ref[b][1][pos, h, l]
     # every byte of a chunk is hit exactly once
     tt, ll = np.meshgrid(np.arange(64), np.arange(L), indexing="ij")
