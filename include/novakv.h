@@ -132,7 +132,8 @@ size_t novakv_decode_workspace_bytes(const novakv_ctx* ctx, int batch);
  * The 2L index bytes go to page page_table[tok_seq[t]][tok_pos[t]/64] at slot tok_pos[t]%64, and
  * seq_lens[tok_seq[t]] becomes max(seq_lens[tok_seq[t]], tok_pos[t]+1).
  *   k_new, v_new  bf16 [n_tokens][Hkv][d]
- *   tok_seq, tok_pos  int32 [n_tokens]; two tokens of one call must not share (seq, pos)
+ *   tok_seq, tok_pos  int32 [n_tokens]; two tokens of one call must not share (seq, pos);
+ *                     tok_seq[t] = -1 marks an unused entry of the list: it is skipped, no status bit
  *   n_tokens = 0 is a no-op.  Out-of-range tokens/pages set device status bits and are skipped.
  */
 novakv_status novakv_encode_append(novakv_ctx* ctx, int layer,
@@ -232,6 +233,34 @@ novakv_status novakv_decode_attention_banded(novakv_ctx* ctx, int layer, const v
     const void* band_k, const void* band_v, int band_cap, int n_sink, const int32_t* band_meta,
     int batch, float sm_scale, void* out, int out_is_fp32, void* workspace, size_t workspace_bytes,
     novakv_stream stream);
+
+/*
+ * Write side of the BF16 band (App. B "Sink-plus-recent band": a new token joins the recent band first;
+ * quantisation is deferred and happens for `block` tokens at a time, eight in the paper): one new token
+ * for every sequence, all bookkeeping in device memory, no host synchronisation.  For sequence b with
+ * band_meta[b] = (sink_cnt, ring_start, ring_len) and ring_cap = band_cap - n_sink:
+ *   - sink_cnt < n_sink: the token goes to slot sink_cnt, sink_cnt grows by one;
+ *   - otherwise it goes to ring slot n_sink + (ring_start + ring_len) % ring_cap and ring_len grows by one;
+ *     if ring_len has reached n_rec + block, the `block` oldest ring tokens are encoded into the index cache
+ *     at positions n_sink + quant_lens[b] .. + block - 1 (the encoder of the format the optional pools
+ *     select: k_scales != NULL the scaled key format, v_meta != NULL as well the deployed format), then
+ *     ring_start = (ring_start + block) % ring_cap, ring_len -= block, quant_lens[b] += block, and
+ *     seq_lens[b] (the index cache's own length, as novakv_encode_append maintains it) follows.
+ * The tokens leaving the band are staged in `staging` together with their (sequence, position) list;
+ * sequences that flush nothing contribute unused entries.
+ *   k_new, v_new   device bf16 [batch][Hkv][d]
+ *   band_k, band_v, band_meta, quant_lens   as in novakv_decode_attention_banded, read and written
+ *   n_rec, block   > 0 with n_rec + block <= band_cap - n_sink; n_sink a multiple of 64
+ *   staging        device, novakv_band_append_staging_bytes(ctx, batch, block) bytes, 256-byte aligned
+ * Returns NOVAKV_EINVAL for inconsistent sizes, NOVAKV_EWORKSPACE for a short or misaligned staging buffer.
+ */
+size_t novakv_band_append_staging_bytes(const novakv_ctx* ctx, int batch, int block);
+novakv_status novakv_band_append(novakv_ctx* ctx, int layer, const void* k_new, const void* v_new, int batch,
+    void* band_k, void* band_v, int band_cap, int n_sink, int n_rec, int block,
+    int32_t* band_meta, int32_t* quant_lens,
+    uint8_t* k_pages, uint8_t* v_pages, void* k_scales, void* v_meta, int n_pages,
+    const int32_t* page_table, int max_pages_per_seq, int32_t* seq_lens,
+    void* staging, size_t staging_bytes, novakv_stream stream);
 
 /*
  * The paper's deployed cache format (Sec. 5 "Bit rate": keys at 2.125 bits per element; values as 2-bit

@@ -25,6 +25,7 @@ EXPORTED = [
     "novakv_decode_attention_sink", "novakv_decode_attention_banded",
     "novakv_value_meta_page_bytes", "novakv_encode_append_deployed", "novakv_decode_attention_deployed",
     "novakv_debug_set_segment_weight", "novakv_debug_set_fused_merge",
+    "novakv_band_append_staging_bytes", "novakv_band_append",
 ]
 
 
@@ -96,6 +97,11 @@ def load_library(path=None):
                                                      c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                                      c_int, c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p,
                                                      c_size_t, c_void_p]
+    lib.novakv_band_append_staging_bytes.argtypes = [c_void_p, c_int, c_int]
+    lib.novakv_band_append_staging_bytes.restype = c_size_t
+    lib.novakv_band_append.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_int,
+                                       c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+                                       c_int, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.novakv_decode_attention_noalloc.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                                     c_int, c_void_p, c_int, c_float, c_void_p, c_int, c_void_p]
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
@@ -260,6 +266,20 @@ class Context:
             _ptr(k_pages), _ptr(v_pages), _ptr(k_scales), _ptr(v_meta), int(k_pages.shape[0]), _ptr(page_table),
             int(page_table.shape[1]), int(page_table.shape[0]), _ptr(seq_lens), _stream()),
             "novakv_encode_append_deployed")
+
+    def novakv_band_append_staging_bytes(self, batch, block):
+        return int(self.lib.novakv_band_append_staging_bytes(self.handle, int(batch), int(block)))
+
+    def novakv_band_append(self, layer, k_new, v_new, band_k, band_v, n_sink, n_rec, block, band_meta, quant_lens,
+                           k_pages, v_pages, k_scales, v_meta, page_table, seq_lens, staging):
+        """One new token per sequence into the BF16 band; blocks that leave it are encoded (all on the device)."""
+        opt = lambda t: _ptr(t) if t is not None else None
+        _check(self.lib, self.lib.novakv_band_append(
+            self.handle, layer, _ptr(k_new), _ptr(v_new), int(k_new.shape[0]), _ptr(band_k), _ptr(band_v),
+            int(band_k.shape[1]), int(n_sink), int(n_rec), int(block), _ptr(band_meta), _ptr(quant_lens),
+            _ptr(k_pages), _ptr(v_pages), opt(k_scales), opt(v_meta), int(k_pages.shape[0]), _ptr(page_table),
+            int(page_table.shape[1]), _ptr(seq_lens), _ptr(staging), int(staging.numel() * staging.element_size()),
+            _stream()), "novakv_band_append")
 
     def novakv_decode_attention_deployed(self, layer, q, k_pages, v_pages, k_scales, v_meta, sink_logits, page_table,
                                          quant_lens, band_k, band_v, n_sink, band_meta, out, workspace, sm_scale=None):

@@ -49,6 +49,8 @@ extern "C" novakv_status novakv_create(novakv_ctx** out, const novakv_config* cf
     novakv_ctx* ctx = new (std::nothrow) novakv_ctx();
     if (!ctx) return NOVAKV_EINVAL;
     ctx->cfg = *cfg;
+    // setting up a segment (score table of 256 x L entries per head) costs about as much as scanning this many pages
+    ctx->seg_weight = cfg->head_dim == 128 ? 40 : 24;
     ctx->hg = cfg->n_q_heads / cfg->n_kv_heads;
     ctx->n_groups = cfg->head_dim / NOVAKV_G;
     ctx->layers.resize(cfg->n_layers);
@@ -374,6 +376,48 @@ extern "C" novakv_status novakv_encode_append_deployed(novakv_ctx* ctx, int laye
                                 tok_seq, tok_pos, n_tokens, k_pages, v_pages, n_pages, page_table,
                                 max_pages_per_seq, n_seq, seq_lens, (cudaStream_t)stream, (__nv_bfloat16*)k_scales,
                                 (__nv_bfloat16*)v_meta);
+}
+
+// staging of novakv_band_append: tokens leaving the band [batch * block][Hkv][d] bf16 for K and for V, then the
+// (sequence, position) list, each part 256-byte aligned
+static size_t band_stage_part(size_t x) { return (x + 255) & ~(size_t)255; }
+extern "C" size_t novakv_band_append_staging_bytes(const novakv_ctx* ctx, int batch, int block) {
+    if (!ctx || batch <= 0 || block <= 0) return 0;
+    const size_t rows = (size_t)batch * block;
+    return 2 * band_stage_part(rows * ctx->cfg.n_kv_heads * ctx->cfg.head_dim * 2) + 2 * band_stage_part(rows * 4);
+}
+
+extern "C" novakv_status novakv_band_append(novakv_ctx* ctx, int layer, const void* k_new, const void* v_new, int batch,
+    void* band_k, void* band_v, int band_cap, int n_sink, int n_rec, int block, int32_t* band_meta, int32_t* quant_lens,
+    uint8_t* k_pages, uint8_t* v_pages, void* k_scales, void* v_meta, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int32_t* seq_lens, void* staging, size_t staging_bytes, novakv_stream stream) {
+    novakv_status st = check_common(ctx, layer);
+    if (st != NOVAKV_OK) return st;
+    if (batch < 0) return NOVAKV_EINVAL;
+    if (batch == 0) return NOVAKV_OK;
+    if (!k_new || !v_new || !band_k || !band_v || !band_meta || !quant_lens || !k_pages || !v_pages || !page_table || !seq_lens)
+        return NOVAKV_EINVAL;
+    if (v_meta != nullptr && k_scales == nullptr) return NOVAKV_EUNSUPPORTED;
+    if (n_sink < 0 || n_sink % NOVAKV_PAGE_TOKENS != 0 || n_rec <= 0 || block <= 0 || (long)n_sink + n_rec + block > band_cap)
+        return NOVAKV_EINVAL;
+    if (n_pages <= 0 || max_pages_per_seq <= 0) return NOVAKV_EPAGE;
+    if (((uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)band_k | (uintptr_t)band_v) & 15) return NOVAKV_EINVAL;
+    if (!staging || staging_bytes < novakv_band_append_staging_bytes(ctx, batch, block) || ((uintptr_t)staging & 255))
+        return NOVAKV_EWORKSPACE;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess) return NOVAKV_ECUDA;
+    const size_t rows = (size_t)batch * block;
+    const size_t tok_bytes = band_stage_part(rows * ctx->cfg.n_kv_heads * ctx->cfg.head_dim * 2);
+    unsigned char* base = (unsigned char*)staging;
+    void* stage_k = base;
+    void* stage_v = base + tok_bytes;
+    int32_t* tok_seq = (int32_t*)(base + 2 * tok_bytes);
+    int32_t* tok_pos = (int32_t*)(base + 2 * tok_bytes + band_stage_part(rows * 4));
+    st = novakv_launch_band_insert(ctx, k_new, v_new, batch, band_k, band_v, band_cap, n_sink, n_rec, block, band_meta,
+                                   quant_lens, stage_k, stage_v, tok_seq, tok_pos, (cudaStream_t)stream);
+    if (st != NOVAKV_OK) return st;
+    return novakv_launch_encode(ctx, ctx->layers[layer], (const __nv_bfloat16*)stage_k, (const __nv_bfloat16*)stage_v,
+                                tok_seq, tok_pos, (int)rows, k_pages, v_pages, n_pages, page_table, max_pages_per_seq,
+                                batch, seq_lens, (cudaStream_t)stream, (__nv_bfloat16*)k_scales, (__nv_bfloat16*)v_meta);
 }
 
 extern "C" novakv_status novakv_decode_attention_deployed(novakv_ctx* ctx, int layer, const void* q,

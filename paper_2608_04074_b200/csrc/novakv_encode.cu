@@ -340,14 +340,21 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
 
+    const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
+    const int tile0 = blockIdx.x * tiles_per_cta;
+    const int n_local = max(0, min(n_tiles, tile0 + tiles_per_cta) - tile0);
+    {
+        // a CTA whose token entries are all unused (sequence -1) has nothing to do
+        int any = 0;
+        const int t_end = min(n_tokens, (tile0 + n_local) * ENC_TILE);
+        for (int t = tile0 * ENC_TILE + threadIdx.x; t < t_end; t += ENC_THREADS) any |= tok_seq[t] != -1;
+        if (!__syncthreads_or(any)) return;
+    }
+
     // codebook of this (head, side) -> shared memory, once per CTA
     if (!(VSQ && side == 1)) fill_codebook_pairs(reinterpret_cast<float*>(cb_s), cb_g, L);
     for (int i = threadIdx.x; i < D; i += ENC_THREADS) mean_s[i] = mean[i];
     __syncthreads();
-
-    const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
-    const int tile0 = blockIdx.x * tiles_per_cta;
-    const int n_local = max(0, min(n_tiles, tile0 + tiles_per_cta) - tile0);
     const bool is_transform = threadIdx.x < NT;
     const int tid = is_transform ? threadIdx.x : threadIdx.x - NT;
 
@@ -391,7 +398,9 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
             int page = -1, slot = 0;
             if (tid < n_valid) {
                 const int sq = tok_seq[t0 + tid], pos = tok_pos[t0 + tid];
-                if (sq < 0 || sq >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
+                if (sq == -1) {
+                    // unused entry of the token list: skipped
+                } else if (sq < 0 || sq >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
                     atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
                 } else {
                     page = page_table[(size_t)sq * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
@@ -623,6 +632,9 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
     for (int t0 = 0; t0 < n_tokens; t0 += tp) {
         const int tkn = t0 + tok_in_pass;
         const bool in_range = tkn < n_tokens;
+        // a pass whose entries are all unused does nothing (the same decision in every warp and CTA: it depends
+        // on the token list alone)
+        if (!__any_sync(0xffffffffu, in_range && tok_seq[tkn] != -1)) continue;
         // this lane's token row (all loads in flight together with the destination lookup)
         uint4 xr[D / 8];
         const uint4* xrow = reinterpret_cast<const uint4*>(x_new + ((size_t)(in_range ? tkn : 0) * n_kv_heads + kvh) * D);
@@ -631,7 +643,9 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
         int page = -1, slot = 0;
         if (in_range) {
             const int s = tok_seq[tkn], pos = tok_pos[tkn];
-            if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
+            if (s == -1) {
+                // unused entry of the token list: skipped
+            } else if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
                 if (reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
             } else {
                 page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
@@ -903,6 +917,70 @@ novakv_status novakv_launch_stage(novakv_ctx* ctx, const novakv_stage_args& a, c
     unsigned blocks = (total + 255) / 256;
     if (blocks > (unsigned)(2 * ctx->n_sm)) blocks = 2 * ctx->n_sm;
     novakv_stage_kernel<<<blocks, 256, 0, stream>>>(a);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
+}
+
+// ------------------------------------------------------------------------------------------------
+// BF16 band, write side: one new token per sequence (App. B "Sink-plus-recent band")
+// ------------------------------------------------------------------------------------------------
+// One block per sequence.  Thread 0 advances the sequence's (sink_cnt, ring_start, ring_len, quantised
+// length); the block copies the new token into its band slot and, when the ring has reached n_rec + block
+// tokens, copies the block oldest ring tokens to the staging rows b * block + i with their (sequence,
+// position) entries.  Rows of sequences that flush nothing get the "unused" marker (sequence -1).
+__global__ void __launch_bounds__(256)
+novakv_band_insert_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ band_k,
+                          uint4* __restrict__ band_v, int band_cap, int n_sink, int n_rec, int block,
+                          int32_t* __restrict__ band_meta, int32_t* __restrict__ quant_lens, int row_u4 /* Hkv * d / 8 */,
+                          uint4* __restrict__ stage_k, uint4* __restrict__ stage_v, int32_t* __restrict__ tok_seq,
+                          int32_t* __restrict__ tok_pos) {
+    const int b = blockIdx.x;
+    const int ring_cap = band_cap - n_sink;
+    __shared__ int s_slot, s_flush, s_rs, s_q;
+    if (threadIdx.x == 0) {
+        int sc = band_meta[b * 3], rs = band_meta[b * 3 + 1], rl = band_meta[b * 3 + 2], q = quant_lens[b];
+        // (state written by this kernel stays in range; a caller's out-of-range state is pulled back into it)
+        sc = min(max(sc, 0), n_sink);
+        rs = min(max(rs, 0), ring_cap - 1);
+        rl = min(max(rl, 0), n_rec + block - 1);
+        q = max(q, 0);
+        int slot;
+        if (sc < n_sink) { slot = sc; ++sc; }
+        else { slot = n_sink + (rs + rl) % ring_cap; ++rl; }
+        const int flush = rl >= n_rec + block;
+        s_slot = slot; s_flush = flush; s_rs = rs; s_q = q;
+        if (flush) { rs = (rs + block) % ring_cap; rl -= block; q += block; }
+        band_meta[b * 3] = sc; band_meta[b * 3 + 1] = rs; band_meta[b * 3 + 2] = rl;
+        quant_lens[b] = q;
+    }
+    __syncthreads();
+    {
+        const size_t dst = ((size_t)b * band_cap + s_slot) * row_u4, src = (size_t)b * row_u4;
+        for (int i = threadIdx.x; i < row_u4; i += blockDim.x) { band_k[dst + i] = k_new[src + i]; band_v[dst + i] = v_new[src + i]; }
+    }
+    if (s_flush) {
+        // the new token's slot is not among the block oldest ones (the ring holds at least n_rec > 0 more)
+        for (int i = threadIdx.x; i < block * row_u4; i += blockDim.x) {
+            const int t = i / row_u4, w = i - t * row_u4;
+            const size_t src = ((size_t)b * band_cap + n_sink + (s_rs + t) % ring_cap) * row_u4 + w;
+            const size_t dst = ((size_t)b * block + t) * row_u4 + w;
+            stage_k[dst] = band_k[src];
+            stage_v[dst] = band_v[src];
+        }
+    }
+    for (int t = threadIdx.x; t < block; t += blockDim.x) {
+        tok_seq[b * block + t] = s_flush ? b : -1;
+        tok_pos[b * block + t] = n_sink + s_q + t;
+    }
+}
+
+novakv_status novakv_launch_band_insert(novakv_ctx* ctx, const void* k_new, const void* v_new, int batch, void* band_k,
+    void* band_v, int band_cap, int n_sink, int n_rec, int block, int32_t* band_meta, int32_t* quant_lens,
+    void* stage_k, void* stage_v, int32_t* tok_seq, int32_t* tok_pos, cudaStream_t stream) {
+    const int row_u4 = ctx->cfg.n_kv_heads * ctx->cfg.head_dim / 8;
+    novakv_band_insert_kernel<<<batch, 256, 0, stream>>>((const uint4*)k_new, (const uint4*)v_new, (uint4*)band_k, (uint4*)band_v,
+                                                        band_cap, n_sink, n_rec, block, band_meta, quant_lens, row_u4,
+                                                        (uint4*)stage_k, (uint4*)stage_v, tok_seq, tok_pos);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
 }

@@ -107,6 +107,9 @@ struct novakv_stage_args {
     int n;
 };
 novakv_status novakv_launch_stage(novakv_ctx* ctx, const novakv_stage_args& a, cudaStream_t stream);
+novakv_status novakv_launch_band_insert(novakv_ctx* ctx, const void* k_new, const void* v_new, int batch, void* band_k,
+    void* band_v, int band_cap, int n_sink, int n_rec, int block, int32_t* band_meta, int32_t* quant_lens,
+    void* stage_k, void* stage_v, int32_t* tok_seq, int32_t* tok_pos, cudaStream_t stream);
 
 // bf16 comparator
 size_t novakv_bf16_ws_bytes(const novakv_ctx* ctx, int batch, int max_pages_per_seq);

@@ -151,6 +151,7 @@ class BandedCache:
         self.ring_len = np.zeros(batch, np.int64)
         self.band_meta = torch.zeros((batch, 3), dtype=torch.int32, device=self.device)
         self.quant_lens = torch.zeros(batch, dtype=torch.int32, device=self.device)
+        self._staging = None
 
     def _sync_meta(self):
         meta = np.stack([np.minimum(self.total, self.n_sink), self.ring_start, self.ring_len], axis=1).astype(np.int32)
@@ -194,22 +195,37 @@ class BandedCache:
         self.total[b], self.quant[b], self.ring_start[b], self.ring_len[b] = n, nq, 0, nrec
         self._sync_meta()
 
-    def append_step(self, layer, k_new: torch.Tensor, v_new: torch.Tensor):
-        """One new token for every sequence (bf16 [batch][Hkv][d]); quantises blocks that leave the band."""
-        flush = []
-        for b in range(self.batch):
-            pos = self.total[b]
-            if pos < self.n_sink:
-                slot = pos
-            else:
-                slot = self.n_sink + (self.ring_start[b] + self.ring_len[b]) % self.ring_cap
-                self.ring_len[b] += 1
-            self.band_k[b, slot] = k_new[b]; self.band_v[b, slot] = v_new[b]
-            self.total[b] += 1
-            if self.ring_len[b] >= self.n_rec + self.block:
-                flush.append((b, self.block))
-        self._flush(layer, flush)
-        self._sync_meta()
+    def append_step(self, layer, k_new: torch.Tensor, v_new: torch.Tensor, mirror: bool = True):
+        """One new token for every sequence (bf16 [batch][Hkv][d]): ``novakv_band_append`` places it, encodes the
+        blocks that leave the band and advances the device-side state.  ``mirror`` keeps the host copies of that
+        state in step by the same rule (bookkeeping for tests; ``refresh_host_state`` reads them back instead)."""
+        if self._staging is None:
+            n = self.ctx.novakv_band_append_staging_bytes(self.batch, self.block)
+            self._staging = torch.empty(n, dtype=torch.uint8, device=self.device)
+        p = self.paged
+        self.ctx.novakv_band_append(layer, k_new, v_new, self.band_k, self.band_v, self.n_sink, self.n_rec, self.block,
+                                    self.band_meta, self.quant_lens, p.k_pages, p.v_pages, p.k_scales,
+                                    p.v_meta if p.int2_values else None, p.page_table, p.seq_lens, self._staging)
+        if not mirror:
+            return
+        self.ring_len += self.total >= self.n_sink
+        self.total += 1
+        fl = self.ring_len >= self.n_rec + self.block
+        self.ring_start[fl] = (self.ring_start[fl] + self.block) % self.ring_cap
+        self.ring_len[fl] -= self.block
+        self.quant[fl] += self.block
+
+    def refresh_host_state(self):
+        """Host copies of the band state from the device (after steps taken with ``mirror=False``)."""
+        meta, quant = self.device_state()
+        self.ring_start[:] = meta[:, 1]
+        self.ring_len[:] = meta[:, 2]
+        self.quant[:] = quant
+        self.total[:] = meta[:, 0].astype(np.int64) + quant + meta[:, 2]
+
+    def device_state(self):
+        """(sink_cnt, ring_start, ring_len) [batch][3] and the quantised lengths [batch] as the device holds them."""
+        return self.band_meta.cpu().numpy(), self.quant_lens.cpu().numpy()
 
     def band_mask(self, b: int) -> np.ndarray:
         """bool [total[b]]: positions held in bf16."""

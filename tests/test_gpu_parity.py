@@ -700,6 +700,12 @@ def test_banded_decode_matches_oracle(name, n_sink, n_rec, request):
     assert case.ctx.novakv_last_device_status() == 0
     assert (cache.total == lens + steps).all()
     assert (cache.ring_len >= 0).all() and (cache.ring_len < n_rec + 8).all()
+    # the device-side state that novakv_band_append advanced equals the rule applied on the host
+    meta, quant = cache.device_state()
+    assert np.array_equal(meta[:, 0], np.minimum(cache.total, n_sink))
+    assert np.array_equal(meta[:, 1], cache.ring_start) and np.array_equal(meta[:, 2], cache.ring_len)
+    assert np.array_equal(quant, cache.quant)
+    assert np.array_equal(cache.paged.seq_lens.cpu().numpy(), np.where(cache.quant > 0, n_sink + cache.quant, 0))
     _, _, q = case.draw(1001, 1, len(lens))
     out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
     assert case.ctx.novakv_last_device_status() == 0
@@ -864,7 +870,7 @@ def test_near_one_hot_and_near_uniform_attention(qwen, factor):
 
 
 # --------------------------------------------------------------------------- work split of the scan
-@pytest.mark.parametrize("weight", [0, 1, 24, 200, 4096])
+@pytest.mark.parametrize("weight", [0, 1, 24, 40, 200, 4096])
 def test_segment_weight_moves_split_points_only(qwen, weight):
     """The cost-weighted split (0 = even in pages; large values push whole pairs to single CTAs) must give
     the same attention output: ragged lengths, empty sequences, pairs much shorter than the weight."""
@@ -881,7 +887,7 @@ def test_segment_weight_moves_split_points_only(qwen, weight):
             outs.append(cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy())
         assert case.ctx.novakv_last_device_status() == 0
     finally:
-        case.ctx.novakv_debug_set_segment_weight(24)
+        case.ctx.novakv_debug_set_segment_weight(40)      # the default at d = 128
         case.ctx.novakv_debug_set_scan_ctas(0)
     for b, n in enumerate(lens):
         for out in outs:
