@@ -59,6 +59,10 @@ constexpr int VCB_COPY_BYTES = 32768;         // 256 codes x 32 slots x 4 bytes
 constexpr int VCB_ROW = 128;
 constexpr int S1_SMEM_BYTES = 229376;         // dynamic shared memory requested (224 KB; the CTA also has a few static words)
 constexpr float M_INIT = -1.0e30f;
+#ifndef NOVAKV_M_SLACK
+#define NOVAKV_M_SLACK 4
+#endif
+constexpr float M_SLACK = (float)NOVAKV_M_SLACK;   // headroom (bits) a running maximum gets when it moves
 constexpr int MAX_SCAN_CTAS = 255;            // scan CTAs (one per SM) the boundary table has room for
 constexpr int PFX_CAP = 511;                  // batches up to this size keep their page / cost prefixes in shared memory
 
@@ -548,8 +552,10 @@ __device__ __noinline__ void fused_merge(float* scratch, const float* part_ml, c
 // binary16 numbers u 2^-24 (subnormal, exact; the tensor core multiplies them exactly).  The same permutation
 // picks the bytes from one of two registers by lane, which undoes the block swap of the odd lane columns.
 // Every NOVAKV_WINDOW tiles, and before any rescaling, the grid centre is removed with the weight sum of
-// the same tokens, which the tensor core accumulates beside the products (an all-ones operand):
-// acc -= 64 2^-24 sum_j w_j leaves 2^-24 sum_j w_j (u_j - 64), so that the long-running sums stay centred.
+// the same tokens (every lane adds up the rounded weights of its own tokens; a shuffle reduction per window
+// gives each lane column the sum of its head): acc -= 64 2^-24 sum_j w_j leaves 2^-24 sum_j w_j (u_j - 64),
+// so that the long-running sums stay centred.  (An all-ones operand on the tensor core gave the same sums at
+// four more matrix instructions per tile, which cost more issue time than the shuffles.)
 template <int D, int HG, bool VM, bool KSC, bool VSQ>
 __global__ void __launch_bounds__(S1_THREADS, 1)
 novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restrict__ cb_k_lut,
@@ -662,7 +668,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
     // ---- per-warp running state
     float m_run[HPAD];                           // running maximum of the logits (base 2), the same in every lane
     float macc[HSETS][NGB][4];                   //  VM: lane (fr, fc): head 4 hs + fc, group 8 gb + fr, 4 coefficients
-    float eacc[HSETS][4];                        //  VM: weight sums of head 4 hs + fc since the last offset removal (four equal numbers)
+    float wsum[HPAD];                            //  VM: this lane's tokens: sums of the (rounded) weights per head since the last offset removal
     float l_run[HPAD];                           //  VM: [hs] weight sum of head 4 hs + fc (every lane); else this lane's tokens, per head
     float lz_run[VSQ ? HPAD : 1];                //  VSQ: running sum_j p_j zero_j per head (this lane's tokens)
     uint64_t acc[VM ? 1 : NGB][VM ? 1 : HPAD][2];  // !VM: lane (fr, fc): group 8 gb + fr, head, 4 coefficients, its own tokens
@@ -677,9 +683,9 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         for (int gb = 0; gb < NGB; ++gb)
 #pragma unroll
             for (int i = 0; i < 4; ++i) macc[hs][gb][i] = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) eacc[hs][i] = 0.f;
     }
+#pragma unroll
+    for (int h = 0; h < HPAD; ++h) wsum[h] = 0.f;
 #pragma unroll
     for (int x = 0; x < (VM ? 1 : NGB); ++x)
 #pragma unroll
@@ -687,16 +693,24 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 
     // remove the offset of the 8-bit grid from the sums of the tiles since the last call (tensor-core value side)
     auto flush_window = [&]() {
+        if (VSQ) return;          // INT2 levels carry no grid centre, and that format sums its normaliser per lane
 #pragma unroll
         for (int hs = 0; hs < HSETS; ++hs) {
-            const float w = eacc[hs][0];
+            // weight sum of head 4 hs + fc over the whole warp's tokens: transposing reduction inside the quad (each
+            // step halves the heads a lane keeps), then a butterfly over the eight quads
+            const float k0 = fc & 1 ? wsum[hs * 4 + 1] : wsum[hs * 4 + 0], s0 = fc & 1 ? wsum[hs * 4 + 0] : wsum[hs * 4 + 1];
+            const float k1 = fc & 1 ? wsum[hs * 4 + 3] : wsum[hs * 4 + 2], s1 = fc & 1 ? wsum[hs * 4 + 2] : wsum[hs * 4 + 3];
+            const float lo = k0 + __shfl_xor_sync(0xffffffffu, s0, 1), hi = k1 + __shfl_xor_sync(0xffffffffu, s1, 1);
+            float w = (fc & 2 ? hi : lo) + __shfl_xor_sync(0xffffffffu, fc & 2 ? lo : hi, 2);
+#pragma unroll
+            for (int o = 4; o <= 16; o <<= 1) w += __shfl_xor_sync(0xffffffffu, w, o);
 #pragma unroll
             for (int gb = 0; gb < NGB; ++gb)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) macc[hs][gb][i] = fmaf(-CEN, w, macc[hs][gb][i]);
-            if (!VSQ) l_run[hs] += w;
+            l_run[hs] += w;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) eacc[hs][i] = 0.f;
+            for (int i = 0; i < 4; ++i) wsum[hs * 4 + i] = 0.f;
         }
     };
 
@@ -847,11 +861,14 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 for (int h = 0; h < HPAD; ++h) up |= zf[h] > m_run[h];
                 if (VSQ) up |= vsmax >= esh_pow;
                 if (__any_sync(0xffffffffu, up)) {
-                    if (VM) flush_window();
                     float alpha[HPAD];
 #pragma unroll
                     for (int h = 0; h < HPAD; ++h) {
-                        const float m_new = fmaxf(m_run[h], warp_max(zf[h]));
+                        // a head whose maximum moved gets M_SLACK bits of headroom above the new maximum: the next
+                        // few record logits then need no update (the reference point of a softmax is free; weights
+                        // stay <= 2^SH, and those below 2^(SH - 24 + M_SLACK) of the maximum vanish)
+                        const float wm = warp_max(zf[h]);
+                        const float m_new = wm > m_run[h] ? wm + M_SLACK : m_run[h];
                         alpha[h] = ex2(m_run[h] - m_new);
                         m_run[h] = m_new;
                     }
@@ -872,7 +889,12 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                             for (int gb = 0; gb < NGB; ++gb)
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) macc[hs][gb][i] *= al * vsc;
-                            if (!VSQ) l_run[hs] *= al;
+                            if (!VSQ) {
+                                l_run[hs] *= al;
+                                // the weight sums still waiting for their window flush move with the accumulators
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) wsum[hs * 4 + i] *= alpha[hs * 4 + i];
+                            }
                         }
                         if (VSQ) {
 #pragma unroll
@@ -909,7 +931,10 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             } else if (VM) {
 #pragma unroll
                 for (int h = 0; h < HPAD; h += 2)
+                {
                     ph[h / 2] = pack_h2(ex2(zf[h] - m_run[h] + SH), ex2(zf[h + 1] - m_run[h + 1] + SH));
+                    flush_h2(ph[h / 2], wsum[h], wsum[h + 1]);       // the rounded weights are what the normaliser sums
+                }
             } else {
 #pragma unroll
                 for (int h = 0; h < HPAD; ++h) { zf[h] = ex2(zf[h] - m_run[h]); l_run[h] += zf[h]; }
@@ -947,7 +972,6 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                             const uint32_t w = t == 0 ? pw[hs].x : (t == 1 ? pw[hs].y : (t == 2 ? pw[hs].z : pw[hs].w));
                             b0[hs] = __byte_perm(w, 0u, sel_b0);
                             b1[hs] = __byte_perm(w, 0u, sel_b1);
-                            mma_f16(eacc[hs], 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b0[hs], b1[hs]);
                         }
                         // gather: X[x][u] = codeword of token 8ts + 4u + fc of the block, group block x ^ (fc & 1), row fr
                         uint32_t X[NGB][2];
