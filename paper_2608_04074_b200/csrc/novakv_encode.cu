@@ -320,7 +320,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
                      uint8_t* __restrict__ k_pages, uint8_t* __restrict__ v_pages,
                      __nv_bfloat16* __restrict__ k_scales, __nv_bfloat16* __restrict__ v_meta, int n_pages,
                      const int32_t* __restrict__ page_table, int max_pages_per_seq, int n_seq,
-                     int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta,
+                     int32_t* __restrict__ seq_lens, int n_kv_heads, int tiles_per_cta_k, int tiles_per_cta_v,
                      uint32_t* __restrict__ dev_status) {
     // rk_d / rv_d: the transforms in tensor-core fragment order [d/4][d][4]; rk_plain / rv_plain: the same
     // matrices row-major [d][d] (read only by the certified search's binary64 recomputation)
@@ -341,6 +341,7 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + (size_t)kvh * L * NOVAKV_C * NOVAKV_G);
 
     const int n_tiles = (n_tokens + ENC_TILE - 1) / ENC_TILE;
+    const int tiles_per_cta = blockIdx.z == 0 ? tiles_per_cta_k : tiles_per_cta_v;     // (the two sides may be cut differently)
     const int tile0 = blockIdx.x * tiles_per_cta;
     const int n_local = max(0, min(n_tiles, tile0 + tiles_per_cta) - tile0);
     {
@@ -858,12 +859,22 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         const double cost = waves * (tp + 1.5);
         if (cost < best) { best = cost; ctas_x = cx; tiles_per_cta = tp; }
     }
+    int tiles_k = tiles_per_cta, tiles_v = tiles_per_cta;
+    if (v_meta != nullptr && ctas_x > 1) {
+        // scalar INT2 values need no codeword search: a value tile costs about 3/8 of a key tile, so the CTAs of a head
+        // are shared out 8 : 3 between the two sides instead of evenly (the value side then takes longer runs)
+        const int per_head = 2 * ctas_x;
+        const int ck = max(1, min(n_tiles, (per_head * 8 + 5) / 11)), cv = max(1, min(n_tiles, per_head - ck));
+        tiles_k = (n_tiles + ck - 1) / ck;
+        tiles_v = (n_tiles + cv - 1) / cv;
+        ctas_x = max((n_tiles + tiles_k - 1) / tiles_k, (n_tiles + tiles_v - 1) / tiles_v);
+    }
     dim3 grid(ctas_x, ctx->cfg.n_kv_heads, 2);
     novakv_prof_scope ps(ctx, 1, stream);
     kern<<<grid, ENC_THREADS, smem, stream>>>(k_new, v_new, tok_seq, tok_pos, n_tokens, ly.rk_d_mma, ly.rv_d_mma,
                                                ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages, k_scales,
                                                v_meta, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
-                                               ctx->cfg.n_kv_heads, tiles_per_cta, ctx->dev_status);
+                                               ctx->cfg.n_kv_heads, tiles_k, tiles_v, ctx->dev_status);
     ps.end();
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? NOVAKV_OK : NOVAKV_ECUDA;
