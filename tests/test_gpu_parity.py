@@ -721,6 +721,51 @@ def test_banded_decode_matches_oracle(name, n_sink, n_rec, request):
     print(f"[{name} sink {n_sink} recent {n_rec}] banded: {n_quant} quantised positions, max|delta|/||o||inf = {worst:.3e}")
 
 
+def test_band_append_block_of_four_scaled_keys_and_argument_checks(qwen_scaled):
+    """Write side of the band with another block size on the scaled key format (the clustered append kernel skips
+    the unused entries of sequences that flush nothing), and its argument checks."""
+    from paper_2608_04074_b200.binding import NovaKVError
+    from paper_2608_04074_b200.runtime import BandedCache
+    case = qwen_scaled
+    lens = np.array([0, 70, 90, 200], np.int32)
+    steps = 19
+    cache = BandedCache(case.ctx, len(lens), int(lens.max()) + steps + 64, n_sink=64, n_rec=16, block=4, seed=21, key_scale=True)
+    ks, vs = [], []
+    for b, n in enumerate(lens):
+        k, v, _ = case.draw(1150 + b, int(n) + steps, 1)
+        ks.append(k); vs.append(v)
+        if n > 0:
+            cache.prefill(0, b, _dev(k[:n], torch.bfloat16), _dev(v[:n], torch.bfloat16))
+    for t in range(steps):
+        cache.append_step(0, _dev(np.stack([ks[b][lens[b] + t] for b in range(len(lens))]), torch.bfloat16),
+                          _dev(np.stack([vs[b][lens[b] + t] for b in range(len(lens))]), torch.bfloat16))
+    assert case.ctx.novakv_last_device_status() == 0
+    meta, quant = cache.device_state()
+    assert np.array_equal(meta[:, 1], cache.ring_start) and np.array_equal(meta[:, 2], cache.ring_len)
+    assert np.array_equal(quant, cache.quant) and (cache.ring_len < 16 + 4).all() and cache.quant.max() > 100
+    _, _, q = case.draw(1151, 1, len(lens))
+    out = cache.decode(0, _dev(q, torch.bfloat16)).cpu().numpy()
+    for b in range(len(lens)):
+        k, v = ks[b].astype(np.float64), vs[b].astype(np.float64)
+        e = case.oracle.encode_scaled(k, v, with_gaps=False)
+        ref = case.oracle.decode_banded(q[b].astype(np.float64), e["kidx"], e["vidx"], k, v, cache.band_mask(b), kscale=e["kscale"])
+        check_output(out[b], ref)
+    # argument checks: ring too small for n_rec + block, sink not a multiple of the page, short staging buffer
+    p = cache.paged
+    k1 = _dev(np.stack([ks[b][0] for b in range(len(lens))]), torch.bfloat16)
+    args = lambda n_sink, n_rec, block, staging: (0, k1, k1, cache.band_k, cache.band_v, n_sink, n_rec, block, cache.band_meta,
+                                                   cache.quant_lens, p.k_pages, p.v_pages, p.k_scales, None, p.page_table,
+                                                   p.seq_lens, staging)
+    with pytest.raises(NovaKVError):
+        case.ctx.novakv_band_append(*args(64, 64, 4, cache._staging))
+    with pytest.raises(NovaKVError):
+        case.ctx.novakv_band_append(*args(32, 16, 4, cache._staging))
+    with pytest.raises(NovaKVError, match="workspace"):
+        case.ctx.novakv_band_append(*args(64, 16, 4, cache._staging[:256]))
+    meta2, quant2 = cache.device_state()
+    assert np.array_equal(meta, meta2) and np.array_equal(quant, quant2)       # refused calls change nothing
+
+
 def test_banded_with_scale_and_sink(qwen_scaled):
     from paper_2608_04074_b200.runtime import BandedCache
     case = qwen_scaled
