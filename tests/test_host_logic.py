@@ -77,6 +77,34 @@ def test_cache_layout_round_trip_and_positions():
         assert sorted(cache_format.value_offset(tt, ll, LL).ravel().tolist()) == list(range(64 * LL))
 
 
+def test_value_codebook_grid_snap():
+    """The declared rounding of value codebooks: every coordinate of a codebook on its own 128-point affine grid
+    between its smallest and largest value; idempotent; at most half a step away from the unsnapped value."""
+    from paper_2608_04074_b200 import calib
+    gen = synth.rng(77)
+    cb = (gen.standard_normal((2, 5, 256, 4)) * np.array([0.01, 1.0, 30.0, 1e-6])).astype(np.float32)
+    cb[0, 0, :, 2] = 0.25                                   # a constant coordinate stays what it is
+    sn = calib.snap_to_byte_grid(cb)
+    assert sn.dtype == np.float32 and sn.shape == cb.shape
+    assert np.array_equal(calib.snap_to_byte_grid(sn), sn)
+    assert np.array_equal(sn[0, 0, :, 2], cb[0, 0, :, 2])
+    lo, hi = cb.min(axis=-2, keepdims=True).astype(np.float64), cb.max(axis=-2, keepdims=True).astype(np.float64)
+    step = np.where(hi > lo, (hi - lo) / calib.GRID_LEVELS, 1.0)
+    assert np.array_equal(sn.min(axis=-2), cb.min(axis=-2)) and np.array_equal(sn.max(axis=-2), cb.max(axis=-2))
+    u = (sn.astype(np.float64) - lo) / step
+    assert np.abs(u - np.rint(u)).max() < 1e-4 and u.min() >= -1e-4 and u.max() <= calib.GRID_LEVELS + 1e-4
+    assert (np.abs(sn.astype(np.float64) - cb) <= 0.5 * step * (1 + 1e-6) + 1e-12).all()
+    for h in range(2):
+        for l in range(5):
+            for i in range(4):
+                assert len(np.unique(sn[h, l, :, i])) <= calib.GRID_LEVELS + 1
+    # the calibrator applies it to the value codebooks only
+    wl = workloads.tiny()
+    cal = wl.calibration(wl.laws())
+    assert np.array_equal(calib.snap_to_byte_grid(cal.cb_v), cal.cb_v)
+    assert not np.array_equal(calib.snap_to_byte_grid(cal.cb_k), cal.cb_k)
+
+
 def test_workloads_have_the_stated_shapes():
     w = workloads.qwen3_8b()
     assert (w.shape.n_q_heads, w.shape.n_kv_heads, w.shape.head_dim, w.batch) == (32, 8, 128, 8)
