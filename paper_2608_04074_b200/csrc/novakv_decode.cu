@@ -48,6 +48,9 @@ namespace {
 #ifndef NOVAKV_CHAIN
 #define NOVAKV_CHAIN 4        // table lookups summed in binary16 before a flush into the binary32 logit
 #endif
+#ifndef NOVAKV_KSC_CHAIN
+#define NOVAKV_KSC_CHAIN 2
+#endif
 #ifndef NOVAKV_WINDOW
 #define NOVAKV_WINDOW 8       // tiles whose tensor-core sums are accumulated before the offset of the 8-bit grid is removed
 #endif
@@ -824,14 +827,17 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 for (int k = 0; k < HPAD / 2; ++k) unpack2(z2[k], zf[2 * k], zf[2 * k + 1]);
             }
             if (HAS16) {
+                // (with a per-token key scale the sum is multiplied by rho afterwards, which carries the rounding of the
+                // binary16 chains into tokens of large norm: shorter chains there)
+                constexpr int CHAIN = KSC ? NOVAKV_KSC_CHAIN : NOVAKV_CHAIN;
                 uint32_t ch[2];
 #pragma unroll
                 for (int j = K32; j < L; ++j) {
                     const uint32_t cw2 = colword15 ^ (uint32_t)(((j & ~1) * 8) | (((j | 1) * 8) << 8));
                     const uint2 v = lds_u64(__byte_perm(cur.kw[j >> 2], cw2, 0x7600u | ((j & 3) << 4) | (4 + (j & 1))));
-                    if ((j - K32) % NOVAKV_CHAIN == 0) { ch[0] = v.x; ch[1] = v.y; }
+                    if ((j - K32) % CHAIN == 0) { ch[0] = v.x; ch[1] = v.y; }
                     else { ch[0] = hadd2(ch[0], v.x); ch[1] = hadd2(ch[1], v.y); }
-                    if ((j - K32) % NOVAKV_CHAIN == NOVAKV_CHAIN - 1 || j == L - 1) {
+                    if ((j - K32) % CHAIN == CHAIN - 1 || j == L - 1) {
                         flush_h2(ch[0], zf[0], zf[1]);
                         flush_h2(ch[1], zf[2], zf[3]);
                     }
