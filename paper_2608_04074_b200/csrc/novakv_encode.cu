@@ -912,12 +912,23 @@ novakv_status novakv_launch_encode(novakv_ctx* ctx, const novakv_layer& ly, cons
 // Gather of up to 5 page-locked host buffers into device staging: every 32-bit word crosses the bus
 // once, consecutive threads take consecutive words (128-byte requests per warp).
 __global__ void __launch_bounds__(256) novakv_stage_kernel(const novakv_stage_args a) {
+    // the kernels behind this one in the stream may start their own prologues (calibration constants) now; they
+    // wait for this grid's completion before they touch the staged inputs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const unsigned stride = gridDim.x * blockDim.x;
 #pragma unroll 1
     for (int sgm = 0; sgm < a.n; ++sgm) {
         const uint32_t* __restrict__ src = a.src[sgm];
         uint32_t* __restrict__ dst = a.dst[sgm];
-        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < a.words[sgm]; i += stride) dst[i] = src[i];
+        const unsigned words = a.words[sgm];
+        if (((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0 && (words & 3) == 0) {
+            // 16 bytes per thread: a quarter of the read requests that cross the bus
+            const uint4* __restrict__ s4 = reinterpret_cast<const uint4*>(src);
+            uint4* __restrict__ d4 = reinterpret_cast<uint4*>(dst);
+            for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < words / 4; i += stride) d4[i] = s4[i];
+        } else {
+            for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < words; i += stride) dst[i] = src[i];
+        }
     }
 }
 
@@ -925,7 +936,8 @@ novakv_status novakv_launch_stage(novakv_ctx* ctx, const novakv_stage_args& a, c
     unsigned total = 0;
     for (int i = 0; i < a.n; ++i) total += a.words[i];
     if (total == 0) return NOVAKV_OK;
-    unsigned blocks = (total + 255) / 256;
+    unsigned blocks = (total / 4 + 255) / 256;          // one 16-byte word per thread where the buffers allow it
+    if (blocks == 0) blocks = 1;
     if (blocks > (unsigned)(2 * ctx->n_sm)) blocks = 2 * ctx->n_sm;
     novakv_stage_kernel<<<blocks, 256, 0, stream>>>(a);
     ctx->launches++;
