@@ -19,7 +19,7 @@
 //                - value side: sum_j p_j * value-codeword_j in the value-transform domain, a dense
 //                  [heads x tokens] x [tokens x d] contraction, run on tensor cores (mma.sync, binary16
 //                  operands, binary32 accumulators) or, as the selectable alternative, on CUDA cores in
-//                  binary32; value codewords are 8-bit grid indices (4 bytes per codeword) that expand to
+//                  binary32; value codewords are 7-bit grid indices (4 bytes per codeword) that expand to
 //                  binary16 with one byte permutation per pair,
 //                - the warps' partial (m, l, acc) are merged and written once per segment.
 //   merge    : exact log-sum-exp merge of the partials of every (sequence, KV head), then the inverse
@@ -52,7 +52,7 @@ namespace {
 #define NOVAKV_KSC_CHAIN 2
 #endif
 #ifndef NOVAKV_WINDOW
-#define NOVAKV_WINDOW 8       // tiles whose tensor-core sums are accumulated before the offset of the 8-bit grid is removed
+#define NOVAKV_WINDOW 8       // tiles whose tensor-core sums are accumulated before the centre of the value grid is removed
 #endif
 constexpr int NCW = NOVAKV_NCW;               // warps of the scan kernel
 constexpr int S1_THREADS = NCW * 32;
@@ -694,7 +694,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 #pragma unroll
         for (int h = 0; h < (VM ? 1 : HPAD); ++h) { acc[x][h][0] = 0ull; acc[x][h][1] = 0ull; }
 
-    // remove the offset of the 8-bit grid from the sums of the tiles since the last call (tensor-core value side)
+    // remove the centre of the value grid from the sums of the tiles since the last call (tensor-core value side)
     auto flush_window = [&]() {
         if (VSQ) return;          // INT2 levels carry no grid centre, and that format sums its normaliser per lane
 #pragma unroll
@@ -950,7 +950,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                 // ---- value side on tensor cores ---------------------------------------------------------
                 // D[m][n] += sum_k A[m][k] B[k][n], m16 n8 k16, per 8-token sub-tile and group block gb:
                 //   k = (token j of the sub-tile, sub-coefficient i in {0,1}),
-                //   A[m][(j,i)] = 1024 + grid index of codeword(token j, group 8gb + (m & 7))[2 (m >> 3) + i]     fp16
+                //   A[m][(j,i)] = 2^-24 x grid index of codeword(token j, group 8gb + (m & 7))[2 (m >> 3) + i]     fp16 (subnormal)
                 //   B[(j,i)][(h,i')] = w_h(token j) * [i == i']                                                fp16
                 //   D[m][(h,i')] = partial of head h, group 8gb + (m & 7), coefficient 2 (m >> 3) + i'
                 // weights -> shared memory as fp16, [head][k-slot pair = token & 3][token >> 3, (token >> 2) & 1]

@@ -34,7 +34,7 @@ struct novakv_layer {
     float* rv_t = nullptr;        // [Hkv][d][d]  transposed R_V: rv_t[c][r] = R_V[r][c]
     float* v_mean = nullptr;      // [Hkv][d]
     float* cb_k_lut = nullptr;    // [Hkv][256][L][4]   key codewords minus k_center, the order the score table is built in
-    uint8_t* cb_v_u8 = nullptr;   // [Hkv][256][32][4]  value codewords as indices of their 8-bit grid, slot = group
+    uint8_t* cb_v_u8 = nullptr;   // [Hkv][256][32][4]  value codewords as indices (0..127) of their 7-bit grid, slot = group
     float* v_scale = nullptr;     // [Hkv][d]  grid step s of each value coefficient: codeword = lo + s u
     float* v_off = nullptr;       // [Hkv][d]  lo + 128 s
 };
