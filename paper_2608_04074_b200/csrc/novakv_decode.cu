@@ -28,10 +28,12 @@
 // Shared-memory gathers are laid out against bank conflicts: byte j of a token's key bytes holds group
 // j ^ (token % 8) (j ^ (token % 16) for j >= 16), so that at every step the lanes of a quarter warp read 8
 // different 16-byte columns of a binary32 table row and the lanes of a half warp 16 different 8-byte
-// columns of a binary16 row (8 for steps 8..15: a two-way conflict on those 8 of 32 steps); on the value
+// columns of a binary16 row (steps 8..15 meet only 8 groups: those groups are stored a second time in the
+// unused first columns of the row and the upper half of a half warp reads the copy); on the value
 // side the 32 lanes of a warp read 32 different 4-byte slots, because the lane columns fc = 0,1 and fc = 2,3
 // use two copies of the value codebook whose slots are rotated by 16, and odd columns take the group
-// blocks in swapped order.
+// blocks in swapped order (the cache stores their bytes in that order, and the byte permutation that widens a
+// codeword for the tensor core picks it from the swapped register).
 // The kernel contains no spin wait.
 #include <math_constants.h>
 #ifdef NOVAKV_TIMING
