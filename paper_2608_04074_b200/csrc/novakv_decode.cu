@@ -410,6 +410,49 @@ __device__ __noinline__ void build_score_table(unsigned char* t32, unsigned char
                                                const float* q_s /* shared: q' of the pair, [HPAD][D] */) {
     using C = S1<D, HG, VM>;
     constexpr int L = C::L, HPAD = C::HPAD, HSETS = C::HSETS, K32 = C::K32;
+    if constexpr (C::HAS16) {
+        // Hybrid table: whole warps take one kind of entry, so that no warp runs both store paths.  Threads
+        // 0 .. 16 K32 - 1 build the binary32 part (group = t % K32, 16 codes per pass), the others the binary16
+        // part (group = K32 + t' % (L - K32), 16 codes per pass); 16 passes either way.
+        static_assert(K32 == 8 && L == 32 && S1_THREADS == 512 && HPAD == 4, "work split of the hybrid table build");
+        constexpr int T32_THREADS = 16 * K32;                   // 128 = 4 warps
+        constexpr int BATCH = 8;
+        const bool is32 = threadIdx.x < T32_THREADS;
+        const int tl = is32 ? threadIdx.x : threadIdx.x - T32_THREADS;
+        const int g = is32 ? tl % K32 : K32 + tl % (L - K32);
+        const int code0 = is32 ? tl / K32 : tl / (L - K32);
+        float4 qs[HPAD];
+#pragma unroll
+        for (int h = 0; h < HPAD; ++h) qs[h] = *reinterpret_cast<const float4*>(q_s + h * D + g * 4);
+        const float4* cbk = reinterpret_cast<const float4*>(cb_k_lut) + g;
+        const uint32_t a32 = smem_u32(t32) + g * 16, a16 = smem_u32(t16) + g * 8;
+#pragma unroll 1
+        for (int it0 = 0; it0 < 16; it0 += BATCH) {
+            float4 cw[BATCH];
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) cw[u] = cbk[(size_t)(code0 + (it0 + u) * 16) * L];
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int code = code0 + (it0 + u) * 16;
+                float o[HPAD];
+#pragma unroll
+                for (int h = 0; h < HPAD; ++h)
+                    o[h] = fmaf(qs[h].w, cw[u].w, fmaf(qs[h].z, cw[u].z, fmaf(qs[h].y, cw[u].y, qs[h].x * cw[u].x)));
+                if (is32) {
+                    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a32 + code * C::ROW32),
+                                 "f"(o[0]), "f"(o[1]), "f"(o[2]), "f"(o[3]) : "memory");
+                } else {
+                    // (a table entry beyond the binary16 range would be a logit share of 2^16 bits; clamped, never inf)
+                    const uint32_t e0 = pack_h2(fminf(fmaxf(o[0], -60000.f), 60000.f), fminf(fmaxf(o[1], -60000.f), 60000.f));
+                    const uint32_t e1 = pack_h2(fminf(fmaxf(o[2], -60000.f), 60000.f), fminf(fmaxf(o[3], -60000.f), 60000.f));
+                    asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(a16 + code * T16_ROW), "r"(e0), "r"(e1) : "memory");
+                    // groups 8..15 a second time in columns 0..7: the 16 lanes of a half warp then read 16 different columns
+                    if (g < 16) asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(a16 + code * T16_ROW - 64), "r"(e0), "r"(e1) : "memory");
+                }
+            }
+        }
+        return;
+    }
     constexpr int CSTEP = S1_THREADS / L;                       // codes per pass of the CTA
     constexpr int NIT = (256 + CSTEP - 1) / CSTEP;
     constexpr int BATCH = 8;                                    // loads in flight per thread
