@@ -106,7 +106,9 @@ struct S1 {
     static constexpr int OFFB_PFX = OFFB_BND + (MAX_SCAN_CTAS + 1) * 8; // int [2][PFX_CAP + 1]: page and cost prefix of small batches
     static constexpr int BELOW_BYTES = OFFB_PFX + 2 * (PFX_CAP + 1) * 4;
     // merge buffer (aliases the larger table once a segment's scan is done)
-    static constexpr int MERGE_ACC_BYTES = NCW * HPAD * D * 4;
+    static constexpr int MROW = D + 4;                                  // floats per (warp, head) row of the merge buffer: 16 bytes of padding
+                                                                        // keep the four head rows a warp writes at once on different banks
+    static constexpr int MERGE_ACC_BYTES = NCW * HPAD * MROW * 4;
     static_assert(MERGE_ACC_BYTES + NCW * HPAD * 16 <= (HAS16 ? T16_BYTES : T32_BYTES), "merge buffer must fit in a table");
     static_assert(BELOW_BYTES + (HAS16 ? T16_BYTES : 0) + 2 * VCB_COPY_BYTES <= S1_SMEM_BYTES, "shared memory budget (before alignment)");
     static_assert(S1_THREADS % L == 0, "table build mapping");
@@ -1106,7 +1108,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
         __syncthreads();                                   // scan done everywhere: the tables are dead
         NOVAKV_TICK(5)
         unsigned char* const merge_p = HAS16 ? t16_p : t32_p;
-        float* m_acc = reinterpret_cast<float*>(merge_p);                              // [NCW][HPAD][D]
+        float* m_acc = reinterpret_cast<float*>(merge_p);                              // [NCW][HPAD][MROW]
         float* m_ml = reinterpret_cast<float*>(merge_p + C::MERGE_ACC_BYTES);          // [NCW][HPAD][2]
         float* m_lz = m_ml + NCW * HPAD * 2;                                           // [NCW][HPAD]  (VSQ)
         if (VM && !VSQ) {
@@ -1141,7 +1143,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
             for (int hs = 0; hs < HSETS; ++hs)
 #pragma unroll
                 for (int gb = 0; gb < NGB; ++gb) {
-                    *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + hs * 4 + fc) * D + (8 * gb + fr) * 4) =
+                    *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + hs * 4 + fc) * C::MROW + (8 * gb + fr) * 4) =
                         make_float4(macc[hs][gb][0] * unsh, macc[hs][gb][1] * unsh, macc[hs][gb][2] * unsh, macc[hs][gb][3] * unsh);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) macc[hs][gb][i] = 0.f;
@@ -1166,7 +1168,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
                         a2 += __shfl_xor_sync(0xffffffffu, a2, o); a3 += __shfl_xor_sync(0xffffffffu, a3, o);
                     }
                     if ((h & 3) == fc)
-                        *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + h) * D + (8 * x + fr) * 4) = make_float4(a0, a1, a2, a3);
+                        *reinterpret_cast<float4*>(m_acc + ((size_t)warp * HPAD + h) * C::MROW + (8 * x + fr) * 4) = make_float4(a0, a1, a2, a3);
                 }
             }
 #pragma unroll
@@ -1187,7 +1189,7 @@ novakv_decode_stage1_kernel(const float* __restrict__ qp, const float* __restric
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
                     const float sc = ex2(m_ml[(w * HPAD + h) * 2] - M);
-                    a = fmaf(sc, m_acc[((size_t)w * HPAD + h) * D + c], a);
+                    a = fmaf(sc, m_acc[((size_t)w * HPAD + h) * C::MROW + c], a);
                     if (VSQ) zsum = fmaf(sc, m_lz[w * HPAD + h], zsum);              // zero-points: the same amount on every coefficient
                     lsum = fmaf(sc, m_ml[(w * HPAD + h) * 2 + 1], lsum);
                 }
