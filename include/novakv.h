@@ -334,8 +334,18 @@ novakv_status novakv_last_device_status(novakv_ctx* ctx, novakv_stream stream, u
  * A buffer in page-locked (pinned, device-mapped) host memory is read or written by the kernels
  * directly across the bus; any other host buffer is staged through `staging` with a copy on `stream`.
  * Either way the step's inputs travel host -> device and its output device -> host inside the call.
+ * novakv_step_host_async enqueues the same work and returns without waiting: the host buffers must stay
+ * valid and out_host must not be read until `stream` has been synchronised (or an event recorded behind
+ * the call has completed); novakv_step_host is that call followed by the synchronisation.
  */
 size_t novakv_step_staging_bytes(const novakv_ctx* ctx, int batch, int n_tokens);
+novakv_status novakv_step_host_async(novakv_ctx* ctx, int layer,
+    const void* k_new_host, const void* v_new_host, const int32_t* tok_seq_host,
+    const int32_t* tok_pos_host, int n_tokens, const void* q_host,
+    uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int32_t* seq_lens, int batch, float sm_scale, float* out_host,
+    void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+    novakv_stream stream);
 novakv_status novakv_step_host(novakv_ctx* ctx, int layer,
     const void* k_new_host, const void* v_new_host, const int32_t* tok_seq_host,
     const int32_t* tok_pos_host, int n_tokens, const void* q_host,

@@ -18,7 +18,7 @@ EXPORTED = [
     "novakv_create", "novakv_destroy", "novakv_status_string", "novakv_load_calibration",
     "novakv_page_bytes", "novakv_decode_workspace_bytes", "novakv_encode_append",
     "novakv_decode_attention", "novakv_last_device_status", "novakv_step_staging_bytes",
-    "novakv_step_host", "novakv_search_coefficients", "novakv_bf16_workspace_bytes",
+    "novakv_step_host", "novakv_step_host_async", "novakv_search_coefficients", "novakv_bf16_workspace_bytes",
     "novakv_bf16_decode_attention", "novakv_profile_enable", "novakv_profile_read",
     "novakv_launch_count", "novakv_debug_set_scan_ctas", "novakv_decode_attention_noalloc", "novakv_debug_set_value_path",
     "novakv_scale_page_bytes", "novakv_encode_append_scaled", "novakv_decode_attention_scaled",
@@ -107,7 +107,7 @@ def load_library(path=None):
     lib.novakv_last_device_status.argtypes = [c_void_p, c_void_p, POINTER(c_uint32)]
     lib.novakv_step_staging_bytes.argtypes = [c_void_p, c_int, c_int]
     lib.novakv_step_staging_bytes.restype = c_size_t
-    lib.novakv_step_host.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
+    lib.novakv_step_host_async.argtypes = lib.novakv_step_host.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p,
                                      c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p, c_int, c_float,
                                      c_void_p, c_void_p, c_size_t, c_void_p, c_size_t, c_void_p]
     lib.novakv_search_coefficients.argtypes = [c_void_p, c_int, c_int, c_void_p, c_int, c_void_p, c_void_p]
@@ -314,12 +314,14 @@ class Context:
         return int(self.lib.novakv_step_staging_bytes(self.handle, batch, n_tokens))
 
     def novakv_step_host(self, layer, k_new_host, v_new_host, tok_seq_host, tok_pos_host, q_host, k_pages,
-                         v_pages, page_table, seq_lens, out_host, staging, workspace, sm_scale=None):
-        """Host tensors (ideally pinned) in, host tensor out; the cache stays on the device."""
+                         v_pages, page_table, seq_lens, out_host, staging, workspace, sm_scale=None, wait=True):
+        """Host tensors (ideally pinned) in, host tensor out; the cache stays on the device.  wait=False enqueues
+        the step without waiting for it (``novakv_step_host_async``): read ``out_host`` after a stream sync."""
         n_tokens = int(k_new_host.shape[0]) if k_new_host is not None else 0
         batch = int(q_host.shape[0])
         scale = float(self.head_dim) ** -0.5 if sm_scale is None else float(sm_scale)
-        _check(self.lib, self.lib.novakv_step_host(
+        fn = self.lib.novakv_step_host if wait else self.lib.novakv_step_host_async
+        _check(self.lib, fn(
             self.handle, layer, _ptr(k_new_host), _ptr(v_new_host), _ptr(tok_seq_host), _ptr(tok_pos_host),
             n_tokens, _ptr(q_host), _ptr(k_pages), _ptr(v_pages), int(k_pages.shape[0]), _ptr(page_table),
             int(page_table.shape[1]), _ptr(seq_lens), batch, scale, _ptr(out_host), _ptr(staging),

@@ -474,7 +474,7 @@ extern "C" size_t novakv_step_staging_bytes(const novakv_ctx* ctx, int batch, in
     return 2 * kv + 2 * tok + q + o + 256;
 }
 
-extern "C" novakv_status novakv_step_host(novakv_ctx* ctx, int layer, const void* k_new_host,
+extern "C" novakv_status novakv_step_host_async(novakv_ctx* ctx, int layer, const void* k_new_host,
     const void* v_new_host, const int32_t* tok_seq_host, const int32_t* tok_pos_host, int n_tokens,
     const void* q_host, uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
     int max_pages_per_seq, int32_t* seq_lens, int batch, float sm_scale, float* out_host, void* staging,
@@ -544,7 +544,20 @@ extern "C" novakv_status novakv_step_host(novakv_ctx* ctx, int layer, const void
                                  seq_lens, batch, sm_scale, uout, 1, workspace, workspace_bytes, stream);
     if (st != NOVAKV_OK) return st;
     if (!out_direct) CUDA_OK(cudaMemcpyAsync(out_host, dout, o_b, cudaMemcpyDeviceToHost, s));
-    CUDA_OK(cudaStreamSynchronize(s));
+    return NOVAKV_OK;
+}
+
+extern "C" novakv_status novakv_step_host(novakv_ctx* ctx, int layer, const void* k_new_host,
+    const void* v_new_host, const int32_t* tok_seq_host, const int32_t* tok_pos_host, int n_tokens,
+    const void* q_host, uint8_t* k_pages, uint8_t* v_pages, int n_pages, const int32_t* page_table,
+    int max_pages_per_seq, int32_t* seq_lens, int batch, float sm_scale, float* out_host, void* staging,
+    size_t staging_bytes, void* workspace, size_t workspace_bytes, novakv_stream stream) {
+    const novakv_status st = novakv_step_host_async(ctx, layer, k_new_host, v_new_host, tok_seq_host, tok_pos_host, n_tokens,
+                                                    q_host, k_pages, v_pages, n_pages, page_table, max_pages_per_seq, seq_lens,
+                                                    batch, sm_scale, out_host, staging, staging_bytes, workspace, workspace_bytes,
+                                                    stream);
+    if (st != NOVAKV_OK) return st;
+    CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
     return NOVAKV_OK;
 }
 

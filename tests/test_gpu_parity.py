@@ -255,6 +255,31 @@ def test_step_host_equals_device_calls(qwen):
 
 
 # --------------------------------------------------------------------------- T7: host-injected faults
+def test_step_host_async_gives_the_same_output(qwen):
+    """novakv_step_host_async enqueues the step; after a stream synchronisation the pinned output equals that of
+    the synchronous call (same launch configuration: bitwise)."""
+    from paper_2608_04074_b200.runtime import PagedCache
+    case = qwen
+    lens = np.array([300, 64, 1], np.int32)
+    outs = []
+    for wait in (True, False):
+        cache = PagedCache(case.ctx, lens, capacity_tokens=lens + 1, seed=4)
+        _fill_with_oracle(case, cache, lens, 830)
+        k1, v1, q = case.draw(831, 3, 3)
+        pin = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(dt) if dt else torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+        kh, vh, qh = pin(k1, torch.bfloat16), pin(v1, torch.bfloat16), pin(q, torch.bfloat16)
+        seq, pos = pin(np.arange(3, dtype=np.int32)), pin(lens.copy())
+        out_h = torch.full((3, case.ctx.n_q_heads, case.ctx.head_dim), float("nan"), dtype=torch.float32).pin_memory()
+        staging = torch.empty(case.ctx.novakv_step_staging_bytes(3, 3), dtype=torch.uint8, device="cuda")
+        case.ctx.novakv_step_host(0, kh, vh, seq, pos, qh, cache.k_pages, cache.v_pages, cache.page_table, cache.seq_lens,
+                                  out_h, staging, cache.workspace, wait=wait)
+        torch.cuda.synchronize()
+        assert case.ctx.novakv_last_device_status() == 0
+        assert np.array_equal(cache.seq_lens.cpu().numpy(), lens + 1)
+        outs.append(out_h.clone())
+    assert torch.isfinite(outs[0]).all() and torch.equal(outs[0], outs[1])
+
+
 def test_faults_are_reported_not_trapped(qwen):
     from paper_2608_04074_b200.binding import Context, NovaKVError
     case = qwen
