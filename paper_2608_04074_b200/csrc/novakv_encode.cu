@@ -11,7 +11,11 @@
 // binary64 by the whole warp (certified search).  The binary32 result is kept only where it provably
 // equals the binary64 one.
 #include <math_constants.h>
+#ifdef NOVAKV_TIMING
+#include <cstdio>
+#endif
 
+#include <atomic>
 #include <cooperative_groups.h>
 
 #include "novakv_internal.cuh"
@@ -565,16 +569,27 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 // group of one (head, side) and stages only its 4 columns of the transform (4 KB of binary64) and its
 // group's codebook (4 KB), so the work spreads over L/4 * Hkv * 2 CTAs.  A pass covers tp tokens
 // (tp = 1, 2, ... 32, the smallest power of two that holds the batch, at most 32): lane = grp * tp + token.
-// The 32 / tp lane groups of a token compute the same coefficients (redundantly) and search disjoint
+// The 32 / tp lane groups of a token share its transform (each takes one block of the input dimension, at most 8
+// blocks; a butterfly adds the partial sums, so every lane holds the same coefficients) and search disjoint
 // ranges of the codebook; their minima are merged with the lowest index winning ties.
 // Everything that depends only on the calibration is staged before the grid-dependency wait, so it
 // overlaps the tail of the preceding kernel in the stream.
-// The coefficients are accumulated in binary64 in index order and the search runs in binary64 throughout
-// (at these sizes the kernel is latency-bound, not ALU-bound), so its indices are the exact nearest codewords.
+// The coefficients are accumulated in binary64 (index order inside a block, then the blocks pairwise) and the
+// search runs in binary64 throughout against a binary64 image of the codebook (at these sizes the kernel is
+// latency-bound, not ALU-bound), so its indices are the exact nearest codewords.
 // KSC (key format with a per-token scale): the L/4 CTAs of a (head, side) form a thread-block cluster;
 // each publishes the sums of squares of its 16 coefficients per token in its shared memory, a cluster
 // barrier makes them visible, and every CTA adds the L/4 x 4 partial sums in the same fixed order through
 // distributed shared memory, so that all of them normalise by the same rho.
+// Dynamic shared memory of the append-sized kernel: the warps' columns of the transform, their groups' codebooks
+// widened to binary64 (once, before the grid-dependency wait, instead of once per comparison), and the mean.
+template <int D>
+struct SmallSmem {
+    static constexpr size_t off_cb = sizeof(double) * 4 * D * 4;
+    static constexpr size_t off_mean = off_cb + sizeof(double) * 4 * NOVAKV_C * 4;
+    static constexpr size_t total = off_mean + sizeof(double) * D;
+};
+
 template <int D, int FMT>
 __global__ void __launch_bounds__(128)
 novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
@@ -589,17 +604,25 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                            int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
     constexpr int L = D / NOVAKV_G;
     constexpr bool KSC = FMT >= 1, VSQ = FMT == 2;
-    __shared__ __align__(16) double R_s[4][D][4];
+    extern __shared__ __align__(16) unsigned char small_smem[];
+    double (*R_s)[D][4] = reinterpret_cast<double (*)[D][4]>(small_smem);                                   // [4 warps][D][4]
+    double (*cb_s)[NOVAKV_C][4] = reinterpret_cast<double (*)[NOVAKV_C][4]>(small_smem + SmallSmem<D>::off_cb);   // [4 warps][256][4]
+    double* mean_s = reinterpret_cast<double*>(small_smem + SmallSmem<D>::off_mean);                        // [D]
     __shared__ double ss_s[4][32];                  // KSC: sum of squares of a warp's 4 coefficients, per token of the pass
     __shared__ float mx_s[4][32];                   // VSQ: maximum of a warp's 4 value coefficients (the minimum rides in ss_s)
-    __shared__ float4 cb_s[4][NOVAKV_C];
-    __shared__ double mean_s[D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int l = blockIdx.x * 4 + warp, kvh = blockIdx.y, side = blockIdx.z;
     const __nv_bfloat16* x_new = side == 0 ? k_new : v_new;
     const double* R = (side == 0 ? rk_d : rv_d) + (size_t)kvh * D * D;
     const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + ((size_t)kvh * L + l) * NOVAKV_C * NOVAKV_G);
+#ifdef NOVAKV_TIMING
+    long long tm[6] = {0, 0, 0, 0, 0, 0};
+    long long t_prev = clock64();
+#define NOVAKV_ETICK(i) { const long long t_now = clock64(); tm[i] += t_now - t_prev; t_prev = t_now; }
+#else
+#define NOVAKV_ETICK(i)
+#endif
     {
         // calibration constants -> shared memory; every load is issued before the first store
         double2 ra[D / 32], rb[D / 32];
@@ -618,65 +641,87 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             *reinterpret_cast<double2*>(&R_s[warp][lane + 32 * k][2]) = rb[k];
         }
 #pragma unroll
-        for (int k = 0; k < NOVAKV_C / 32; ++k) cb_s[warp][lane + 32 * k] = cw[k];
+        for (int k = 0; k < NOVAKV_C / 32; ++k) {
+            *reinterpret_cast<double2*>(&cb_s[warp][lane + 32 * k][0]) = make_double2((double)cw[k].x, (double)cw[k].y);
+            *reinterpret_cast<double2*>(&cb_s[warp][lane + 32 * k][2]) = make_double2((double)cw[k].z, (double)cw[k].w);
+        }
         if (threadIdx.x < D) mean_s[threadIdx.x] = mv;
     }
     __syncthreads();
+    NOVAKV_ETICK(0)
     novakv_grid_dependency_wait();           // inputs and the cache may be written by preceding kernels
+    NOVAKV_ETICK(1)
 
     const int tp = 1 << tp_log2;
     const int tok_in_pass = lane & (tp - 1), grp = lane >> tp_log2;
     const int codes_per_grp = NOVAKV_C >> (5 - tp_log2);
     const int c0 = grp * codes_per_grp;
     const bool reporter = blockIdx.x == 0 && warp == 0 && kvh == 0 && side == 0 && grp == 0;
+    // the lane groups of a token also share its transform: each takes one block of the input dimension
+    // (at most 8 blocks), and a butterfly over the lane groups adds the partial sums
+    const int ts_log2 = min(5 - tp_log2, 3);
+    const int part = grp & ((1 << ts_log2) - 1);
+    const int per = (D / 8) >> ts_log2;             // 16-byte chunks of the token row per lane (>= 1)
 
     for (int t0 = 0; t0 < n_tokens; t0 += tp) {
         const int tkn = t0 + tok_in_pass;
         const bool in_range = tkn < n_tokens;
+        int s = -1, pos = 0;
+        if (in_range) { s = tok_seq[tkn]; pos = tok_pos[tkn]; }
+        // this lane's block of its token's row (the loads are in flight together with the token list's)
+        uint4 xr[D / 8];
+        const uint4* xrow = reinterpret_cast<const uint4*>(x_new + ((size_t)(in_range ? tkn : 0) * n_kv_heads + kvh) * D) + part * per;
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c)
+            if (c < per) xr[c] = xrow[c];
         // a pass whose entries are all unused does nothing (the same decision in every warp and CTA: it depends
         // on the token list alone)
-        if (!__any_sync(0xffffffffu, in_range && tok_seq[tkn] != -1)) continue;
-        // this lane's token row (all loads in flight together with the destination lookup)
-        uint4 xr[D / 8];
-        const uint4* xrow = reinterpret_cast<const uint4*>(x_new + ((size_t)(in_range ? tkn : 0) * n_kv_heads + kvh) * D);
+        if (!__any_sync(0xffffffffu, s != -1)) continue;
+        // destination: the page-table entry is requested here and looked at after the transform
+        const bool ok = s >= 0 && s < n_seq && pos >= 0 && pos / NOVAKV_PAGE_TOKENS < max_pages_per_seq;
+        if (s != -1 && !ok && reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
+        int page_raw = -1;
+        if (ok) page_raw = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
+        const int slot = pos % NOVAKV_PAGE_TOKENS;
+        NOVAKV_ETICK(2)
+        // coefficients of group l in binary64: every block of the input dimension in index order, then the blocks
+        // pairwise (neighbours first); all lanes of a token end with the same bits
+        double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
 #pragma unroll
-        for (int i8 = 0; i8 < D / 8; ++i8) xr[i8] = xrow[i8];
-        int page = -1, slot = 0;
-        if (in_range) {
-            const int s = tok_seq[tkn], pos = tok_pos[tkn];
-            if (s == -1) {
-                // unused entry of the token list: skipped
-            } else if (s < 0 || s >= n_seq || pos < 0 || pos / NOVAKV_PAGE_TOKENS >= max_pages_per_seq) {
-                if (reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_TOKEN);
-            } else {
-                page = page_table[(size_t)s * max_pages_per_seq + pos / NOVAKV_PAGE_TOKENS];
-                slot = pos % NOVAKV_PAGE_TOKENS;
-                if (page < 0 || page >= n_pages) {
-                    if (reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
-                    page = -1;
-                } else if (reporter) {
-                    atomicMax(&seq_lens[s], pos + 1);
+        for (int c = 0; c < D / 8; ++c) {
+            if (c < per) {
+                const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&xr[c]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int i = (part * per + c) * 8 + j;
+                    const double xc = (double)__bfloat162float(xb[j]) - mean_s[i];
+                    const double2 r01 = *reinterpret_cast<const double2*>(&R_s[warp][i][0]);
+                    const double2 r23 = *reinterpret_cast<const double2*>(&R_s[warp][i][2]);
+                    acc0 = fma(xc, r01.x, acc0);
+                    acc1 = fma(xc, r01.y, acc1);
+                    acc2 = fma(xc, r23.x, acc2);
+                    acc3 = fma(xc, r23.y, acc3);
                 }
             }
         }
-        // coefficients of group l: binary64 accumulation over the input dimension in index order
-        double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
-#pragma unroll
-        for (int i8 = 0; i8 < D / 8; ++i8) {
-            const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&xr[i8]);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int i = i8 * 8 + j;
-                const double xc = (double)__bfloat162float(xb[j]) - mean_s[i];
-                const double2 r01 = *reinterpret_cast<const double2*>(&R_s[warp][i][0]);
-                const double2 r23 = *reinterpret_cast<const double2*>(&R_s[warp][i][2]);
-                acc0 = fma(xc, r01.x, acc0);
-                acc1 = fma(xc, r01.y, acc1);
-                acc2 = fma(xc, r23.x, acc2);
-                acc3 = fma(xc, r23.y, acc3);
+        for (int b = 0; b < ts_log2; ++b) {
+            const int off = tp << b;
+            acc0 += __shfl_xor_sync(0xffffffffu, acc0, off);
+            acc1 += __shfl_xor_sync(0xffffffffu, acc1, off);
+            acc2 += __shfl_xor_sync(0xffffffffu, acc2, off);
+            acc3 += __shfl_xor_sync(0xffffffffu, acc3, off);
+        }
+        int page = -1;
+        if (ok) {
+            if (page_raw < 0 || page_raw >= n_pages) {
+                if (reporter) atomicOr(dev_status, NOVAKV_DEV_BAD_PAGE);
+            } else {
+                page = page_raw;
+                if (reporter) atomicMax(&seq_lens[s], pos + 1);
             }
         }
         float4 r = make_float4((float)acc0, (float)acc1, (float)acc2, (float)acc3);
+        NOVAKV_ETICK(3)
         int vsq_byte = 0;
         if (KSC) {
             namespace cg = cooperative_groups;
@@ -738,8 +783,9 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
         // The vector to encode is the binary64 coefficient; for normalised keys it is the binary32 quotient.
         double rd[4] = {acc0, acc1, acc2, acc3};
         if (KSC && side == 0) { rd[0] = (double)r.x; rd[1] = (double)r.y; rd[2] = (double)r.z; rd[3] = (double)r.w; }
-        auto dist_d = [&](const float4 c) {
-            const double e0 = rd[0] - (double)c.x, e1 = rd[1] - (double)c.y, e2 = rd[2] - (double)c.z, e3 = rd[3] - (double)c.w;
+        auto dist_d = [&](const double* c) {
+            const double2 c01 = *reinterpret_cast<const double2*>(c), c23 = *reinterpret_cast<const double2*>(c + 2);
+            const double e0 = rd[0] - c01.x, e1 = rd[1] - c01.y, e2 = rd[2] - c23.x, e3 = rd[3] - c23.y;
             return __dadd_rn(__dadd_rn(__dadd_rn(__dmul_rn(e0, e0), __dmul_rn(e1, e1)), __dmul_rn(e2, e2)), __dmul_rn(e3, e3));
         };
         double best = dist_d(cb_s[warp][c0]);
@@ -755,6 +801,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
             if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
         }
+        NOVAKV_ETICK(4)
         if (VSQ && side == 1) bi = vsq_byte;             // scalar codec: the byte holds four levels, no search result
         if (grp == 0 && page >= 0) {
             const size_t base = ((size_t)page * n_kv_heads + kvh) * (NOVAKV_PAGE_TOKENS * L);
@@ -762,6 +809,12 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             else v_pages[base + novakv_v_offset<L>(slot, l)] = (uint8_t)bi;
         }
     }
+#ifdef NOVAKV_TIMING
+    NOVAKV_ETICK(5)
+    if (threadIdx.x == 0 && blockIdx.y == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
+        printf("append cta (%d,%d,%d) clocks: constants %lld dependency wait %lld rows+lookup %lld transform %lld scale+search %lld store %lld\n",
+               blockIdx.x, blockIdx.y, blockIdx.z, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5]);
+#endif
 }
 
 // Search only, from given binary32 coefficients [n][Hkv][D]; logical indices out [n][Hkv][L].
@@ -808,8 +861,23 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         novakv_prof_scope ps(ctx, 1, stream);
         int tp_log2 = 0;
         while ((1 << tp_log2) < n_tokens && tp_log2 < 5) ++tp_log2;
+        auto small = v_meta ? novakv_encode_small_kernel<D, 2>
+                            : (k_scales ? novakv_encode_small_kernel<D, 1> : novakv_encode_small_kernel<D, 0>);
+        {
+            // more than 48 KB of dynamic shared memory: opted in once per kernel and device
+            static std::atomic<uint64_t> opted[3];
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess) return NOVAKV_ECUDA;
+            const int f = v_meta ? 2 : (k_scales ? 1 : 0);
+            const uint64_t bit = 1ull << (dev & 63);
+            if (!(opted[f].load(std::memory_order_acquire) & bit)) {
+                if (cudaFuncSetAttribute(small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmallSmem<D>::total) != cudaSuccess)
+                    return NOVAKV_ECUDA;
+                opted[f].fetch_or(bit, std::memory_order_release);
+            }
+        }
         if (k_scales == nullptr) {
-            novakv_launch_pdl(novakv_encode_small_kernel<D, 0>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos,
+            novakv_launch_pdl(novakv_encode_small_kernel<D, 0>, grid, dim3(128), SmallSmem<D>::total, stream, k_new, v_new, tok_seq, tok_pos,
                               n_tokens, tp_log2, ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages,
                               (__nv_bfloat16*)nullptr, (__nv_bfloat16*)nullptr, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
                               ctx->cfg.n_kv_heads, ctx->dev_status);
@@ -818,6 +886,7 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = grid;
             cfg.blockDim = dim3(128);
+            cfg.dynamicSmemBytes = SmallSmem<D>::total;
             cfg.stream = stream;
             cudaLaunchAttribute attr[2];
             attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -829,7 +898,6 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
             cfg.attrs = attr;
             cfg.numAttrs = 2;
             const int hkv = ctx->cfg.n_kv_heads;
-            auto small = v_meta ? novakv_encode_small_kernel<D, 2> : novakv_encode_small_kernel<D, 1>;
             if (cudaLaunchKernelEx(&cfg, small, k_new, v_new, tok_seq, tok_pos, n_tokens, tp_log2,
                                    (const double*)ly.rk_d, (const double*)ly.rv_d, (const double*)ly.k_mean_d,
                                    (const double*)ly.v_mean_d, (const float*)ly.cb_k, (const float*)ly.cb_v, k_pages, v_pages,
