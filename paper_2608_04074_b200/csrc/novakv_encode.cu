@@ -15,7 +15,6 @@
 #include <cstdio>
 #endif
 
-#include <atomic>
 #include <cooperative_groups.h>
 
 #include "novakv_internal.cuh"
@@ -574,21 +573,36 @@ novakv_encode_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat1
 // ranges of the codebook; their minima are merged with the lowest index winning ties.
 // Everything that depends only on the calibration is staged before the grid-dependency wait, so it
 // overlaps the tail of the preceding kernel in the stream.
-// The coefficients are accumulated in binary64 (index order inside a block, then the blocks pairwise) and the
-// search runs in binary64 throughout against a binary64 image of the codebook (at these sizes the kernel is
-// latency-bound, not ALU-bound), so its indices are the exact nearest codewords.
+// The coefficients are accumulated in binary64 (index order inside a block, then the blocks pairwise).  The
+// search is the certified one of the tiled kernel: binary32 ranking, and a binary64 search by the whole warp
+// wherever the two nearest codewords are closer than binary32 rounding can resolve (the binary64 pipe is the
+// slowest unit of the SM: a binary64 search of every token was 60 % of this kernel's time after the launch).
 // KSC (key format with a per-token scale): the L/4 CTAs of a (head, side) form a thread-block cluster;
 // each publishes the sums of squares of its 16 coefficients per token in its shared memory, a cluster
 // barrier makes them visible, and every CTA adds the L/4 x 4 partial sums in the same fixed order through
 // distributed shared memory, so that all of them normalise by the same rho.
-// Dynamic shared memory of the append-sized kernel: the warps' columns of the transform, their groups' codebooks
-// widened to binary64 (once, before the grid-dependency wait, instead of once per comparison), and the mean.
-template <int D>
-struct SmallSmem {
-    static constexpr size_t off_cb = sizeof(double) * 4 * D * 4;
-    static constexpr size_t off_mean = off_cb + sizeof(double) * 4 * NOVAKV_C * 4;
-    static constexpr size_t total = off_mean + sizeof(double) * D;
-};
+// Binary64 search of one coefficient vector (the same in every lane) against a group's 256 codewords by the
+// whole warp: lane i takes codewords i, i + 32, ... in ascending order with a strict '<'; the lanes' minima are
+// merged with the lowest index winning ties.  The distance is the plain sum of the four squares, every
+// operation rounded to binary64.
+__device__ __forceinline__ int exact_search_warp(const double (&rd)[4], const float4* cb /* shared, [256] */, int lane) {
+    double best = CUDART_INF;
+    int bi = lane;
+#pragma unroll
+    for (int j = 0; j < NOVAKV_C / 32; ++j) {
+        const float4 c = cb[lane + 32 * j];
+        const double e0 = rd[0] - (double)c.x, e1 = rd[1] - (double)c.y, e2 = rd[2] - (double)c.z, e3 = rd[3] - (double)c.w;
+        const double dd = __dadd_rn(__dadd_rn(__dadd_rn(__dmul_rn(e0, e0), __dmul_rn(e1, e1)), __dmul_rn(e2, e2)), __dmul_rn(e3, e3));
+        if (dd < best) { best = dd; bi = lane + 32 * j; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    return bi;
+}
 
 template <int D, int FMT>
 __global__ void __launch_bounds__(128)
@@ -604,10 +618,9 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                            int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
     constexpr int L = D / NOVAKV_G;
     constexpr bool KSC = FMT >= 1, VSQ = FMT == 2;
-    extern __shared__ __align__(16) unsigned char small_smem[];
-    double (*R_s)[D][4] = reinterpret_cast<double (*)[D][4]>(small_smem);                                   // [4 warps][D][4]
-    double (*cb_s)[NOVAKV_C][4] = reinterpret_cast<double (*)[NOVAKV_C][4]>(small_smem + SmallSmem<D>::off_cb);   // [4 warps][256][4]
-    double* mean_s = reinterpret_cast<double*>(small_smem + SmallSmem<D>::off_mean);                        // [D]
+    __shared__ __align__(16) double R_s[4][D][4];
+    __shared__ float4 cb_s[4][NOVAKV_C];
+    __shared__ double mean_s[D];
     __shared__ double ss_s[4][32];                  // KSC: sum of squares of a warp's 4 coefficients, per token of the pass
     __shared__ float mx_s[4][32];                   // VSQ: maximum of a warp's 4 value coefficients (the minimum rides in ss_s)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -641,10 +654,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             *reinterpret_cast<double2*>(&R_s[warp][lane + 32 * k][2]) = rb[k];
         }
 #pragma unroll
-        for (int k = 0; k < NOVAKV_C / 32; ++k) {
-            *reinterpret_cast<double2*>(&cb_s[warp][lane + 32 * k][0]) = make_double2((double)cw[k].x, (double)cw[k].y);
-            *reinterpret_cast<double2*>(&cb_s[warp][lane + 32 * k][2]) = make_double2((double)cw[k].z, (double)cw[k].w);
-        }
+        for (int k = 0; k < NOVAKV_C / 32; ++k) cb_s[warp][lane + 32 * k] = cw[k];
         if (threadIdx.x < D) mean_s[threadIdx.x] = mv;
     }
     __syncthreads();
@@ -779,27 +789,47 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             }
             cluster.sync();                             // partial sums may be overwritten by the next pass / CTAs may exit
         }
-        // this lane group's range of the codebook in binary64, ascending with a strict '<' (first minimum).
         // The vector to encode is the binary64 coefficient; for normalised keys it is the binary32 quotient.
         double rd[4] = {acc0, acc1, acc2, acc3};
         if (KSC && side == 0) { rd[0] = (double)r.x; rd[1] = (double)r.y; rd[2] = (double)r.z; rd[3] = (double)r.w; }
-        auto dist_d = [&](const double* c) {
-            const double2 c01 = *reinterpret_cast<const double2*>(c), c23 = *reinterpret_cast<const double2*>(c + 2);
-            const double e0 = rd[0] - c01.x, e1 = rd[1] - c01.y, e2 = rd[2] - c23.x, e3 = rd[3] - c23.y;
-            return __dadd_rn(__dadd_rn(__dadd_rn(__dmul_rn(e0, e0), __dmul_rn(e1, e1)), __dmul_rn(e2, e2)), __dmul_rn(e3, e3));
-        };
-        double best = dist_d(cb_s[warp][c0]);
+        // Certified search, as in the tiled kernel: this lane group's range of the codebook is ranked in binary32
+        // from the coefficient rounded to binary32 (ascending, strict '<': first minimum), with the second-smallest
+        // distance tracked beside the smallest (equal distances count as two: their gap is zero).
+        float best = CUDART_INF_F, sec = CUDART_INF_F;
         int bi = c0;
 #pragma unroll 4
-        for (int c = 1; c < codes_per_grp; ++c) {
-            const double dd = dist_d(cb_s[warp][c0 + c]);
+        for (int c = 0; c < codes_per_grp; ++c) {
+            const float4 cw = cb_s[warp][c0 + c];
+            const float e0 = r.x - cw.x, e1 = r.y - cw.y, e2 = r.z - cw.z, e3 = r.w - cw.w;
+            const float dd = fmaf(e3, e3, fmaf(e2, e2, fmaf(e1, e1, e0 * e0)));
+            sec = fminf(sec, fmaxf(best, dd));
             if (dd < best) { best = dd; bi = c0 + c; }
         }
         // merge the groups of a token: smaller distance wins, equal distances keep the lower index
         for (int off = tp; off < 32; off <<= 1) {
-            const double ob = __shfl_xor_sync(0xffffffffu, best, off);
+            const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+            const float os = __shfl_xor_sync(0xffffffffu, sec, off);
             const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            sec = fminf(fminf(sec, os), fmaxf(best, ob));
             if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        }
+        // Where binary32 rounding (of the coefficient: at most 2^-24 per component, none for the quotient, which is
+        // a binary32 number; and of the distance) can have changed the order of the two nearest codewords, the whole
+        // warp searches that token's group again in binary64.
+        {
+            float delta = 0.f;
+            if (!(KSC && side == 0))
+                delta = 5.97e-8f * sqrtf(fmaf(r.x, r.x, fmaf(r.y, r.y, fmaf(r.z, r.z, r.w * r.w)))) * 1.0001f;
+            const bool need = grp == 0 && s != -1 && !(VSQ && side == 1) && needs_exact_search(best, sec, delta);
+            unsigned todo = __ballot_sync(0xffffffffu, need);
+            while (todo) {
+                const int src = __ffs(todo) - 1;             // (a lane of lane group 0: its index is the token's)
+                todo &= todo - 1;
+                const double rs[4] = {__shfl_sync(0xffffffffu, rd[0], src), __shfl_sync(0xffffffffu, rd[1], src),
+                                      __shfl_sync(0xffffffffu, rd[2], src), __shfl_sync(0xffffffffu, rd[3], src)};
+                const int res = exact_search_warp(rs, cb_s[warp], lane);
+                if (tok_in_pass == src) bi = res;
+            }
         }
         NOVAKV_ETICK(4)
         if (VSQ && side == 1) bi = vsq_byte;             // scalar codec: the byte holds four levels, no search result
@@ -863,21 +893,8 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
         while ((1 << tp_log2) < n_tokens && tp_log2 < 5) ++tp_log2;
         auto small = v_meta ? novakv_encode_small_kernel<D, 2>
                             : (k_scales ? novakv_encode_small_kernel<D, 1> : novakv_encode_small_kernel<D, 0>);
-        {
-            // more than 48 KB of dynamic shared memory: opted in once per kernel and device
-            static std::atomic<uint64_t> opted[3];
-            int dev = 0;
-            if (cudaGetDevice(&dev) != cudaSuccess) return NOVAKV_ECUDA;
-            const int f = v_meta ? 2 : (k_scales ? 1 : 0);
-            const uint64_t bit = 1ull << (dev & 63);
-            if (!(opted[f].load(std::memory_order_acquire) & bit)) {
-                if (cudaFuncSetAttribute(small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmallSmem<D>::total) != cudaSuccess)
-                    return NOVAKV_ECUDA;
-                opted[f].fetch_or(bit, std::memory_order_release);
-            }
-        }
         if (k_scales == nullptr) {
-            novakv_launch_pdl(novakv_encode_small_kernel<D, 0>, grid, dim3(128), SmallSmem<D>::total, stream, k_new, v_new, tok_seq, tok_pos,
+            novakv_launch_pdl(novakv_encode_small_kernel<D, 0>, grid, dim3(128), 0, stream, k_new, v_new, tok_seq, tok_pos,
                               n_tokens, tp_log2, ly.rk_d, ly.rv_d, ly.k_mean_d, ly.v_mean_d, ly.cb_k, ly.cb_v, k_pages, v_pages,
                               (__nv_bfloat16*)nullptr, (__nv_bfloat16*)nullptr, n_pages, page_table, max_pages_per_seq, n_seq, seq_lens,
                               ctx->cfg.n_kv_heads, ctx->dev_status);
@@ -886,7 +903,6 @@ novakv_status launch_encode_t(novakv_ctx* ctx, const novakv_layer& ly, const __n
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = grid;
             cfg.blockDim = dim3(128);
-            cfg.dynamicSmemBytes = SmallSmem<D>::total;
             cfg.stream = stream;
             cudaLaunchAttribute attr[2];
             attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
