@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 from gpu_common import Case, check_indices, check_output, NEAR_TIE
-from paper_2608_04074_b200 import synth, workloads
+from paper_2608_04074_b200 import calib, synth, workloads
 
 pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
@@ -104,6 +104,47 @@ def test_encode_append_matches_oracle_indices(name, add, request):
     if add[3] > 0:
         kk, _ = cache.load_logical(3, 0, 130)
         assert not kk.any()
+
+
+@pytest.mark.parametrize("name", ["tiny", "qwen"])
+def test_equal_codewords_lowest_index_wins(name, request):
+    """Exact ties (Alg. 1 line 7 with the lowest index winning): the upper half of every codebook is made a copy
+    of the lower half, so every search ends in an exact tie between c and c + 128.  Both kernels of the write path
+    (8 tokens: the per-group append kernel; 300 tokens: the tiled kernel) must store the lower index - a tie is a
+    zero gap in the binary32 ranking, so every group goes through the binary64 re-search of the certified search.
+    The oracle's gaps are all zero here; the near-tie band comes from a second oracle whose upper half is moved far
+    away instead (same decisions, gap = distance between the two nearest different codewords)."""
+    import dataclasses
+    from oracle import novakv_oracle as O
+    from paper_2608_04074_b200.binding import Context
+    from paper_2608_04074_b200.runtime import PagedCache
+    base = request.getfixturevalue(name)
+    cal = dataclasses.replace(base.cal, cb_k=base.cal.cb_k.copy(), cb_v=base.cal.cb_v.copy())
+    cal.cb_k[:, :, 128:] = cal.cb_k[:, :, :128]
+    cal.cb_v[:, :, 128:] = cal.cb_v[:, :, :128]
+    cal.cb_v = calib.snap_to_byte_grid(cal.cb_v)     # (the extremes may have gone with the upper half: new grid)
+    assert np.array_equal(cal.cb_v[:, :, 128:], cal.cb_v[:, :, :128])
+    far = dataclasses.replace(base.cal, cb_k=cal.cb_k.copy(), cb_v=cal.cb_v.copy())
+    far.cb_k[:, :, 128:] += 1.0e3 * np.abs(cal.cb_k).max()
+    far.cb_v[:, :, 128:] += 1.0e3 * np.abs(cal.cb_v).max()
+    oracle, oracle_far = O.Oracle.from_calibration(cal), O.Oracle.from_calibration(far)
+    shape = base.wl.shape
+    ctx = Context(shape.n_q_heads, shape.n_kv_heads, shape.head_dim)
+    ctx.novakv_load_calibration(0, cal)
+    for n in (8, 300):
+        k, v, _ = base.draw(900 + n, n, 1)
+        cache = PagedCache(ctx, np.zeros(1, np.int32), capacity_tokens=np.array([n], np.int32), seed=3)
+        cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(np.zeros(n, np.int32)),
+                     _dev(np.arange(n, dtype=np.int32)))
+        assert ctx.novakv_last_device_status() == 0
+        enc = oracle.encode(k.astype(np.float64), v.astype(np.float64))
+        enc_far = oracle_far.encode(k.astype(np.float64), v.astype(np.float64))
+        got_k, got_v = cache.load_logical(0, 0, n)
+        for which, got in (("k", got_k), ("v", got_v)):
+            assert (enc[which + "idx"] < 128).all() and not enc[which + "gap"].any()     # the oracle: ties, lower index
+            assert np.array_equal(enc[which + "idx"], enc_far[which + "idx"])
+            assert (got < 128).all(), f"{which}, {n} tokens: the higher index of two equal codewords was stored"
+            check_indices(got, enc_far, which)
 
 
 # --------------------------------------------------------------------------- T3/T5: decode on the oracle's indices
