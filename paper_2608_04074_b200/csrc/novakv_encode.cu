@@ -618,9 +618,13 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                            int32_t* __restrict__ seq_lens, int n_kv_heads, uint32_t* __restrict__ dev_status) {
     constexpr int L = D / NOVAKV_G;
     constexpr bool KSC = FMT >= 1, VSQ = FMT == 2;
-    __shared__ __align__(16) double R_s[4][D][4];
+    // Rows of the transform and the mean are indexed by i + i / (D / 4): one row of padding after every quarter of
+    // the input dimension, so that lane groups working on different blocks of it read different banks.
+    constexpr int DP = D + 4;
+    auto padded = [](int i) { return i + i / (D / 4); };
+    __shared__ __align__(16) double R_s[4][DP][4];
     __shared__ float4 cb_s[4][NOVAKV_C];
-    __shared__ double mean_s[D];
+    __shared__ double mean_s[DP];
     __shared__ double ss_s[4][32];                  // KSC: sum of squares of a warp's 4 coefficients, per token of the pass
     __shared__ float mx_s[4][32];                   // VSQ: maximum of a warp's 4 value coefficients (the minimum rides in ss_s)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -630,7 +634,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
     const double* mean = (side == 0 ? k_mean_d : v_mean_d) + (size_t)kvh * D;
     const float4* cb_g = reinterpret_cast<const float4*>((side == 0 ? cb_k : cb_v) + ((size_t)kvh * L + l) * NOVAKV_C * NOVAKV_G);
 #ifdef NOVAKV_TIMING
-    long long tm[6] = {0, 0, 0, 0, 0, 0};
+    long long tm[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     long long t_prev = clock64();
 #define NOVAKV_ETICK(i) { const long long t_now = clock64(); tm[i] += t_now - t_prev; t_prev = t_now; }
 #else
@@ -650,12 +654,12 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
         const double mv = threadIdx.x < D ? mean[threadIdx.x] : 0.0;
 #pragma unroll
         for (int k = 0; k < D / 32; ++k) {
-            *reinterpret_cast<double2*>(&R_s[warp][lane + 32 * k][0]) = ra[k];
-            *reinterpret_cast<double2*>(&R_s[warp][lane + 32 * k][2]) = rb[k];
+            *reinterpret_cast<double2*>(&R_s[warp][padded(lane + 32 * k)][0]) = ra[k];
+            *reinterpret_cast<double2*>(&R_s[warp][padded(lane + 32 * k)][2]) = rb[k];
         }
 #pragma unroll
         for (int k = 0; k < NOVAKV_C / 32; ++k) cb_s[warp][lane + 32 * k] = cw[k];
-        if (threadIdx.x < D) mean_s[threadIdx.x] = mv;
+        if (threadIdx.x < D) mean_s[padded(threadIdx.x)] = mv;
     }
     __syncthreads();
     NOVAKV_ETICK(0)
@@ -703,7 +707,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                 const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(&xr[c]);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const int i = (part * per + c) * 8 + j;
+                    const int i = padded((part * per + c) * 8 + j);
                     const double xc = (double)__bfloat162float(xb[j]) - mean_s[i];
                     const double2 r01 = *reinterpret_cast<const double2*>(&R_s[warp][i][0]);
                     const double2 r23 = *reinterpret_cast<const double2*>(&R_s[warp][i][2]);
@@ -793,18 +797,46 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
         double rd[4] = {acc0, acc1, acc2, acc3};
         if (KSC && side == 0) { rd[0] = (double)r.x; rd[1] = (double)r.y; rd[2] = (double)r.z; rd[3] = (double)r.w; }
         // Certified search, as in the tiled kernel: this lane group's range of the codebook is ranked in binary32
-        // from the coefficient rounded to binary32 (ascending, strict '<': first minimum), with the second-smallest
+        // from the coefficient rounded to binary32 (first minimum in ascending order), with the second-smallest
         // distance tracked beside the smallest (equal distances count as two: their gap is zero).
+        // The range is a whole number of blocks of 8 codewords.  Per block the 8 distances are independent; the block
+        // minimum updates the running minimum with a strict '<' (keeps the first block that attains it), and the
+        // larger of the two feeds the second-smallest value.  The winning block is then evaluated again (same
+        // instructions, same bits): its first distance equal to the minimum gives the index, the others are the
+        // remaining candidates for the second-smallest value.
+        const float4* cbw = &cb_s[warp][c0];
+        auto dist8 = [&](int blk, float (&d)[8]) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float4 cw = cbw[blk * 8 + k];
+                const float e0 = r.x - cw.x, e1 = r.y - cw.y, e2 = r.z - cw.z, e3 = r.w - cw.w;
+                d[k] = fmaf(e3, e3, fmaf(e2, e2, fmaf(e1, e1, e0 * e0)));
+            }
+        };
         float best = CUDART_INF_F, sec = CUDART_INF_F;
-        int bi = c0;
-#pragma unroll 4
-        for (int c = 0; c < codes_per_grp; ++c) {
-            const float4 cw = cb_s[warp][c0 + c];
-            const float e0 = r.x - cw.x, e1 = r.y - cw.y, e2 = r.z - cw.z, e3 = r.w - cw.w;
-            const float dd = fmaf(e3, e3, fmaf(e2, e2, fmaf(e1, e1, e0 * e0)));
-            sec = fminf(sec, fmaxf(best, dd));
-            if (dd < best) { best = dd; bi = c0 + c; }
+        int bblk = 0;
+#pragma unroll 2
+        for (int blk = 0; blk < codes_per_grp / 8; ++blk) {
+            float d[8];
+            dist8(blk, d);
+            const float m = fminf(fminf(fminf(d[0], d[1]), fminf(d[2], d[3])), fminf(fminf(d[4], d[5]), fminf(d[6], d[7])));
+            sec = fminf(sec, fmaxf(best, m));
+            if (m < best) { best = m; bblk = blk; }
         }
+        int bi;
+        {
+            float d[8];
+            dist8(bblk, d);
+            int kb = 7;
+#pragma unroll
+            for (int k = 6; k >= 0; --k)
+                if (d[k] == best) kb = k;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k != kb) sec = fminf(sec, d[k]);
+            bi = c0 + bblk * 8 + kb;
+        }
+        NOVAKV_ETICK(6)
         // merge the groups of a token: smaller distance wins, equal distances keep the lower index
         for (int off = tp; off < 32; off <<= 1) {
             const float ob = __shfl_xor_sync(0xffffffffu, best, off);
@@ -813,6 +845,7 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
             sec = fminf(fminf(sec, os), fmaxf(best, ob));
             if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
         }
+        NOVAKV_ETICK(7)
         // Where binary32 rounding (of the coefficient: at most 2^-24 per component, none for the quotient, which is
         // a binary32 number; and of the distance) can have changed the order of the two nearest codewords, the whole
         // warp searches that token's group again in binary64.
@@ -822,6 +855,9 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
                 delta = 5.97e-8f * sqrtf(fmaf(r.x, r.x, fmaf(r.y, r.y, fmaf(r.z, r.z, r.w * r.w)))) * 1.0001f;
             const bool need = grp == 0 && s != -1 && !(VSQ && side == 1) && needs_exact_search(best, sec, delta);
             unsigned todo = __ballot_sync(0xffffffffu, need);
+#ifdef NOVAKV_TIMING
+            tm[8] += __popc(todo);
+#endif
             while (todo) {
                 const int src = __ffs(todo) - 1;             // (a lane of lane group 0: its index is the token's)
                 todo &= todo - 1;
@@ -842,8 +878,8 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
 #ifdef NOVAKV_TIMING
     NOVAKV_ETICK(5)
     if (threadIdx.x == 0 && blockIdx.y == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
-        printf("append cta (%d,%d,%d) clocks: constants %lld dependency wait %lld rows+lookup %lld transform %lld scale+search %lld store %lld\n",
-               blockIdx.x, blockIdx.y, blockIdx.z, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5]);
+        printf("append cta (%d,%d,%d) clocks: constants %lld dependency wait %lld rows+lookup %lld transform %lld ranking %lld merge %lld certificate+re-search %lld (%lld re-searches) store %lld\n",
+               blockIdx.x, blockIdx.y, blockIdx.z, tm[0], tm[1], tm[2], tm[3], tm[6], tm[7], tm[4], tm[8], tm[5]);
 #endif
 }
 
