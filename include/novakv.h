@@ -121,11 +121,12 @@ size_t novakv_decode_workspace_bytes(const novakv_ctx* ctx, int batch);
 /*
  * Write path (Algorithm 1 line 7; Sec. 4 "Complexity"): for each new token t and KV head,
  *     r = (k_t - k_mean) rk,   s = (v_t - v_mean) rv          exact products accumulated in binary64
- * (in index order for append-sized batches, in blocks of four input dimensions on the fp64 tensor path
- * for larger ones: the two differ by less than an ulp of binary64), then for every group l the index of
+ * (append-sized batches: blocks of the input dimension in index order, the blocks added pairwise; larger
+ * ones: blocks of four input dimensions on the fp64 tensor path; the results differ by less than an ulp of
+ * binary64), then for every group l the index of
  * the nearest codeword: exact Euclidean search (Sec. 2.2 "Quantization", App. B "Calibration"), the
  * lowest index winning a tie.  The stored index is the minimiser of the binary64 squared distance
- * sum_i (coef_i - codeword_i)^2 of the binary64 coefficient.  (Large batches evaluate the 256 distances
+ * sum_i (coef_i - codeword_i)^2 of the binary64 coefficient.  (Both kernels evaluate the 256 distances
  * in binary32 first and keep that result only where the two smallest distances are further apart than
  * binary32 rounding can have moved them; every other group is searched again in binary64.  The result
  * can differ from a binary64 reference only where the two nearest codewords are within ~1e-12 relative.)
