@@ -826,7 +826,7 @@ def run_profile_case(args):
         wl = workloads.gpt_oss_20b(batch=args.batch, seq_len=args.seq_len, calib_tokens=2048, lloyd_iters=2)
     elif name == "mix":
         wl = workloads.paged_mix(calib_tokens=2048, lloyd_iters=2)
-    elif name in ("qwen", "encode"):
+    elif name in ("qwen", "encode", "append"):
         wl = workloads.qwen3_8b(batch=args.batch, seq_len=args.seq_len, calib_tokens=2048, lloyd_iters=2)
     else:
         raise SystemExit(f"unknown profile case {name}")
@@ -835,9 +835,16 @@ def run_profile_case(args):
     s = wl.shape
     ctx = Context(s.n_q_heads, s.n_kv_heads, s.head_dim)
     ctx.novakv_load_calibration(0, cal)
-    cache = PagedCache(ctx, wl.seq_lens, seed=3)
+    cache = PagedCache(ctx, wl.seq_lens, capacity_tokens=wl.seq_lens + 1 if name == "append" else None, seed=3)
     times = []
-    if name == "encode":
+    if name == "append":
+        # one new token per sequence at the end of its context (the append of a decode step)
+        k, v = synth.draw_kv(laws, 7300, wl.batch)
+        kd, vd = bf16_tensor(k), bf16_tensor(v)
+        ts = torch.arange(wl.batch, dtype=torch.int32, device="cuda")
+        tp = torch.from_numpy(wl.seq_lens.astype(np.int32)).cuda()
+        fn = lambda: cache.append(0, kd, vd, ts, tp)
+    elif name == "encode":
         T = int(wl.seq_lens.sum())
         k, v = synth.draw_kv(laws, 7200, T)
         kd, vd = bf16_tensor(k), bf16_tensor(v)
@@ -882,7 +889,7 @@ def main():
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--seq-len", type=int, default=16384)
     ap.add_argument("--no-sweep", action="store_true")
-    ap.add_argument("--profile-case", default=None, choices=["qwen", "gptoss", "mix", "encode"],
+    ap.add_argument("--profile-case", default=None, choices=["qwen", "gptoss", "mix", "encode", "append"],
                     help="profiling helper: short decode-only (encode-only) loop of one workload shape")
     ap.add_argument("--calib-tokens", type=int, default=8192, help="calibration tokens per KV head (set-up cost only)")
     ap.add_argument("--lloyd-iters", type=int, default=12, help="Lloyd iterations of the calibration (set-up cost only)")
