@@ -141,6 +141,10 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
                       int32_t* __restrict__ pair_count /* [Hkv * batch] arrival counters of the fused merge, or null */,
                       void* __restrict__ out_fused /* outputs, when the scan kernel itself merges */, int out_is_fp32) {
     const int blk = blockIdx.x;
+#ifdef NOVAKV_TIMING
+    unsigned long long g_p0, g_p1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_p0));
+#endif
     constexpr int PARTS = 512 / D, ROWS = D / PARTS;
     const int b = blk / n_kv_heads, kvh = blk - b * n_kv_heads;
     const int c = threadIdx.x % D, part = threadIdx.x / D;
@@ -200,6 +204,10 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
             }
             if (threadIdx.x == 0) { page_prefix[batch] = carry; cost_prefix[batch] = carry + seg_weight * carry_ne; }
         }
+#ifdef NOVAKV_TIMING
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_p1));
+        if (threadIdx.x == 0) printf("prepare prefix block | ns start %llu end %llu\n", g_p0, g_p1);
+#endif
         return;
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -251,6 +259,11 @@ novakv_prepare_kernel(const __nv_bfloat16* __restrict__ q, const float* __restri
             if (lane == 0) qc[(size_t)b * n_q_heads + kvh * HG + h] = acc;
         }
     }
+#ifdef NOVAKV_TIMING
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_p1));
+    if (threadIdx.x == 0 && (blk == 0 || blk == batch * n_kv_heads - 1))
+        printf("prepare block %d | ns start %llu end %llu\n", blk, g_p0, g_p1);
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1280,7 +1293,14 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
     float vm[(HG * D + NT - 1) / NT];
 #pragma unroll
     for (int k = 0; k < (HG * D + NT - 1) / NT; ++k) vm[k] = v_mean[(size_t)kvh * D + (threadIdx.x + k * NT) % D];
+#ifdef NOVAKV_TIMING
+    unsigned long long g_m0, g_m1, g_m2;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_m0));
+#endif
     novakv_grid_dependency_wait();
+#ifdef NOVAKV_TIMING
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_m1));
+#endif
     const int len = clamp_len(seq_lens[b], max_pages_per_seq);
     const int pages_b = (len + NOVAKV_PAGE_TOKENS - 1) / NOVAKV_PAGE_TOKENS;
     const long P = page_prefix[batch];
@@ -1389,6 +1409,11 @@ novakv_decode_merge_kernel(const float* __restrict__ part_ml, const float* __res
         if (out_is_fp32) reinterpret_cast<float*>(out)[oi] = o;
         else reinterpret_cast<__nv_bfloat16*>(out)[oi] = __float2bfloat16_rn(o);
     }
+#ifdef NOVAKV_TIMING
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_m2));
+    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
+        printf("merge block %d | ns start %llu after-wait %llu end %llu\n", blockIdx.x, g_m0, g_m1, g_m2);
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -636,6 +636,8 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
 #ifdef NOVAKV_TIMING
     long long tm[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     long long t_prev = clock64();
+    unsigned long long g_a0, g_a1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_a0));
 #define NOVAKV_ETICK(i) { const long long t_now = clock64(); tm[i] += t_now - t_prev; t_prev = t_now; }
 #else
 #define NOVAKV_ETICK(i)
@@ -877,9 +879,10 @@ novakv_encode_small_kernel(const __nv_bfloat16* __restrict__ k_new, const __nv_b
     }
 #ifdef NOVAKV_TIMING
     NOVAKV_ETICK(5)
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g_a1));
     if (threadIdx.x == 0 && blockIdx.y == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
-        printf("append cta (%d,%d,%d) clocks: constants %lld dependency wait %lld rows+lookup %lld transform %lld ranking %lld merge %lld certificate+re-search %lld (%lld re-searches) store %lld\n",
-               blockIdx.x, blockIdx.y, blockIdx.z, tm[0], tm[1], tm[2], tm[3], tm[6], tm[7], tm[4], tm[8], tm[5]);
+        printf("append cta (%d,%d,%d) clocks: constants %lld dependency wait %lld rows+lookup %lld transform %lld ranking %lld merge %lld certificate+re-search %lld (%lld re-searches) store %lld | ns start %llu end %llu\n",
+               blockIdx.x, blockIdx.y, blockIdx.z, tm[0], tm[1], tm[2], tm[3], tm[6], tm[7], tm[4], tm[8], tm[5], g_a0, g_a1);
 #endif
 }
 
