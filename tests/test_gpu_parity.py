@@ -106,6 +106,31 @@ def test_encode_append_matches_oracle_indices(name, add, request):
         assert not kk.any()
 
 
+@pytest.mark.parametrize("n", [2, 3, 5, 8, 9, 16, 17])
+@pytest.mark.parametrize("name", ["qwen", "gptoss"])
+def test_append_kernel_every_split_of_the_transform(name, n, request):
+    """The per-group append kernel covers n tokens in passes of tp = 2, 4, 8, 8, 16, 16, 32 lanes here; the 32 / tp lane
+    groups of a token share its transform in 8, 8, 4, 4, 2, 2, 1 blocks of the input dimension (d = 128; d = 64
+    likewise) and split the codebook.  Every split must give the oracle's indices."""
+    case = request.getfixturevalue(name)
+    lens0 = np.array([61, 0, 64], np.int32)              # appended tokens cross a page boundary in sequence 0
+    add = np.array([n - n // 2, 0, n // 2], np.int32)
+    cache = _cache(case, lens0, capacity=lens0 + add)
+    k, v, _ = case.draw(7000 + n, n, 1)
+    tok_seq = np.concatenate([np.full(a, b, np.int32) for b, a in enumerate(add)])
+    tok_pos = np.concatenate([lens0[b] + np.arange(a, dtype=np.int32) for b, a in enumerate(add)])
+    cache.append(0, _dev(k, torch.bfloat16), _dev(v, torch.bfloat16), _dev(tok_seq), _dev(tok_pos))
+    assert case.ctx.novakv_last_device_status() == 0
+    assert np.array_equal(cache.seq_lens.cpu().numpy(), lens0 + add)
+    enc = case.oracle.encode(k.astype(np.float64), v.astype(np.float64))
+    got_k = np.empty_like(enc["kidx"]); got_v = np.empty_like(enc["vidx"])
+    for t in range(n):
+        kk, vv = cache.load_logical(int(tok_seq[t]), int(tok_pos[t]), 1)
+        got_k[t], got_v[t] = kk[0], vv[0]
+    check_indices(got_k, enc, "k")
+    check_indices(got_v, enc, "v")
+
+
 @pytest.mark.parametrize("name", ["tiny", "qwen"])
 def test_equal_codewords_lowest_index_wins(name, request):
     """Exact ties (Alg. 1 line 7 with the lowest index winning): the upper half of every codebook is made a copy
